@@ -1,0 +1,167 @@
+"""ctypes front end of the CPU oracle (TEST INFRASTRUCTURE ONLY).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline / reference leg may import this
+package.  It compiles ``w4a4_oracle.cpp`` with gcc (single thread, ``-O2 -ffp-contract=off``) into a
+shared library next to the source and marshals numpy arrays into it.  Nothing here touches CUDA and
+nothing in the CUDA package imports it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "w4a4_oracle.cpp")
+_LIB = os.path.join(_HERE, "libw4a4_oracle.so")
+CXXFLAGS = ["-O2", "-std=c++17", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared"]
+GROUP = 64
+
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle if the shared library is missing or older than its source."""
+    with _lock:
+        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+            tmp = _LIB + ".tmp%d" % os.getpid()
+            subprocess.run(["g++", *CXXFLAGS, "-o", tmp, _SRC], check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.oracle_f32_to_bf16.restype = ctypes.c_uint16
+        _lib.oracle_f32_to_bf16.argtypes = [ctypes.c_float]
+    return _lib
+
+
+def _p(a, dtype):
+    """Pointer to a C-contiguous numpy array of the given dtype (None -> NULL)."""
+    if a is None:
+        return None
+    assert isinstance(a, np.ndarray) and a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _as(a, dtype):
+    return None if a is None else np.ascontiguousarray(a, dtype=dtype)
+
+
+def f32_to_bf16(x: float) -> int:
+    return int(_load().oracle_f32_to_bf16(ctypes.c_float(x)))
+
+
+def quantize(X_bits, lam, rho, want_xhat=False):
+    """Eq. 3-5, 8-9 on every row.  X_bits: [M, K] uint16 BF16 patterns.  -> codes int8 [M,K], scales f32 [M,G]."""
+    X_bits = _as(X_bits, np.uint16)
+    lam = _as(lam, np.float32)
+    M, K = X_bits.shape
+    q = np.empty((M, K), np.int8)
+    s = np.empty((M, K // GROUP), np.float32)
+    xh = np.empty((M, K), np.float32) if want_xhat else None
+    rc = _load().oracle_quantize(_p(X_bits, np.uint16), _p(lam, np.float32), ctypes.c_float(rho), M, K,
+                                 _p(q, np.int8), _p(s, np.float32), _p(xh, np.float32))
+    assert rc == 0
+    return (q, s, xh) if want_xhat else (q, s)
+
+
+def lowrank_down(X_bits, lam, L1_bits):
+    """T = X-hat L1 (Eq. 7), FP64 accumulation, returned as FP32 [M, r]."""
+    X_bits = _as(X_bits, np.uint16)
+    lam = _as(lam, np.float32)
+    L1_bits = _as(L1_bits, np.uint16)
+    M, K = X_bits.shape
+    r = L1_bits.shape[1]
+    T = np.empty((M, r), np.float32)
+    rc = _load().oracle_lowrank_down(_p(X_bits, np.uint16), _p(lam, np.float32), _p(L1_bits, np.uint16), M, K, r,
+                                     _p(T, np.float32))
+    assert rc == 0
+    return T
+
+
+def partials(q, qw):
+    """Per-group integer partial sums P[m, g, n] (Eq. 7, 4-bit branch before rescaling)."""
+    q = _as(q, np.int8)
+    qw = _as(qw, np.int8)
+    M, K = q.shape
+    N = qw.shape[1]
+    P = np.empty((M, K // GROUP, N), np.int32)
+    rc = _load().oracle_partials(_p(q, np.int8), _p(qw, np.int8), M, K, N, _p(P, np.int32))
+    assert rc == 0
+    return P
+
+
+def assemble(P, s, sw, T, L2_bits, bias):
+    """Eq. 7/11: Y64 [M,N] and its BF16 rounding from partials, scales, low-rank pieces and bias."""
+    P = _as(P, np.int32)
+    s = _as(s, np.float32)
+    sw = _as(sw, np.float32)
+    M, G, N = P.shape
+    K = G * GROUP
+    r = 0 if T is None else T.shape[1]
+    T = _as(T, np.float32)
+    L2_bits = _as(L2_bits, np.uint16)
+    bias = _as(bias, np.float32)
+    Y = np.empty((M, N), np.float64)
+    Yb = np.empty((M, N), np.uint16)
+    rc = _load().oracle_assemble(_p(P, np.int32), _p(s, np.float32), _p(sw, np.float32), _p(T, np.float32),
+                                 _p(L2_bits, np.uint16), _p(bias, np.float32), M, K, N, r, _p(Y, np.float64),
+                                 _p(Yb, np.uint16))
+    assert rc == 0
+    return Y, Yb
+
+
+def forward_rows(X_bits, rows, lam, rho, L1_bits, L2_bits, qw, sw, bias, want_partials=False):
+    """Whole layer on the chosen rows of X.  Returns a dict with q, s, T, (P), Y64, Ybf16 indexed by position in rows."""
+    X_bits = _as(X_bits, np.uint16)
+    rows = _as(rows, np.int32)
+    lam = _as(lam, np.float32)
+    qw = _as(qw, np.int8)
+    sw = _as(sw, np.float32)
+    bias = _as(bias, np.float32)
+    M, K = X_bits.shape
+    N = qw.shape[1]
+    G = K // GROUP
+    r = 0 if L1_bits is None else L1_bits.shape[1]
+    L1_bits = _as(L1_bits, np.uint16)
+    L2_bits = _as(L2_bits, np.uint16)
+    n = rows.shape[0]
+    assert rows.min(initial=0) >= 0 and rows.max(initial=0) < max(M, 1)
+    out = dict(q=np.empty((n, K), np.int8), s=np.empty((n, G), np.float32),
+               T=np.empty((n, r), np.float32) if r > 0 else None,
+               P=np.empty((n, G, N), np.int32) if want_partials else None,
+               Y64=np.empty((n, N), np.float64), Ybf16=np.empty((n, N), np.uint16))
+    rc = _load().oracle_forward_rows(_p(X_bits, np.uint16), _p(rows, np.int32), n, K, N, r, _p(lam, np.float32),
+                                     ctypes.c_float(rho), _p(L1_bits, np.uint16), _p(L2_bits, np.uint16),
+                                     _p(qw, np.int8), _p(sw, np.float32), _p(bias, np.float32),
+                                     _p(out["q"], np.int8), _p(out["s"], np.float32), _p(out["T"], np.float32),
+                                     _p(out["P"], np.int32), _p(out["Y64"], np.float64), _p(out["Ybf16"], np.uint16))
+    assert rc == 0
+    return out
+
+
+def forward_noquant(X, lam, L1, L2, R, bias):
+    """Eq. 5-7 with both quantizers off, FP64 throughout: (X/lam) L1 L2 + (X/lam) R + b."""
+    X = _as(X, np.float64)
+    lam = _as(lam, np.float64)
+    R = _as(R, np.float64)
+    M, K = X.shape
+    N = R.shape[1]
+    r = 0 if L1 is None else L1.shape[1]
+    L1 = _as(L1, np.float64)
+    L2 = _as(L2, np.float64)
+    bias = _as(bias, np.float64)
+    Y = np.empty((M, N), np.float64)
+    rc = _load().oracle_forward_noquant(_p(X, np.float64), _p(lam, np.float64), _p(L1, np.float64), _p(L2, np.float64),
+                                        _p(R, np.float64), _p(bias, np.float64), M, K, N, r, _p(Y, np.float64))
+    assert rc == 0
+    return Y
