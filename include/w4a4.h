@@ -1,0 +1,124 @@
+/*
+ * libw4a4 -- W4A4 + low-rank linear layer forward for NVIDIA B200 (sm_100a).
+ *
+ * The layer computed here is the inference-time form of the paper's quantized linear (Eq. 7 and
+ * Eq. 11 of "Timestep-Aware SVDQuant-GPTQ for W4A4 Quantization of Wan2.2-I2V"):
+ *
+ *     Y = Q_A(Xh; rho[expert, layer, bin]) * Qw  +  (Xh * L1) * L2  +  b ,     Xh = X * diag(lambda)^-1
+ *
+ * Xh is the smoothed activation (Eq. 5), Q_A the symmetric 4-bit quantizer of Eq. 3-4 applied per
+ * token and per group of 64 consecutive input channels with the clip threshold of Eq. 8-9
+ * (threshold = rho * group absolute maximum, scale = threshold / 7, codes clipped to [-8, 7],
+ * round half to even), Qw the 4-bit residual weight with one FP32 scale per (64-row group, output
+ * column) (Eq. 6), and L1 (K x r), L2 (r x N) the BF16 low-rank pair (Eq. 6).  rho is fetched on the
+ * device from a table indexed by (expert, layer, timestep bin) (Sec. III-C, last paragraph).
+ *
+ * Every step runs in hand-written CUDA kernels; there is no CPU fallback.  All entry points return
+ * a status code, never throw and never abort.  Unless stated otherwise pointers are DEVICE pointers
+ * owned by the caller, 16-byte aligned, and only read/written during the call (asynchronously, on
+ * the given stream, for the forward calls).
+ */
+#ifndef W4A4_H_
+#define W4A4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  W4A4_OK = 0,
+  W4A4_ERR_INVALID_ARG = 1, /* NULL pointer, out-of-range expert / bin / layer, misaligned buffer */
+  W4A4_ERR_SHAPE = 2,       /* unsupported K, N, r, group or M beyond the context's limits */
+  W4A4_ERR_ALLOC = 3,       /* device or host allocation failed (setup calls only) */
+  W4A4_ERR_CUDA = 4,        /* a CUDA runtime / driver call or a kernel launch failed */
+  W4A4_ERR_ARCH = 5,        /* the device is not compute capability 10.x */
+  W4A4_ERR_TIMEOUT = 6      /* a kernel gave up on a bounded wait and returned early (see w4a4_query_status) */
+} w4a4_status_t;
+
+typedef struct w4a4_ctx* w4a4_ctx_t;      /* per-stream workspace: activation codes, scales, low-rank intermediate */
+typedef struct w4a4_layer* w4a4_handle_t; /* one layer position: packed constants of all its experts */
+
+/*
+ * Constants of one layer position for all experts (Eq. 5-6; Sec. I: one weight set per expert).
+ * Arrays are indexed by expert.  With pointers_on_device == 0 the inner pointers are HOST pointers,
+ * with 1 they are DEVICE pointers; the outer arrays are always host arrays.  Everything is copied /
+ * repacked during w4a4_pack_weights and may be freed when it returns.
+ */
+typedef struct {
+  int K;           /* input channels C_in, multiple of 64 */
+  int N;           /* output channels C_out, multiple of 128 */
+  int r;           /* low-rank width: 0, 16, 32 or 64 */
+  int group;       /* quantization group along K: must be 64 */
+  int num_experts; /* >= 1 */
+  int num_bins;    /* timestep bins per (expert, layer) in the clip table */
+  int num_layers;  /* layers per expert in the clip table */
+  int layer_id;    /* this layer's index into the clip table */
+  int pointers_on_device;
+  const int8_t* const* qweight;  /* [E] -> K x N row-major, one code per byte, values in [-8, 7] */
+  const float* const* wscale;    /* [E] -> (K/64) x N row-major FP32 */
+  const float* const* lambda;    /* [E] -> K FP32, > 0 (diagonal of the smoothing matrix D_l) */
+  const uint16_t* const* L1;     /* [E] -> K x r row-major BF16 bit patterns (ignored if r == 0) */
+  const uint16_t* const* L2;     /* [E] -> r x N row-major BF16 bit patterns (ignored if r == 0) */
+  const float* const* bias;      /* [E] -> N FP32; the array or an entry may be NULL (no bias) */
+} w4a4_weight_desc_t;
+
+/* Creates a context on `device` whose workspace fits M <= max_M tokens, K <= max_K, r <= max_r.
+ * One context serves one stream at a time (calls on it reuse the same workspace in stream order).
+ * Sec. III (whole forward) -- the workspace holds Q_A(Xh), its scales and Xh*L1 between the two kernels. */
+w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_ctx_t* out);
+void w4a4_ctx_destroy(w4a4_ctx_t ctx);
+
+/* Copies and repacks one layer's constants (Eq. 5-6) into the library's own device layout:
+ * reciprocal smoothing vector, nibble-packed K-interleaved residual codes, scales, low-rank factors
+ * in tensor-core fragment order, bias.  Synchronous; allocates device memory owned by the handle. */
+w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* desc, w4a4_handle_t* out);
+void w4a4_destroy(w4a4_handle_t h);
+
+/* The layer forward, Eq. 11:  Y = Q_A(Xh; rho) Qw + (Xh L1) L2 + b  with rho =
+ * clip_table[(expert_id * num_layers + layer_id) * num_bins + timestep_bin], read on the device.
+ *   X   device BF16 [M, K] row-major (leading dimension K), 16-byte aligned
+ *   Y   device BF16 [M, N] row-major, 16-byte aligned
+ *   clip_table  device FP32 [num_experts, num_layers, num_bins], values in [1e-4, 1]
+ *   stream      a cudaStream_t (as void*); two kernels are enqueued, no host synchronisation.
+ * M may be 0 (nothing is launched).  Errors: INVALID_ARG, SHAPE (M > max_M), CUDA. */
+w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                  const float* clip_table, void* Y, void* stream);
+
+/* The two halves of w4a4_linear_forward, exposed so that each kernel can be timed on its own.
+ * w4a4_quantize_activations: Eq. 3-5, 8-9 and the first factor of Eq. 7's low-rank term, into the
+ * context workspace.  w4a4_gemm_from_workspace: the rest of Eq. 7/11 from that workspace into Y. */
+w4a4_status_t w4a4_quantize_activations(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                        const float* clip_table, void* stream);
+w4a4_status_t w4a4_gemm_from_workspace(w4a4_handle_t h, int M, int expert_id, void* Y, void* stream);
+
+/* Parity taps (tests only; same kernels, extra stores).
+ * w4a4_debug_quantize: runs the activation kernel and decodes its outputs to plain layouts:
+ *   codes  device int8 [M, K] (logical 4-bit codes, Eq. 3), scales device FP32 [M, K/64] (Eq. 9),
+ *   T      device FP32 [M, r] (Xh L1 as the GEMM will see it: the sum of its BF16 high and low parts); may be NULL.
+ * w4a4_debug_partials: runs the whole forward and additionally stores the per-group integer partial
+ *   sums (Eq. 7's 4-bit product before rescaling) of the output tile whose first row is m0 and first
+ *   column is n0 (multiples of the tile sizes reported by w4a4_tile_shape):
+ *   P device int32 [tile_m, K/64, tile_n];  Y as in the forward. */
+w4a4_status_t w4a4_debug_quantize(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                  const float* clip_table, int8_t* codes, float* scales, float* T, void* stream);
+w4a4_status_t w4a4_debug_partials(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                  const float* clip_table, void* Y, int m0, int n0, int32_t* P, void* stream);
+void w4a4_tile_shape(int* tile_m, int* tile_n);
+
+/* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
+ * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
+w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);
+
+/* Bytes of device memory held by a handle / a context. */
+size_t w4a4_handle_bytes(w4a4_handle_t h);
+size_t w4a4_ctx_bytes(w4a4_ctx_t ctx);
+
+const char* w4a4_status_string(w4a4_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W4A4_H_ */

@@ -1,0 +1,200 @@
+// Kernel 1: fused smoothing + per-(token, 64-channel group) 4-bit quantization + nibble packing
+// + low-rank down-projection, one streaming pass over the BF16 activations (HBM bound).
+//
+//   Eq. 5      xh = f32(x) * (1/lambda)                      one FP32 multiply per element
+//   Eq. 8      a  = max |xh| over the 64-channel group       quad shuffles
+//   Eq. 9 / 4  s  = (rho * a) / 7 ,  is = 1 / s              IEEE divides, once per (row, group)
+//   Eq. 3      q  = clip(rint(xh * is), -8, 7)               rounding by the 1.5*2^23 magic add (ties to even)
+//   Eq. 7      T  = bf16(xh) L1                              mma.sync m16n8k16 BF16, FP32 accumulate
+//
+// Work split: a CTA of 4 warps owns 16 consecutive token rows; warp w owns the groups g = w, w+4, ...
+// so the four warps together stream 512 contiguous bytes of every row per step.  Inside a warp,
+// lane = 4*i + j owns rows i and i+8 and, within the group, channels
+//      32*(j/2) + 8*(j%2) + [0,8)     and the same + 16,
+// which is exactly the pair of 8-channel runs that fill two whole 32-bit words of the packed layout
+// below, so no lane exchange is needed to pack.  The tensor-core K order is free (a dot product does
+// not care about order), so the lane's 16 channels are used as-is as A-fragment slots and the L1
+// fragments are laid out at pack time to match (see l1_fragment_channel()).
+//
+// Packed activation layout (shared with kernel 2's unpack): per row, per 32 consecutive channels
+// [32c, 32c+32) one 16-byte chunk of four 32-bit words; word w, byte b holds channel 32c + 4w + b in
+// its LOW nibble and channel 32c + 16 + 4w + b in its HIGH nibble (two's complement nibbles).  With
+// that interleave `word & 0xF0F0F0F0` and `(word << 4) & 0xF0F0F0F0` are each four signed bytes equal
+// to 16 x code, i.e. two K-contiguous runs ready for the integer tensor core.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace w4a4 {
+
+constexpr int kQuantRows = 16;      // token rows per CTA
+constexpr int kQuantWarps = 4;      // warps per CTA, each owning every 4th group
+constexpr int kQuantThreads = 32 * kQuantWarps;
+
+// Channel (within its 64-group) that lane-in-quad j holds as its e-th element, e in [0,16).
+__host__ __device__ constexpr int l1_fragment_channel(int j, int e) {
+  return 32 * (j >> 1) + 8 * (j & 1) + (e < 8 ? e : e + 8);
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint4 ldg_stream_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// Smooth 8 BF16 values (one 16-byte load) with 8 reciprocals.
+__device__ __forceinline__ void smooth8(const uint4& raw, const float4& r0, const float4& r1, float* xh) {
+  xh[0] = __fmul_rn(__uint_as_float(raw.x << 16), r0.x);
+  xh[1] = __fmul_rn(__uint_as_float(raw.x & 0xffff0000u), r0.y);
+  xh[2] = __fmul_rn(__uint_as_float(raw.y << 16), r0.z);
+  xh[3] = __fmul_rn(__uint_as_float(raw.y & 0xffff0000u), r0.w);
+  xh[4] = __fmul_rn(__uint_as_float(raw.z << 16), r1.x);
+  xh[5] = __fmul_rn(__uint_as_float(raw.z & 0xffff0000u), r1.y);
+  xh[6] = __fmul_rn(__uint_as_float(raw.w << 16), r1.z);
+  xh[7] = __fmul_rn(__uint_as_float(raw.w & 0xffff0000u), r1.w);
+}
+
+// Quantize the lane's 16 smoothed values of one row and return its two packed words.
+// `s_out` receives the group scale (identical on the 4 lanes of the quad).
+__device__ __forceinline__ uint2 quantize16(const float* xh, float rho, float& s_out) {
+  float a = 0.0f;
+#pragma unroll
+  for (int e = 0; e < 16; ++e) a = fmaxf(a, fabsf(xh[e]));
+  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
+  float s = 0.0f, is = 0.0f;
+  if (a > 0.0f) {
+    s = __fdiv_rn(__fmul_rn(rho, a), 7.0f);
+    is = __fdiv_rn(1.0f, s);
+  }
+  s_out = s;
+  // code + 8 in [0, 15]:  (float bits of z + 1.5*2^23 + 8) - bits(1.5*2^23), clamped.
+  uint32_t u[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    const float f = __fadd_rn(__fmul_rn(xh[e], is), 12582920.0f);
+    u[e] = static_cast<uint32_t>(__viaddmin_s32_relu(__float_as_int(f), -0x4B400000, 15));
+  }
+  uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    w0 |= (u[b] | (u[8 + b] << 4)) << (8 * b);
+    w1 |= (u[4 + b] | (u[12 + b] << 4)) << (8 * b);
+  }
+  return make_uint2(w0 ^ 0x88888888u, w1 ^ 0x88888888u);  // offset-binary -> two's complement nibbles
+}
+
+template <int R>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
+                const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
+                uint8_t* __restrict__ codes, float* __restrict__ scales, uint16_t* __restrict__ t_hilo) {
+  constexpr int NT = R / 8;  // n-tiles of the m16n8k16 MMA
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qi = lane >> 2, qj = lane & 3;
+  const int G = K >> 6;
+  const int row0 = blockIdx.x * kQuantRows;
+  const int rowA = row0 + qi, rowB = rowA + 8;
+  const bool okA = rowA < M, okB = rowB < M;
+  const float rho = __ldg(clip_table + clip_index);
+  const int coff = 32 * (qj >> 1) + 8 * (qj & 1);  // lane's first channel inside a group
+
+  const uint16_t* xa = X + static_cast<size_t>(okA ? rowA : 0) * K + coff;
+  const uint16_t* xb = X + static_cast<size_t>(okB ? rowB : 0) * K + coff;
+
+  float acc[NT > 0 ? NT : 1][4];
+#pragma unroll
+  for (int nt = 0; nt < (NT > 0 ? NT : 1); ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
+
+  const uint4 zero4 = make_uint4(0, 0, 0, 0);
+  uint4 ra0 = zero4, ra1 = zero4, rb0 = zero4, rb1 = zero4;
+  int g = warp;
+  if (g < G) {
+    if (okA) { ra0 = ldg_stream_v4(xa + 64 * g); ra1 = ldg_stream_v4(xa + 64 * g + 16); }
+    if (okB) { rb0 = ldg_stream_v4(xb + 64 * g); rb1 = ldg_stream_v4(xb + 64 * g + 16); }
+  }
+  for (; g < G; g += kQuantWarps) {
+    const uint4 ca0 = ra0, ca1 = ra1, cb0 = rb0, cb1 = rb1;
+    const int gn = g + kQuantWarps;
+    if (gn < G) {  // prefetch the next group's activations before touching this one
+      if (okA) { ra0 = ldg_stream_v4(xa + 64 * gn); ra1 = ldg_stream_v4(xa + 64 * gn + 16); }
+      if (okB) { rb0 = ldg_stream_v4(xb + 64 * gn); rb1 = ldg_stream_v4(xb + 64 * gn + 16); }
+    }
+    const float4* rl = reinterpret_cast<const float4*>(rlam + 64 * g + coff);
+    const float4 l0 = __ldg(rl), l1 = __ldg(rl + 1), l4 = __ldg(rl + 4), l5 = __ldg(rl + 5);
+    float xhA[16], xhB[16];
+    smooth8(ca0, l0, l1, xhA);
+    smooth8(ca1, l4, l5, xhA + 8);
+    smooth8(cb0, l0, l1, xhB);
+    smooth8(cb1, l4, l5, xhB + 8);
+
+    float sA, sB;
+    const uint2 wA = quantize16(xhA, rho, sA);
+    const uint2 wB = quantize16(xhB, rho, sB);
+    const size_t cpitch = static_cast<size_t>(K >> 1);
+    if (okA) *reinterpret_cast<uint2*>(codes + rowA * cpitch + 32 * g + 8 * qj) = wA;
+    if (okB) *reinterpret_cast<uint2*>(codes + rowB * cpitch + 32 * g + 8 * qj) = wB;
+    if (qj == 0 && okA) scales[static_cast<size_t>(rowA) * G + g] = sA;
+    if (qj == 1 && okB) scales[static_cast<size_t>(rowB) * G + g] = sB;
+
+    if constexpr (NT > 0) {
+      const uint2* lf = l1frag + (static_cast<size_t>(g) * 4 * NT) * 32 + lane;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint32_t a[4];
+        a[0] = pack_bf16x2(xhA[4 * i], xhA[4 * i + 1]);
+        a[1] = pack_bf16x2(xhB[4 * i], xhB[4 * i + 1]);
+        a[2] = pack_bf16x2(xhA[4 * i + 2], xhA[4 * i + 3]);
+        a[3] = pack_bf16x2(xhB[4 * i + 2], xhB[4 * i + 3]);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const uint2 b = __ldg(lf + (i * NT + nt) * 32);
+          mma_bf16_16816(acc[nt], a, b.x, b.y);
+        }
+      }
+    }
+  }
+
+  if constexpr (NT > 0) {
+    __shared__ float tred[kQuantWarps][kQuantRows][R];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int c = 8 * nt + 2 * qj;
+      tred[warp][qi][c] = acc[nt][0];
+      tred[warp][qi][c + 1] = acc[nt][1];
+      tred[warp][qi + 8][c] = acc[nt][2];
+      tred[warp][qi + 8][c + 1] = acc[nt][3];
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < kQuantRows * R; idx += kQuantThreads) {
+      const int rr = idx / R, c = idx % R;
+      const int row = row0 + rr;
+      if (row < M) {
+        const float t = (tred[0][rr][c] + tred[1][rr][c]) + (tred[2][rr][c] + tred[3][rr][c]);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(t);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(t - __bfloat162float(hi));
+        uint16_t* dst = t_hilo + static_cast<size_t>(row) * (2 * R);
+        dst[c] = *reinterpret_cast<const uint16_t*>(&hi);
+        dst[R + c] = *reinterpret_cast<const uint16_t*>(&lo);
+      }
+    }
+  }
+}
+
+}  // namespace w4a4

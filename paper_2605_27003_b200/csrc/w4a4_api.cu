@@ -1,0 +1,550 @@
+// C-ABI entry points of libw4a4: context / handle management, weight repacking and the launches of
+// the two forward kernels.  Host code only does argument checks, descriptor set-up and launches.
+#include "../../include/w4a4.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "gemm_kernel.cuh"
+#include "quantize_kernel.cuh"
+
+namespace w4a4 {
+
+// ------------------------------------------------------------------------------------ setup kernels
+// lambda -> 1/lambda (Eq. 5), IEEE FP32 division, once.
+__global__ void reciprocal_kernel(const float* __restrict__ lam, float* __restrict__ out, int K) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < K) out[k] = __fdiv_rn(1.0f, lam[k]);
+}
+
+// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed, K-interleaved (see quantize_kernel.cuh).
+// One thread builds one 16-byte chunk (32 consecutive K of one output channel).
+__global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __restrict__ out, int K, int N,
+                                   int* __restrict__ bad) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int c = blockIdx.y;
+  if (n >= N) return;
+  uint32_t w[4] = {0, 0, 0, 0};
+  bool oob = false;
+  for (int o = 0; o < 32; ++o) {
+    const int v = q[static_cast<size_t>(32 * c + o) * N + n];
+    oob |= (v < -8 || v > 7);
+    const uint32_t nib = static_cast<uint32_t>(v) & 0xFu;
+    const int word = (o & 15) >> 2, byte = o & 3, hi = o >> 4;
+    w[word] |= nib << (8 * byte + 4 * hi);
+  }
+  if (oob) atomicOr(bad, 1);
+  *reinterpret_cast<uint4*>(out + static_cast<size_t>(n) * (K >> 1) + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// L1 [K, r] BF16 -> B fragments of mma.sync m16n8k16 in the K order the activation kernel uses.
+__global__ void l1_fragment_kernel(const uint16_t* __restrict__ L1, uint2* __restrict__ out, int K, int r) {
+  const int NT = r / 8;
+  const size_t total = static_cast<size_t>(K / 64) * 4 * NT * 32;
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int lane = idx & 31;
+  const int nt = (idx >> 5) % NT;
+  const int i = ((idx >> 5) / NT) & 3;
+  const int g = (idx >> 5) / NT / 4;
+  const int j = lane & 3, n = 8 * nt + (lane >> 2);
+  uint16_t v[4];
+  for (int e = 0; e < 4; ++e) {
+    const int ch = 64 * g + l1_fragment_channel(j, 4 * i + e);
+    v[e] = L1[static_cast<size_t>(ch) * r + n];
+  }
+  out[idx] = make_uint2(static_cast<uint32_t>(v[0]) | (static_cast<uint32_t>(v[1]) << 16),
+                        static_cast<uint32_t>(v[2]) | (static_cast<uint32_t>(v[3]) << 16));
+}
+
+// L2 [r, N] BF16 -> [N, 2r]: the transposed factor twice, matching the [T_hi | T_lo] split of T.
+__global__ void l2_dup_kernel(const uint16_t* __restrict__ L2, uint16_t* __restrict__ out, int r, int N) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(N) * 2 * r) return;
+  const int c = idx % (2 * r);
+  const int n = idx / (2 * r);
+  out[idx] = L2[static_cast<size_t>(c % r) * N + n];
+}
+
+// Test-only decoders of the activation kernel's outputs.
+__global__ void decode_codes_kernel(const uint8_t* __restrict__ packed, int8_t* __restrict__ codes, int M, int K) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(M) * K) return;
+  const int k = idx % K;
+  const size_t m = idx / K;
+  const int c = k >> 5, o = k & 31;
+  const uint8_t b = packed[m * (K >> 1) + 16 * c + 4 * ((o & 15) >> 2) + (o & 3)];
+  const int nib = (o >> 4) ? (b >> 4) : (b & 0xF);
+  codes[idx] = static_cast<int8_t>((nib ^ 8) - 8);
+}
+__global__ void decode_t_kernel(const uint16_t* __restrict__ thl, float* __restrict__ T, int M, int r) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(M) * r) return;
+  const int c = idx % r;
+  const size_t m = idx / r;
+  const float hi = __uint_as_float(static_cast<uint32_t>(thl[m * 2 * r + c]) << 16);
+  const float lo = __uint_as_float(static_cast<uint32_t>(thl[m * 2 * r + r + c]) << 16);
+  T[idx] = hi + lo;
+}
+
+}  // namespace w4a4
+
+using namespace w4a4;
+
+// ------------------------------------------------------------------------------------ host objects
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct w4a4_ctx {
+  int device = 0;
+  int max_M = 0, max_K = 0, max_r = 0;
+  uint8_t* codes = nullptr;   // [max_M, K/2] packed activation codes (pitch K/2 of the running layer)
+  float* scales = nullptr;    // [max_M, K/64]
+  uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
+  int* d_err = nullptr;       // device error word
+  size_t bytes = 0;
+  EncodeTiledFn encode = nullptr;
+};
+
+struct ExpertData {
+  uint8_t* bpacked = nullptr;  // [N, K/2]
+  float* wscale = nullptr;     // [G, N]
+  float* rlam = nullptr;       // [K]
+  uint2* l1frag = nullptr;
+  uint16_t* l2dup = nullptr;   // [N, 2r]
+  float* bias = nullptr;       // [N] or null
+  CUtensorMap tmB, tmL2;
+};
+
+struct w4a4_layer {
+  w4a4_ctx* ctx = nullptr;
+  int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0;
+  std::vector<ExpertData> experts;
+  CUtensorMap tmA, tmT;
+  size_t bytes = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
+    if (ok && prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+w4a4_status_t dev_alloc(T** p, size_t count, size_t* tally) {
+  *p = nullptr;
+  if (count == 0) return W4A4_OK;
+  void* q = nullptr;
+  if (cudaMalloc(&q, count * sizeof(T)) != cudaSuccess) {
+    cudaGetLastError();
+    return W4A4_ERR_ALLOC;
+  }
+  *p = static_cast<T*>(q);
+  if (tally) *tally += count * sizeof(T);
+  return W4A4_OK;
+}
+
+bool encode_2d(EncodeTiledFn fn, CUtensorMap* tm, CUtensorMapDataType dt, size_t elem, void* base, uint64_t inner,
+               uint64_t outer, uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle sw) {
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {box_inner, box_outer};
+  const cuuint32_t es[2] = {1, 1};
+  (void)elem;
+  return fn(tm, dt, 2, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+void free_expert(ExpertData& e) {
+  cudaFree(e.bpacked);
+  cudaFree(e.wscale);
+  cudaFree(e.rlam);
+  cudaFree(e.l1frag);
+  cudaFree(e.l2dup);
+  cudaFree(e.bias);
+  e = ExpertData();
+}
+
+// Brings `count` elements at `src` (host or device) into a fresh device staging buffer when needed.
+template <typename T>
+w4a4_status_t stage_in(const T* src, size_t count, bool on_device, const T** dev, T** owned) {
+  *owned = nullptr;
+  if (on_device) {
+    *dev = src;
+    return W4A4_OK;
+  }
+  w4a4_status_t st = dev_alloc(owned, count, nullptr);
+  if (st != W4A4_OK) return st;
+  if (cudaMemcpy(*owned, src, count * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return W4A4_ERR_CUDA;
+  *dev = *owned;
+  return W4A4_OK;
+}
+
+w4a4_status_t check_forward_args(w4a4_handle_t h, const void* X, int M, int expert_id, int bin,
+                                 const float* clip_table, bool need_x) {
+  if (!h || !h->ctx) return W4A4_ERR_INVALID_ARG;
+  if (M < 0) return W4A4_ERR_INVALID_ARG;
+  if (M > h->ctx->max_M) return W4A4_ERR_SHAPE;
+  if (expert_id < 0 || expert_id >= h->E) return W4A4_ERR_INVALID_ARG;
+  if (need_x) {
+    if (bin < 0 || bin >= h->B) return W4A4_ERR_INVALID_ARG;
+    if (M > 0 && (!X || !aligned16(X))) return W4A4_ERR_INVALID_ARG;
+    if (!clip_table) return W4A4_ERR_INVALID_ARG;
+  }
+  return W4A4_OK;
+}
+
+w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_id, int bin, const float* clip_table,
+                              cudaStream_t stream) {
+  if (M == 0) return W4A4_OK;
+  w4a4_ctx* ctx = h->ctx;
+  const ExpertData& e = h->experts[expert_id];
+  const int clip_index = (expert_id * h->L + h->layer_id) * h->B + bin;
+  const dim3 grid((M + kQuantRows - 1) / kQuantRows), block(kQuantThreads);
+  const uint16_t* x = static_cast<const uint16_t*>(X);
+#define W4A4_LAUNCH_Q(R)                                                                                         \
+  quantize_kernel<R><<<grid, block, 0, stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
+                                                 ctx->scales, ctx->t_hilo)
+  switch (h->r) {
+    case 0: W4A4_LAUNCH_Q(0); break;
+    case 16: W4A4_LAUNCH_Q(16); break;
+    case 32: W4A4_LAUNCH_Q(32); break;
+    case 64: W4A4_LAUNCH_Q(64); break;
+    default: return W4A4_ERR_SHAPE;
+  }
+#undef W4A4_LAUNCH_Q
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream, int32_t* dbg_P,
+                          int dbg_m0, int dbg_n0) {
+  if (M == 0) return W4A4_OK;
+  w4a4_ctx* ctx = h->ctx;
+  const ExpertData& e = h->experts[expert_id];
+  GemmParams p;
+  p.sa = ctx->scales;
+  p.sw = e.wscale;
+  p.bias = e.bias;
+  p.Y = static_cast<uint16_t*>(Y);
+  p.M = M;
+  p.N = h->N;
+  p.K = h->K;
+  p.r = h->r;
+  p.err = ctx->d_err;
+  p.dbg_P = dbg_P;
+  p.dbg_m0 = dbg_m0;
+  p.dbg_n0 = dbg_n0;
+  const dim3 grid(h->N / kBN, (M + kBM - 1) / kBM), block(kGemmThreads);
+  const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
+  const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
+  if (dbg_P) {
+    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
+  } else {
+    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
+  }
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------ C ABI
+extern "C" {
+
+const char* w4a4_status_string(w4a4_status_t s) {
+  switch (s) {
+    case W4A4_OK: return "ok";
+    case W4A4_ERR_INVALID_ARG: return "invalid argument";
+    case W4A4_ERR_SHAPE: return "unsupported shape";
+    case W4A4_ERR_ALLOC: return "allocation failed";
+    case W4A4_ERR_CUDA: return "CUDA error";
+    case W4A4_ERR_ARCH: return "device is not compute capability 10.x";
+    case W4A4_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+  }
+  return "unknown status";
+}
+
+void w4a4_tile_shape(int* tile_m, int* tile_n) {
+  if (tile_m) *tile_m = kBM;
+  if (tile_n) *tile_n = kBN;
+}
+
+w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_ctx_t* out) {
+  if (!out) return W4A4_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (max_M <= 0 || max_K <= 0 || max_K % 64 != 0 || max_r < 0 || max_r > 64) return W4A4_ERR_SHAPE;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+    cudaGetLastError();
+    return W4A4_ERR_CUDA;
+  }
+  if (device < 0 || device >= ndev) return W4A4_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return W4A4_ERR_CUDA;
+  if (prop.major != 10) return W4A4_ERR_ARCH;
+  DeviceGuard guard(device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+
+  w4a4_ctx* ctx = new (std::nothrow) w4a4_ctx();
+  if (!ctx) return W4A4_ERR_ALLOC;
+  ctx->device = device;
+  ctx->max_M = max_M;
+  ctx->max_K = max_K;
+  ctx->max_r = max_r;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete ctx;
+    return W4A4_ERR_CUDA;
+  }
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  w4a4_status_t st = dev_alloc(&ctx->codes, static_cast<size_t>(max_M) * (max_K / 2), &ctx->bytes);
+  if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(max_M) * (max_K / 64), &ctx->bytes);
+  if (st == W4A4_OK) st = dev_alloc(&ctx->t_hilo, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8), &ctx->bytes);
+  if (st == W4A4_OK) st = dev_alloc(&ctx->d_err, 1, &ctx->bytes);
+  if (st == W4A4_OK && cudaMemset(ctx->d_err, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
+  // The workspace is read by TMA for rows up to max_M even when fewer are valid: start it defined.
+  if (st == W4A4_OK && cudaMemset(ctx->codes, 0, static_cast<size_t>(max_M) * (max_K / 2)) != cudaSuccess) st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK &&
+      cudaMemset(ctx->t_hilo, 0, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8) * sizeof(uint16_t)) != cudaSuccess)
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK) {
+    cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+    cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+    if (e1 != cudaSuccess || e2 != cudaSuccess) {
+      cudaGetLastError();
+      st = W4A4_ERR_CUDA;
+    }
+  }
+  if (st != W4A4_OK) {
+    w4a4_ctx_destroy(ctx);
+    return st;
+  }
+  *out = ctx;
+  return W4A4_OK;
+}
+
+void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
+  if (!ctx) return;
+  DeviceGuard guard(ctx->device);
+  cudaFree(ctx->codes);
+  cudaFree(ctx->scales);
+  cudaFree(ctx->t_hilo);
+  cudaFree(ctx->d_err);
+  delete ctx;
+}
+
+size_t w4a4_ctx_bytes(w4a4_ctx_t ctx) { return ctx ? ctx->bytes : 0; }
+size_t w4a4_handle_bytes(w4a4_handle_t h) { return h ? h->bytes : 0; }
+
+void w4a4_destroy(w4a4_handle_t h) {
+  if (!h) return;
+  if (h->ctx) {
+    DeviceGuard guard(h->ctx->device);
+    for (auto& e : h->experts) free_expert(e);
+  }
+  delete h;
+}
+
+w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a4_handle_t* out) {
+  if (!out) return W4A4_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !d) return W4A4_ERR_INVALID_ARG;
+  if (d->group != 64 || d->K <= 0 || d->K % 64 != 0 || d->N <= 0 || d->N % kBN != 0) return W4A4_ERR_SHAPE;
+  if (!(d->r == 0 || d->r == 16 || d->r == 32 || d->r == 64)) return W4A4_ERR_SHAPE;
+  if (d->K > ctx->max_K || d->r > ctx->max_r) return W4A4_ERR_SHAPE;
+  if (d->num_experts < 1 || d->num_bins < 1 || d->num_layers < 1 || d->layer_id < 0 || d->layer_id >= d->num_layers)
+    return W4A4_ERR_INVALID_ARG;
+  if (!d->qweight || !d->wscale || !d->lambda || (d->r > 0 && (!d->L1 || !d->L2))) return W4A4_ERR_INVALID_ARG;
+  for (int e = 0; e < d->num_experts; ++e) {
+    if (!d->qweight[e] || !d->wscale[e] || !d->lambda[e] || (d->r > 0 && (!d->L1[e] || !d->L2[e])))
+      return W4A4_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+
+  w4a4_layer* h = new (std::nothrow) w4a4_layer();
+  if (!h) return W4A4_ERR_ALLOC;
+  h->ctx = ctx;
+  h->K = d->K;
+  h->N = d->N;
+  h->r = d->r;
+  h->E = d->num_experts;
+  h->B = d->num_bins;
+  h->L = d->num_layers;
+  h->layer_id = d->layer_id;
+  h->experts.resize(d->num_experts);
+  const int K = d->K, N = d->N, r = d->r, G = K / 64;
+  const bool dev = d->pointers_on_device != 0;
+  w4a4_status_t st = W4A4_OK;
+  int* d_bad = nullptr;
+  st = dev_alloc(&d_bad, 1, nullptr);
+  if (st == W4A4_OK && cudaMemset(d_bad, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
+
+  for (int ei = 0; st == W4A4_OK && ei < d->num_experts; ++ei) {
+    ExpertData& e = h->experts[ei];
+    st = dev_alloc(&e.bpacked, static_cast<size_t>(N) * (K / 2), &h->bytes);
+    if (st == W4A4_OK) st = dev_alloc(&e.wscale, static_cast<size_t>(G) * N, &h->bytes);
+    if (st == W4A4_OK) st = dev_alloc(&e.rlam, static_cast<size_t>(K), &h->bytes);
+    if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l1frag, static_cast<size_t>(G) * 4 * (r / 8) * 32, &h->bytes);
+    if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l2dup, static_cast<size_t>(N) * 2 * r, &h->bytes);
+    const float* bias_src = d->bias ? d->bias[ei] : nullptr;
+    if (st == W4A4_OK && bias_src) st = dev_alloc(&e.bias, static_cast<size_t>(N), &h->bytes);
+    if (st != W4A4_OK) break;
+
+    const cudaMemcpyKind kind = dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    if (cudaMemcpy(e.wscale, d->wscale[ei], sizeof(float) * G * N, kind) != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK && bias_src && cudaMemcpy(e.bias, bias_src, sizeof(float) * N, kind) != cudaSuccess)
+      st = W4A4_ERR_CUDA;
+    if (st != W4A4_OK) break;
+
+    const int8_t* q_dev = nullptr;
+    int8_t* q_own = nullptr;
+    const float* lam_dev = nullptr;
+    float* lam_own = nullptr;
+    const uint16_t *l1_dev = nullptr, *l2_dev = nullptr;
+    uint16_t *l1_own = nullptr, *l2_own = nullptr;
+    st = stage_in(d->qweight[ei], static_cast<size_t>(K) * N, dev, &q_dev, &q_own);
+    if (st == W4A4_OK) st = stage_in(d->lambda[ei], static_cast<size_t>(K), dev, &lam_dev, &lam_own);
+    if (st == W4A4_OK && r > 0) st = stage_in(d->L1[ei], static_cast<size_t>(K) * r, dev, &l1_dev, &l1_own);
+    if (st == W4A4_OK && r > 0) st = stage_in(d->L2[ei], static_cast<size_t>(r) * N, dev, &l2_dev, &l2_own);
+    if (st == W4A4_OK) {
+      reciprocal_kernel<<<(K + 255) / 256, 256>>>(lam_dev, e.rlam, K);
+      pack_weight_kernel<<<dim3((N + 127) / 128, K / 32), 128>>>(q_dev, e.bpacked, K, N, d_bad);
+      if (r > 0) {
+        const size_t nf = static_cast<size_t>(G) * 4 * (r / 8) * 32;
+        l1_fragment_kernel<<<static_cast<unsigned>((nf + 255) / 256), 256>>>(l1_dev, e.l1frag, K, r);
+        const size_t nl = static_cast<size_t>(N) * 2 * r;
+        l2_dup_kernel<<<static_cast<unsigned>((nl + 255) / 256), 256>>>(l2_dev, e.l2dup, r, N);
+      }
+      if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) st = W4A4_ERR_CUDA;
+    }
+    cudaFree(q_own);
+    cudaFree(lam_own);
+    cudaFree(l1_own);
+    cudaFree(l2_own);
+    if (st != W4A4_OK) break;
+
+    if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, kBK / 2, kBN,
+                   CU_TENSOR_MAP_SWIZZLE_NONE))
+      st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK && r > 0 &&
+        !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kBN,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+      st = W4A4_ERR_CUDA;
+  }
+  if (st == W4A4_OK) {
+    int bad = 0;
+    if (cudaMemcpy(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) st = W4A4_ERR_CUDA;
+    else if (bad) st = W4A4_ERR_INVALID_ARG;  // a residual code outside [-8, 7]
+  }
+  cudaFree(d_bad);
+  if (st == W4A4_OK &&
+      !encode_2d(ctx->encode, &h->tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->codes, K / 2, ctx->max_M, K / 2, kBK / 2,
+                 kBM, CU_TENSOR_MAP_SWIZZLE_NONE))
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && r > 0 &&
+      !encode_2d(ctx->encode, &h->tmT, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo, 2 * r, ctx->max_M, 4 * r, 64,
+                 kBM, CU_TENSOR_MAP_SWIZZLE_128B))
+    st = W4A4_ERR_CUDA;
+  if (st != W4A4_OK) {
+    cudaGetLastError();
+    w4a4_destroy(h);
+    return st;
+  }
+  *out = h;
+  return W4A4_OK;
+}
+
+w4a4_status_t w4a4_quantize_activations(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                        const float* clip_table, void* stream) {
+  w4a4_status_t st = check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  DeviceGuard guard(h->ctx->device);
+  return launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, static_cast<cudaStream_t>(stream));
+}
+
+w4a4_status_t w4a4_gemm_from_workspace(w4a4_handle_t h, int M, int expert_id, void* Y, void* stream) {
+  w4a4_status_t st = check_forward_args(h, nullptr, M, expert_id, 0, nullptr, false);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!Y || !aligned16(Y))) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(h->ctx->device);
+  return launch_gemm(h, M, expert_id, Y, static_cast<cudaStream_t>(stream), nullptr, 0, 0);
+}
+
+w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                  const float* clip_table, void* Y, void* stream) {
+  w4a4_status_t st = check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!Y || !aligned16(Y))) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(h->ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
+  if (st != W4A4_OK) return st;
+  return launch_gemm(h, M, expert_id, Y, s, nullptr, 0, 0);
+}
+
+w4a4_status_t w4a4_debug_quantize(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                  const float* clip_table, int8_t* codes, float* scales, float* T, void* stream) {
+  w4a4_status_t st = check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!codes || !scales)) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(h->ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
+  if (st != W4A4_OK || M == 0) return st;
+  const size_t nc = static_cast<size_t>(M) * h->K;
+  decode_codes_kernel<<<static_cast<unsigned>((nc + 255) / 256), 256, 0, s>>>(h->ctx->codes, codes, M, h->K);
+  if (cudaMemcpyAsync(scales, h->ctx->scales, sizeof(float) * M * (h->K / 64), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return W4A4_ERR_CUDA;
+  if (T && h->r > 0) {
+    const size_t nt = static_cast<size_t>(M) * h->r;
+    decode_t_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, s>>>(h->ctx->t_hilo, T, M, h->r);
+  }
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+w4a4_status_t w4a4_debug_partials(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                  const float* clip_table, void* Y, int m0, int n0, int32_t* P, void* stream) {
+  w4a4_status_t st = check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!Y || !aligned16(Y) || !P)) return W4A4_ERR_INVALID_ARG;
+  if (m0 < 0 || n0 < 0 || m0 % kBM != 0 || n0 % kBN != 0 || n0 >= h->N || (M > 0 && m0 >= M)) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(h->ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
+  if (st != W4A4_OK) return st;
+  return launch_gemm(h, M, expert_id, Y, s, P, m0, n0);
+}
+
+w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx) {
+  if (!ctx) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (cudaDeviceSynchronize() != cudaSuccess) return W4A4_ERR_CUDA;
+  int err = 0;
+  if (cudaMemcpy(&err, ctx->d_err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return W4A4_ERR_CUDA;
+  if (err != 0) {
+    cudaMemset(ctx->d_err, 0, sizeof(int));
+    return W4A4_ERR_TIMEOUT;
+  }
+  return W4A4_OK;
+}
+
+}  // extern "C"

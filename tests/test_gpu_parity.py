@@ -1,0 +1,228 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Bars: integer codes, group scales and per-group int32 partial sums bit-exact; the BF16 output within
+|Y_gpu - Y_oracle| <= 2^-7 |Y_oracle| + 1e-3 rms(Y_oracle) (rms over the compared rows); the low-rank
+intermediate T (FP32 accumulation on the GPU, FP64 in the oracle) within 1e-4 relative to the row's
+largest |T|.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_27003_b200 as w4
+from paper_2605_27003_b200 import build as pkg_build
+from workloads import generator as gen
+
+pytestmark = pytest.mark.gpu
+G = 64
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    pkg_build.build()
+    w4.load_library()
+
+
+def bits(t):
+    return gen.bf16_bits(t.cpu()).numpy().view(np.uint16)
+
+
+def y_within_tolerance(y_gpu_bf16: torch.Tensor, y64: np.ndarray):
+    got = y_gpu_bf16.to(torch.float64).cpu().numpy()
+    rms = float(np.sqrt(np.mean(y64 ** 2)))
+    bound = 2.0 ** -7 * np.abs(y64) + 1e-3 * rms
+    err = np.abs(got - y64)
+    worst = float((err / bound).max()) if err.size else 0.0
+    return worst, rms
+
+
+def oracle_rows(x_rows: torch.Tensor, layer, rho: float, want_partials=False):
+    rows = np.arange(x_rows.shape[0], dtype=np.int32)
+    return oracle.forward_rows(
+        bits(x_rows), rows, layer.lam.cpu().numpy(), rho,
+        None if layer.L1 is None else bits(layer.L1), None if layer.L2 is None else bits(layer.L2),
+        layer.qweight.cpu().numpy(), layer.wscale.cpu().numpy(),
+        None if layer.bias is None else layer.bias.cpu().numpy(), want_partials=want_partials)
+
+
+def run_case(x: torch.Tensor, experts, clip: torch.Tensor, expert_id: int, bin_id: int, rows=None,
+             check_partials_tiles=(), layer_id=0, num_layers=1, max_M=None):
+    """Runs quantize tap + forward (+ partial taps) on the GPU and compares with the oracle on `rows`."""
+    M, K = x.shape
+    lay = experts[expert_id]
+    N, r = lay.N, lay.r
+    ctx = w4.Context(0, max_M or max(M, 1), K, r)
+    L = w4.Layer(ctx, [e.to(DEV) for e in experts], num_bins=clip.shape[2], num_layers=num_layers, layer_id=layer_id)
+    clip_d = clip.to(DEV)
+    rho = float(clip[expert_id, layer_id, bin_id])
+    xd = x.to(DEV)
+    codes = torch.full((M, K), 99, dtype=torch.int8, device=DEV)
+    scales = torch.full((M, K // G), -1.0, dtype=torch.float32, device=DEV)
+    T = torch.zeros((M, max(r, 1)), dtype=torch.float32, device=DEV)
+    w4.w4a4_debug_quantize(L.ptr, xd, M, expert_id, bin_id, clip_d, codes, scales, T if r > 0 else None)
+    Y = L.forward(xd, expert_id, bin_id, clip_d)
+    torch.cuda.synchronize()
+    ctx.check()
+    if rows is None:
+        rows = np.arange(M)
+    rows = np.asarray(rows)
+    ref = oracle_rows(x[rows], lay, rho, want_partials=bool(check_partials_tiles))
+    rt = torch.from_numpy(rows).to(DEV)
+    assert np.array_equal(codes[rt].cpu().numpy(), ref["q"]), "activation codes differ"
+    assert np.array_equal(scales[rt].cpu().numpy().view(np.uint32), ref["s"].view(np.uint32)), "scales differ"
+    if r > 0:
+        t_gpu = T[rt].cpu().numpy().astype(np.float64)
+        t_ref = ref["T"].astype(np.float64)
+        tol = 1e-4 * np.abs(t_ref).max(axis=1, keepdims=True) + 1e-30
+        assert np.all(np.abs(t_gpu - t_ref) <= tol), "low-rank intermediate differs"
+    worst, rms = y_within_tolerance(Y[rt], ref["Y64"])
+    assert worst <= 1.0, f"output outside tolerance: worst err/bound = {worst:.3f} (rms {rms:.4g})"
+    bm, bn = w4.w4a4_tile_shape()
+    for (m0, n0) in check_partials_tiles:
+        P = torch.zeros((bm, K // G, bn), dtype=torch.int32, device=DEV)
+        Y2 = torch.empty_like(Y)
+        w4.w4a4_debug_partials(L.ptr, xd, M, expert_id, bin_id, clip_d, Y2, m0, n0, P)
+        torch.cuda.synchronize()
+        ctx.check()
+        assert torch.equal(Y2, Y), "the debug-tap forward must give the same output"
+        sel = [(i, int(rw)) for i, rw in enumerate(rows) if m0 <= rw < min(m0 + bm, M)]
+        assert sel, "no compared row falls into the requested tile"
+        Pg = P.cpu().numpy()
+        for i, rw in sel:
+            assert np.array_equal(Pg[rw - m0], ref["P"][i][:, n0:n0 + bn]), f"partials differ at row {rw}"
+    L.close()
+    ctx.close()
+    return worst
+
+
+def tiny_inputs(M=256, K=512, N=512, r=16, seed=0, bias=False):
+    idx = gen.outlier_channels(K, 0, seed, count=4)
+    x = gen.make_activations(M, K, outlier_idx=idx, outlier_gain=40.0, seed=seed)
+    layer = gen.make_layer_svd(K, N, r, x, seed=seed + 1, bias_std=0.01 if bias else None)
+    return x, layer
+
+
+def test_tiny_config_full_parity():
+    # M=256, K=N=512, r=16, one bin with rho=0.9, no bias; every row, every tile's partial sums.
+    x, layer = tiny_inputs()
+    clip = torch.full((1, 1, 1), 0.9, dtype=torch.float32)
+    tiles = [(m0, n0) for m0 in (0, 128) for n0 in (0, 128, 256, 384)]
+    run_case(x, [layer], clip, 0, 0, check_partials_tiles=tiles)
+
+
+@pytest.mark.parametrize("M,K,N,r,bias", [
+    (333, 640, 256, 32, True),    # ragged M, G=10 (not a multiple of 4)
+    (200, 704, 128, 64, True),    # G=11: odd group count -> half-filled last stage; r=64 -> two low-rank stages
+    (129, 512, 384, 0, True),     # no low-rank branch
+    (1, 128, 128, 16, False),     # a single token, a single stage
+    (127, 1024, 256, 32, False),
+])
+def test_ragged_shapes_and_ranks(M, K, N, r, bias):
+    x, layer = tiny_inputs(M, K, N, r, seed=10 + r + M, bias=bias)
+    clip = gen.make_clip_table(1, 3, 4, [(0.6, 1.0)], seed=M)
+    last_tile_m0 = ((M - 1) // 128) * 128
+    run_case(x, [layer], clip, 0, 2, check_partials_tiles=[(0, 0), (last_tile_m0, N - 128)], layer_id=1, num_layers=3,
+             max_M=M + 77)
+
+
+def test_two_experts_and_bins_select_their_own_constants():
+    M, K, N, r = 160, 512, 256, 16
+    x, e0 = tiny_inputs(M, K, N, r, seed=3, bias=True)
+    e1 = gen.make_layer_direct(K, N, r, seed=4)
+    clip = gen.make_clip_table(2, 2, 8, [(0.6, 1.0), (0.8, 1.0)], seed=5)
+    for expert, b in ((0, 0), (1, 7), (1, 3)):
+        run_case(x, [e0, e1], clip, expert, b, layer_id=1, num_layers=2)
+
+
+def test_degenerate_inputs_zero_rows_and_exact_grid():
+    M, K, N, r = 140, 256, 128, 16
+    x, layer = tiny_inputs(M, K, N, r, seed=6)
+    x = x.clone()
+    x[5] = 0          # an all-zero token
+    x[7, 64:128] = 0  # an all-zero group
+    xi = torch.randint(-7, 8, (K,), generator=torch.Generator().manual_seed(1)).to(torch.float32)
+    xi[::64] = 7.0
+    x[9] = (xi * layer.lam * 0.25).to(torch.bfloat16)  # roughly on-grid row
+    clip = torch.tensor([[[1.0, 0.5]]], dtype=torch.float32)
+    run_case(x, [layer], clip, 0, 0, check_partials_tiles=[(0, 0)])
+    run_case(x, [layer], clip, 0, 1, check_partials_tiles=[(128, 0)])
+
+
+def test_empty_batch_and_argument_errors():
+    x, layer = tiny_inputs(64, 128, 128, 16, seed=8)
+    ctx = w4.Context(0, 64, 128, 16)
+    L = w4.Layer(ctx, [layer.to(DEV)], num_bins=2)
+    clip = torch.ones(1, 1, 2, device=DEV)
+    Y = torch.empty(64, 128, dtype=torch.bfloat16, device=DEV)
+    w4.w4a4_linear_forward(L.ptr, x.to(DEV), 0, 0, 0, clip, Y)  # M = 0: nothing launched, no error
+    for kwargs, status in ((dict(M=65), 2), (dict(expert=1), 1), (dict(bin=2), 1)):
+        with pytest.raises(w4.W4A4Error) as ei:
+            w4.w4a4_linear_forward(L.ptr, x.to(DEV), kwargs.get("M", 64), kwargs.get("expert", 0),
+                                   kwargs.get("bin", 0), clip, Y)
+        assert ei.value.status == status
+    bad = gen.make_layer_direct(128, 128, 16, seed=1)
+    bad.qweight[3, 5] = 9
+    with pytest.raises(w4.W4A4Error) as ei:
+        w4.Layer(ctx, [bad.to(DEV)], num_bins=2)
+    assert ei.value.status == 1
+    with pytest.raises(w4.W4A4Error) as ei:
+        w4.Layer(ctx, [gen.make_layer_direct(256, 128, 16, seed=1).to(DEV)], num_bins=2)  # K beyond the context
+    assert ei.value.status == 2
+    torch.cuda.synchronize()
+    ctx.check()
+    L.close()
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- full-size workloads, sampled rows
+def sampled_rows(M, n_random, seed):
+    fixed = [0, 127, 128, M - 1, (M - 1) // 128 * 128, (M - 1) // 128 * 128 - 1]
+    rng = np.random.default_rng(seed)
+    rnd = rng.choice(M, size=n_random, replace=False).tolist()
+    return np.array(sorted(set(r for r in fixed + rnd if 0 <= r < M)))
+
+
+def big_layer(K, N, r, x_calib, seed):
+    return gen.make_layer_svd(K, N, r, x_calib, seed=seed, bias_std=0.01, device=DEV, exact_svd=False,
+                              keep_float64=False).to("cpu")
+
+
+def test_attention_projection_full_size_sampled_rows():
+    # M = 32760 (21 x 30 x 52 latent grid), K = N = 5120, r = 32; sigma decays over 8 bins; 1% outlier channels x50.
+    M, K, N, r = 32760, 5120, 5120, 32
+    idx = gen.outlier_channels(K, 0.01, 2)
+    clip = gen.make_clip_table(1, 1, 8, [(0.6, 1.0)], seed=2)
+    calib = gen.make_activations(1024, K, sigma=gen.sigma_for_bin(0), outlier_idx=idx, outlier_gain=50.0, seed=2000,
+                                 device=DEV)
+    layer = big_layer(K, N, r, calib, 2001)
+    for b in (0, 5):
+        x = gen.make_activations(M, K, sigma=gen.sigma_for_bin(b), outlier_idx=idx, outlier_gain=50.0, seed=2002 + b,
+                                 device=DEV).cpu()
+        rows = sampled_rows(M, 24, b)
+        last = (M - 1) // 128 * 128
+        run_case(x, [layer], clip, 0, b, rows=rows, check_partials_tiles=[(0, 0), (last, N - 128)])
+
+
+def test_ffn_pair_full_size_sampled_rows():
+    # up 5120 -> 13824 and down 13824 -> 5120 at M = 32760; the down input is GELU of a Gaussian with
+    # 1% outlier channels x80; two experts with their own clip tables.
+    M, r = 32760, 32
+    clip = gen.make_clip_table(2, 1, 8, [(0.6, 1.0), (0.8, 1.0)], seed=3)
+    # up projection
+    K, N = 5120, 13824
+    idx = gen.outlier_channels(K, 0.01, 3)
+    calib = gen.make_activations(1024, K, sigma=1.0, outlier_idx=idx, outlier_gain=50.0, seed=3000, device=DEV)
+    up = big_layer(K, N, r, calib, 3001)
+    x = gen.make_activations(M, K, sigma=1.0, outlier_idx=idx, outlier_gain=50.0, seed=3002, device=DEV).cpu()
+    rows = sampled_rows(M, 10, 31)
+    run_case(x, [up, up], clip, 1, 4, rows=rows, check_partials_tiles=[((M - 1) // 128 * 128, 0)])
+    del x, up
+    # down projection
+    K, N = 13824, 5120
+    idx = gen.outlier_channels(K, 0.01, 4)
+    calib = gen.make_activations(1024, K, dist="gelu", outlier_idx=idx, outlier_gain=80.0, seed=3003, device=DEV)
+    down = big_layer(K, N, r, calib, 3004)
+    x = gen.make_activations(M, K, dist="gelu", outlier_idx=idx, outlier_gain=80.0, seed=3005, device=DEV).cpu()
+    run_case(x, [down, down], clip, 0, 1, rows=rows, check_partials_tiles=[(0, N - 128)])
