@@ -3,18 +3,27 @@
 //   Eq. 7 / 11    Y[m,n] = sum_g  P[m,g,n] * s[m,g] * sw[g,n]  +  sum_j T[m,j] L2[j,n]  +  b[n]
 //                 P[m,g,n] = sum_{k in group g} q[m,k] qw[k,n]            (exact int32)
 //
-// One CTA computes a 128 x 128 output tile.  Warp roles (16 warps):
+// Persistent kernel: one CTA per SM walks over 128 x 128 output tiles (column tile fastest, so the
+// CTAs running at any moment share a few row blocks of A and all of B through L2).  Warp roles:
 //   warp 0        TMA producer: nibble-packed A (activation codes) and B (weight codes) tiles of
-//                 128 K-codes (= two quantization groups) per stage into the "packed" ring.
-//   warp 1        MMA issuer (one lane): tcgen05.mma kind::i8, two K=32 instructions per group into a
-//                 fresh 128-column TMEM buffer per group (4 buffers), so that every group's int32
-//                 partial sums stay separate; kind::f16 for the low-rank product (first buffer of the tile).
+//                 128 K-codes (= two quantization groups) per stage into the "packed" ring, and the
+//                 matching 2 x 128 block of weight scales into the "sw" ring.
+//   warp 1        MMA issuer (one lane): per stage four tcgen05.mma kind::i8 (K=32 each), two per group,
+//                 each group into its own 128-column half of a 256-column TMEM slot (2 slots), so that
+//                 every group's int32 partial sums stay separate; kind::f16 for the low-rank product
+//                 (first slot of a tile).  One barrier round trip per stage, not per group: a single
+//                 thread needs ~300 cycles per wait/issue/commit cycle, more than one group's MMA time.
 //   warp 2        TMEM allocation / release.
 //   warps 4-7     unpack: packed ring -> signed bytes (16 x code, see quantize_kernel.cuh) written with
 //                 the 128-byte swizzle the tensor core expects, into the "s8" ring; they also fetch the
 //                 ready-made BF16 low-rank operands straight into an s8 slot by TMA.
-//   warps 8-15    epilogue: TMEM -> registers, int -> float, * s[m,g] * sw[g,n] into FP32 accumulators
-//                 (thread = output row, 64 columns each), finally * 2^-8 (undoing 16 x 16), + bias, BF16.
+//   warps 8-15    epilogue: TMEM -> registers (accumulator-fragment shape: 4 rows x 16 channels per
+//                 thread), int -> float, * sw[g,n] * s[m,g] into FP32 accumulators, finally * 2^-8
+//                 (undoing 16 x 16), + bias, BF16.
+//
+// The epilogue's FP32 work (one convert, one multiply, one fused multiply-add per partial sum, all with
+// distinct register operands) is what bounds this kernel, not the tensor core; its loop is therefore
+// written one stage (two groups) per iteration with all ring bookkeeping kept incremental.
 //
 // Every wait on an mbarrier is bounded: after kWaitLimitNs without progress (or as soon as another
 // CTA has reported an error) the role leaves its loop, the CTA records a code in *err and exits
@@ -33,10 +42,12 @@ constexpr int kBN = 128;            // output tile columns (output channels)
 constexpr int kBK = 128;            // K codes per pipeline stage = 2 quantization groups
 constexpr int kPackedStages = 4;    // ring of nibble-packed tiles (TMA destination)
 constexpr int kS8Stages = 3;        // ring of unpacked signed-byte tiles (tensor core source)
-constexpr int kTmemBufs = 4;        // kBN-column accumulator buffers in TMEM
+constexpr int kSwStages = 8;        // ring of weight-scale blocks (2 groups x kBN floats)
+constexpr int kTmemSlots = 2;       // TMEM slots of 2 x kBN columns: one per stage in flight
 constexpr int kGemmThreads = 512;
 constexpr int kUnpackWarp0 = 4, kUnpackWarps = 4;
 constexpr int kEpiWarp0 = 8, kEpiWarps = 8;
+constexpr int kRegsControl = 56, kRegsUnpack = 80, kRegsEpilogue = 184;   // setmaxnreg budgets per role
 
 constexpr uint32_t kPackedATile = kBM * (kBK / 2);   // 8 KiB
 constexpr uint32_t kPackedBTile = kBN * (kBK / 2);   // 8 KiB
@@ -44,9 +55,11 @@ constexpr uint32_t kPackedStageBytes = kPackedATile + kPackedBTile;
 constexpr uint32_t kS8ATile = kBM * kBK;             // 16 KiB
 constexpr uint32_t kS8BTile = kBN * kBK;             // 16 KiB
 constexpr uint32_t kS8StageBytes = kS8ATile + kS8BTile;
-constexpr uint32_t kNumBarriers = 2 * kPackedStages + 2 * kS8Stages + 2 * kTmemBufs;
-constexpr uint32_t kGemmSmemBytes =
-    1024 /*alignment slack*/ + kS8Stages * kS8StageBytes + kPackedStages * kPackedStageBytes + kNumBarriers * 8 + 16;
+constexpr uint32_t kSwStageBytes = 2 * kBN * 4;      // 1 KiB
+constexpr uint32_t kNumBarriers = 2 * kPackedStages + 2 * kS8Stages + 2 * kSwStages + 2 * kTmemSlots;
+constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kS8Stages * kS8StageBytes +
+                                    kPackedStages * kPackedStageBytes + kSwStages * kSwStageBytes +
+                                    kNumBarriers * 8 + 16;
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // 2 s
 
@@ -63,64 +76,154 @@ struct WaitEnv {
   volatile int* s_abort;     // CTA-local abort flag in shared memory
 };
 
-// Bounded wait.  Returns false if the CTA should give up.
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, const WaitEnv& env, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
+// Slow path of a bounded wait, kept out of line so that the callers' loops stay small.
+template <int BACKOFF_NS>
+__device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, int* g_err, volatile int* s_abort,
+                                               int code) {
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);  // roles that run ahead poll lazily: issue slots belong to the epilogue
     if ((++spins & 31u) == 0) {
-      if (*env.s_abort) return false;
-      if (*reinterpret_cast<volatile int*>(env.g_err) != 0) {
-        *env.s_abort = 1;
+      if (*s_abort) return false;
+      if (*reinterpret_cast<volatile int*>(g_err) != 0) {
+        *s_abort = 1;
         return false;
       }
       if (global_timer_ns() - t0 > kWaitLimitNs) {
-        atomicCAS(env.g_err, 0, code);
-        *env.s_abort = 1;
+        atomicCAS(g_err, 0, code);
+        *s_abort = 1;
         return false;
       }
     }
   }
 }
 
+// Bounded wait.  Returns false if the CTA should give up.
+template <int BACKOFF_NS = 0>
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, const WaitEnv& env, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return bounded_wait_slow<BACKOFF_NS>(bar, parity, env.g_err, env.s_abort, code);
+}
+
+// Position in a ring of N mbarrier pairs: slot index and the parity of the phase a consumer waits
+// for (a producer waits for parity ^ 1).  Advanced incrementally: no division in the hot loops.
+template <int N>
+struct Ring {
+  uint32_t slot = 0, parity = 0;
+  __device__ __forceinline__ void advance() {
+    if (++slot == N) {
+      slot = 0;
+      parity ^= 1u;
+    }
+  }
+};
+
+template <int N>
+__device__ __forceinline__ void set_max_regs_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void set_max_regs_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 struct GemmParams {
   const float* sa;      // [*, G] activation scales (row pitch G)
-  const float* sw;      // [G, N] weight scales
   const float* bias;    // [N] or nullptr
   uint16_t* Y;          // [M, N] BF16
   int M, N, K, r;
+  int tiles_m, tiles_n;
   int* err;
   int32_t* dbg_P;       // debug tap: [kBM, G, kBN] or nullptr
   int dbg_m0, dbg_n0;
 };
 
+// Output-channel order inside every 64-column block of a tile.  The epilogue reads TMEM with the
+// accumulator-fragment shape (16 lanes x 256 bits), where a thread (r = lane / 4, q = lane % 4) sees
+// columns 8 j + 2 q + e.  The packed weights (and the low-rank factor) are laid out at pack time so
+// that TMEM column c = 8 j + 2 q + e holds output channel 16 q + 2 j + e: every thread then owns 16
+// consecutive channels, reads its 16 weight scales with four conflict-free 128-bit loads, and
+// stores 32 contiguous bytes per output row.
+__host__ __device__ constexpr int tile_column_to_channel(int c) {
+  return 16 * ((c >> 1) & 3) + 2 * (c >> 3) + (c & 1);
+}
+
+// Rescales one fragment (16 TMEM lanes x 64 columns: two rows x 16 channels per thread) of a group's
+// int32 partial sums (256 x P) into the FP32 accumulators:  acc += float(P) * sw[channel] * sa[row].
+//   v     the fragment as loaded by tmem_ld_16x256b_x8
+//   w     the thread's 16 weight scales, channel order
+//   sa_t  activation scales of the thread's two rows (r and r + 8 of the 16-lane half)
+//   acc   [0..8): first row, [8..16): second row
+template <bool DEBUG>
+__device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[32], const float4 (&w)[4], float sa_t0,
+                                                 float sa_t1, float2* acc, int32_t* dbg_row0, int32_t* dbg_row1) {
+  const float2 s0 = make_float2(sa_t0, sa_t0), s1 = make_float2(sa_t1, sa_t1);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float2 wj = (j & 1) ? make_float2(w[j >> 1].z, w[j >> 1].w) : make_float2(w[j >> 1].x, w[j >> 1].y);
+    const float2 p0 = make_float2(static_cast<float>(static_cast<int32_t>(v[4 * j])),
+                                  static_cast<float>(static_cast<int32_t>(v[4 * j + 1])));
+    const float2 p1 = make_float2(static_cast<float>(static_cast<int32_t>(v[4 * j + 2])),
+                                  static_cast<float>(static_cast<int32_t>(v[4 * j + 3])));
+    acc[j] = __ffma2_rn(__fmul2_rn(p0, wj), s0, acc[j]);
+    acc[8 + j] = __ffma2_rn(__fmul2_rn(p1, wj), s1, acc[8 + j]);
+    if (DEBUG) {
+      if (dbg_row0 != nullptr) {
+        dbg_row0[2 * j] = static_cast<int32_t>(v[4 * j]) >> 8;
+        dbg_row0[2 * j + 1] = static_cast<int32_t>(v[4 * j + 1]) >> 8;
+        dbg_row1[2 * j] = static_cast<int32_t>(v[4 * j + 2]) >> 8;
+        dbg_row1[2 * j + 1] = static_cast<int32_t>(v[4 * j + 3]) >> 8;
+      }
+    }
+  }
+}
+
+// One 16-byte packed chunk (32 codes) -> two 16-byte runs of signed bytes (16 x code), shared to shared.
+template <int SRC_OFF, int DST_OFF>
+__device__ __forceinline__ void unpack_chunk(uint32_t src, uint32_t dst_lo, uint32_t dst_hi) {
+  uint32_t w0, w1, w2, w3;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
+               : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
+               : "r"(src), "n"(SRC_OFF));
+  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_lo), "n"(DST_OFF), "r"((w0 << 4) & 0xF0F0F0F0u),
+               "r"((w1 << 4) & 0xF0F0F0F0u), "r"((w2 << 4) & 0xF0F0F0F0u), "r"((w3 << 4) & 0xF0F0F0F0u)
+               : "memory");
+  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_hi), "n"(DST_OFF), "r"(w0 & 0xF0F0F0F0u),
+               "r"(w1 & 0xF0F0F0F0u), "r"(w2 & 0xF0F0F0F0u), "r"(w3 & 0xF0F0F0F0u)
+               : "memory");
+}
+
 template <bool DEBUG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL2, const GemmParams p) {
+            const __grid_constant__ CUtensorMap tmSW, const __grid_constant__ CUtensorMap tmT,
+            const __grid_constant__ CUtensorMap tmL2, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t s8_base = smem_base;
   const uint32_t packed_base = s8_base + kS8Stages * kS8StageBytes;
-  const uint32_t bar_base = packed_base + kPackedStages * kPackedStageBytes;
+  const uint32_t sw_base = packed_base + kPackedStages * kPackedStageBytes;
+  const uint32_t bar_base = sw_base + kSwStages * kSwStageBytes;
   const uint32_t bar_packed_full = bar_base;
   const uint32_t bar_packed_empty = bar_packed_full + 8 * kPackedStages;
   const uint32_t bar_s8_full = bar_packed_empty + 8 * kPackedStages;
   const uint32_t bar_s8_empty = bar_s8_full + 8 * kS8Stages;
-  const uint32_t bar_tmem_full = bar_s8_empty + 8 * kS8Stages;
-  const uint32_t bar_tmem_empty = bar_tmem_full + 8 * kTmemBufs;
-  const uint32_t misc_off = (bar_tmem_empty + 8 * kTmemBufs) - smem_base;
+  const uint32_t bar_sw_full = bar_s8_empty + 8 * kS8Stages;
+  const uint32_t bar_sw_empty = bar_sw_full + 8 * kSwStages;
+  const uint32_t bar_tmem_full = bar_sw_empty + 8 * kSwStages;
+  const uint32_t bar_tmem_empty = bar_tmem_full + 8 * kTmemSlots;
+  const uint32_t misc_off = (bar_tmem_empty + 8 * kTmemSlots) - smem_base;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * kBN, m0 = blockIdx.y * kBM;
   const int G = p.K >> 6;
   const int n_int_stages = (G + 1) >> 1;
   const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
+  const int num_tiles = p.tiles_m * p.tiles_n;
   const WaitEnv env{p.err, s_abort};
 
   if (threadIdx.x == 0) {
@@ -133,7 +236,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_init(bar_s8_full + 8 * i, kUnpackWarps);
       mbar_init(bar_s8_empty + 8 * i, 1);
     }
-    for (int i = 0; i < kTmemBufs; ++i) {
+    for (int i = 0; i < kSwStages; ++i) {
+      mbar_init(bar_sw_full + 8 * i, 1);
+      mbar_init(bar_sw_empty + 8 * i, kEpiWarps);
+    }
+    for (int i = 0; i < kTmemSlots; ++i) {
       mbar_init(bar_tmem_full + 8 * i, 1);
       mbar_init(bar_tmem_empty + 8 * i, kEpiWarps);
     }
@@ -141,6 +248,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    tma_prefetch_desc(&tmSW);
     if (p.r > 0) {
       tma_prefetch_desc(&tmT);
       tma_prefetch_desc(&tmL2);
@@ -154,231 +262,326 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  const bool live = (*s_abort == 0);
 
-  if (!*s_abort) {
-    if (warp == 0) {
+  // Per tile the TMEM slots are used by: [one slot for the low-rank product, if r > 0] followed by
+  // one slot per K stage (two groups, 128 columns each).
+  if (warp < kUnpackWarp0) {
+    set_max_regs_dec<kRegsControl>();
+    if (live && warp == 0 && lane == 0) {
       // ------------------------------------------------------------------ TMA producer
-      if (lane == 0) {
-        for (int pi = 0; pi < n_int_stages; ++pi) {
-          const int ps = pi % kPackedStages;
-          const uint32_t ph = (pi / kPackedStages) & 1;
-          if (!bounded_wait(bar_packed_empty + 8 * ps, ph ^ 1u, env, kErrProducerWait)) break;
-          const uint32_t full = bar_packed_full + 8 * ps;
-          const uint32_t dst = packed_base + ps * kPackedStageBytes;
+      Ring<kPackedStages> pk;
+      Ring<kSwStages> sw;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+        for (int st = 0; st < n_int_stages; ++st) {
+          ok = bounded_wait<128>(bar_packed_empty + 8 * pk.slot, pk.parity ^ 1u, env, kErrProducerWait) &&
+               bounded_wait<128>(bar_sw_empty + 8 * sw.slot, sw.parity ^ 1u, env, kErrProducerWait);
+          if (!ok) break;
+          const uint32_t full = bar_packed_full + 8 * pk.slot;
+          const uint32_t dst = packed_base + pk.slot * kPackedStageBytes;
           mbar_arrive_expect_tx(full, kPackedStageBytes);
-          tma_load_2d(dst, &tmA, full, pi * (kBK / 2), m0);
-          tma_load_2d(dst + kPackedATile, &tmB, full, pi * (kBK / 2), n0);
+          tma_load_2d(dst, &tmA, full, st * (kBK / 2), m0);
+          tma_load_2d(dst + kPackedATile, &tmB, full, st * (kBK / 2), n0);
+          const uint32_t swfull = bar_sw_full + 8 * sw.slot;
+          mbar_arrive_expect_tx(swfull, kSwStageBytes);
+          tma_load_2d(sw_base + sw.slot * kSwStageBytes, &tmSW, swfull, n0, 2 * st);
+          pk.advance();
+          sw.advance();
         }
       }
-    } else if (warp == 1) {
+    } else if (live && warp == 1 && lane == 0) {
       // ------------------------------------------------------------------ MMA issuer
-      if (lane == 0) {
-        constexpr uint32_t idesc_i8 = umma_idesc(2, 1, kBM, kBN);
-        constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
-        int si = 0, unit = 0;
-        bool ok = true;
+      constexpr uint32_t idesc_i8 = umma_idesc(2, 1, kBM, kBN);
+      constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
+      Ring<kS8Stages> s8;
+      Ring<kTmemSlots> tm;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         if (n_lr_stages > 0) {
-          ok = bounded_wait(bar_tmem_empty, 1u, env, kErrMmaWait);
-          for (int l = 0; ok && l < n_lr_stages; ++l, ++si) {
-            const int ss = si % kS8Stages;
-            ok = bounded_wait(bar_s8_full + 8 * ss, (si / kS8Stages) & 1, env, kErrMmaWait);
+          ok = bounded_wait<32>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait);
+          for (int l = 0; ok && l < n_lr_stages; ++l) {
+            ok = bounded_wait<32>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t a = s8_base + ss * kS8StageBytes, b = a + kS8ATile;
+            const uint32_t a = s8_base + s8.slot * kS8StageBytes, b = a + kS8ATile;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-              umma_f16(tmem_base, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_bf16,
-                       (l > 0 || kk > 0) ? 1u : 0u);
+              umma_f16(tmem_base + tm.slot * 2 * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk),
+                       idesc_bf16, (l > 0 || kk > 0) ? 1u : 0u);
             }
-            umma_commit(bar_s8_empty + 8 * ss);
+            umma_commit(bar_s8_empty + 8 * s8.slot);
+            s8.advance();
           }
-          if (ok) umma_commit(bar_tmem_full);
-          unit = 1;
-        }
-        for (int g = 0; ok && g < G; ++g, ++unit) {
-          const int buf = unit % kTmemBufs;
-          ok = bounded_wait(bar_tmem_empty + 8 * buf, ((unit / kTmemBufs) & 1) ^ 1u, env, kErrMmaWait);
           if (!ok) break;
-          const int ss = si % kS8Stages;
-          const int half = g & 1;
-          if (half == 0) {
-            ok = bounded_wait(bar_s8_full + 8 * ss, (si / kS8Stages) & 1, env, kErrMmaWait);
-            if (!ok) break;
-          }
+          umma_commit(bar_tmem_full + 8 * tm.slot);
+          tm.advance();
+        }
+        for (int st = 0; ok && st < n_int_stages; ++st) {
+          ok = bounded_wait<32>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait) &&
+               bounded_wait<32>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
+          if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t a = s8_base + ss * kS8StageBytes, b = a + kS8ATile;
-          const uint32_t d = tmem_base + buf * kBN;
+          const uint32_t a = s8_base + s8.slot * kS8StageBytes, b = a + kS8ATile;
+          const uint32_t d = tmem_base + tm.slot * 2 * kBN;
+          const int groups = (2 * st + 1 < G) ? 2 : 1;
 #pragma unroll
-          for (int kk = 0; kk < 2; ++kk) {
-            const uint32_t off = 64 * half + 32 * kk;
-            umma_i8(d, umma_desc_k_sw128(a, off), umma_desc_k_sw128(b, off), idesc_i8, kk);
+          for (int kk = 0; kk < 4; ++kk) {  // bytes [32 kk, 32 kk + 32) of every row: group kk / 2, K half kk % 2
+            if (kk < 2 * groups) {
+              umma_i8(d + (kk >> 1) * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_i8,
+                      kk & 1);
+            }
           }
-          if (half == 1 || g == G - 1) {
-            umma_commit(bar_s8_empty + 8 * ss);
-            ++si;
-          }
-          umma_commit(bar_tmem_full + 8 * buf);
+          umma_commit(bar_s8_empty + 8 * s8.slot);
+          umma_commit(bar_tmem_full + 8 * tm.slot);
+          s8.advance();
+          tm.advance();
         }
       }
-    } else if (warp >= kUnpackWarp0 && warp < kUnpackWarp0 + kUnpackWarps) {
+    }
+  } else if (warp < kEpiWarp0) {
+    set_max_regs_dec<kRegsUnpack>();
+    if (live) {
       // ------------------------------------------------------------------ unpack warps
       const int ut = threadIdx.x - 32 * kUnpackWarp0;  // 0..127
-      const int total = n_lr_stages + n_int_stages;
-      for (int si = 0; si < total; ++si) {
-        const int ss = si % kS8Stages;
-        if (!bounded_wait(bar_s8_empty + 8 * ss, ((si / kS8Stages) & 1) ^ 1u, env, kErrUnpackWait)) break;
-        const uint32_t s8a = s8_base + ss * kS8StageBytes;
-        const uint32_t full = bar_s8_full + 8 * ss;
-        if (si < n_lr_stages) {
-          // BF16 low-rank operands are tensor-core ready: fetch them straight into the s8 slot.
-          if (ut == 0) {
-            mbar_arrive_expect_tx(full, kS8StageBytes);
-            tma_load_2d(s8a, &tmT, full, si * 64, m0);
-            tma_load_2d(s8a + kS8ATile, &tmL2, full, si * 64, n0);
-          } else if (lane == 0) {
-            mbar_arrive(full);
-          }
-          continue;
-        }
-        const int pi = si - n_lr_stages;
-        const int ps = pi % kPackedStages;
-        if (!bounded_wait(bar_packed_full + 8 * ps, (pi / kPackedStages) & 1, env, kErrUnpackWait)) break;
-        const uint32_t pk = packed_base + ps * kPackedStageBytes;
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int id = it * 128 + ut;
-          const int tileB = id >> 9;
-          const int rid = id & 511;
-          const int row = rid >> 2, c = rid & 3;
-          const uint32_t src = pk + tileB * kPackedATile + row * 64 + c * 16;
-          uint32_t w0, w1, w2, w3;
-          asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(src));
-          const uint32_t dst_row = s8a + tileB * kS8ATile + row * 128;
-          const uint32_t sw = row & 7;
-          const uint32_t d_lo = dst_row + (((2 * c) ^ sw) << 4);
-          const uint32_t d_hi = dst_row + (((2 * c + 1) ^ sw) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d_lo), "r"((w0 << 4) & 0xF0F0F0F0u),
-                       "r"((w1 << 4) & 0xF0F0F0F0u), "r"((w2 << 4) & 0xF0F0F0F0u), "r"((w3 << 4) & 0xF0F0F0F0u)
-                       : "memory");
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(d_hi), "r"(w0 & 0xF0F0F0F0u),
-                       "r"(w1 & 0xF0F0F0F0u), "r"(w2 & 0xF0F0F0F0u), "r"(w3 & 0xF0F0F0F0u)
-                       : "memory");
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(full);
-          mbar_arrive(bar_packed_empty + 8 * ps);
-        }
-      }
-    } else if (warp >= kEpiWarp0) {
-      // ------------------------------------------------------------------ epilogue warps
-      const int ew = warp - kEpiWarp0;
-      const int quarter = ew & 3, colhalf = ew >> 2;
-      const int row = m0 + 32 * quarter + lane;
-      const bool row_ok = row < p.M;
-      const int col0 = n0 + 64 * colhalf;
-      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colhalf;
-      float2 acc[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) acc[j] = make_float2(0.0f, 0.0f);
-      int unit = 0;
+      // Thread ut owns packed chunk (ut & 3) of rows (ut >> 2) + 32 * j, j = 0..3, of A and of B:
+      // every address is a per-thread base plus a compile-time constant.
+      const uint32_t src_off = (ut >> 2) * 64 + (ut & 3) * 16;
+      const uint32_t swz = (ut >> 2) & 7;
+      const uint32_t dst_lo_off = (ut >> 2) * 128 + (((2 * (ut & 3)) ^ swz) << 4);
+      const uint32_t dst_hi_off = (ut >> 2) * 128 + (((2 * (ut & 3) + 1) ^ swz) << 4);
+      Ring<kS8Stages> s8;
+      Ring<kPackedStages> pk;
       bool ok = true;
-      if (n_lr_stages > 0) {
-        ok = bounded_wait(bar_tmem_full, 0u, env, kErrEpilogueWait);
-        if (ok) {
-          tc_fence_after_sync();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t v[16];
-            tmem_ld_32x32b_x16(t_lane + 16 * c, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              acc[8 * c + j] = make_float2(__uint_as_float(v[2 * j]) * 256.0f, __uint_as_float(v[2 * j + 1]) * 256.0f);
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+        for (int st = 0; ok && st < n_lr_stages + n_int_stages; ++st) {
+          ok = bounded_wait<64>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrUnpackWait);
+          if (!ok) break;
+          const uint32_t s8a = s8_base + s8.slot * kS8StageBytes;
+          const uint32_t full = bar_s8_full + 8 * s8.slot;
+          s8.advance();
+          if (st < n_lr_stages) {
+            // BF16 low-rank operands are tensor-core ready: fetch them straight into the s8 slot.
+            if (ut == 0) {
+              mbar_arrive_expect_tx(full, kS8StageBytes);
+              tma_load_2d(s8a, &tmT, full, st * 64, m0);
+              tma_load_2d(s8a + kS8ATile, &tmL2, full, st * 64, n0);
+            } else if (lane == 0) {
+              mbar_arrive(full);
             }
+            continue;
           }
-          tc_fence_before_sync();
+          ok = bounded_wait<64>(bar_packed_full + 8 * pk.slot, pk.parity, env, kErrUnpackWait);
+          if (!ok) break;
+          const uint32_t src = packed_base + pk.slot * kPackedStageBytes + src_off;
+          const uint32_t dlo = s8a + dst_lo_off, dhi = s8a + dst_hi_off;
+          unpack_chunk<0 * 2048, 0 * 4096>(src, dlo, dhi);
+          unpack_chunk<1 * 2048, 1 * 4096>(src, dlo, dhi);
+          unpack_chunk<2 * 2048, 2 * 4096>(src, dlo, dhi);
+          unpack_chunk<3 * 2048, 3 * 4096>(src, dlo, dhi);
+          unpack_chunk<kPackedATile + 0 * 2048, kS8ATile + 0 * 4096>(src, dlo, dhi);
+          unpack_chunk<kPackedATile + 1 * 2048, kS8ATile + 1 * 4096>(src, dlo, dhi);
+          unpack_chunk<kPackedATile + 2 * 2048, kS8ATile + 2 * 4096>(src, dlo, dhi);
+          unpack_chunk<kPackedATile + 3 * 2048, kS8ATile + 3 * 4096>(src, dlo, dhi);
+          fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_tmem_empty);
-        }
-        unit = 1;
-      }
-      const float* sa_row = p.sa + static_cast<size_t>(row_ok ? row : 0) * G;
-      const bool vec4 = (G & 3) == 0;
-      float4 sa_cur = make_float4(0.f, 0.f, 0.f, 0.f), sa_nxt = sa_cur;
-      if (vec4 && row_ok) sa_nxt = __ldg(reinterpret_cast<const float4*>(sa_row));
-      for (int g = 0; ok && g < G; ++g, ++unit) {
-        float sa;
-        if (vec4) {
-          if ((g & 3) == 0) {
-            sa_cur = sa_nxt;
-            if (row_ok && g + 4 < G) sa_nxt = __ldg(reinterpret_cast<const float4*>(sa_row + g + 4));
+          if (lane == 0) {
+            mbar_arrive(full);
+            mbar_arrive(bar_packed_empty + 8 * pk.slot);
           }
-          const int gi = g & 3;
-          sa = gi == 0 ? sa_cur.x : gi == 1 ? sa_cur.y : gi == 2 ? sa_cur.z : sa_cur.w;
-        } else {
-          sa = row_ok ? __ldg(sa_row + g) : 0.0f;
+          pk.advance();
         }
-        const float4* swp = reinterpret_cast<const float4*>(p.sw + static_cast<size_t>(g) * p.N + col0);
-        const int buf = unit % kTmemBufs;
-        ok = bounded_wait(bar_tmem_full + 8 * buf, (unit / kTmemBufs) & 1, env, kErrEpilogueWait);
+      }
+    }
+  } else {
+    set_max_regs_inc<kRegsEpilogue>();
+    if (live) {
+      // ------------------------------------------------------------------ epilogue warps
+      // Warp ew owns TMEM lanes 32 * (ew % 4) .. +31 (token rows) and the 64-column block ew / 4.  A
+      // thread (r = lane / 4, q = lane % 4) owns rows r, r + 8, r + 16, r + 24 of that quarter and the 16
+      // consecutive output channels 16 q .. 16 q + 15 of the block (see tile_column_to_channel).
+      // Software pipeline over 16-lane fragments: while one fragment is being rescaled the next TMEM
+      // load (and, at stage boundaries, the barrier wait in front of it) is already in flight.
+      const int ew = warp - kEpiWarp0;
+      const int quarter = ew & 3, colblk = ew >> 2;
+      const int fr = lane >> 2, fq = lane & 3;
+      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colblk;
+      constexpr uint32_t kHalf = 16u << 16;  // second 16-lane half of the quarter
+      const float* sw_thread = reinterpret_cast<const float*>(smem + (sw_base - smem_base)) + 64 * colblk + 16 * fq;
+      const bool sa_vec2 = (G & 1) == 0;  // rows of the scale matrix are 8-byte aligned: load two groups at once
+      Ring<kTmemSlots> tm;
+      Ring<kSwStages> sw;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+        const int row0 = m0 + 32 * quarter + fr;  // the thread's rows are row0 + 8 t, t = 0..3
+        const int ch0 = n0 + 64 * colblk + 16 * fq;
+        const bool dbg_tile = DEBUG && p.dbg_P != nullptr && m0 == p.dbg_m0 && n0 == p.dbg_n0;
+        float2 acc[32];  // [t][j]: row row0 + 8 t, channels ch0 + 2 j, ch0 + 2 j + 1
+        uint32_t vA[32], vB[32];
+        // First slot of the tile.
+        ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
         if (!ok) break;
         tc_fence_after_sync();
-        const float2 sa2 = make_float2(sa, sa);
+        tmem_ld_16x256b_x8(t_lane + tm.slot * 2 * kBN, vA);
+        tmem_wait_ld();
+        if (n_lr_stages > 0) {
+          // The low-rank product T L2 (FP32) seeds the accumulators, scaled like the integer part.
+          tmem_ld_16x256b_x8(t_lane + kHalf + tm.slot * 2 * kBN, vB);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {  // 16 columns at a time keeps the live registers under the 128 budget
-          uint32_t v[16];
-          tmem_ld_32x32b_x16(t_lane + buf * kBN + 16 * c, v);
-          float4 w[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) w[i] = __ldg(swp + 4 * c + i);
-          tmem_wait_ld();
-          if (DEBUG) {
-            if (p.dbg_P != nullptr && m0 == p.dbg_m0 && n0 == p.dbg_n0) {
-              int32_t* dst = p.dbg_P + (static_cast<size_t>(32 * quarter + lane) * G + g) * kBN + 64 * colhalf + 16 * c;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) dst[j] = static_cast<int32_t>(v[j]) >> 8;
-            }
+          for (int j = 0; j < 8; ++j) {
+            acc[j] = make_float2(__uint_as_float(vA[4 * j]) * 256.0f, __uint_as_float(vA[4 * j + 1]) * 256.0f);
+            acc[8 + j] = make_float2(__uint_as_float(vA[4 * j + 2]) * 256.0f, __uint_as_float(vA[4 * j + 3]) * 256.0f);
           }
+          tmem_wait_ld();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
+          tm.advance();
+          ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
+          if (!ok) break;
+          tc_fence_after_sync();
+          tmem_ld_16x256b_x8(t_lane + tm.slot * 2 * kBN, vA);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 sc0 = __fmul2_rn(sa2, make_float2(w[i].x, w[i].y));
-            const float2 sc1 = __fmul2_rn(sa2, make_float2(w[i].z, w[i].w));
-            const float2 p0 = make_float2(static_cast<float>(static_cast<int32_t>(v[4 * i])),
-                                          static_cast<float>(static_cast<int32_t>(v[4 * i + 1])));
-            const float2 p1 = make_float2(static_cast<float>(static_cast<int32_t>(v[4 * i + 2])),
-                                          static_cast<float>(static_cast<int32_t>(v[4 * i + 3])));
-            acc[8 * c + 2 * i] = __ffma2_rn(p0, sc0, acc[8 * c + 2 * i]);
-            acc[8 * c + 2 * i + 1] = __ffma2_rn(p1, sc1, acc[8 * c + 2 * i + 1]);
+          for (int j = 0; j < 8; ++j) {
+            acc[16 + j] = make_float2(__uint_as_float(vB[4 * j]) * 256.0f, __uint_as_float(vB[4 * j + 1]) * 256.0f);
+            acc[24 + j] = make_float2(__uint_as_float(vB[4 * j + 2]) * 256.0f, __uint_as_float(vB[4 * j + 3]) * 256.0f);
+          }
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) acc[j] = make_float2(0.0f, 0.0f);
+        }
+        // Activation scales of the thread's four rows, one stage (two groups) ahead.  Rows past M read
+        // row 0 (their results are never stored).
+        const float* sa_p[4];
+        float2 sa_nxt[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int rw = row0 + 8 * t;
+          sa_p[t] = p.sa + static_cast<size_t>(rw < p.M ? rw : 0) * G;
+          if (sa_vec2) {
+            sa_nxt[t] = __ldg(reinterpret_cast<const float2*>(sa_p[t]));
+          } else {
+            sa_nxt[t] = make_float2(__ldg(sa_p[t]), G > 1 ? __ldg(sa_p[t] + 1) : 0.0f);
           }
         }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * buf);
-      }
-      if (ok && row_ok) {
-        uint4* yrow = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + col0);
-        const float4* bp = p.bias ? reinterpret_cast<const float4*>(p.bias + col0) : nullptr;
+        // Invariant at the top of each iteration: the stage's TMEM slot has been waited for and vA
+        // holds the first 16-lane fragment of its first group.
+        float2 (&acc_lo)[16] = *reinterpret_cast<float2(*)[16]>(&acc[0]);   // rows row0, row0 + 8
+        float2 (&acc_hi)[16] = *reinterpret_cast<float2(*)[16]>(&acc[16]);  // rows row0 + 16, row0 + 24
+        for (int st = 0; st < n_int_stages; ++st) {
+          const int g0 = 2 * st;
+          const bool two = g0 + 1 < G;
+          const bool last_stage = st + 1 == n_int_stages;
+          float2 sa[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {  // 8 output columns per 16-byte store
-          float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-          if (bp) {
-            b0 = __ldg(bp + 2 * i);
-            b1 = __ldg(bp + 2 * i + 1);
+          for (int t = 0; t < 4; ++t) {
+            sa[t] = sa_nxt[t];
+            if (!last_stage) {
+              if (sa_vec2) {
+                sa_nxt[t] = __ldg(reinterpret_cast<const float2*>(sa_p[t] + g0 + 2));
+              } else {
+                sa_nxt[t] = make_float2(__ldg(sa_p[t] + g0 + 2), g0 + 3 < G ? __ldg(sa_p[t] + g0 + 3) : 0.0f);
+              }
+            }
           }
-          const float k = 0.00390625f;  // 2^-8: the codes were fed to the tensor core as 16 x code on both sides
-          const float2 a0 = acc[4 * i], a1 = acc[4 * i + 1], a2 = acc[4 * i + 2], a3 = acc[4 * i + 3];
-          __nv_bfloat162 o0 = __floats2bfloat162_rn(fmaf(a0.x, k, b0.x), fmaf(a0.y, k, b0.y));
-          __nv_bfloat162 o1 = __floats2bfloat162_rn(fmaf(a1.x, k, b0.z), fmaf(a1.y, k, b0.w));
-          __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(a2.x, k, b1.x), fmaf(a2.y, k, b1.y));
-          __nv_bfloat162 o3 = __floats2bfloat162_rn(fmaf(a3.x, k, b1.z), fmaf(a3.y, k, b1.w));
-          uint4 o;
-          o.x = *reinterpret_cast<uint32_t*>(&o0);
-          o.y = *reinterpret_cast<uint32_t*>(&o1);
-          o.z = *reinterpret_cast<uint32_t*>(&o2);
-          o.w = *reinterpret_cast<uint32_t*>(&o3);
-          yrow[i] = o;
+          const uint32_t t_grp = t_lane + tm.slot * 2 * kBN;
+          tmem_ld_16x256b_x8_before(t_grp + kHalf, vB, vA[0]);
+          ok = bounded_wait(bar_sw_full + 8 * sw.slot, sw.parity, env, kErrEpilogueWait);
+          if (!ok) break;
+          const float4* swp = reinterpret_cast<const float4*>(sw_thread + sw.slot * (2 * kBN));
+          float4 w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) w[i] = swp[i];
+          int32_t *d0 = nullptr, *d1 = nullptr, *d2 = nullptr, *d3 = nullptr;
+          if (DEBUG) {
+            if (dbg_tile) {
+              const size_t rs = static_cast<size_t>(8) * G * kBN;
+              d0 = p.dbg_P + (static_cast<size_t>(32 * quarter + fr) * G + g0) * kBN + 64 * colblk + 16 * fq;
+              d1 = d0 + rs;
+              d2 = d1 + rs;
+              d3 = d2 + rs;
+            }
+          }
+          // ---- group g0
+          rescale_fragment<DEBUG>(vA, w, sa[0].x, sa[1].x, acc, d0, d1);
+          tmem_wait_ld_after(acc_lo);
+          if (two) {
+            tmem_ld_16x256b_x8_before(t_grp + kBN, vA, vB[0]);
+          } else {
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
+          }
+          rescale_fragment<DEBUG>(vB, w, sa[2].x, sa[3].x, acc + 16, d2, d3);
+          if (two) {
+            // ---- group g0 + 1
+            tmem_wait_ld_after(acc_hi);
+            tmem_ld_16x256b_x8_before(t_grp + kBN + kHalf, vB, vA[0]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) w[i] = swp[kBN / 4 + i];
+            if (DEBUG) {
+              if (dbg_tile) {
+                d0 += kBN;
+                d1 += kBN;
+                d2 += kBN;
+                d3 += kBN;
+              }
+            }
+            rescale_fragment<DEBUG>(vA, w, sa[0].y, sa[1].y, acc, d0, d1);
+            tmem_wait_ld_after(acc_lo);
+            // The whole slot is in registers: hand it back to the MMA warp.
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
+          }
+          tm.advance();
+          if (!last_stage) {
+            ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
+            if (!ok) break;
+            tc_fence_after_sync();
+            tmem_ld_16x256b_x8_before(t_lane + tm.slot * 2 * kBN, vA, vB[0]);
+          }
+          if (two) rescale_fragment<DEBUG>(vB, w, sa[2].y, sa[3].y, acc + 16, d2, d3);
+          if (!last_stage) tmem_wait_ld_after(acc_hi);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_sw_empty + 8 * sw.slot);
+          sw.advance();
+        }
+        if (!ok) break;
+        {
+          float4 bv[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            bv[i] = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+          const float k = 0.00390625f;  // 2^-8: the codes went through the tensor core as 16 x code on both sides
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const int rw = row0 + 8 * t;
+            if (rw < p.M) {
+              uint4* yrow = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(rw) * p.N + ch0);
+#pragma unroll
+              for (int i = 0; i < 2; ++i) {  // 8 channels per 16-byte store
+                const float2 a0 = acc[8 * t + 4 * i], a1 = acc[8 * t + 4 * i + 1], a2 = acc[8 * t + 4 * i + 2],
+                             a3 = acc[8 * t + 4 * i + 3];
+                const float4 b0 = bv[2 * i], b1 = bv[2 * i + 1];
+                __nv_bfloat162 o0 = __floats2bfloat162_rn(fmaf(a0.x, k, b0.x), fmaf(a0.y, k, b0.y));
+                __nv_bfloat162 o1 = __floats2bfloat162_rn(fmaf(a1.x, k, b0.z), fmaf(a1.y, k, b0.w));
+                __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(a2.x, k, b1.x), fmaf(a2.y, k, b1.y));
+                __nv_bfloat162 o3 = __floats2bfloat162_rn(fmaf(a3.x, k, b1.z), fmaf(a3.y, k, b1.w));
+                uint4 o;
+                o.x = *reinterpret_cast<uint32_t*>(&o0);
+                o.y = *reinterpret_cast<uint32_t*>(&o1);
+                o.z = *reinterpret_cast<uint32_t*>(&o2);
+                o.w = *reinterpret_cast<uint32_t*>(&o3);
+                yrow[i] = o;
+              }
+            }
+          }
         }
       }
     }

@@ -133,6 +133,50 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&v)
       : "memory");
 }
 
+// 16 lanes x (8 repetitions of 256 bits): the accumulator-fragment shape.  With r = laneid / 4 and
+// q = laneid % 4, register 4 j + 2 t + e of a thread holds TMEM lane (base_lane + r + 8 t), column
+// (base_col + 8 j + 2 q + e),  j = 0..7, t = 0..1, e = 0..1.
+__device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Scheduling pins.  The compiler is free to move register-only arithmetic across the (volatile)
+// TMEM load and wait instructions, which would serialise "load the next fragment" and "rescale the
+// current one".  `pin` (a register the following arithmetic reads) makes that arithmetic stay below
+// the load; tmem_wait_ld_after() takes the arithmetic's results as operands so that the wait stays
+// below it.  Neither adds an instruction.
+__device__ __forceinline__ void tmem_ld_16x256b_x8_before(uint32_t taddr, uint32_t (&v)[32], uint32_t& pin) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "+r"(pin)
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld_after(float2 (&a)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+f"(a[0].x), "+f"(a[0].y), "+f"(a[1].x), "+f"(a[1].y), "+f"(a[2].x), "+f"(a[2].y), "+f"(a[3].x),
+                 "+f"(a[3].y), "+f"(a[4].x), "+f"(a[4].y), "+f"(a[5].x), "+f"(a[5].y), "+f"(a[6].x), "+f"(a[6].y),
+                 "+f"(a[7].x), "+f"(a[7].y), "+f"(a[8].x), "+f"(a[8].y), "+f"(a[9].x), "+f"(a[9].y), "+f"(a[10].x),
+                 "+f"(a[10].y), "+f"(a[11].x), "+f"(a[11].y), "+f"(a[12].x), "+f"(a[12].y), "+f"(a[13].x),
+                 "+f"(a[13].y), "+f"(a[14].x), "+f"(a[14].y), "+f"(a[15].x), "+f"(a[15].y)
+               :
+               : "memory");
+}
+
 // Shared-memory operand descriptor, K-major tile with the 128-byte swizzle: rows of 128 bytes,
 // 8-row swizzle atoms of 1024 bytes stacked along M/N (stride-byte-offset 1024), tile base aligned
 // to 1024 bytes.  `byte_offset_in_row` selects the K slice (multiple of 32 bytes) inside the row.

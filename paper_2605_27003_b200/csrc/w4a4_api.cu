@@ -22,17 +22,19 @@ __global__ void reciprocal_kernel(const float* __restrict__ lam, float* __restri
   if (k < K) out[k] = __fdiv_rn(1.0f, lam[k]);
 }
 
-// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed, K-interleaved (see quantize_kernel.cuh).
+// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed, K-interleaved (see quantize_kernel.cuh),
+// rows in the tile order of tile_column_to_channel (see gemm_kernel.cuh).
 // One thread builds one 16-byte chunk (32 consecutive K of one output channel).
 __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __restrict__ out, int K, int N,
                                    int* __restrict__ bad) {
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;  // packed row = position in the tile
   const int c = blockIdx.y;
   if (n >= N) return;
+  const int ch = (n & ~63) + tile_column_to_channel(n & 63);  // output channel stored at that position
   uint32_t w[4] = {0, 0, 0, 0};
   bool oob = false;
   for (int o = 0; o < 32; ++o) {
-    const int v = q[static_cast<size_t>(32 * c + o) * N + n];
+    const int v = q[static_cast<size_t>(32 * c + o) * N + ch];
     oob |= (v < -8 || v > 7);
     const uint32_t nib = static_cast<uint32_t>(v) & 0xFu;
     const int word = (o & 15) >> 2, byte = o & 3, hi = o >> 4;
@@ -62,13 +64,15 @@ __global__ void l1_fragment_kernel(const uint16_t* __restrict__ L1, uint2* __res
                         static_cast<uint32_t>(v[2]) | (static_cast<uint32_t>(v[3]) << 16));
 }
 
-// L2 [r, N] BF16 -> [N, 2r]: the transposed factor twice, matching the [T_hi | T_lo] split of T.
+// L2 [r, N] BF16 -> [N, 2r]: the transposed factor twice, matching the [T_hi | T_lo] split of T,
+// rows in the same tile order as the packed weights.
 __global__ void l2_dup_kernel(const uint16_t* __restrict__ L2, uint16_t* __restrict__ out, int r, int N) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(N) * 2 * r) return;
   const int c = idx % (2 * r);
   const int n = idx / (2 * r);
-  out[idx] = L2[static_cast<size_t>(c % r) * N + n];
+  const int ch = (n & ~63) + tile_column_to_channel(n & 63);
+  out[idx] = L2[static_cast<size_t>(c % r) * N + ch];
 }
 
 // Test-only decoders of the activation kernel's outputs.
@@ -109,6 +113,7 @@ struct w4a4_ctx {
   uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
   int* d_err = nullptr;       // device error word
   size_t bytes = 0;
+  int num_sms = 0;
   EncodeTiledFn encode = nullptr;
 };
 
@@ -119,7 +124,7 @@ struct ExpertData {
   uint2* l1frag = nullptr;
   uint16_t* l2dup = nullptr;   // [N, 2r]
   float* bias = nullptr;       // [N] or null
-  CUtensorMap tmB, tmL2;
+  CUtensorMap tmB, tmSW, tmL2;
 };
 
 struct w4a4_layer {
@@ -240,24 +245,26 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   const ExpertData& e = h->experts[expert_id];
   GemmParams p;
   p.sa = ctx->scales;
-  p.sw = e.wscale;
   p.bias = e.bias;
   p.Y = static_cast<uint16_t*>(Y);
   p.M = M;
   p.N = h->N;
   p.K = h->K;
   p.r = h->r;
+  p.tiles_m = (M + kBM - 1) / kBM;
+  p.tiles_n = h->N / kBN;
   p.err = ctx->d_err;
   p.dbg_P = dbg_P;
   p.dbg_m0 = dbg_m0;
   p.dbg_n0 = dbg_n0;
-  const dim3 grid(h->N / kBN, (M + kBM - 1) / kBM), block(kGemmThreads);
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
   if (dbg_P) {
-    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
+    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, tmT, tmL2, p);
   } else {
-    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
+    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, tmT, tmL2, p);
   }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
@@ -307,6 +314,7 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   ctx->max_M = max_M;
   ctx->max_K = max_K;
   ctx->max_r = max_r;
+  ctx->num_sms = prop.multiProcessorCount;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -444,6 +452,10 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
 
     if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, kBK / 2, kBN,
                    CU_TENSOR_MAP_SWIZZLE_NONE))
+      st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK &&
+        !encode_2d(ctx->encode, &e.tmSW, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, e.wscale, N, G, static_cast<uint64_t>(N) * 4,
+                   kBN, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
       st = W4A4_ERR_CUDA;
     if (st == W4A4_OK && r > 0 &&
         !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kBN,
