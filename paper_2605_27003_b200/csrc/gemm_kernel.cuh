@@ -7,7 +7,8 @@
 // CTAs running at any moment share a few row blocks of A and all of B through L2).  Warp roles:
 //   warp 0        TMA producer: nibble-packed A (activation codes) and B (weight codes) tiles of
 //                 128 K-codes (= two quantization groups) per stage into the "packed" ring, and the
-//                 matching 2 x 128 block of weight scales into the "sw" ring.
+//                 matching 2 x 128 blocks of weight scales and of activation scales into the "scale"
+//                 ring (same mbarrier; that ring is deep enough to need no barriers of its own).
 //   warp 1        MMA issuer (one lane): per stage four tcgen05.mma kind::i8 (K=32 each), two per group,
 //                 each group into its own 128-column half of a 256-column TMEM slot (2 slots), so that
 //                 every group's int32 partial sums stay separate; kind::f16 for the low-rank product
@@ -42,7 +43,8 @@ constexpr int kBN = 128;            // output tile columns (output channels)
 constexpr int kBK = 128;            // K codes per pipeline stage = 2 quantization groups
 constexpr int kPackedStages = 4;    // ring of nibble-packed tiles (TMA destination)
 constexpr int kS8Stages = 3;        // ring of unpacked signed-byte tiles (tensor core source)
-constexpr int kSwStages = 8;        // ring of weight-scale blocks (2 groups x kBN floats)
+constexpr int kScaleStages = 16;   // ring of scale blocks (2 groups x (kBN weight scales + kBM activation scales));
+                                   // deeper than the TMA producer can ever run ahead of the epilogue, so it needs no barriers
 constexpr int kTmemSlots = 2;       // TMEM slots of 2 x kBN columns: one per stage in flight
 constexpr int kGemmThreads = 512;
 constexpr int kUnpackWarp0 = 4, kUnpackWarps = 4;
@@ -55,10 +57,10 @@ constexpr uint32_t kPackedStageBytes = kPackedATile + kPackedBTile;
 constexpr uint32_t kS8ATile = kBM * kBK;             // 16 KiB
 constexpr uint32_t kS8BTile = kBN * kBK;             // 16 KiB
 constexpr uint32_t kS8StageBytes = kS8ATile + kS8BTile;
-constexpr uint32_t kSwStageBytes = 2 * kBN * 4;      // 1 KiB
-constexpr uint32_t kNumBarriers = 2 * kPackedStages + 2 * kS8Stages + 2 * kSwStages + 2 * kTmemSlots;
+constexpr uint32_t kScaleStageBytes = 2 * (kBN + kBM) * 4;   // 2 KiB: sw[2][kBN] then sa[2][kBM]
+constexpr uint32_t kNumBarriers = 2 * kPackedStages + 2 * kS8Stages + 2 * kTmemSlots;
 constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kS8Stages * kS8StageBytes +
-                                    kPackedStages * kPackedStageBytes + kSwStages * kSwStageBytes +
+                                    kPackedStages * kPackedStageBytes + kScaleStages * kScaleStageBytes +
                                     kNumBarriers * 8 + 16;
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // 2 s
@@ -130,7 +132,6 @@ __device__ __forceinline__ void set_max_regs_dec() {
 }
 
 struct GemmParams {
-  const float* sa;      // [*, G] activation scales (row pitch G)
   const float* bias;    // [N] or nullptr
   uint16_t* Y;          // [M, N] BF16
   int M, N, K, r;
@@ -198,22 +199,21 @@ __device__ __forceinline__ void unpack_chunk(uint32_t src, uint32_t dst_lo, uint
 template <bool DEBUG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const __grid_constant__ CUtensorMap tmSW, const __grid_constant__ CUtensorMap tmT,
+            const __grid_constant__ CUtensorMap tmSW, const __grid_constant__ CUtensorMap tmSA,
+            const __grid_constant__ CUtensorMap tmT,
             const __grid_constant__ CUtensorMap tmL2, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t s8_base = smem_base;
   const uint32_t packed_base = s8_base + kS8Stages * kS8StageBytes;
-  const uint32_t sw_base = packed_base + kPackedStages * kPackedStageBytes;
-  const uint32_t bar_base = sw_base + kSwStages * kSwStageBytes;
+  const uint32_t scale_base = packed_base + kPackedStages * kPackedStageBytes;
+  const uint32_t bar_base = scale_base + kScaleStages * kScaleStageBytes;
   const uint32_t bar_packed_full = bar_base;
   const uint32_t bar_packed_empty = bar_packed_full + 8 * kPackedStages;
   const uint32_t bar_s8_full = bar_packed_empty + 8 * kPackedStages;
   const uint32_t bar_s8_empty = bar_s8_full + 8 * kS8Stages;
-  const uint32_t bar_sw_full = bar_s8_empty + 8 * kS8Stages;
-  const uint32_t bar_sw_empty = bar_sw_full + 8 * kSwStages;
-  const uint32_t bar_tmem_full = bar_sw_empty + 8 * kSwStages;
+  const uint32_t bar_tmem_full = bar_s8_empty + 8 * kS8Stages;
   const uint32_t bar_tmem_empty = bar_tmem_full + 8 * kTmemSlots;
   const uint32_t misc_off = (bar_tmem_empty + 8 * kTmemSlots) - smem_base;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
@@ -236,10 +236,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_init(bar_s8_full + 8 * i, kUnpackWarps);
       mbar_init(bar_s8_empty + 8 * i, 1);
     }
-    for (int i = 0; i < kSwStages; ++i) {
-      mbar_init(bar_sw_full + 8 * i, 1);
-      mbar_init(bar_sw_empty + 8 * i, kEpiWarps);
-    }
     for (int i = 0; i < kTmemSlots; ++i) {
       mbar_init(bar_tmem_full + 8 * i, 1);
       mbar_init(bar_tmem_empty + 8 * i, kEpiWarps);
@@ -249,6 +245,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
     tma_prefetch_desc(&tmSW);
+    tma_prefetch_desc(&tmSA);
     if (p.r > 0) {
       tma_prefetch_desc(&tmT);
       tma_prefetch_desc(&tmL2);
@@ -271,24 +268,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (live && warp == 0 && lane == 0) {
       // ------------------------------------------------------------------ TMA producer
       Ring<kPackedStages> pk;
-      Ring<kSwStages> sw;
+      Ring<kScaleStages> sc;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
         for (int st = 0; st < n_int_stages; ++st) {
-          ok = bounded_wait<128>(bar_packed_empty + 8 * pk.slot, pk.parity ^ 1u, env, kErrProducerWait) &&
-               bounded_wait<128>(bar_sw_empty + 8 * sw.slot, sw.parity ^ 1u, env, kErrProducerWait);
+          ok = bounded_wait<256>(bar_packed_empty + 8 * pk.slot, pk.parity ^ 1u, env, kErrProducerWait);
           if (!ok) break;
           const uint32_t full = bar_packed_full + 8 * pk.slot;
           const uint32_t dst = packed_base + pk.slot * kPackedStageBytes;
-          mbar_arrive_expect_tx(full, kPackedStageBytes);
+          const uint32_t sdst = scale_base + sc.slot * kScaleStageBytes;
+          mbar_arrive_expect_tx(full, kPackedStageBytes + kScaleStageBytes);
           tma_load_2d(dst, &tmA, full, st * (kBK / 2), m0);
           tma_load_2d(dst + kPackedATile, &tmB, full, st * (kBK / 2), n0);
-          const uint32_t swfull = bar_sw_full + 8 * sw.slot;
-          mbar_arrive_expect_tx(swfull, kSwStageBytes);
-          tma_load_2d(sw_base + sw.slot * kSwStageBytes, &tmSW, swfull, n0, 2 * st);
+          tma_load_2d(sdst, &tmSW, full, n0, 2 * st);
+          tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * st);
           pk.advance();
-          sw.advance();
+          sc.advance();
         }
       }
     } else if (live && warp == 1 && lane == 0) {
@@ -300,9 +296,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         if (n_lr_stages > 0) {
-          ok = bounded_wait<32>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait);
+          ok = bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait);
           for (int l = 0; ok && l < n_lr_stages; ++l) {
-            ok = bounded_wait<32>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
+            ok = bounded_wait<64>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t a = s8_base + s8.slot * kS8StageBytes, b = a + kS8ATile;
@@ -319,8 +315,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tm.advance();
         }
         for (int st = 0; ok && st < n_int_stages; ++st) {
-          ok = bounded_wait<32>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait) &&
-               bounded_wait<32>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
+          ok = bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait) &&
+               bounded_wait<64>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t a = s8_base + s8.slot * kS8StageBytes, b = a + kS8ATile;
@@ -357,7 +353,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
         for (int st = 0; ok && st < n_lr_stages + n_int_stages; ++st) {
-          ok = bounded_wait<64>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrUnpackWait);
+          ok = bounded_wait<128>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrUnpackWait);
           if (!ok) break;
           const uint32_t s8a = s8_base + s8.slot * kS8StageBytes;
           const uint32_t full = bar_s8_full + 8 * s8.slot;
@@ -373,7 +369,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             continue;
           }
-          ok = bounded_wait<64>(bar_packed_full + 8 * pk.slot, pk.parity, env, kErrUnpackWait);
+          ok = bounded_wait<128>(bar_packed_full + 8 * pk.slot, pk.parity, env, kErrUnpackWait);
           if (!ok) break;
           const uint32_t src = packed_base + pk.slot * kPackedStageBytes + src_off;
           const uint32_t dlo = s8a + dst_lo_off, dhi = s8a + dst_hi_off;
@@ -409,10 +405,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int fr = lane >> 2, fq = lane & 3;
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colblk;
       constexpr uint32_t kHalf = 16u << 16;  // second 16-lane half of the quarter
-      const float* sw_thread = reinterpret_cast<const float*>(smem + (sw_base - smem_base)) + 64 * colblk + 16 * fq;
-      const bool sa_vec2 = (G & 1) == 0;  // rows of the scale matrix are 8-byte aligned: load two groups at once
+      // Per scale stage: sw[2][kBN] then sa[2][kBM] floats.  The thread's 16 weight scales start at
+      // float 64 colblk + 16 q, its four activation scales at float 2 kBN + 32 quarter + r + 8 t.
+      const float* sw_thread = reinterpret_cast<const float*>(smem + (scale_base - smem_base)) + 64 * colblk + 16 * fq;
+      const float* sa_thread = reinterpret_cast<const float*>(smem + (scale_base - smem_base)) + 2 * kBN + 32 * quarter + fr;
       Ring<kTmemSlots> tm;
-      Ring<kSwStages> sw;
+      Ring<kScaleStages> sc;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
@@ -454,20 +452,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int j = 0; j < 32; ++j) acc[j] = make_float2(0.0f, 0.0f);
         }
-        // Activation scales of the thread's four rows, one stage (two groups) ahead.  Rows past M read
-        // row 0 (their results are never stored).
-        const float* sa_p[4];
-        float2 sa_nxt[4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const int rw = row0 + 8 * t;
-          sa_p[t] = p.sa + static_cast<size_t>(rw < p.M ? rw : 0) * G;
-          if (sa_vec2) {
-            sa_nxt[t] = __ldg(reinterpret_cast<const float2*>(sa_p[t]));
-          } else {
-            sa_nxt[t] = make_float2(__ldg(sa_p[t]), G > 1 ? __ldg(sa_p[t] + 1) : 0.0f);
-          }
-        }
         // Invariant at the top of each iteration: the stage's TMEM slot has been waited for and vA
         // holds the first 16-lane fragment of its first group.
         float2 (&acc_lo)[16] = *reinterpret_cast<float2(*)[16]>(&acc[0]);   // rows row0, row0 + 8
@@ -476,23 +460,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int g0 = 2 * st;
           const bool two = g0 + 1 < G;
           const bool last_stage = st + 1 == n_int_stages;
-          float2 sa[4];
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            sa[t] = sa_nxt[t];
-            if (!last_stage) {
-              if (sa_vec2) {
-                sa_nxt[t] = __ldg(reinterpret_cast<const float2*>(sa_p[t] + g0 + 2));
-              } else {
-                sa_nxt[t] = make_float2(__ldg(sa_p[t] + g0 + 2), g0 + 3 < G ? __ldg(sa_p[t] + g0 + 3) : 0.0f);
-              }
-            }
-          }
           const uint32_t t_grp = t_lane + tm.slot * 2 * kBN;
           tmem_ld_16x256b_x8_before(t_grp + kHalf, vB, vA[0]);
-          ok = bounded_wait(bar_sw_full + 8 * sw.slot, sw.parity, env, kErrEpilogueWait);
-          if (!ok) break;
-          const float4* swp = reinterpret_cast<const float4*>(sw_thread + sw.slot * (2 * kBN));
+          // The stage's scales landed before the MMA that produced this slot was even issued (they ride
+          // on the packed tiles' mbarrier), so they can be read without a wait of their own.
+          const float4* swp = reinterpret_cast<const float4*>(sw_thread + sc.slot * (kScaleStageBytes / 4));
+          const float* sap = sa_thread + sc.slot * (kScaleStageBytes / 4);
+          float2 sa[4];  // .x: group g0, .y: group g0 + 1
+#pragma unroll
+          for (int t = 0; t < 4; ++t) sa[t] = make_float2(sap[8 * t], sap[kBM + 8 * t]);
           float4 w[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) w[i] = swp[i];
@@ -547,9 +523,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           if (two) rescale_fragment<DEBUG>(vB, w, sa[2].y, sa[3].y, acc + 16, d2, d3);
           if (!last_stage) tmem_wait_ld_after(acc_hi);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_sw_empty + 8 * sw.slot);
-          sw.advance();
+          sc.advance();
         }
         if (!ok) break;
         {

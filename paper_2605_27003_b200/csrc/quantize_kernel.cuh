@@ -104,7 +104,8 @@ template <int R>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
-                uint8_t* __restrict__ codes, float* __restrict__ scales, uint16_t* __restrict__ t_hilo) {
+                uint8_t* __restrict__ codes, float* __restrict__ scales, int scales_ld,
+                uint16_t* __restrict__ t_hilo) {
   constexpr int NT = R / 8;  // n-tiles of the m16n8k16 MMA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qi = lane >> 2, qj = lane & 3;
@@ -150,8 +151,9 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     const size_t cpitch = static_cast<size_t>(K >> 1);
     if (okA) *reinterpret_cast<uint2*>(codes + rowA * cpitch + 32 * g + 8 * qj) = wA;
     if (okB) *reinterpret_cast<uint2*>(codes + rowB * cpitch + 32 * g + 8 * qj) = wB;
-    if (qj == 0 && okA) scales[static_cast<size_t>(rowA) * G + g] = sA;
-    if (qj == 1 && okB) scales[static_cast<size_t>(rowB) * G + g] = sB;
+    // Scales are stored group-major ([G][scales_ld]): kernel 2 fetches a (2 groups x 128 rows) block by TMA.
+    if (qj == 0 && okA) scales[static_cast<size_t>(g) * scales_ld + rowA] = sA;
+    if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = sB;
 
     if constexpr (NT > 0) {
       const uint2* lf = l1frag + (static_cast<size_t>(g) * 4 * NT) * 32 + lane;

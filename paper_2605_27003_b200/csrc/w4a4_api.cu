@@ -86,6 +86,14 @@ __global__ void decode_codes_kernel(const uint8_t* __restrict__ packed, int8_t* 
   const int nib = (o >> 4) ? (b >> 4) : (b & 0xF);
   codes[idx] = static_cast<int8_t>((nib ^ 8) - 8);
 }
+// Group-major workspace scales -> [M, G].
+__global__ void decode_scales_kernel(const float* __restrict__ ws, int ld, float* __restrict__ out, int M, int G) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(M) * G) return;
+  const int g = idx % G;
+  const size_t m = idx / G;
+  out[idx] = ws[static_cast<size_t>(g) * ld + m];
+}
 __global__ void decode_t_kernel(const uint16_t* __restrict__ thl, float* __restrict__ T, int M, int r) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(M) * r) return;
@@ -109,7 +117,8 @@ struct w4a4_ctx {
   int device = 0;
   int max_M = 0, max_K = 0, max_r = 0;
   uint8_t* codes = nullptr;   // [max_M, K/2] packed activation codes (pitch K/2 of the running layer)
-  float* scales = nullptr;    // [max_M, K/64]
+  float* scales = nullptr;    // [K/64, scales_ld] group-major activation scales
+  int scales_ld = 0;          // max_M rounded up to a multiple of 4 (16-byte rows for TMA)
   uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
   int* d_err = nullptr;       // device error word
   size_t bytes = 0;
@@ -131,7 +140,7 @@ struct w4a4_layer {
   w4a4_ctx* ctx = nullptr;
   int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0;
   std::vector<ExpertData> experts;
-  CUtensorMap tmA, tmT;
+  CUtensorMap tmA, tmSA, tmT;
   size_t bytes = 0;
 };
 
@@ -226,7 +235,7 @@ w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define W4A4_LAUNCH_Q(R)                                                                                         \
   quantize_kernel<R><<<grid, block, 0, stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
-                                                 ctx->scales, ctx->t_hilo)
+                                                 ctx->scales, ctx->scales_ld, ctx->t_hilo)
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
     case 16: W4A4_LAUNCH_Q(16); break;
@@ -244,7 +253,6 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   w4a4_ctx* ctx = h->ctx;
   const ExpertData& e = h->experts[expert_id];
   GemmParams p;
-  p.sa = ctx->scales;
   p.bias = e.bias;
   p.Y = static_cast<uint16_t*>(Y);
   p.M = M;
@@ -262,9 +270,9 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
   if (dbg_P) {
-    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, tmT, tmL2, p);
+    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
   } else {
-    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, tmT, tmL2, p);
+    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
   }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
@@ -315,6 +323,7 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   ctx->max_K = max_K;
   ctx->max_r = max_r;
   ctx->num_sms = prop.multiProcessorCount;
+  ctx->scales_ld = (max_M + 3) & ~3;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -324,7 +333,8 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   }
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   w4a4_status_t st = dev_alloc(&ctx->codes, static_cast<size_t>(max_M) * (max_K / 2), &ctx->bytes);
-  if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(max_M) * (max_K / 64), &ctx->bytes);
+  if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(ctx->scales_ld) * (max_K / 64), &ctx->bytes);
+  if (st == W4A4_OK && cudaMemset(ctx->scales, 0, sizeof(float) * ctx->scales_ld * (max_K / 64)) != cudaSuccess) st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) st = dev_alloc(&ctx->t_hilo, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8), &ctx->bytes);
   if (st == W4A4_OK) st = dev_alloc(&ctx->d_err, 1, &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->d_err, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
@@ -472,6 +482,10 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
       !encode_2d(ctx->encode, &h->tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->codes, K / 2, ctx->max_M, K / 2, kBK / 2,
                  kBM, CU_TENSOR_MAP_SWIZZLE_NONE))
     st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK &&
+      !encode_2d(ctx->encode, &h->tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ctx->scales, ctx->scales_ld, G,
+                 static_cast<uint64_t>(ctx->scales_ld) * 4, kBM, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
+    st = W4A4_ERR_CUDA;
   if (st == W4A4_OK && r > 0 &&
       !encode_2d(ctx->encode, &h->tmT, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo, 2 * r, ctx->max_M, 4 * r, 64,
                  kBM, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -524,8 +538,9 @@ w4a4_status_t w4a4_debug_quantize(w4a4_handle_t h, const void* X, int M, int exp
   if (st != W4A4_OK || M == 0) return st;
   const size_t nc = static_cast<size_t>(M) * h->K;
   decode_codes_kernel<<<static_cast<unsigned>((nc + 255) / 256), 256, 0, s>>>(h->ctx->codes, codes, M, h->K);
-  if (cudaMemcpyAsync(scales, h->ctx->scales, sizeof(float) * M * (h->K / 64), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
-    return W4A4_ERR_CUDA;
+  const size_t ns = static_cast<size_t>(M) * (h->K / 64);
+  decode_scales_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256, 0, s>>>(h->ctx->scales, h->ctx->scales_ld, scales, M,
+                                                                               h->K / 64);
   if (T && h->r > 0) {
     const size_t nt = static_cast<size_t>(M) * h->r;
     decode_t_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, s>>>(h->ctx->t_hilo, T, M, h->r);
