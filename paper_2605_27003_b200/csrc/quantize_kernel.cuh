@@ -70,20 +70,32 @@ __device__ __forceinline__ void smooth8(const uint4& raw, const float4& r0, cons
   xh[7] = __fmul_rn(__uint_as_float(raw.w & 0xffff0000u), r1.w);
 }
 
-// Quantize the lane's 16 smoothed values of one row and return its two packed words.
-// `s_out` receives the group scale (identical on the 4 lanes of the quad).
-__device__ __forceinline__ uint2 quantize16(const float* xh, float rho, float& s_out) {
-  float a = 0.0f;
+// Group absolute maximum of the lane's 16 smoothed values, combined over the quad (= 64 channels).
+__device__ __forceinline__ float quad_absmax16(const float* xh) {
+  float a0 = fmaxf(fabsf(xh[0]), fabsf(xh[1])), a1 = fmaxf(fabsf(xh[2]), fabsf(xh[3]));
 #pragma unroll
-  for (int e = 0; e < 16; ++e) a = fmaxf(a, fabsf(xh[e]));
+  for (int e = 4; e < 16; e += 2) {
+    a0 = fmaxf(a0, fabsf(xh[e]));
+    a1 = fmaxf(a1, fabsf(xh[e + 1]));
+  }
+  float a = fmaxf(a0, a1);
   a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
   a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-  float s = 0.0f, is = 0.0f;
+  return a;
+}
+
+// Eq. 8-9 / Eq. 4: s = (rho * a) / 7 and its reciprocal, both correctly rounded (IEEE); a == 0 -> 0, 0.
+__device__ __forceinline__ void group_scale(float rho, float a, float& s, float& is) {
+  s = 0.0f;
+  is = 0.0f;
   if (a > 0.0f) {
     s = __fdiv_rn(__fmul_rn(rho, a), 7.0f);
-    is = __fdiv_rn(1.0f, s);
+    is = __frcp_rn(s);  // == 1.0f / s, round to nearest
   }
-  s_out = s;
+}
+
+// Quantize the lane's 16 smoothed values of one row (Eq. 3) and return its two packed words.
+__device__ __forceinline__ uint2 quantize16(const float* xh, float is) {
   // code + 8 in [0, 15]:  (float bits of z + 1.5*2^23 + 8) - bits(1.5*2^23), clamped.
   uint32_t u[16];
 #pragma unroll
@@ -91,11 +103,16 @@ __device__ __forceinline__ uint2 quantize16(const float* xh, float rho, float& s
     const float f = __fadd_rn(__fmul_rn(xh[e], is), 12582920.0f);
     u[e] = static_cast<uint32_t>(__viaddmin_s32_relu(__float_as_int(f), -0x4B400000, 15));
   }
-  uint32_t w0 = 0, w1 = 0;
+  // One shift-add per code places its nibble: word w, byte b = low nibble u[4w+b], high nibble u[8+4w+b].
+  uint32_t w0 = u[0], w1 = u[4];
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
-    w0 |= (u[b] | (u[8 + b] << 4)) << (8 * b);
-    w1 |= (u[4 + b] | (u[12 + b] << 4)) << (8 * b);
+    if (b > 0) {
+      w0 += u[b] << (8 * b);
+      w1 += u[4 + b] << (8 * b);
+    }
+    w0 += u[8 + b] << (8 * b + 4);
+    w1 += u[12 + b] << (8 * b + 4);
   }
   return make_uint2(w0 ^ 0x88888888u, w1 ^ 0x88888888u);  // offset-binary -> two's complement nibbles
 }
@@ -137,6 +154,21 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
       if (okA) { ra0 = ldg_stream_v4(xa + 64 * gn); ra1 = ldg_stream_v4(xa + 64 * gn + 16); }
       if (okB) { rb0 = ldg_stream_v4(xb + 64 * gn); rb1 = ldg_stream_v4(xb + 64 * gn + 16); }
     }
+    if constexpr (NT > 0) {
+      // Pull the next group's L1 fragments (NT * 128 bytes per lane-line) into L1 while this group computes:
+      // every warp needs all of L1 once per 16 rows, far more bytes than it reads from X, and an L2 hit
+      // in front of every MMA would stall the warp.
+      if (gn < G) {
+        const char* nf = reinterpret_cast<const char*>(l1frag) + static_cast<size_t>(gn) * (4 * NT * 32 * 8);
+#pragma unroll
+        for (int c = 0; c < (4 * NT * 32 * 8) / 4096; ++c) {
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(nf + c * 4096 + lane * 128));
+        }
+        if ((4 * NT * 32 * 8) % 4096 != 0 && lane < ((4 * NT * 32 * 8) % 4096) / 128) {
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(nf + ((4 * NT * 32 * 8) / 4096) * 4096 + lane * 128));
+        }
+      }
+    }
     const float4* rl = reinterpret_cast<const float4*>(rlam + 64 * g + coff);
     const float4 l0 = __ldg(rl), l1 = __ldg(rl + 1), l4 = __ldg(rl + 4), l5 = __ldg(rl + 5);
     float xhA[16], xhB[16];
@@ -145,18 +177,24 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     smooth8(cb0, l0, l1, xhB);
     smooth8(cb1, l4, l5, xhB + 8);
 
-    float sA, sB;
-    const uint2 wA = quantize16(xhA, rho, sA);
-    const uint2 wB = quantize16(xhB, rho, sB);
+    // Even lanes of the quad derive row A's scale, odd lanes row B's; one shuffle shares the reciprocals.
+    const float aA = quad_absmax16(xhA), aB = quad_absmax16(xhB);
+    float s_mine, is_mine;
+    group_scale(rho, (qj & 1) ? aB : aA, s_mine, is_mine);
+    const float is_other = __shfl_xor_sync(0xffffffffu, is_mine, 1);
+    const float isA = (qj & 1) ? is_other : is_mine, isB = (qj & 1) ? is_mine : is_other;
+    const uint2 wA = quantize16(xhA, isA);
+    const uint2 wB = quantize16(xhB, isB);
     const size_t cpitch = static_cast<size_t>(K >> 1);
     if (okA) *reinterpret_cast<uint2*>(codes + rowA * cpitch + 32 * g + 8 * qj) = wA;
     if (okB) *reinterpret_cast<uint2*>(codes + rowB * cpitch + 32 * g + 8 * qj) = wB;
     // Scales are stored group-major ([G][scales_ld]): kernel 2 fetches a (2 groups x 128 rows) block by TMA.
-    if (qj == 0 && okA) scales[static_cast<size_t>(g) * scales_ld + rowA] = sA;
-    if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = sB;
+    if (qj == 0 && okA) scales[static_cast<size_t>(g) * scales_ld + rowA] = s_mine;
+    if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = s_mine;
 
     if constexpr (NT > 0) {
-      const uint2* lf = l1frag + (static_cast<size_t>(g) * 4 * NT) * 32 + lane;
+      // Fragment storage: [group][i][n-tile pair][lane] as uint4 = (b0, b1) of n-tile 2p, (b0, b1) of n-tile 2p + 1.
+      const uint4* lf = reinterpret_cast<const uint4*>(l1frag) + (static_cast<size_t>(g) * 4 * (NT / 2)) * 32 + lane;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         uint32_t a[4];
@@ -165,9 +203,10 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
         a[2] = pack_bf16x2(xhA[4 * i + 2], xhA[4 * i + 3]);
         a[3] = pack_bf16x2(xhB[4 * i + 2], xhB[4 * i + 3]);
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          const uint2 b = __ldg(lf + (i * NT + nt) * 32);
-          mma_bf16_16816(acc[nt], a, b.x, b.y);
+        for (int np = 0; np < NT / 2; ++np) {
+          const uint4 b = __ldg(lf + (i * (NT / 2) + np) * 32);
+          mma_bf16_16816(acc[2 * np], a, b.x, b.y);
+          mma_bf16_16816(acc[2 * np + 1], a, b.z, b.w);
         }
       }
     }

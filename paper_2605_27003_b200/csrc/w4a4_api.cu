@@ -44,16 +44,19 @@ __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __rest
   *reinterpret_cast<uint4*>(out + static_cast<size_t>(n) * (K >> 1) + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// L1 [K, r] BF16 -> B fragments of mma.sync m16n8k16 in the K order the activation kernel uses.
+// L1 [K, r] BF16 -> B fragments of mma.sync m16n8k16 in the K order the activation kernel uses,
+// stored [group][i][n-tile pair][lane][n-tile of the pair] so that one 16-byte load feeds two MMAs.
 __global__ void l1_fragment_kernel(const uint16_t* __restrict__ L1, uint2* __restrict__ out, int K, int r) {
   const int NT = r / 8;
   const size_t total = static_cast<size_t>(K / 64) * 4 * NT * 32;
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= total) return;
-  const int lane = idx & 31;
-  const int nt = (idx >> 5) % NT;
-  const int i = ((idx >> 5) / NT) & 3;
-  const int g = (idx >> 5) / NT / 4;
+  const int sub = idx & 1;             // n-tile inside the pair
+  const int lane = (idx >> 1) & 31;
+  const int np = (idx >> 6) % (NT / 2);
+  const int i = ((idx >> 6) / (NT / 2)) & 3;
+  const int g = (idx >> 6) / (NT / 2) / 4;
+  const int nt = 2 * np + sub;
   const int j = lane & 3, n = 8 * nt + (lane >> 2);
   uint16_t v[4];
   for (int e = 0; e < 4; ++e) {
