@@ -108,6 +108,26 @@ w4a4_status_t w4a4_debug_partials(w4a4_handle_t h, const void* X, int M, int exp
                                   const float* clip_table, void* Y, int m0, int n0, int32_t* P, void* stream);
 void w4a4_tile_shape(int* tile_m, int* tile_n);
 
+/* Activation quantization for callers that cannot allocate (the paper has no counterpart: this entry
+ * point exists for deployment, not for the method).  Code that runs in a host callback, under a runtime
+ * whose memory pool owns the whole device, or on a latency-critical path where the implicit device
+ * synchronisation of cudaMalloc is not acceptable cannot create a context or a handle.  This call needs
+ * neither: it computes Xh = X / lambda, the per-(token, 64-channel group) scales and the 4-bit codes
+ * (Eq. 3-5, 8-9; no low-rank branch) with its scratch held in a fixed array inside the library image
+ * (about 2.3 MiB of device memory on every GPU that loads the library, for the life of the process).
+ *   X       device BF16 [M, K] row-major, 16-byte aligned          lambda  device FP32 [K], > 0
+ *   clip_table / clip_index   device FP32 table and the index of the ratio to use (read on the device)
+ *   codes   device int8 [M, K], one code per byte in [-8, 7]       scales  device FP32 [M, K/64]
+ * Limits: K a multiple of 64, K <= 16384 and M * K <= 4194304; anything larger returns W4A4_ERR_SHAPE.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  The first call on each device
+ * looks up the scratch's device address (cudaGetSymbolAddress) with that device current, so make that
+ * first call outside any stream capture.  All calls share the one scratch array: every byte a call reads
+ * it has written itself first (nothing relies on old contents or on zeros), but two calls that overlap
+ * on the GPU (different streams, or threads) race on it -- serialise them.  Work is enqueued on `stream`;
+ * the call does not synchronise. */
+w4a4_status_t w4a4_quantize_noalloc(const void* X, int M, int K, const float* lambda, const float* clip_table,
+                                    int clip_index, int8_t* codes, float* scales, void* stream);
+
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
  * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
 w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_ALLOC", 4
 EXPORTED_SYMBOLS = (
     "w4a4_ctx_create", "w4a4_ctx_destroy", "w4a4_pack_weights", "w4a4_destroy", "w4a4_linear_forward",
     "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
-    "w4a4_tile_shape", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
+    "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
 
@@ -68,6 +68,7 @@ def _lib():
         lib.w4a4_gemm_from_workspace.argtypes = [vp, ci, ci, vp, vp]
         lib.w4a4_debug_quantize.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.w4a4_debug_partials.argtypes = [vp, vp, ci, ci, ci, vp, vp, ci, ci, vp, vp]
+        lib.w4a4_quantize_noalloc.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp]
         lib.w4a4_tile_shape.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
         lib.w4a4_tile_shape.restype = None
         lib.w4a4_query_status.argtypes = [vp]
@@ -185,6 +186,12 @@ def w4a4_debug_quantize(handle, X, M, expert_id, timestep_bin, clip_table, codes
 def w4a4_debug_partials(handle, X, M, expert_id, timestep_bin, clip_table, Y, m0, n0, P, stream=None):
     _check(_lib().w4a4_debug_partials(handle, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table), _ptr(Y), m0, n0,
                                       _ptr(P), _stream(stream)), "w4a4_debug_partials")
+
+
+def w4a4_quantize_noalloc(X, M, K, lam, clip_table, clip_index, codes, scales, stream=None):
+    """Context-free activation quantization into caller buffers; the library's built-in scratch is used."""
+    _check(_lib().w4a4_quantize_noalloc(_ptr(X), M, K, _ptr(lam), _ptr(clip_table), clip_index, _ptr(codes),
+                                        _ptr(scales), _stream(stream)), "w4a4_quantize_noalloc")
 
 
 def w4a4_query_status(ctx) -> int:

@@ -1,0 +1,56 @@
+"""The allocation-free activation-quantization entry point against the regular one.
+
+Callers that may not allocate device memory (host callbacks, latency-critical paths, runtimes that own all
+device memory through their own pool) use w4a4_quantize_noalloc, whose scratch is a fixed array inside the library.  Here
+it is called twice in a row through the C ABI, on different inputs, and each result must equal what the
+context-based tap (w4a4_debug_quantize) returns for the same input: integer codes and FP32 scales
+bit for bit, the bar the other parity tests use for these quantities.  The file name keeps this test last
+in collection order.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2605_27003_b200 as w4
+from paper_2605_27003_b200 import build as pkg_build
+from workloads import generator as gen
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def test_noalloc_quantize_matches_context_path_on_two_calls_in_a_row():
+    pkg_build.build()
+    w4.load_library()
+    M, K, N = 200, 1024, 128
+    layer = gen.make_layer_direct(K, N, 0, seed=11).to(DEV)
+    ctx = w4.Context(0, M, K, 0)
+    L = w4.Layer(ctx, [layer], num_bins=4)
+    clip = torch.tensor([[[1.0, 0.9, 0.75, 0.6]]], dtype=torch.float32, device=DEV)
+    idx = gen.outlier_channels(K, 0.01, 5)
+    for call, (seed, b) in enumerate(((21, 2), (22, 0))):
+        x = gen.make_activations(M, K, sigma=1.5, outlier_idx=idx, outlier_gain=30.0, seed=seed, device=DEV)
+        if call == 1:
+            x[3] = 0  # an all-zero token: scales 0, codes 0
+        codes_ref = torch.full((M, K), 99, dtype=torch.int8, device=DEV)
+        scales_ref = torch.full((M, K // 64), -1.0, dtype=torch.float32, device=DEV)
+        w4.w4a4_debug_quantize(L.ptr, x, M, 0, b, clip, codes_ref, scales_ref, None)
+        codes = torch.full((M, K), 77, dtype=torch.int8, device=DEV)
+        scales = torch.full((M, K // 64), -2.0, dtype=torch.float32, device=DEV)
+        w4.w4a4_quantize_noalloc(x, M, K, layer.lam, clip, b, codes, scales)
+        torch.cuda.synchronize()
+        assert torch.equal(codes, codes_ref), f"call {call}: codes differ"
+        assert np.array_equal(scales.cpu().numpy().view(np.uint32), scales_ref.cpu().numpy().view(np.uint32)), \
+            f"call {call}: scales differ"
+        assert codes.abs().max() <= 8 and codes.max() <= 7
+    # sizes beyond the built-in scratch are refused with a clear status, nothing is launched
+    big = torch.empty(1, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(w4.W4A4Error) as ei:
+        w4.w4a4_quantize_noalloc(big, 8192, 1024, layer.lam, clip, 0, codes, scales)  # M * K > 4 Mi
+    assert ei.value.status == 2
+    with pytest.raises(w4.W4A4Error) as ei:
+        w4.w4a4_quantize_noalloc(big, 1, 32768, layer.lam, clip, 0, codes, scales)  # K > 16384
+    assert ei.value.status == 2
+    ctx.check()
+    L.close()
+    ctx.close()
