@@ -143,12 +143,14 @@ struct GemmParams {
 
 // Output-channel order inside every 64-column block of a tile.  The epilogue reads TMEM with the
 // accumulator-fragment shape (16 lanes x 256 bits), where a thread (r = lane / 4, q = lane % 4) sees
-// columns 8 j + 2 q + e.  The packed weights (and the low-rank factor) are laid out at pack time so
-// that TMEM column c = 8 j + 2 q + e holds output channel 16 q + 2 j + e: every thread then owns 16
-// consecutive channels, reads its 16 weight scales with four conflict-free 128-bit loads, and
-// stores 32 contiguous bytes per output row.
+// columns 8 j + 2 q + e, j = 0..7, e = 0..1.  The packed weights (and the low-rank factor) are laid out
+// at pack time so that those 16 columns are the 16 consecutive output channels 16 q .. 16 q + 15:
+// column 8 j + 2 q + e holds channel 16 q + 4 ((j / 2) xor (q / 2)) + 2 (j % 2) + e.  Every thread then
+// reads its 16 weight scales with four 128-bit shared loads and stores 32 contiguous bytes per output
+// row; the xor makes the four addresses of each of those loads (q = 0..3, 64 bytes apart) fall into
+// different 16-byte bank groups, which a plain "16 q + 2 j + e" order would not.
 __host__ __device__ constexpr int tile_column_to_channel(int c) {
-  return 16 * ((c >> 1) & 3) + 2 * (c >> 3) + (c & 1);
+  return 16 * ((c >> 1) & 3) + 4 * (((c >> 4) & 3) ^ ((c >> 2) & 1)) + 2 * ((c >> 3) & 1) + (c & 1);
 }
 
 // Rescales one fragment (16 TMEM lanes x 64 columns: two rows x 16 channels per thread) of a group's
@@ -157,9 +159,11 @@ __host__ __device__ constexpr int tile_column_to_channel(int c) {
 //   w     the thread's 16 weight scales, channel order
 //   sa_t  activation scales of the thread's two rows (r and r + 8 of the 16-lane half)
 //   acc   [0..8): first row, [8..16): second row
+//   w[i]  holds the thread's channels 4 (i xor swap) .. + 3 (see tile_column_to_channel), swap = q / 2
 template <bool DEBUG>
 __device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[32], const float4 (&w)[4], float sa_t0,
-                                                 float sa_t1, float2* acc, int32_t* dbg_row0, int32_t* dbg_row1) {
+                                                 float sa_t1, float2* acc, int32_t* dbg_row0, int32_t* dbg_row1,
+                                                 int swap = 0) {
   const float2 s0 = make_float2(sa_t0, sa_t0), s1 = make_float2(sa_t1, sa_t1);
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
@@ -172,10 +176,11 @@ __device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[32], const 
     acc[8 + j] = __ffma2_rn(__fmul2_rn(p1, wj), s1, acc[8 + j]);
     if (DEBUG) {
       if (dbg_row0 != nullptr) {
-        dbg_row0[2 * j] = static_cast<int32_t>(v[4 * j]) >> 8;
-        dbg_row0[2 * j + 1] = static_cast<int32_t>(v[4 * j + 1]) >> 8;
-        dbg_row1[2 * j] = static_cast<int32_t>(v[4 * j + 2]) >> 8;
-        dbg_row1[2 * j + 1] = static_cast<int32_t>(v[4 * j + 3]) >> 8;
+        const int o = 4 * ((j >> 1) ^ swap) + 2 * (j & 1);  // channel offset of columns (j, 0), (j, 1)
+        dbg_row0[o] = static_cast<int32_t>(v[4 * j]) >> 8;
+        dbg_row0[o + 1] = static_cast<int32_t>(v[4 * j + 1]) >> 8;
+        dbg_row1[o] = static_cast<int32_t>(v[4 * j + 2]) >> 8;
+        dbg_row1[o + 1] = static_cast<int32_t>(v[4 * j + 3]) >> 8;
       }
     }
   }
@@ -403,6 +408,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int ew = warp - kEpiWarp0;
       const int quarter = ew & 3, colblk = ew >> 2;
       const int fr = lane >> 2, fq = lane & 3;
+      const int swap = fq >> 1;  // see tile_column_to_channel
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colblk;
       constexpr uint32_t kHalf = 16u << 16;  // second 16-lane half of the quarter
       // Per scale stage: sw[2][kBN] then sa[2][kBM] floats.  The thread's 16 weight scales start at
@@ -471,7 +477,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int t = 0; t < 4; ++t) sa[t] = make_float2(sap[8 * t], sap[kBM + 8 * t]);
           float4 w[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) w[i] = swp[i];
+          for (int i = 0; i < 4; ++i) w[i] = swp[i ^ swap];
           int32_t *d0 = nullptr, *d1 = nullptr, *d2 = nullptr, *d3 = nullptr;
           if (DEBUG) {
             if (dbg_tile) {
@@ -483,7 +489,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           }
           // ---- group g0
-          rescale_fragment<DEBUG>(vA, w, sa[0].x, sa[1].x, acc, d0, d1);
+          rescale_fragment<DEBUG>(vA, w, sa[0].x, sa[1].x, acc, d0, d1, swap);
           tmem_wait_ld_after(acc_lo);
           if (two) {
             tmem_ld_16x256b_x8_before(t_grp + kBN, vA, vB[0]);
@@ -492,13 +498,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
           }
-          rescale_fragment<DEBUG>(vB, w, sa[2].x, sa[3].x, acc + 16, d2, d3);
+          rescale_fragment<DEBUG>(vB, w, sa[2].x, sa[3].x, acc + 16, d2, d3, swap);
           if (two) {
             // ---- group g0 + 1
             tmem_wait_ld_after(acc_hi);
             tmem_ld_16x256b_x8_before(t_grp + kBN + kHalf, vB, vA[0]);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) w[i] = swp[kBN / 4 + i];
+            for (int i = 0; i < 4; ++i) w[i] = swp[kBN / 4 + (i ^ swap)];
             if (DEBUG) {
               if (dbg_tile) {
                 d0 += kBN;
@@ -507,7 +513,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 d3 += kBN;
               }
             }
-            rescale_fragment<DEBUG>(vA, w, sa[0].y, sa[1].y, acc, d0, d1);
+            rescale_fragment<DEBUG>(vA, w, sa[0].y, sa[1].y, acc, d0, d1, swap);
             tmem_wait_ld_after(acc_lo);
             // The whole slot is in registers: hand it back to the MMA warp.
             tc_fence_before_sync();
@@ -521,7 +527,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             tc_fence_after_sync();
             tmem_ld_16x256b_x8_before(t_lane + tm.slot * 2 * kBN, vA, vB[0]);
           }
-          if (two) rescale_fragment<DEBUG>(vB, w, sa[2].y, sa[3].y, acc + 16, d2, d3);
+          if (two) rescale_fragment<DEBUG>(vB, w, sa[2].y, sa[3].y, acc + 16, d2, d3, swap);
           if (!last_stage) tmem_wait_ld_after(acc_hi);
           sc.advance();
         }
@@ -540,8 +546,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               uint4* yrow = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(rw) * p.N + ch0);
 #pragma unroll
               for (int i = 0; i < 2; ++i) {  // 8 channels per 16-byte store
-                const float2 a0 = acc[8 * t + 4 * i], a1 = acc[8 * t + 4 * i + 1], a2 = acc[8 * t + 4 * i + 2],
-                             a3 = acc[8 * t + 4 * i + 3];
+                // acc[8 t + j] holds channels 4 ((j / 2) xor swap) + 2 (j % 2) + {0, 1}: undo the swap here.
+                const float2 x0 = acc[8 * t + 4 * i], x1 = acc[8 * t + 4 * i + 1], x2 = acc[8 * t + 4 * i + 2],
+                             x3 = acc[8 * t + 4 * i + 3];
+                const float2 a0 = swap ? x2 : x0, a1 = swap ? x3 : x1, a2 = swap ? x0 : x2, a3 = swap ? x1 : x3;
                 const float4 b0 = bv[2 * i], b1 = bv[2 * i + 1];
                 __nv_bfloat162 o0 = __floats2bfloat162_rn(fmaf(a0.x, k, b0.x), fmaf(a0.y, k, b0.y));
                 __nv_bfloat162 o1 = __floats2bfloat162_rn(fmaf(a1.x, k, b0.z), fmaf(a1.y, k, b0.w));
