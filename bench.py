@@ -35,7 +35,7 @@ NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_HBM_GBS = 7700.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries (profiles/);
 # None until a capture exists for that kernel and workload.
-NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): None, ("quantize", "attn_proj"): None}
+NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 403.4e6, ("quantize", "attn_proj"): 381.3e6}
 
 
 def load_peaks():
