@@ -38,6 +38,26 @@ NOMINAL_HBM_GBS = 7700.0
 NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 403.4e6, ("quantize", "attn_proj"): 381.3e6}
 
 
+def max_over_ranks(ms: float, dist, device="cpu") -> float:
+    """Device time of the slowest rank (the whole job is as slow as its slowest replica)."""
+    if dist is None:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(ops_per_step_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Aggregate effective TOPS of `world` independent replicas that each do ops_per_step_per_rank per step."""
+    return world * ops_per_step_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
+def dit_step_layers(blocks: int = 40):
+    """(K, N) of the quantized linears of one denoising step: per block q, k, v, o, cross q, cross o, ffn up, ffn down."""
+    per_block = [(5120, 5120)] * 6 + [(5120, 13824), (13824, 5120)]
+    return per_block * blocks
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -178,12 +198,148 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def time_layer(w4, layer, xs, bins, expert, clip, Y, M, iters, warmup, stream):
+    """Mean (quantize ms, gemm ms) of one layer over `iters` forwards, CUDA events on `stream`."""
+    for i in range(warmup):
+        w4.w4a4_linear_forward(layer.ptr, xs[i % len(xs)], M, expert, bins[i % len(xs)], clip, Y, stream)
+    torch.cuda.synchronize()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(iters)]
+    for i in range(iters):
+        b = i % len(xs)
+        ev[i][0].record(stream)
+        w4.w4a4_quantize_activations(layer.ptr, xs[b], M, expert, bins[b], clip, stream)
+        ev[i][1].record(stream)
+        w4.w4a4_gemm_from_workspace(layer.ptr, M, expert, Y, stream)
+        ev[i][2].record(stream)
+    torch.cuda.synchronize()
+    return (statistics.mean(e[0].elapsed_time(e[1]) for e in ev), statistics.mean(e[1].elapsed_time(e[2]) for e in ev))
+
+
+def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks):
+    """One denoising step's quantized linears of a 40-block, 5120-hidden DiT at M = 32760, r = 32, with both
+    experts' weight sets resident; step s uses expert (s >= 20) and timestep bin s // 5 (40-step schedule)."""
+    M, r, bins, experts = 32760, 32, 8, 2
+    shapes = dit_step_layers(args.blocks)
+    L = len(shapes)
+    ctx = w4.Context(local_rank, M, 13824, r)
+    layers = []
+    for li, (K, N) in enumerate(shapes):
+        ex = [gen.make_layer_direct(K, N, r, seed=4000 + 2 * li + e, device=dev) for e in range(experts)]
+        layers.append(w4.Layer(ctx, ex, num_bins=bins, num_layers=L, layer_id=li))
+        del ex
+    weight_bytes = sum(w4.w4a4_handle_bytes(l.ptr) for l in layers)
+    clip = gen.make_clip_table(experts, L, bins, [(0.6, 1.0), (0.8, 1.0)], seed=4).to(dev)
+    idx = {K: gen.outlier_channels(K, 0.01, 40 + K) for K in (5120, 13824)}
+    xs = {5120: [gen.make_activations(M, 5120, sigma=1.0, outlier_idx=idx[5120], outlier_gain=50.0, seed=4100 + i,
+                                      device=dev) for i in range(3)],
+          13824: [gen.make_activations(M, 13824, dist="gelu", outlier_idx=idx[13824], outlier_gain=80.0, seed=4200 + i,
+                                       device=dev) for i in range(3)]}
+    Y = {n: torch.empty(M, n, dtype=torch.bfloat16, device=dev) for n in (5120, 13824)}
+    stream = torch.cuda.current_stream()
+
+    def step(s):
+        expert, b = (1 if (s % 40) >= 20 else 0), (s % 40) // 5
+        for li, (K, N) in enumerate(shapes):
+            w4.w4a4_linear_forward(layers[li].ptr, xs[K][(s + li) % 3], M, expert, b, clip, Y[N], stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for s in range(args.warmup):
+        step(s)
+    barrier()
+    ctx.check()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for s in range(args.steps):
+        step(18 + s)  # straddles the expert switch at step 20
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ctx.check()
+    total_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    ms_per_step = total_ms / args.steps
+    ops = sum(2.0 * M * K * N for (K, N) in shapes)
+    if rank == 0:
+        int8_peak = 2.0 * peaks["bf16_sustained"]
+        tops = whole_job_tops(ops, world, ms_per_step)
+        line = dict(metric=METRIC, value=tops, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="s8",
+                    data="synthetic",
+                    config=dict(workload="dit_step", M=M, r=r, group=64, blocks=args.blocks, linears=L, experts=experts,
+                                bins=bins, resident_weight_gb=weight_bytes / 1e9, tera_ops_per_step=ops / 1e12,
+                                l2="inputs larger than L2: 3 rotating activation buffers per shape (335 / 906 MB)",
+                                parallelism="replicas" if world > 1 else "single"),
+                    ms_per_dit_step=ms_per_step,
+                    roofline=dict(bound="tensor", achieved=tops / world, peak=int8_peak, unit="TOP/s",
+                                  frac=tops / world / int8_peak, traffic=None, kernel="quantize + gemm, whole step",
+                                  peak_source=f"{peaks['source']} sustained BF16 x 2"),
+                    gpu_launches=2 * L * args.steps, clocks=clocks)
+        print(json.dumps(line), flush=True)
+    for l in layers:
+        l.close()
+    ctx.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_sweep(args, w4, dev, local_rank, rank, peaks):
+    """Shape sweep: M x (K, N) x r x outlier fraction x clip ratio, TOPS and roofline fractions per point."""
+    if rank != 0:
+        return
+    int8_peak = 2.0 * peaks["bf16_sustained"]
+    rows = []
+    stream = torch.cuda.current_stream()
+    for (K, N) in ((5120, 5120), (5120, 13824), (13824, 5120)):
+        for r in (0, 16, 32, 64):
+            for M in (1560, 32760, 75600):
+                ctx = w4.Context(local_rank, M, K, r)
+                layer = w4.Layer(ctx, [gen.make_layer_direct(K, N, r, seed=5000 + r + K // 64, device=dev)], num_bins=2)
+                clip = torch.tensor([[[0.7, 1.0]]], dtype=torch.float32, device=dev)
+                Y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+                for frac in (0.0, 0.01, 0.05):
+                    n_x = 2 if M * K * 2 > 64e6 else 4
+                    xs = [gen.make_activations(M, K, outlier_idx=gen.outlier_channels(K, frac, 50 + i), outlier_gain=50.0,
+                                               seed=5100 + i, device=dev) for i in range(n_x)]
+                    for b, alpha in ((0, 0.7), (1, 1.0)):
+                        tq, tg = time_layer(w4, layer, xs, [b] * n_x, 0, clip, Y, M, args.steps, max(3, args.warmup), stream)
+                        ops = 2.0 * M * K * N
+                        qb = M * (2.5625 * K + 2.0 * r)
+                        rows.append(dict(M=M, K=K, N=N, r=r, outlier_fraction=frac, alpha=alpha, quantize_ms=tq, gemm_ms=tg,
+                                         layer_tops=ops / ((tq + tg) * 1e-3) / 1e12, gemm_tops=ops / (tg * 1e-3) / 1e12,
+                                         gemm_frac=ops / (tg * 1e-3) / 1e12 / int8_peak,
+                                         quantize_gbs=qb / (tq * 1e-3) / 1e9, quantize_frac=qb / (tq * 1e-3) / 1e9 / peaks["hbm_gbs"]))
+                    del xs
+                ctx.check()
+                layer.close()
+                ctx.close()
+                del Y
+                torch.cuda.empty_cache()
+    out = args.out or os.path.join(ROOT, "gpurun_out", "sweep.json")
+    os.makedirs(os.path.dirname(out), exist_ok=True)
+    with open(out, "w") as f:
+        json.dump(rows, f)
+    best = max(rows, key=lambda x: x["gemm_tops"])
+    print(json.dumps(dict(metric=METRIC, unit=UNIT, value=statistics.mean(x["layer_tops"] for x in rows), n_gpus=1,
+                          steps=args.steps, warmup=args.warmup, higher_is_better=True, scaling="weak", vs_baseline=None,
+                          dtype="s8", data="synthetic", config=dict(workload="sweep", points=len(rows), table=out),
+                          best_point=best, gpu_launches=2 * args.steps * len(rows))), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES))
+    ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep"])
+    ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
+    ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -215,6 +371,12 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     peaks = load_peaks()
+    if args.workload == "dit_step":
+        run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks)
+        return
+    if args.workload == "sweep":
+        run_sweep(args, w4, dev, local_rank, rank, peaks)
+        return
     n_buf = 4
     w = workload_inputs(args.workload, dev, n_buf)
     M, K, N, r = w["M"], w["K"], w["N"], w["r"]
@@ -248,16 +410,12 @@ def main():
     barrier()
     clocks = sampler.stop()
     ctx.check()
-    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    total_ms = max_over_ranks(ev[0][0].elapsed_time(ev[-1][2]), dist, dev)
     t_q = [e[0].elapsed_time(e[1]) for e in ev]
     t_g = [e[1].elapsed_time(e[2]) for e in ev]
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
     ops = 2.0 * M * K * N
-    value = world * ops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(ops, world, ms_per_step)
 
     # -------------------------------------------------------------- end to end from pinned host memory
     e2e_steps = max(1, min(args.e2e_steps, args.steps))
@@ -279,12 +437,8 @@ def main():
         e2e_step(i)
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * ops / (e2e_ms / e2e_steps * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    e2e_value = whole_job_tops(ops, world, e2e_ms / e2e_steps)
     ctx.check()
 
     if rank == 0:

@@ -226,3 +226,33 @@ def test_ffn_pair_full_size_sampled_rows():
     down = big_layer(K, N, r, calib, 3004)
     x = gen.make_activations(M, K, dist="gelu", outlier_idx=idx, outlier_gain=80.0, seed=3005, device=DEV).cpu()
     run_case(x, [down, down], clip, 0, 1, rows=rows, check_partials_tiles=[(0, N - 128)])
+
+
+def test_dit_step_layers_both_experts_sampled_rows():
+    # Layers of one denoising step (direct-recipe constants, two resident experts, 8 bins, several layers in
+    # the clip table): the step index picks expert (s >= 20) and bin s // 5; parity per distinct shape.
+    M, r = 32760, 32
+    clip = gen.make_clip_table(2, 4, 8, [(0.6, 1.0), (0.8, 1.0)], seed=4)
+    rows = sampled_rows(M, 6, 41)
+    for layer_id, (K, N, step) in enumerate(((5120, 5120, 3), (5120, 13824, 22), (13824, 5120, 39))):
+        expert, b = (1 if step >= 20 else 0), step // 5
+        experts = [gen.make_layer_direct(K, N, r, seed=4000 + 2 * layer_id + e, device=DEV).to("cpu") for e in range(2)]
+        dist = "gelu" if K == 13824 else "normal"
+        x = gen.make_activations(M, K, dist=dist, outlier_idx=gen.outlier_channels(K, 0.01, 40 + K), outlier_gain=50.0,
+                                 seed=4100 + layer_id, device=DEV).cpu()
+        run_case(x, experts, clip, expert, b, rows=rows, layer_id=layer_id, num_layers=4,
+                 check_partials_tiles=[((M - 1) // 128 * 128, N - 128)])
+        del x, experts
+
+
+@pytest.mark.parametrize("M,K,N,r,frac,alpha", [
+    (1560, 5120, 5120, 0, 0.0, 0.7),      # one latent frame, no low-rank branch, no outliers
+    (1560, 13824, 5120, 64, 0.05, 1.0),   # widest K, widest rank, 5% outlier channels
+    (75600, 5120, 13824, 16, 0.01, 0.7),  # the largest token count (21 x 45 x 80 grid)
+])
+def test_sweep_points_sampled_rows(M, K, N, r, frac, alpha):
+    layer = gen.make_layer_direct(K, N, r, seed=5000 + r + K // 64, device=DEV).to("cpu")
+    x = gen.make_activations(M, K, outlier_idx=gen.outlier_channels(K, frac, 50), outlier_gain=50.0, seed=5100,
+                             device=DEV).cpu()
+    clip = torch.tensor([[[alpha]]], dtype=torch.float32)
+    run_case(x, [layer], clip, 0, 0, rows=sampled_rows(M, 6, 51), check_partials_tiles=[(0, 0)])
