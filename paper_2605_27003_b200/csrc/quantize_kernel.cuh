@@ -7,8 +7,8 @@
 //   Eq. 3      q  = clip(rint(xh * is), -8, 7)               rounding by the 1.5*2^23 magic add (ties to even)
 //   Eq. 7      T  = bf16(xh) L1                              mma.sync m16n8k16 BF16, FP32 accumulate
 //
-// Work split: a CTA of 4 warps owns 16 consecutive token rows; warp w owns the groups g = w, w+4, ...
-// so the four warps together stream 512 contiguous bytes of every row per step.  Inside a warp,
+// Work split: a CTA of kQuantWarps warps owns 16 consecutive token rows per warp; all warps walk the K groups
+// together, so the group's L1 fragments and smoothing factors are staged once per CTA.  Inside a warp,
 // lane = 4*i + j owns rows i and i+8 and, within the group, channels
 //      32*(j/2) + 8*(j%2) + [0,8)     and the same + 16,
 // which is exactly the pair of 8-channel runs that fill two whole 32-bit words of the packed layout
@@ -30,8 +30,16 @@
 namespace w4a4 {
 
 constexpr int kQuantRows = 16;      // token rows per CTA
-constexpr int kQuantWarps = 4;      // warps per CTA, each owning every 4th group
-constexpr int kQuantThreads = 32 * kQuantWarps;
+// Warps per CTA (16 rows each).  Small CTAs spread evenly over the 148 SMs; the widest rank shares its
+// larger L1 fragments among more warps.
+constexpr int quantize_warps(int R) { return R >= 64 ? 4 : 2; }
+constexpr int kStages = 3;          // depth of the cp.async rings (groups in flight = kStages - 1)
+
+// Dynamic shared memory of quantize_kernel<R>: activation rings, smoothing-factor ring, L1 fragment ring.
+constexpr size_t quantize_smem_bytes(int R) {
+  return static_cast<size_t>(quantize_warps(R)) * kStages * 4 * 32 * 16 + kStages * 64 * 4 +
+         static_cast<size_t>(kStages) * (4 * (R / 8) * 32 * 8);
+}
 
 // Channel (within its 64-group) that lane-in-quad j holds as its e-th element, e in [0,16).
 __host__ __device__ constexpr int l1_fragment_channel(int j, int e) {
@@ -117,17 +125,19 @@ __device__ __forceinline__ uint2 quantize16(const float* xh, float is) {
   return make_uint2(w0 ^ 0x88888888u, w1 ^ 0x88888888u);  // offset-binary -> two's complement nibbles
 }
 
-template <int R>
-__global__ void __launch_bounds__(kQuantThreads)
+template <int R, int WARPS>
+__global__ void __launch_bounds__(32 * WARPS)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
                 uint8_t* __restrict__ codes, float* __restrict__ scales, int scales_ld,
                 uint16_t* __restrict__ t_hilo) {
-  constexpr int NT = R / 8;  // n-tiles of the m16n8k16 MMA
+  constexpr int NT = R / 8;                          // n-tiles of the m16n8k16 MMA
+  constexpr int kFragBytes = 4 * NT * 32 * 8;        // L1 fragments of one group (4 KiB at r = 32)
+  constexpr int kFragChunks = kFragBytes / 16;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qi = lane >> 2, qj = lane & 3;
   const int G = K >> 6;
-  const int row0 = blockIdx.x * kQuantRows;
+  const int row0 = (blockIdx.x * WARPS + warp) * kQuantRows;
   const int rowA = row0 + qi, rowB = rowA + 8;
   const bool okA = rowA < M, okB = rowB < M;
   const float rho = __ldg(clip_table + clip_index);
@@ -140,37 +150,61 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
 #pragma unroll
   for (int nt = 0; nt < (NT > 0 ? NT : 1); ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
 
-  const uint4 zero4 = make_uint4(0, 0, 0, 0);
-  uint4 ra0 = zero4, ra1 = zero4, rb0 = zero4, rb1 = zero4;
-  int g = warp;
-  if (g < G) {
-    if (okA) { ra0 = ldg_stream_v4(xa + 64 * g); ra1 = ldg_stream_v4(xa + 64 * g + 16); }
-    if (okB) { rb0 = ldg_stream_v4(xb + 64 * g); rb1 = ldg_stream_v4(xb + 64 * g + 16); }
-  }
-  for (; g < G; g += kQuantWarps) {
-    const uint4 ca0 = ra0, ca1 = ra1, cb0 = rb0, cb1 = rb1;
-    const int gn = g + kQuantWarps;
-    if (gn < G) {  // prefetch the next group's activations before touching this one
-      if (okA) { ra0 = ldg_stream_v4(xa + 64 * gn); ra1 = ldg_stream_v4(xa + 64 * gn + 16); }
-      if (okB) { rb0 = ldg_stream_v4(xb + 64 * gn); rb1 = ldg_stream_v4(xb + 64 * gn + 16); }
-    }
+  // Everything a group needs is streamed through shared-memory rings with cp.async, kStages - 1 groups
+  // ahead of the one being processed:
+  //   xring   per warp: the 16 rows x 64 channels of activations (2 KiB); every lane reads back only the
+  //           4 x 16 bytes it requested itself ([piece][lane] layout, conflict free, no barrier needed);
+  //   fring   per CTA: the group's L1 fragments, shared by the CTA's warps (they all walk the same groups,
+  //           each on its own 16 rows), so L1 crosses L2 once per 64 rows instead of once per 16;
+  //   lring   per CTA: the group's 64 reciprocal smoothing factors.
+  extern __shared__ __align__(16) uint8_t quant_smem[];
+  typedef uint4 (*XRing)[kStages][4][32];
+  typedef uint4 (*FRing)[kFragChunks > 0 ? kFragChunks : 1];
+  typedef float (*LRing)[64];
+  XRing xring = reinterpret_cast<XRing>(quant_smem);
+  LRing lring = reinterpret_cast<LRing>(quant_smem + WARPS * kStages * 4 * 32 * 16);
+  FRing fring = reinterpret_cast<FRing>(quant_smem + WARPS * kStages * 4 * 32 * 16 + kStages * 64 * 4);
+  const uint32_t xring0 = static_cast<uint32_t>(__cvta_generic_to_shared(&xring[warp][0][0][lane]));
+  auto issue = [&](int gg, int stage) {
+    const uint32_t dst = xring0 + stage * (4 * 32 * 16);
+    const uint32_t szA = okA ? 16u : 0u, szB = okB ? 16u : 0u;  // rows past M are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(xa + 64 * gg), "r"(szA) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 512), "l"(xa + 64 * gg + 16), "r"(szA) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 1024), "l"(xb + 64 * gg), "r"(szB) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + 1536), "l"(xb + 64 * gg + 16), "r"(szB) : "memory");
     if constexpr (NT > 0) {
-      // Pull the next group's L1 fragments (NT * 128 bytes per lane-line) into L1 while this group computes:
-      // every warp needs all of L1 once per 16 rows, far more bytes than it reads from X, and an L2 hit
-      // in front of every MMA would stall the warp.
-      if (gn < G) {
-        const char* nf = reinterpret_cast<const char*>(l1frag) + static_cast<size_t>(gn) * (4 * NT * 32 * 8);
-#pragma unroll
-        for (int c = 0; c < (4 * NT * 32 * 8) / 4096; ++c) {
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(nf + c * 4096 + lane * 128));
-        }
-        if ((4 * NT * 32 * 8) % 4096 != 0 && lane < ((4 * NT * 32 * 8) % 4096) / 128) {
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(nf + ((4 * NT * 32 * 8) / 4096) * 4096 + lane * 128));
-        }
+      const uint4* src = reinterpret_cast<const uint4*>(l1frag) + static_cast<size_t>(gg) * kFragChunks;
+      for (int c = threadIdx.x; c < kFragChunks; c += (32 * WARPS)) {
+        const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(&fring[stage][c]));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + c) : "memory");
       }
     }
-    const float4* rl = reinterpret_cast<const float4*>(rlam + 64 * g + coff);
-    const float4 l0 = __ldg(rl), l1 = __ldg(rl + 1), l4 = __ldg(rl + 4), l5 = __ldg(rl + 5);
+    if (threadIdx.x < 16) {
+      const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(&lring[stage][4 * threadIdx.x]));
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(rlam + 64 * gg + 4 * threadIdx.x) : "memory");
+    }
+  };
+#pragma unroll
+  for (int d = 0; d < kStages - 1; ++d) {
+    if (d < G) issue(d, d);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  int stage = 0;
+  for (int g = 0; g < G; ++g) {
+    // This thread's copies for group g have landed; after the barrier so have everyone's, and every warp
+    // has finished group g - 1, whose ring slot the prefetch below overwrites.
+    asm volatile("cp.async.wait_group %0;" ::"n"(kStages - 2) : "memory");
+    __syncthreads();
+    {
+      int pstage = stage + kStages - 1;
+      if (pstage >= kStages) pstage -= kStages;
+      if (g + kStages - 1 < G) issue(g + kStages - 1, pstage);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    const uint4* slot = &xring[warp][stage][0][lane];
+    const uint4 ca0 = slot[0], ca1 = slot[32], cb0 = slot[64], cb1 = slot[96];
+    const float4* rl = reinterpret_cast<const float4*>(&lring[stage][coff]);
+    const float4 l0 = rl[0], l1 = rl[1], l4 = rl[4], l5 = rl[5];
     float xhA[16], xhB[16];
     smooth8(ca0, l0, l1, xhA);
     smooth8(ca1, l4, l5, xhA + 8);
@@ -193,8 +227,8 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = s_mine;
 
     if constexpr (NT > 0) {
-      // Fragment storage: [group][i][n-tile pair][lane] as uint4 = (b0, b1) of n-tile 2p, (b0, b1) of n-tile 2p + 1.
-      const uint4* lf = reinterpret_cast<const uint4*>(l1frag) + (static_cast<size_t>(g) * 4 * (NT / 2)) * 32 + lane;
+      // Fragment storage: [i][n-tile pair][lane] as uint4 = (b0, b1) of n-tile 2p, (b0, b1) of n-tile 2p + 1.
+      const uint4* lf = &fring[stage][lane];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         uint32_t a[4];
@@ -204,35 +238,33 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
         a[3] = pack_bf16x2(xhB[4 * i + 2], xhB[4 * i + 3]);
 #pragma unroll
         for (int np = 0; np < NT / 2; ++np) {
-          const uint4 b = __ldg(lf + (i * (NT / 2) + np) * 32);
+          const uint4 b = lf[(i * (NT / 2) + np) * 32];
           mma_bf16_16816(acc[2 * np], a, b.x, b.y);
           mma_bf16_16816(acc[2 * np + 1], a, b.z, b.w);
         }
       }
     }
+    if (++stage == kStages) stage = 0;
   }
 
   if constexpr (NT > 0) {
-    __shared__ float tred[kQuantWarps][kQuantRows][R];
+    // Each warp owns its 16 rows over all of K: T is complete in its accumulators.  Store it as a BF16
+    // high part and the BF16 rounding of the remainder ([T_hi | T_lo], two values per 32-bit store).
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int c = 8 * nt + 2 * qj;
-      tred[warp][qi][c] = acc[nt][0];
-      tred[warp][qi][c + 1] = acc[nt][1];
-      tred[warp][qi + 8][c] = acc[nt][2];
-      tred[warp][qi + 8][c + 1] = acc[nt][3];
-    }
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < kQuantRows * R; idx += kQuantThreads) {
-      const int rr = idx / R, c = idx % R;
-      const int row = row0 + rr;
-      if (row < M) {
-        const float t = (tred[0][rr][c] + tred[1][rr][c]) + (tred[2][rr][c] + tred[3][rr][c]);
-        const __nv_bfloat16 hi = __float2bfloat16_rn(t);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(t - __bfloat162float(hi));
-        uint16_t* dst = t_hilo + static_cast<size_t>(row) * (2 * R);
-        dst[c] = *reinterpret_cast<const uint16_t*>(&hi);
-        dst[R + c] = *reinterpret_cast<const uint16_t*>(&lo);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int row = h ? rowB : rowA;
+        if (row < M) {
+          const float t0 = acc[nt][2 * h], t1 = acc[nt][2 * h + 1];
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(t0), h1 = __float2bfloat16_rn(t1);
+          const uint32_t hi = pack_bf16x2(__bfloat162float(h0), __bfloat162float(h1));
+          const uint32_t lo = pack_bf16x2(t0 - __bfloat162float(h0), t1 - __bfloat162float(h1));
+          uint16_t* dst = t_hilo + static_cast<size_t>(row) * (2 * R);
+          *reinterpret_cast<uint32_t*>(dst + c) = hi;
+          *reinterpret_cast<uint32_t*>(dst + R + c) = lo;
+        }
       }
     }
   }

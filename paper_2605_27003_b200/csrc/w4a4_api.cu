@@ -234,10 +234,11 @@ w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_
   w4a4_ctx* ctx = h->ctx;
   const ExpertData& e = h->experts[expert_id];
   const int clip_index = (expert_id * h->L + h->layer_id) * h->B + bin;
-  const dim3 grid((M + kQuantRows - 1) / kQuantRows), block(kQuantThreads);
+  const int rows_per_cta = kQuantRows * quantize_warps(h->r);
+  const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define W4A4_LAUNCH_Q(R)                                                                                         \
-  quantize_kernel<R><<<grid, block, 0, stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
+  quantize_kernel<R, quantize_warps(R)><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
                                                  ctx->scales, ctx->scales_ld, ctx->t_hilo)
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
@@ -347,6 +348,8 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
       cudaMemset(ctx->t_hilo, 0, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8) * sizeof(uint16_t)) != cudaSuccess)
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) {
+    cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64)>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         static_cast<int>(quantize_smem_bytes(64)));
     cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
