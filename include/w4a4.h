@@ -87,6 +87,19 @@ void w4a4_destroy(w4a4_handle_t h);
 w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
                                   const float* clip_table, void* Y, void* stream);
 
+/* The same layer (Eq. 11) with X and Y in HOST memory (pinned memory recommended; pageable works but the
+ * copies then serialise).  M is split into chunks of `chunk_rows` tokens that flow through three internal
+ * streams -- host-to-device copy, the two kernels, device-to-host copy -- so that the copies of neighbouring
+ * chunks overlap the kernels (rows are independent, so chunking does not change any result).  The whole
+ * operation is ordered after the work already enqueued on `stream`, and `stream` waits for its completion;
+ * the call itself does not synchronise the host.  w4a4_ctx_enable_host_io must have been called once on the
+ * context (it allocates the staging buffers: 2 x chunk_rows x (max_K + max_N) BF16 values, plus streams and
+ * events); the forward itself allocates nothing.  clip_table stays a DEVICE pointer.
+ * Errors: INVALID_ARG (host I/O not enabled, NULL pointers), SHAPE (M > max_M, N > max_N), CUDA. */
+w4a4_status_t w4a4_ctx_enable_host_io(w4a4_ctx_t ctx, int chunk_rows, int max_N);
+w4a4_status_t w4a4_linear_forward_host(w4a4_handle_t h, const void* X_host, int M, int expert_id, int timestep_bin,
+                                       const float* clip_table, void* Y_host, void* stream);
+
 /* The two halves of w4a4_linear_forward, exposed so that each kernel can be timed on its own.
  * w4a4_quantize_activations: Eq. 3-5, 8-9 and the first factor of Eq. 7's low-rank term, into the
  * context workspace.  w4a4_gemm_from_workspace: the rest of Eq. 7/11 from that workspace into Y. */

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_ALLOC", 4
 # Every symbol include/w4a4.h declares.
 EXPORTED_SYMBOLS = (
     "w4a4_ctx_create", "w4a4_ctx_destroy", "w4a4_pack_weights", "w4a4_destroy", "w4a4_linear_forward",
-    "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
+    "w4a4_ctx_enable_host_io", "w4a4_linear_forward_host", "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
     "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
@@ -64,6 +64,8 @@ def _lib():
         lib.w4a4_destroy.argtypes = [vp]
         lib.w4a4_destroy.restype = None
         lib.w4a4_linear_forward.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
+        lib.w4a4_ctx_enable_host_io.argtypes = [vp, ci, ci]
+        lib.w4a4_linear_forward_host.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
         lib.w4a4_quantize_activations.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         lib.w4a4_gemm_from_workspace.argtypes = [vp, ci, ci, vp, vp]
         lib.w4a4_debug_quantize.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
@@ -167,6 +169,18 @@ def w4a4_linear_forward(handle, X: torch.Tensor, M: int, expert_id: int, timeste
                         clip_table: torch.Tensor, Y: torch.Tensor, stream=None):
     _check(_lib().w4a4_linear_forward(handle, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table), _ptr(Y),
                                       _stream(stream)), "w4a4_linear_forward")
+
+
+def w4a4_ctx_enable_host_io(ctx, chunk_rows: int, max_N: int):
+    _check(_lib().w4a4_ctx_enable_host_io(ctx, chunk_rows, max_N), "w4a4_ctx_enable_host_io")
+
+
+def w4a4_linear_forward_host(handle, X_host: torch.Tensor, M: int, expert_id: int, timestep_bin: int,
+                             clip_table: torch.Tensor, Y_host: torch.Tensor, stream=None):
+    """X_host / Y_host are CPU tensors (pinned for overlap); clip_table is a CUDA tensor."""
+    assert not X_host.is_cuda and not Y_host.is_cuda and clip_table.is_cuda
+    _check(_lib().w4a4_linear_forward_host(handle, _ptr(X_host), M, expert_id, timestep_bin, _ptr(clip_table),
+                                           _ptr(Y_host), _stream(stream)), "w4a4_linear_forward_host")
 
 
 def w4a4_quantize_activations(handle, X, M, expert_id, timestep_bin, clip_table, stream=None):

@@ -127,6 +127,13 @@ struct w4a4_ctx {
   size_t bytes = 0;
   int num_sms = 0;
   EncodeTiledFn encode = nullptr;
+  // Host-buffer forward (w4a4_linear_forward_host): staging buffers, copy streams and events.
+  int host_chunk_rows = 0, host_max_N = 0;
+  uint16_t* hx[2] = {nullptr, nullptr};  // device staging of an activation chunk (double buffered)
+  uint16_t* hy[2] = {nullptr, nullptr};  // device staging of an output chunk
+  cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
 };
 
 struct ExpertData {
@@ -372,6 +379,18 @@ void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
   cudaFree(ctx->scales);
   cudaFree(ctx->t_hilo);
   cudaFree(ctx->d_err);
+  for (int i = 0; i < 2; ++i) {
+    cudaFree(ctx->hx[i]);
+    cudaFree(ctx->hy[i]);
+    if (ctx->ev_in[i]) cudaEventDestroy(ctx->ev_in[i]);
+    if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+    if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
+  }
+  if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
+  if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
+  if (ctx->s_h2d) cudaStreamDestroy(ctx->s_h2d);
+  if (ctx->s_compute) cudaStreamDestroy(ctx->s_compute);
+  if (ctx->s_d2h) cudaStreamDestroy(ctx->s_d2h);
   delete ctx;
 }
 
@@ -531,6 +550,83 @@ w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int exp
   st = launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
   if (st != W4A4_OK) return st;
   return launch_gemm(h, M, expert_id, Y, s, nullptr, 0, 0);
+}
+
+w4a4_status_t w4a4_ctx_enable_host_io(w4a4_ctx_t ctx, int chunk_rows, int max_N) {
+  if (!ctx) return W4A4_ERR_INVALID_ARG;
+  if (chunk_rows <= 0 || chunk_rows > ctx->max_M || max_N <= 0) return W4A4_ERR_SHAPE;
+  if (ctx->host_chunk_rows != 0) return W4A4_ERR_INVALID_ARG;  // already enabled
+  DeviceGuard guard(ctx->device);
+  w4a4_status_t st = W4A4_OK;
+  for (int i = 0; st == W4A4_OK && i < 2; ++i) {
+    st = dev_alloc(&ctx->hx[i], static_cast<size_t>(chunk_rows) * ctx->max_K, &ctx->bytes);
+    if (st == W4A4_OK) st = dev_alloc(&ctx->hy[i], static_cast<size_t>(chunk_rows) * max_N, &ctx->bytes);
+    if (st == W4A4_OK && (cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) != cudaSuccess ||
+                          cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming) != cudaSuccess ||
+                          cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming) != cudaSuccess))
+      st = W4A4_ERR_CUDA;
+  }
+  if (st == W4A4_OK && (cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaStreamCreateWithFlags(&ctx->s_compute, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&ctx->ev_begin, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&ctx->ev_end, cudaEventDisableTiming) != cudaSuccess))
+    st = W4A4_ERR_CUDA;
+  if (st != W4A4_OK) {
+    cudaGetLastError();
+    return st;
+  }
+  ctx->host_chunk_rows = chunk_rows;
+  ctx->host_max_N = max_N;
+  return W4A4_OK;
+}
+
+w4a4_status_t w4a4_linear_forward_host(w4a4_handle_t h, const void* X_host, int M, int expert_id, int timestep_bin,
+                                       const float* clip_table, void* Y_host, void* stream) {
+  w4a4_status_t st = check_forward_args(h, X_host, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  w4a4_ctx* ctx = h->ctx;
+  if (ctx->host_chunk_rows == 0) return W4A4_ERR_INVALID_ARG;  // w4a4_ctx_enable_host_io was not called
+  if (h->N > ctx->host_max_N) return W4A4_ERR_SHAPE;
+  if (M > 0 && !Y_host) return W4A4_ERR_INVALID_ARG;
+  if (M == 0) return W4A4_OK;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t user = static_cast<cudaStream_t>(stream);
+  const int C = ctx->host_chunk_rows;
+  const int chunks = (M + C - 1) / C;
+  const uint16_t* xh = static_cast<const uint16_t*>(X_host);
+  uint16_t* yh = static_cast<uint16_t*>(Y_host);
+  bool ok = cudaEventRecord(ctx->ev_begin, user) == cudaSuccess &&
+            cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_begin, 0) == cudaSuccess &&
+            cudaStreamWaitEvent(ctx->s_compute, ctx->ev_begin, 0) == cudaSuccess &&
+            cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_begin, 0) == cudaSuccess;
+  // Three streams: chunk i is copied in while chunk i-1 is computed and chunk i-2 is copied out.
+  for (int i = 0; ok && i < chunks; ++i) {
+    const int b = i & 1;
+    const int rows = (i + 1 < chunks) ? C : M - i * C;
+    if (i >= 2) ok = cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_done[b], 0) == cudaSuccess;  // staging X[b] consumed
+    ok = ok && cudaMemcpyAsync(ctx->hx[b], xh + static_cast<size_t>(i) * C * h->K, sizeof(uint16_t) * rows * h->K,
+                               cudaMemcpyHostToDevice, ctx->s_h2d) == cudaSuccess &&
+         cudaEventRecord(ctx->ev_in[b], ctx->s_h2d) == cudaSuccess &&
+         cudaStreamWaitEvent(ctx->s_compute, ctx->ev_in[b], 0) == cudaSuccess;
+    if (ok && i >= 2) ok = cudaStreamWaitEvent(ctx->s_compute, ctx->ev_out[b], 0) == cudaSuccess;  // staging Y[b] drained
+    if (!ok) break;
+    st = launch_quantize(h, ctx->hx[b], rows, expert_id, timestep_bin, clip_table, ctx->s_compute);
+    if (st == W4A4_OK) st = launch_gemm(h, rows, expert_id, ctx->hy[b], ctx->s_compute, nullptr, 0, 0);
+    if (st != W4A4_OK) return st;
+    ok = cudaEventRecord(ctx->ev_done[b], ctx->s_compute) == cudaSuccess &&
+         cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_done[b], 0) == cudaSuccess &&
+         cudaMemcpyAsync(yh + static_cast<size_t>(i) * C * h->N, ctx->hy[b], sizeof(uint16_t) * rows * h->N,
+                         cudaMemcpyDeviceToHost, ctx->s_d2h) == cudaSuccess &&
+         cudaEventRecord(ctx->ev_out[b], ctx->s_d2h) == cudaSuccess;
+  }
+  ok = ok && cudaEventRecord(ctx->ev_end, ctx->s_d2h) == cudaSuccess &&
+       cudaStreamWaitEvent(user, ctx->ev_end, 0) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return W4A4_ERR_CUDA;
+  }
+  return W4A4_OK;
 }
 
 w4a4_status_t w4a4_debug_quantize(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,

@@ -256,3 +256,26 @@ def test_sweep_points_sampled_rows(M, K, N, r, frac, alpha):
                              device=DEV).cpu()
     clip = torch.tensor([[[alpha]]], dtype=torch.float32)
     run_case(x, [layer], clip, 0, 0, rows=sampled_rows(M, 6, 51), check_partials_tiles=[(0, 0)])
+
+
+def test_host_buffer_forward_equals_device_forward():
+    # X and Y in pinned host memory, M split into chunks with a ragged last chunk: rows are independent, so
+    # the chunked three-stream pipeline must reproduce the device-resident forward bit for bit.
+    M, K, N, r = 1000, 512, 256, 16
+    x, layer = tiny_inputs(M, K, N, r, seed=12, bias=True)
+    ctx = w4.Context(0, M, K, r)
+    L = w4.Layer(ctx, [layer.to(DEV)], num_bins=2)
+    clip = torch.tensor([[[0.9, 0.7]]], dtype=torch.float32, device=DEV)
+    y_dev = L.forward(x.to(DEV), 0, 1, clip)
+    with pytest.raises(w4.W4A4Error):  # host I/O has to be enabled first
+        w4.w4a4_linear_forward_host(L.ptr, x.pin_memory(), M, 0, 1, clip, torch.empty(M, N, dtype=torch.bfloat16).pin_memory())
+    w4.w4a4_ctx_enable_host_io(ctx.ptr, 384, N)
+    xh = x.pin_memory()
+    for _ in range(2):
+        yh = torch.zeros(M, N, dtype=torch.bfloat16).pin_memory()
+        w4.w4a4_linear_forward_host(L.ptr, xh, M, 0, 1, clip, yh)
+        torch.cuda.synchronize()
+        assert torch.equal(yh, y_dev.cpu())
+    ctx.check()
+    L.close()
+    ctx.close()
