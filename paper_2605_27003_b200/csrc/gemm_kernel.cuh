@@ -1,30 +1,36 @@
 // Kernel 2: fused W4A4 GEMM + per-group rescale + low-rank up-projection + bias + BF16 store.
 //
 //   Eq. 7 / 11    Y[m,n] = sum_g  P[m,g,n] * s[m,g] * sw[g,n]  +  sum_j T[m,j] L2[j,n]  +  b[n]
-//                 P[m,g,n] = sum_{k in group g} q[m,k] qw[k,n]            (exact int32)
+//                 P[m,g,n] = sum_{k in group g} q[m,k] qw[k,n]            (exact: integers in FP32)
+//
+// The 4-bit codes go through the tensor core as E4M3 bytes (fp8_codes.cuh): tcgen05.mma kind::f8f6f4 runs
+// at the 8-bit rate and leaves every group's partial sums in TMEM as exact integers already in FP32, so
+// the epilogue needs no int -> float conversion.
 //
 // Persistent kernel: one CTA per SM walks over 128 x 128 output tiles (column tile fastest, so the
 // CTAs running at any moment share a few row blocks of A and all of B through L2).  Warp roles:
-//   warp 0        TMA producer: nibble-packed A (activation codes) and B (weight codes) tiles of
-//                 128 K-codes (= two quantization groups) per stage into the "packed" ring, and the
-//                 matching 2 x 128 blocks of weight scales and of activation scales into the "scale"
-//                 ring (same mbarrier; that ring is deep enough to need no barriers of its own).
-//   warp 1        MMA issuer (one lane): per stage four tcgen05.mma kind::i8 (K=32 each), two per group,
+//   warp 0        weight producer (one lane): nibble-packed B (weight codes) tiles of 128 K-codes (= two
+//                 quantization groups) per stage into the "packed" ring by TMA, and the matching 2 x 128
+//                 blocks of weight scales and of activation scales into the "scale" ring (same mbarrier;
+//                 that ring is deep enough to need no barriers of its own).
+//   warp 3        activation producer (one lane): the activation codes arrive from kernel 1 as E4M3 bytes,
+//                 so TMA drops the 128 x 128-byte A tile of a stage straight into the "op" ring with the
+//                 128-byte swizzle the tensor core expects; likewise the BF16 low-rank intermediate T.
+//   warp 1        MMA issuer (one lane): per stage four tcgen05.mma kind::f8f6f4 (K=32 each), two per group,
 //                 each group into its own 128-column half of a 256-column TMEM slot (2 slots), so that
-//                 every group's int32 partial sums stay separate; kind::f16 for the low-rank product
+//                 every group's partial sums stay separate; kind::f16 for the low-rank product
 //                 (first slot of a tile).  One barrier round trip per stage, not per group: a single
 //                 thread needs ~300 cycles per wait/issue/commit cycle, more than one group's MMA time.
 //   warp 2        TMEM allocation / release.
-//   warps 4-7     unpack: packed ring -> signed bytes (16 x code, see quantize_kernel.cuh) written with
-//                 the 128-byte swizzle the tensor core expects, into the "s8" ring; they also fetch the
-//                 ready-made BF16 low-rank operands straight into an s8 slot by TMA.
+//   warps 4-7     unpack: packed weight nibbles -> E4M3 bytes (byte-permute lookup), written with the
+//                 128-byte swizzle into the B half of the stage's "op" slot; for the low-rank stages they
+//                 fetch the ready-made BF16 factor there by TMA instead.
 //   warps 8-15    epilogue: TMEM -> registers (accumulator-fragment shape: 4 rows x 16 channels per
-//                 thread), int -> float, * sw[g,n] * s[m,g] into FP32 accumulators, finally * 2^-8
-//                 (undoing 16 x 16), + bias, BF16.
+//                 thread), * sw[g,n] * s[m,g] into FP32 accumulators, finally + bias, BF16.
 //
-// The epilogue's FP32 work (one convert, one multiply, one fused multiply-add per partial sum, all with
-// distinct register operands) is what bounds this kernel, not the tensor core; its loop is therefore
-// written one stage (two groups) per iteration with all ring bookkeeping kept incremental.
+// The epilogue's FP32 work (one multiply and one fused multiply-add per partial sum, all with distinct
+// register operands) is what bounds this kernel, not the tensor core; its loop is therefore written one
+// stage (two groups) per iteration with all ring bookkeeping kept incremental.
 //
 // Every wait on an mbarrier is bounded: after kWaitLimitNs without progress (or as soon as another
 // CTA has reported an error) the role leaves its loop, the CTA records a code in *err and exits
@@ -34,6 +40,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include "fp8_codes.cuh"
 #include "ptx.cuh"
 
 namespace w4a4 {
@@ -41,8 +48,8 @@ namespace w4a4 {
 constexpr int kBM = 128;            // output tile rows (tokens)
 constexpr int kBN = 128;            // output tile columns (output channels)
 constexpr int kBK = 128;            // K codes per pipeline stage = 2 quantization groups
-constexpr int kPackedStages = 4;    // ring of nibble-packed tiles (TMA destination)
-constexpr int kS8Stages = 3;        // ring of unpacked signed-byte tiles (tensor core source)
+constexpr int kPackedStages = 4;    // ring of nibble-packed weight tiles (TMA destination)
+constexpr int kS8Stages = 4;        // "op" ring: tensor-core operand tiles, A (by TMA) and B (unpacked), one byte per code
 constexpr int kScaleStages = 16;   // ring of scale blocks (2 groups x (kBN weight scales + kBM activation scales));
                                    // deeper than the TMA producer can ever run ahead of the epilogue, so it needs no barriers
 constexpr int kTmemSlots = 2;       // TMEM slots of 2 x kBN columns: one per stage in flight
@@ -51,9 +58,8 @@ constexpr int kUnpackWarp0 = 4, kUnpackWarps = 4;
 constexpr int kEpiWarp0 = 8, kEpiWarps = 8;
 constexpr int kRegsControl = 56, kRegsUnpack = 80, kRegsEpilogue = 184;   // setmaxnreg budgets per role
 
-constexpr uint32_t kPackedATile = kBM * (kBK / 2);   // 8 KiB
 constexpr uint32_t kPackedBTile = kBN * (kBK / 2);   // 8 KiB
-constexpr uint32_t kPackedStageBytes = kPackedATile + kPackedBTile;
+constexpr uint32_t kPackedStageBytes = kPackedBTile;
 constexpr uint32_t kS8ATile = kBM * kBK;             // 16 KiB
 constexpr uint32_t kS8BTile = kBN * kBK;             // 16 KiB
 constexpr uint32_t kS8StageBytes = kS8ATile + kS8BTile;
@@ -154,7 +160,7 @@ __host__ __device__ constexpr int tile_column_to_channel(int c) {
 }
 
 // Rescales one fragment (16 TMEM lanes x 64 columns: two rows x 16 channels per thread) of a group's
-// int32 partial sums (256 x P) into the FP32 accumulators:  acc += float(P) * sw[channel] * sa[row].
+// partial sums P (integers held in FP32) into the FP32 accumulators:  acc += P * sw[channel] * sa[row].
 //   v     the fragment as loaded by tmem_ld_16x256b_x8
 //   w     the thread's 16 weight scales, channel order
 //   sa_t  activation scales of the thread's two rows (r and r + 8 of the 16-lane half)
@@ -168,36 +174,37 @@ __device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[32], const 
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const float2 wj = (j & 1) ? make_float2(w[j >> 1].z, w[j >> 1].w) : make_float2(w[j >> 1].x, w[j >> 1].y);
-    const float2 p0 = make_float2(static_cast<float>(static_cast<int32_t>(v[4 * j])),
-                                  static_cast<float>(static_cast<int32_t>(v[4 * j + 1])));
-    const float2 p1 = make_float2(static_cast<float>(static_cast<int32_t>(v[4 * j + 2])),
-                                  static_cast<float>(static_cast<int32_t>(v[4 * j + 3])));
+    const float2 p0 = make_float2(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]));
+    const float2 p1 = make_float2(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
     acc[j] = __ffma2_rn(__fmul2_rn(p0, wj), s0, acc[j]);
     acc[8 + j] = __ffma2_rn(__fmul2_rn(p1, wj), s1, acc[8 + j]);
     if (DEBUG) {
       if (dbg_row0 != nullptr) {
         const int o = 4 * ((j >> 1) ^ swap) + 2 * (j & 1);  // channel offset of columns (j, 0), (j, 1)
-        dbg_row0[o] = static_cast<int32_t>(v[4 * j]) >> 8;
-        dbg_row0[o + 1] = static_cast<int32_t>(v[4 * j + 1]) >> 8;
-        dbg_row1[o] = static_cast<int32_t>(v[4 * j + 2]) >> 8;
-        dbg_row1[o + 1] = static_cast<int32_t>(v[4 * j + 3]) >> 8;
+        dbg_row0[o] = static_cast<int32_t>(p0.x);
+        dbg_row0[o + 1] = static_cast<int32_t>(p0.y);
+        dbg_row1[o] = static_cast<int32_t>(p1.x);
+        dbg_row1[o + 1] = static_cast<int32_t>(p1.y);
       }
     }
   }
 }
 
-// One 16-byte packed chunk (32 codes) -> two 16-byte runs of signed bytes (16 x code), shared to shared.
+// One 16-byte packed weight chunk (32 codes, stored as code + 8) -> two 16-byte runs of E4M3 bytes, shared to
+// shared.  Word w of the chunk holds codes 4 w .. 4 w + 3 in its low four nibbles and codes 16 + 4 w .. + 3 in
+// its high four, so each half-word is one byte-permute selector and becomes one word of a run.
 template <int SRC_OFF, int DST_OFF>
 __device__ __forceinline__ void unpack_chunk(uint32_t src, uint32_t dst_lo, uint32_t dst_hi) {
   uint32_t w0, w1, w2, w3;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
                : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
                : "r"(src), "n"(SRC_OFF));
-  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_lo), "n"(DST_OFF), "r"((w0 << 4) & 0xF0F0F0F0u),
-               "r"((w1 << 4) & 0xF0F0F0F0u), "r"((w2 << 4) & 0xF0F0F0F0u), "r"((w3 << 4) & 0xF0F0F0F0u)
+  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_lo), "n"(DST_OFF), "r"(e4m3_of_offset_nibbles4(w0)),
+               "r"(e4m3_of_offset_nibbles4(w1)), "r"(e4m3_of_offset_nibbles4(w2)), "r"(e4m3_of_offset_nibbles4(w3))
                : "memory");
-  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_hi), "n"(DST_OFF), "r"(w0 & 0xF0F0F0F0u),
-               "r"(w1 & 0xF0F0F0F0u), "r"(w2 & 0xF0F0F0F0u), "r"(w3 & 0xF0F0F0F0u)
+  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_hi), "n"(DST_OFF),
+               "r"(e4m3_of_offset_nibbles4(w0 >> 16)), "r"(e4m3_of_offset_nibbles4(w1 >> 16)),
+               "r"(e4m3_of_offset_nibbles4(w2 >> 16)), "r"(e4m3_of_offset_nibbles4(w3 >> 16))
                : "memory");
 }
 
@@ -238,7 +245,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_init(bar_packed_empty + 8 * i, kUnpackWarps);
     }
     for (int i = 0; i < kS8Stages; ++i) {
-      mbar_init(bar_s8_full + 8 * i, kUnpackWarps);
+      mbar_init(bar_s8_full + 8 * i, kUnpackWarps + 1);  // the unpack warps (B half) and the activation producer (A half)
       mbar_init(bar_s8_empty + 8 * i, 1);
     }
     for (int i = 0; i < kTmemSlots; ++i) {
@@ -271,7 +278,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp < kUnpackWarp0) {
     set_max_regs_dec<kRegsControl>();
     if (live && warp == 0 && lane == 0) {
-      // ------------------------------------------------------------------ TMA producer
+      // ------------------------------------------------------------------ weight / scale producer
       Ring<kPackedStages> pk;
       Ring<kScaleStages> sc;
       bool ok = true;
@@ -284,17 +291,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t dst = packed_base + pk.slot * kPackedStageBytes;
           const uint32_t sdst = scale_base + sc.slot * kScaleStageBytes;
           mbar_arrive_expect_tx(full, kPackedStageBytes + kScaleStageBytes);
-          tma_load_2d(dst, &tmA, full, st * (kBK / 2), m0);
-          tma_load_2d(dst + kPackedATile, &tmB, full, st * (kBK / 2), n0);
+          tma_load_2d(dst, &tmB, full, st * (kBK / 2), n0);
           tma_load_2d(sdst, &tmSW, full, n0, 2 * st);
           tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * st);
           pk.advance();
           sc.advance();
         }
       }
+    } else if (live && warp == 3 && lane == 0) {
+      // ------------------------------------------------------------------ activation producer
+      // A halves of the op ring, in the order the MMA warp consumes the slots: per tile the low-rank
+      // stages (T) first, then the code stages.
+      Ring<kS8Stages> s8;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * kBM;
+        for (int st = 0; st < n_lr_stages + n_int_stages; ++st) {
+          ok = bounded_wait<256>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrProducerWait);
+          if (!ok) break;
+          const uint32_t full = bar_s8_full + 8 * s8.slot;
+          const uint32_t dst = s8_base + s8.slot * kS8StageBytes;
+          mbar_arrive_expect_tx(full, kS8ATile);
+          if (st < n_lr_stages) {
+            tma_load_2d(dst, &tmT, full, st * 64, m0);
+          } else {
+            tma_load_2d(dst, &tmA, full, (st - n_lr_stages) * kBK, m0);
+          }
+          s8.advance();
+        }
+      }
     } else if (live && warp == 1 && lane == 0) {
       // ------------------------------------------------------------------ MMA issuer
-      constexpr uint32_t idesc_i8 = umma_idesc(2, 1, kBM, kBN);
+      constexpr uint32_t idesc_f8 = umma_idesc(1, 0, kBM, kBN);
       constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
       Ring<kS8Stages> s8;
       Ring<kTmemSlots> tm;
@@ -330,7 +358,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {  // bytes [32 kk, 32 kk + 32) of every row: group kk / 2, K half kk % 2
             if (kk < 2 * groups) {
-              umma_i8(d + (kk >> 1) * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_i8,
+              umma_f8(d + (kk >> 1) * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_f8,
                       kk & 1);
             }
           }
@@ -346,7 +374,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (live) {
       // ------------------------------------------------------------------ unpack warps
       const int ut = threadIdx.x - 32 * kUnpackWarp0;  // 0..127
-      // Thread ut owns packed chunk (ut & 3) of rows (ut >> 2) + 32 * j, j = 0..3, of A and of B:
+      // Thread ut owns packed chunk (ut & 3) of rows (ut >> 2) + 32 * j, j = 0..3, of the weight tile:
       // every address is a per-thread base plus a compile-time constant.
       const uint32_t src_off = (ut >> 2) * 64 + (ut & 3) * 16;
       const uint32_t swz = (ut >> 2) & 7;
@@ -356,7 +384,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       Ring<kPackedStages> pk;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+        const int n0 = (tile % p.tiles_n) * kBN;
         for (int st = 0; ok && st < n_lr_stages + n_int_stages; ++st) {
           ok = bounded_wait<128>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrUnpackWait);
           if (!ok) break;
@@ -364,10 +392,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t full = bar_s8_full + 8 * s8.slot;
           s8.advance();
           if (st < n_lr_stages) {
-            // BF16 low-rank operands are tensor-core ready: fetch them straight into the s8 slot.
+            // The BF16 low-rank factor is tensor-core ready: fetch it straight into the slot's B half.
             if (ut == 0) {
-              mbar_arrive_expect_tx(full, kS8StageBytes);
-              tma_load_2d(s8a, &tmT, full, st * 64, m0);
+              mbar_arrive_expect_tx(full, kS8BTile);
               tma_load_2d(s8a + kS8ATile, &tmL2, full, st * 64, n0);
             } else if (lane == 0) {
               mbar_arrive(full);
@@ -378,14 +405,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (!ok) break;
           const uint32_t src = packed_base + pk.slot * kPackedStageBytes + src_off;
           const uint32_t dlo = s8a + dst_lo_off, dhi = s8a + dst_hi_off;
-          unpack_chunk<0 * 2048, 0 * 4096>(src, dlo, dhi);
-          unpack_chunk<1 * 2048, 1 * 4096>(src, dlo, dhi);
-          unpack_chunk<2 * 2048, 2 * 4096>(src, dlo, dhi);
-          unpack_chunk<3 * 2048, 3 * 4096>(src, dlo, dhi);
-          unpack_chunk<kPackedATile + 0 * 2048, kS8ATile + 0 * 4096>(src, dlo, dhi);
-          unpack_chunk<kPackedATile + 1 * 2048, kS8ATile + 1 * 4096>(src, dlo, dhi);
-          unpack_chunk<kPackedATile + 2 * 2048, kS8ATile + 2 * 4096>(src, dlo, dhi);
-          unpack_chunk<kPackedATile + 3 * 2048, kS8ATile + 3 * 4096>(src, dlo, dhi);
+          unpack_chunk<0 * 2048, kS8ATile + 0 * 4096>(src, dlo, dhi);
+          unpack_chunk<1 * 2048, kS8ATile + 1 * 4096>(src, dlo, dhi);
+          unpack_chunk<2 * 2048, kS8ATile + 2 * 4096>(src, dlo, dhi);
+          unpack_chunk<3 * 2048, kS8ATile + 3 * 4096>(src, dlo, dhi);
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
@@ -432,12 +455,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tmem_ld_16x256b_x8(t_lane + tm.slot * 2 * kBN, vA);
         tmem_wait_ld();
         if (n_lr_stages > 0) {
-          // The low-rank product T L2 (FP32) seeds the accumulators, scaled like the integer part.
+          // The low-rank product T L2 (FP32) seeds the accumulators.
           tmem_ld_16x256b_x8(t_lane + kHalf + tm.slot * 2 * kBN, vB);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            acc[j] = make_float2(__uint_as_float(vA[4 * j]) * 256.0f, __uint_as_float(vA[4 * j + 1]) * 256.0f);
-            acc[8 + j] = make_float2(__uint_as_float(vA[4 * j + 2]) * 256.0f, __uint_as_float(vA[4 * j + 3]) * 256.0f);
+            acc[j] = make_float2(__uint_as_float(vA[4 * j]), __uint_as_float(vA[4 * j + 1]));
+            acc[8 + j] = make_float2(__uint_as_float(vA[4 * j + 2]), __uint_as_float(vA[4 * j + 3]));
           }
           tmem_wait_ld();
           tc_fence_before_sync();
@@ -450,8 +473,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           tmem_ld_16x256b_x8(t_lane + tm.slot * 2 * kBN, vA);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            acc[16 + j] = make_float2(__uint_as_float(vB[4 * j]) * 256.0f, __uint_as_float(vB[4 * j + 1]) * 256.0f);
-            acc[24 + j] = make_float2(__uint_as_float(vB[4 * j + 2]) * 256.0f, __uint_as_float(vB[4 * j + 3]) * 256.0f);
+            acc[16 + j] = make_float2(__uint_as_float(vB[4 * j]), __uint_as_float(vB[4 * j + 1]));
+            acc[24 + j] = make_float2(__uint_as_float(vB[4 * j + 2]), __uint_as_float(vB[4 * j + 3]));
           }
           tmem_wait_ld();
         } else {
@@ -538,7 +561,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int i = 0; i < 4; ++i) {
             bv[i] = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
           }
-          const float k = 0.00390625f;  // 2^-8: the codes went through the tensor core as 16 x code on both sides
 #pragma unroll
           for (int t = 0; t < 4; ++t) {
             const int rw = row0 + 8 * t;
@@ -551,10 +573,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                              x3 = acc[8 * t + 4 * i + 3];
                 const float2 a0 = swap ? x2 : x0, a1 = swap ? x3 : x1, a2 = swap ? x0 : x2, a3 = swap ? x1 : x3;
                 const float4 b0 = bv[2 * i], b1 = bv[2 * i + 1];
-                __nv_bfloat162 o0 = __floats2bfloat162_rn(fmaf(a0.x, k, b0.x), fmaf(a0.y, k, b0.y));
-                __nv_bfloat162 o1 = __floats2bfloat162_rn(fmaf(a1.x, k, b0.z), fmaf(a1.y, k, b0.w));
-                __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(a2.x, k, b1.x), fmaf(a2.y, k, b1.y));
-                __nv_bfloat162 o3 = __floats2bfloat162_rn(fmaf(a3.x, k, b1.z), fmaf(a3.y, k, b1.w));
+                __nv_bfloat162 o0 = __floats2bfloat162_rn(a0.x + b0.x, a0.y + b0.y);
+                __nv_bfloat162 o1 = __floats2bfloat162_rn(a1.x + b0.z, a1.y + b0.w);
+                __nv_bfloat162 o2 = __floats2bfloat162_rn(a2.x + b1.x, a2.y + b1.y);
+                __nv_bfloat162 o3 = __floats2bfloat162_rn(a3.x + b1.z, a3.y + b1.w);
                 uint4 o;
                 o.x = *reinterpret_cast<uint32_t*>(&o0);
                 o.y = *reinterpret_cast<uint32_t*>(&o1);

@@ -106,6 +106,18 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// kind::f8f6f4 with 8-bit operands: same shared-memory layout and K = 32 per instruction as kind::i8.
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
   asm volatile(
@@ -207,7 +219,8 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t tile_smem_addr, u
 }
 
 // Instruction descriptor for dense, K-major A and B, M x N tile.
-//   c_format: 1 = F32, 2 = S32;  ab_format: kind::i8 -> 1 = signed 8-bit; kind::f16 -> 1 = BF16.
+//   c_format: 1 = F32, 2 = S32;  ab_format: kind::i8 -> 1 = signed 8-bit; kind::f16 -> 1 = BF16;
+//   kind::f8f6f4 -> 0 = E4M3.
 __host__ __device__ constexpr uint32_t umma_idesc(uint32_t c_format, uint32_t ab_format, uint32_t M, uint32_t N) {
   return (c_format << 4) | (ab_format << 7) | (ab_format << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }

@@ -1,4 +1,4 @@
-// Kernel 1: fused smoothing + per-(token, 64-channel group) 4-bit quantization + nibble packing
+// Kernel 1: fused smoothing + per-(token, 64-channel group) 4-bit quantization + code output
 // + low-rank down-projection, one streaming pass over the BF16 activations (HBM bound).
 //
 //   Eq. 5      xh = f32(x) * (1/lambda)                      one FP32 multiply per element
@@ -16,16 +16,22 @@
 // not care about order), so the lane's 16 channels are used as-is as A-fragment slots and the L1
 // fragments are laid out at pack time to match (see l1_fragment_channel()).
 //
-// Packed activation layout (shared with kernel 2's unpack): per row, per 32 consecutive channels
+// Code output, two formats (template parameter BYTES):
+//   BYTES = true   one E4M3 byte per code, row-major [M, K]: the tensor-core operand of kernel 2 as it is
+//                  (fp8_codes.cuh), fetched by TMA straight into the swizzled operand tile;
+//   BYTES = false  nibble-packed, half the bytes, for callers that want the compact form.
+// Packed activation layout: per row, per 32 consecutive channels
 // [32c, 32c+32) one 16-byte chunk of four 32-bit words; word w, byte b holds channel 32c + 4w + b in
 // its LOW nibble and channel 32c + 16 + 4w + b in its HIGH nibble (two's complement nibbles).  With
-// that interleave `word & 0xF0F0F0F0` and `(word << 4) & 0xF0F0F0F0` are each four signed bytes equal
-// to 16 x code, i.e. two K-contiguous runs ready for the integer tensor core.
+// that interleave `word & 0x0F0F0F0F` and `(word >> 4) & 0x0F0F0F0F` are each four K-contiguous codes,
+// one per byte.
 #pragma once
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include "fp8_codes.cuh"
 
 namespace w4a4 {
 
@@ -102,15 +108,35 @@ __device__ __forceinline__ void group_scale(float rho, float a, float& s, float&
   }
 }
 
-// Quantize the lane's 16 smoothed values of one row (Eq. 3) and return its two packed words.
-__device__ __forceinline__ uint2 quantize16(const float* xh, float is) {
-  // code + 8 in [0, 15]:  (float bits of z + 1.5*2^23 + 8) - bits(1.5*2^23), clamped.
-  uint32_t u[16];
+// Eq. 3 for the lane's 16 smoothed values of one row: code + 8 in [0, 15].
+__device__ __forceinline__ void quantize16_offset(const float* xh, float is, uint32_t (&u)[16]) {
+  // (float bits of z + 1.5*2^23 + 8) - bits(1.5*2^23), clamped.
 #pragma unroll
   for (int e = 0; e < 16; ++e) {
     const float f = __fadd_rn(__fmul_rn(xh[e], is), 12582920.0f);
     u[e] = static_cast<uint32_t>(__viaddmin_s32_relu(__float_as_int(f), -0x4B400000, 15));
   }
+}
+
+// Quantize the lane's 16 values and return them as E4M3 bytes: .x/.y = elements 0..7 (channels coff .. +7),
+// .z/.w = elements 8..15 (channels coff + 16 .. +23).
+__device__ __forceinline__ uint4 quantize16_bytes(const float* xh, float is) {
+  uint32_t u[16];
+  quantize16_offset(xh, is, u);
+  uint32_t n0 = u[0], n1 = u[8];  // eight nibbles each, element e in nibble e % 8
+#pragma unroll
+  for (int e = 1; e < 8; ++e) {
+    n0 += u[e] << (4 * e);
+    n1 += u[8 + e] << (4 * e);
+  }
+  return make_uint4(e4m3_of_offset_nibbles4(n0), e4m3_of_offset_nibbles4(n0 >> 16), e4m3_of_offset_nibbles4(n1),
+                    e4m3_of_offset_nibbles4(n1 >> 16));
+}
+
+// Quantize the lane's 16 smoothed values of one row (Eq. 3) and return its two packed words.
+__device__ __forceinline__ uint2 quantize16(const float* xh, float is) {
+  uint32_t u[16];
+  quantize16_offset(xh, is, u);
   // One shift-add per code places its nibble: word w, byte b = low nibble u[4w+b], high nibble u[8+4w+b].
   uint32_t w0 = u[0], w1 = u[4];
 #pragma unroll
@@ -125,7 +151,7 @@ __device__ __forceinline__ uint2 quantize16(const float* xh, float is) {
   return make_uint2(w0 ^ 0x88888888u, w1 ^ 0x88888888u);  // offset-binary -> two's complement nibbles
 }
 
-template <int R, int WARPS>
+template <int R, int WARPS, bool BYTES>
 __global__ void __launch_bounds__(32 * WARPS)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
@@ -217,11 +243,26 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     group_scale(rho, (qj & 1) ? aB : aA, s_mine, is_mine);
     const float is_other = __shfl_xor_sync(0xffffffffu, is_mine, 1);
     const float isA = (qj & 1) ? is_other : is_mine, isB = (qj & 1) ? is_mine : is_other;
-    const uint2 wA = quantize16(xhA, isA);
-    const uint2 wB = quantize16(xhB, isB);
-    const size_t cpitch = static_cast<size_t>(K >> 1);
-    if (okA) *reinterpret_cast<uint2*>(codes + rowA * cpitch + 32 * g + 8 * qj) = wA;
-    if (okB) *reinterpret_cast<uint2*>(codes + rowB * cpitch + 32 * g + 8 * qj) = wB;
+    if constexpr (BYTES) {
+      const uint4 bA = quantize16_bytes(xhA, isA);
+      const uint4 bB = quantize16_bytes(xhB, isB);
+      uint8_t* ca = codes + static_cast<size_t>(rowA) * K + 64 * g + coff;
+      uint8_t* cb = codes + static_cast<size_t>(rowB) * K + 64 * g + coff;
+      if (okA) {
+        *reinterpret_cast<uint2*>(ca) = make_uint2(bA.x, bA.y);
+        *reinterpret_cast<uint2*>(ca + 16) = make_uint2(bA.z, bA.w);
+      }
+      if (okB) {
+        *reinterpret_cast<uint2*>(cb) = make_uint2(bB.x, bB.y);
+        *reinterpret_cast<uint2*>(cb + 16) = make_uint2(bB.z, bB.w);
+      }
+    } else {
+      const uint2 wA = quantize16(xhA, isA);
+      const uint2 wB = quantize16(xhB, isB);
+      const size_t cpitch = static_cast<size_t>(K >> 1);
+      if (okA) *reinterpret_cast<uint2*>(codes + rowA * cpitch + 32 * g + 8 * qj) = wA;
+      if (okB) *reinterpret_cast<uint2*>(codes + rowB * cpitch + 32 * g + 8 * qj) = wB;
+    }
     // Scales are stored group-major ([G][scales_ld]): kernel 2 fetches a (2 groups x 128 rows) block by TMA.
     if (qj == 0 && okA) scales[static_cast<size_t>(g) * scales_ld + rowA] = s_mine;
     if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = s_mine;

@@ -22,9 +22,10 @@ __global__ void reciprocal_kernel(const float* __restrict__ lam, float* __restri
   if (k < K) out[k] = __fdiv_rn(1.0f, lam[k]);
 }
 
-// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed, K-interleaved (see quantize_kernel.cuh),
-// rows in the tile order of tile_column_to_channel (see gemm_kernel.cuh).
-// One thread builds one 16-byte chunk (32 consecutive K of one output channel).
+// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed as code + 8, rows in the tile order of
+// tile_column_to_channel, nibbles in the order kernel 2's unpack_chunk expects (see gemm_kernel.cuh): in the
+// 16-byte chunk of 32 consecutive K, word w holds K offsets 4 w .. 4 w + 3 in its low four nibbles and
+// 16 + 4 w .. + 3 in its high four.  One thread builds one chunk.
 __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __restrict__ out, int K, int N,
                                    int* __restrict__ bad) {
   const int n = blockIdx.x * blockDim.x + threadIdx.x;  // packed row = position in the tile
@@ -36,9 +37,9 @@ __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __rest
   for (int o = 0; o < 32; ++o) {
     const int v = q[static_cast<size_t>(32 * c + o) * N + ch];
     oob |= (v < -8 || v > 7);
-    const uint32_t nib = static_cast<uint32_t>(v) & 0xFu;
-    const int word = (o & 15) >> 2, byte = o & 3, hi = o >> 4;
-    w[word] |= nib << (8 * byte + 4 * hi);
+    const uint32_t nib = static_cast<uint32_t>(v + 8) & 0xFu;
+    const int word = (o & 15) >> 2, pos = o & 3, hi = o >> 4;
+    w[word] |= nib << (4 * pos + 16 * hi);
   }
   if (oob) atomicOr(bad, 1);
   *reinterpret_cast<uint4*>(out + static_cast<size_t>(n) * (K >> 1) + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -79,15 +80,10 @@ __global__ void l2_dup_kernel(const uint16_t* __restrict__ L2, uint16_t* __restr
 }
 
 // Test-only decoders of the activation kernel's outputs.
-__global__ void decode_codes_kernel(const uint8_t* __restrict__ packed, int8_t* __restrict__ codes, int M, int K) {
+__global__ void decode_codes_kernel(const uint8_t* __restrict__ e4m3, int8_t* __restrict__ codes, int M, int K) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(M) * K) return;
-  const int k = idx % K;
-  const size_t m = idx / K;
-  const int c = k >> 5, o = k & 31;
-  const uint8_t b = packed[m * (K >> 1) + 16 * c + 4 * ((o & 15) >> 2) + (o & 3)];
-  const int nib = (o >> 4) ? (b >> 4) : (b & 0xF);
-  codes[idx] = static_cast<int8_t>((nib ^ 8) - 8);
+  codes[idx] = static_cast<int8_t>(e4m3_integer_value(e4m3[idx]));
 }
 // Group-major workspace scales -> [M, G].
 __global__ void decode_scales_kernel(const float* __restrict__ ws, int ld, float* __restrict__ out, int M, int G) {
@@ -119,7 +115,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct w4a4_ctx {
   int device = 0;
   int max_M = 0, max_K = 0, max_r = 0;
-  uint8_t* codes = nullptr;   // [max_M, K/2] packed activation codes (pitch K/2 of the running layer)
+  uint8_t* codes = nullptr;   // [max_M, K] activation codes, one E4M3 byte each (pitch K of the running layer)
   float* scales = nullptr;    // [K/64, scales_ld] group-major activation scales
   int scales_ld = 0;          // max_M rounded up to a multiple of 4 (16-byte rows for TMA)
   uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
@@ -245,7 +241,7 @@ w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_
   const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define W4A4_LAUNCH_Q(R)                                                                                         \
-  quantize_kernel<R, quantize_warps(R)><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
+  quantize_kernel<R, quantize_warps(R), true><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
                                                  ctx->scales, ctx->scales_ld, ctx->t_hilo)
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
@@ -343,19 +339,19 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
     return W4A4_ERR_CUDA;
   }
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  w4a4_status_t st = dev_alloc(&ctx->codes, static_cast<size_t>(max_M) * (max_K / 2), &ctx->bytes);
+  w4a4_status_t st = dev_alloc(&ctx->codes, static_cast<size_t>(max_M) * max_K, &ctx->bytes);
   if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(ctx->scales_ld) * (max_K / 64), &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->scales, 0, sizeof(float) * ctx->scales_ld * (max_K / 64)) != cudaSuccess) st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) st = dev_alloc(&ctx->t_hilo, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8), &ctx->bytes);
   if (st == W4A4_OK) st = dev_alloc(&ctx->d_err, 1, &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->d_err, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
   // The workspace is read by TMA for rows up to max_M even when fewer are valid: start it defined.
-  if (st == W4A4_OK && cudaMemset(ctx->codes, 0, static_cast<size_t>(max_M) * (max_K / 2)) != cudaSuccess) st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && cudaMemset(ctx->codes, 0, static_cast<size_t>(max_M) * max_K) != cudaSuccess) st = W4A4_ERR_CUDA;
   if (st == W4A4_OK &&
       cudaMemset(ctx->t_hilo, 0, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8) * sizeof(uint16_t)) != cudaSuccess)
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) {
-    cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64)>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          static_cast<int>(quantize_smem_bytes(64)));
     cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
@@ -504,8 +500,8 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
   }
   cudaFree(d_bad);
   if (st == W4A4_OK &&
-      !encode_2d(ctx->encode, &h->tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->codes, K / 2, ctx->max_M, K / 2, kBK / 2,
-                 kBM, CU_TENSOR_MAP_SWIZZLE_NONE))
+      !encode_2d(ctx->encode, &h->tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->codes, K, ctx->max_M, K, kBK, kBM,
+                 CU_TENSOR_MAP_SWIZZLE_128B))
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK &&
       !encode_2d(ctx->encode, &h->tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ctx->scales, ctx->scales_ld, G,
