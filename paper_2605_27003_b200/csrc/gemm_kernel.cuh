@@ -8,24 +8,24 @@
 // the epilogue needs no int -> float conversion.
 //
 // Persistent kernel: one CTA per SM walks over 128 x 128 output tiles (column tile fastest, so the
-// CTAs running at any moment share a few row blocks of A and all of B through L2).  Warp roles:
-//   warp 0        weight producer (one lane): nibble-packed B (weight codes) tiles of 128 K-codes (= two
-//                 quantization groups) per stage into the "packed" ring by TMA, and the matching 2 x 128
-//                 blocks of weight scales and of activation scales into the "scale" ring (same mbarrier;
-//                 that ring is deep enough to need no barriers of its own).
-//   warp 3        activation producer (one lane): the activation codes arrive from kernel 1 as E4M3 bytes,
-//                 so TMA drops the 128 x 128-byte A tile of a stage straight into the "op" ring with the
-//                 128-byte swizzle the tensor core expects; likewise the BF16 low-rank intermediate T.
+// CTAs running at any moment share a few row blocks of A and all of B through L2).  Both operands arrive
+// as E4M3 bytes: the activation codes straight from kernel 1, the weight codes from expand_weight_kernel,
+// which runs right before this kernel and turns the layer's nibble-packed weights (their format at rest)
+// into an N x K byte image that stays in L2 for the duration of the GEMM.  Nothing is unpacked on the SM:
+// its issue slots and shared-memory port belong to the epilogue.  Warp roles:
+//   warp 0        producer (one lane): per stage (128 K-codes = two quantization groups) one TMA for the
+//                 128 x 128-byte A tile and one for the B tile, both with the 128-byte swizzle the tensor
+//                 core expects, into a slot of the operand ring, plus the matching 2 x 128 blocks of weight
+//                 scales and of activation scales into the "scale" ring (same mbarrier; that ring is deep
+//                 enough to need no barriers of its own).  The BF16 low-rank operands T and L2 use the
+//                 same ring.
 //   warp 1        MMA issuer (one lane): per stage four tcgen05.mma kind::f8f6f4 (K=32 each), two per group,
 //                 each group into its own 128-column half of a 256-column TMEM slot (2 slots), so that
 //                 every group's partial sums stay separate; kind::f16 for the low-rank product
 //                 (first slot of a tile).  One barrier round trip per stage, not per group: a single
 //                 thread needs ~300 cycles per wait/issue/commit cycle, more than one group's MMA time.
 //   warp 2        TMEM allocation / release.
-//   warps 4-7     unpack: packed weight nibbles -> E4M3 bytes (byte-permute lookup), written with the
-//                 128-byte swizzle into the B half of the stage's "op" slot; for the low-rank stages they
-//                 fetch the ready-made BF16 factor there by TMA instead.
-//   warps 8-15    epilogue: TMEM -> registers (accumulator-fragment shape: 4 rows x 16 channels per
+//   warps 4-11    epilogue: TMEM -> registers (accumulator-fragment shape: 4 rows x 16 channels per
 //                 thread), * sw[g,n] * s[m,g] into FP32 accumulators, finally + bias, BF16.
 //
 // The epilogue's FP32 work (one multiply and one fused multiply-add per partial sum, all with distinct
@@ -48,33 +48,27 @@ namespace w4a4 {
 constexpr int kBM = 128;            // output tile rows (tokens)
 constexpr int kBN = 128;            // output tile columns (output channels)
 constexpr int kBK = 128;            // K codes per pipeline stage = 2 quantization groups
-constexpr int kPackedStages = 4;    // ring of nibble-packed weight tiles (TMA destination)
-constexpr int kS8Stages = 4;        // "op" ring: tensor-core operand tiles, A (by TMA) and B (unpacked), one byte per code
-constexpr int kScaleStages = 16;   // ring of scale blocks (2 groups x (kBN weight scales + kBM activation scales));
+constexpr int kS8Stages = 6;        // operand ring: A and B tiles of one stage, one byte per code, tensor-core ready
+constexpr int kScaleStages = 12;   // ring of scale blocks (2 groups x (kBN weight scales + kBM activation scales));
                                    // deeper than the TMA producer can ever run ahead of the epilogue, so it needs no barriers
 constexpr int kTmemSlots = 2;       // TMEM slots of 2 x kBN columns: one per stage in flight
-constexpr int kGemmThreads = 512;
-constexpr int kUnpackWarp0 = 4, kUnpackWarps = 4;
-constexpr int kEpiWarp0 = 8, kEpiWarps = 8;
-constexpr int kRegsControl = 56, kRegsUnpack = 80, kRegsEpilogue = 184;   // setmaxnreg budgets per role
+constexpr int kGemmThreads = 384;
+constexpr int kEpiWarp0 = 4, kEpiWarps = 8;
+constexpr int kRegsControl = 56, kRegsEpilogue = 216;   // setmaxnreg budgets per role (4 x 32 x 56 + 8 x 32 x 216 <= 64 K)
 
-constexpr uint32_t kPackedBTile = kBN * (kBK / 2);   // 8 KiB
-constexpr uint32_t kPackedStageBytes = kPackedBTile;
 constexpr uint32_t kS8ATile = kBM * kBK;             // 16 KiB
 constexpr uint32_t kS8BTile = kBN * kBK;             // 16 KiB
 constexpr uint32_t kS8StageBytes = kS8ATile + kS8BTile;
 constexpr uint32_t kScaleStageBytes = 2 * (kBN + kBM) * 4;   // 2 KiB: sw[2][kBN] then sa[2][kBM]
-constexpr uint32_t kNumBarriers = 2 * kPackedStages + 2 * kS8Stages + 2 * kTmemSlots;
+constexpr uint32_t kNumBarriers = 2 * kS8Stages + 2 * kTmemSlots;
 constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kS8Stages * kS8StageBytes +
-                                    kPackedStages * kPackedStageBytes + kScaleStages * kScaleStageBytes +
-                                    kNumBarriers * 8 + 16;
+                                    kScaleStages * kScaleStageBytes + kNumBarriers * 8 + 16;
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // 2 s
 
 enum GemmErr : int {
   kErrNone = 0,
   kErrProducerWait = 101,
-  kErrUnpackWait = 102,
   kErrMmaWait = 103,
   kErrEpilogueWait = 104,
 };
@@ -190,22 +184,17 @@ __device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[32], const 
   }
 }
 
-// One 16-byte packed weight chunk (32 codes, stored as code + 8) -> two 16-byte runs of E4M3 bytes, shared to
-// shared.  Word w of the chunk holds codes 4 w .. 4 w + 3 in its low four nibbles and codes 16 + 4 w .. + 3 in
-// its high four, so each half-word is one byte-permute selector and becomes one word of a run.
-template <int SRC_OFF, int DST_OFF>
-__device__ __forceinline__ void unpack_chunk(uint32_t src, uint32_t dst_lo, uint32_t dst_hi) {
-  uint32_t w0, w1, w2, w3;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
-               : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-               : "r"(src), "n"(SRC_OFF));
-  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_lo), "n"(DST_OFF), "r"(e4m3_of_offset_nibbles4(w0)),
-               "r"(e4m3_of_offset_nibbles4(w1)), "r"(e4m3_of_offset_nibbles4(w2)), "r"(e4m3_of_offset_nibbles4(w3))
-               : "memory");
-  asm volatile("st.shared.v4.u32 [%0+%1], {%2,%3,%4,%5};" ::"r"(dst_hi), "n"(DST_OFF),
-               "r"(e4m3_of_offset_nibbles4(w0 >> 16)), "r"(e4m3_of_offset_nibbles4(w1 >> 16)),
-               "r"(e4m3_of_offset_nibbles4(w2 >> 16)), "r"(e4m3_of_offset_nibbles4(w3 >> 16))
-               : "memory");
+// Weight codes at rest -> the E4M3 byte image kernel 2 reads: [N, K/2] packed as code + 8 (byte j of a row holds
+// K offsets 2 j in its low nibble and 2 j + 1 in its high nibble) -> [N, K] bytes.  One thread turns 32 codes
+// (16 bytes in) into 32 bytes out; each half-word of an input word is one byte-permute selector.
+__global__ void expand_weight_kernel(const uint4* __restrict__ packed, uint4* __restrict__ out, size_t chunks) {
+  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= chunks) return;
+  const uint4 w = __ldg(packed + i);
+  out[2 * i] = make_uint4(e4m3_of_offset_nibbles4(w.x), e4m3_of_offset_nibbles4(w.x >> 16), e4m3_of_offset_nibbles4(w.y),
+                          e4m3_of_offset_nibbles4(w.y >> 16));
+  out[2 * i + 1] = make_uint4(e4m3_of_offset_nibbles4(w.z), e4m3_of_offset_nibbles4(w.z >> 16),
+                              e4m3_of_offset_nibbles4(w.w), e4m3_of_offset_nibbles4(w.w >> 16));
 }
 
 template <bool DEBUG>
@@ -218,12 +207,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t s8_base = smem_base;
-  const uint32_t packed_base = s8_base + kS8Stages * kS8StageBytes;
-  const uint32_t scale_base = packed_base + kPackedStages * kPackedStageBytes;
+  const uint32_t scale_base = s8_base + kS8Stages * kS8StageBytes;
   const uint32_t bar_base = scale_base + kScaleStages * kScaleStageBytes;
-  const uint32_t bar_packed_full = bar_base;
-  const uint32_t bar_packed_empty = bar_packed_full + 8 * kPackedStages;
-  const uint32_t bar_s8_full = bar_packed_empty + 8 * kPackedStages;
+  const uint32_t bar_s8_full = bar_base;
   const uint32_t bar_s8_empty = bar_s8_full + 8 * kS8Stages;
   const uint32_t bar_tmem_full = bar_s8_empty + 8 * kS8Stages;
   const uint32_t bar_tmem_empty = bar_tmem_full + 8 * kTmemSlots;
@@ -240,12 +226,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
-    for (int i = 0; i < kPackedStages; ++i) {
-      mbar_init(bar_packed_full + 8 * i, 1);
-      mbar_init(bar_packed_empty + 8 * i, kUnpackWarps);
-    }
     for (int i = 0; i < kS8Stages; ++i) {
-      mbar_init(bar_s8_full + 8 * i, kUnpackWarps + 1);  // the unpack warps (B half) and the activation producer (A half)
+      mbar_init(bar_s8_full + 8 * i, 1);
       mbar_init(bar_s8_empty + 8 * i, 1);
     }
     for (int i = 0; i < kTmemSlots; ++i) {
@@ -275,47 +257,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   // Per tile the TMEM slots are used by: [one slot for the low-rank product, if r > 0] followed by
   // one slot per K stage (two groups, 128 columns each).
-  if (warp < kUnpackWarp0) {
+  if (warp < kEpiWarp0) {
     set_max_regs_dec<kRegsControl>();
     if (live && warp == 0 && lane == 0) {
-      // ------------------------------------------------------------------ weight / scale producer
-      Ring<kPackedStages> pk;
+      // ------------------------------------------------------------------ TMA producer
+      // Slots of the operand ring in the order the MMA warp consumes them: per tile the low-rank stages
+      // (T and the duplicated L2 factor, BF16) first, then the code stages with their scales.
+      Ring<kS8Stages> s8;
       Ring<kScaleStages> sc;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
-        for (int st = 0; st < n_int_stages; ++st) {
-          ok = bounded_wait<256>(bar_packed_empty + 8 * pk.slot, pk.parity ^ 1u, env, kErrProducerWait);
-          if (!ok) break;
-          const uint32_t full = bar_packed_full + 8 * pk.slot;
-          const uint32_t dst = packed_base + pk.slot * kPackedStageBytes;
-          const uint32_t sdst = scale_base + sc.slot * kScaleStageBytes;
-          mbar_arrive_expect_tx(full, kPackedStageBytes + kScaleStageBytes);
-          tma_load_2d(dst, &tmB, full, st * (kBK / 2), n0);
-          tma_load_2d(sdst, &tmSW, full, n0, 2 * st);
-          tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * st);
-          pk.advance();
-          sc.advance();
-        }
-      }
-    } else if (live && warp == 3 && lane == 0) {
-      // ------------------------------------------------------------------ activation producer
-      // A halves of the op ring, in the order the MMA warp consumes the slots: per tile the low-rank
-      // stages (T) first, then the code stages.
-      Ring<kS8Stages> s8;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * kBM;
         for (int st = 0; st < n_lr_stages + n_int_stages; ++st) {
-          ok = bounded_wait<256>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrProducerWait);
+          ok = bounded_wait<128>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrProducerWait);
           if (!ok) break;
           const uint32_t full = bar_s8_full + 8 * s8.slot;
           const uint32_t dst = s8_base + s8.slot * kS8StageBytes;
-          mbar_arrive_expect_tx(full, kS8ATile);
           if (st < n_lr_stages) {
+            mbar_arrive_expect_tx(full, kS8StageBytes);
             tma_load_2d(dst, &tmT, full, st * 64, m0);
+            tma_load_2d(dst + kS8ATile, &tmL2, full, st * 64, n0);
           } else {
-            tma_load_2d(dst, &tmA, full, (st - n_lr_stages) * kBK, m0);
+            const int ks = st - n_lr_stages;
+            const uint32_t sdst = scale_base + sc.slot * kScaleStageBytes;
+            mbar_arrive_expect_tx(full, kS8StageBytes + kScaleStageBytes);
+            tma_load_2d(dst, &tmA, full, ks * kBK, m0);
+            tma_load_2d(dst + kS8ATile, &tmB, full, ks * kBK, n0);
+            tma_load_2d(sdst, &tmSW, full, n0, 2 * ks);
+            tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * ks);
+            sc.advance();
           }
           s8.advance();
         }
@@ -366,56 +336,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           umma_commit(bar_tmem_full + 8 * tm.slot);
           s8.advance();
           tm.advance();
-        }
-      }
-    }
-  } else if (warp < kEpiWarp0) {
-    set_max_regs_dec<kRegsUnpack>();
-    if (live) {
-      // ------------------------------------------------------------------ unpack warps
-      const int ut = threadIdx.x - 32 * kUnpackWarp0;  // 0..127
-      // Thread ut owns packed chunk (ut & 3) of rows (ut >> 2) + 32 * j, j = 0..3, of the weight tile:
-      // every address is a per-thread base plus a compile-time constant.
-      const uint32_t src_off = (ut >> 2) * 64 + (ut & 3) * 16;
-      const uint32_t swz = (ut >> 2) & 7;
-      const uint32_t dst_lo_off = (ut >> 2) * 128 + (((2 * (ut & 3)) ^ swz) << 4);
-      const uint32_t dst_hi_off = (ut >> 2) * 128 + (((2 * (ut & 3) + 1) ^ swz) << 4);
-      Ring<kS8Stages> s8;
-      Ring<kPackedStages> pk;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int n0 = (tile % p.tiles_n) * kBN;
-        for (int st = 0; ok && st < n_lr_stages + n_int_stages; ++st) {
-          ok = bounded_wait<128>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrUnpackWait);
-          if (!ok) break;
-          const uint32_t s8a = s8_base + s8.slot * kS8StageBytes;
-          const uint32_t full = bar_s8_full + 8 * s8.slot;
-          s8.advance();
-          if (st < n_lr_stages) {
-            // The BF16 low-rank factor is tensor-core ready: fetch it straight into the slot's B half.
-            if (ut == 0) {
-              mbar_arrive_expect_tx(full, kS8BTile);
-              tma_load_2d(s8a + kS8ATile, &tmL2, full, st * 64, n0);
-            } else if (lane == 0) {
-              mbar_arrive(full);
-            }
-            continue;
-          }
-          ok = bounded_wait<128>(bar_packed_full + 8 * pk.slot, pk.parity, env, kErrUnpackWait);
-          if (!ok) break;
-          const uint32_t src = packed_base + pk.slot * kPackedStageBytes + src_off;
-          const uint32_t dlo = s8a + dst_lo_off, dhi = s8a + dst_hi_off;
-          unpack_chunk<0 * 2048, kS8ATile + 0 * 4096>(src, dlo, dhi);
-          unpack_chunk<1 * 2048, kS8ATile + 1 * 4096>(src, dlo, dhi);
-          unpack_chunk<2 * 2048, kS8ATile + 2 * 4096>(src, dlo, dhi);
-          unpack_chunk<3 * 2048, kS8ATile + 3 * 4096>(src, dlo, dhi);
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(full);
-            mbar_arrive(bar_packed_empty + 8 * pk.slot);
-          }
-          pk.advance();
         }
       }
     }
@@ -492,7 +412,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const uint32_t t_grp = t_lane + tm.slot * 2 * kBN;
           tmem_ld_16x256b_x8_before(t_grp + kHalf, vB, vA[0]);
           // The stage's scales landed before the MMA that produced this slot was even issued (they ride
-          // on the packed tiles' mbarrier), so they can be read without a wait of their own.
+          // on the operand tiles' mbarrier), so they can be read without a wait of their own.
           const float4* swp = reinterpret_cast<const float4*>(sw_thread + sc.slot * (kScaleStageBytes / 4));
           const float* sap = sa_thread + sc.slot * (kScaleStageBytes / 4);
           float2 sa[4];  // .x: group g0, .y: group g0 + 1

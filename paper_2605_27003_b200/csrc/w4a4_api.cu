@@ -22,10 +22,9 @@ __global__ void reciprocal_kernel(const float* __restrict__ lam, float* __restri
   if (k < K) out[k] = __fdiv_rn(1.0f, lam[k]);
 }
 
-// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed as code + 8, rows in the tile order of
-// tile_column_to_channel, nibbles in the order kernel 2's unpack_chunk expects (see gemm_kernel.cuh): in the
-// 16-byte chunk of 32 consecutive K, word w holds K offsets 4 w .. 4 w + 3 in its low four nibbles and
-// 16 + 4 w .. + 3 in its high four.  One thread builds one chunk.
+// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed as code + 8 (the weights' format at rest), rows
+// in the tile order of tile_column_to_channel (see gemm_kernel.cuh); byte j of a row holds K offsets 2 j (low
+// nibble) and 2 j + 1 (high nibble).  One thread builds one 16-byte chunk (32 consecutive K).
 __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __restrict__ out, int K, int N,
                                    int* __restrict__ bad) {
   const int n = blockIdx.x * blockDim.x + threadIdx.x;  // packed row = position in the tile
@@ -38,8 +37,7 @@ __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __rest
     const int v = q[static_cast<size_t>(32 * c + o) * N + ch];
     oob |= (v < -8 || v > 7);
     const uint32_t nib = static_cast<uint32_t>(v + 8) & 0xFu;
-    const int word = (o & 15) >> 2, pos = o & 3, hi = o >> 4;
-    w[word] |= nib << (4 * pos + 16 * hi);
+    w[o >> 3] |= nib << (4 * (o & 7));
   }
   if (oob) atomicOr(bad, 1);
   *reinterpret_cast<uint4*>(out + static_cast<size_t>(n) * (K >> 1) + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -119,6 +117,8 @@ struct w4a4_ctx {
   float* scales = nullptr;    // [K/64, scales_ld] group-major activation scales
   int scales_ld = 0;          // max_M rounded up to a multiple of 4 (16-byte rows for TMA)
   uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
+  uint8_t* b8 = nullptr;      // [N, K] E4M3 image of the running layer's weight codes (rewritten by every forward)
+  size_t b8_bytes = 0;        // grows to the largest N x K packed on this context
   int* d_err = nullptr;       // device error word
   size_t bytes = 0;
   int num_sms = 0;
@@ -139,14 +139,15 @@ struct ExpertData {
   uint2* l1frag = nullptr;
   uint16_t* l2dup = nullptr;   // [N, 2r]
   float* bias = nullptr;       // [N] or null
-  CUtensorMap tmB, tmSW, tmL2;
+  CUtensorMap tmSW, tmL2;
 };
 
 struct w4a4_layer {
   w4a4_ctx* ctx = nullptr;
   int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0;
   std::vector<ExpertData> experts;
-  CUtensorMap tmA, tmSA, tmT;
+  CUtensorMap tmA, tmSA, tmT, tmB;
+  const uint8_t* tmB_base = nullptr;  // the context's weight-byte scratch this handle's tmB was encoded for
   size_t bytes = 0;
 };
 
@@ -274,12 +275,22 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   p.dbg_n0 = dbg_n0;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
+  // The context's weight-byte scratch may have been reallocated (a larger layer packed since): re-aim the map.
+  if (h->tmB_base != ctx->b8) {
+    if (!encode_2d(ctx->encode, &h->tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->b8, h->K, h->N, h->K, kBK, kBN,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+      return W4A4_ERR_CUDA;
+    h->tmB_base = ctx->b8;
+  }
+  const size_t chunks = static_cast<size_t>(h->N) * h->K / 32;
+  expand_weight_kernel<<<static_cast<unsigned>((chunks + 255) / 256), 256, 0, stream>>>(
+      reinterpret_cast<const uint4*>(e.bpacked), reinterpret_cast<uint4*>(ctx->b8), chunks);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
-  const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
+  const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : h->tmB;
   if (dbg_P) {
-    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
+    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
   } else {
-    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, e.tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
+    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
   }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
@@ -372,6 +383,7 @@ void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
   if (!ctx) return;
   DeviceGuard guard(ctx->device);
   cudaFree(ctx->codes);
+  cudaFree(ctx->b8);
   cudaFree(ctx->scales);
   cudaFree(ctx->t_hilo);
   cudaFree(ctx->d_err);
@@ -433,8 +445,21 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
   const int K = d->K, N = d->N, r = d->r, G = K / 64;
   const bool dev = d->pointers_on_device != 0;
   w4a4_status_t st = W4A4_OK;
+  // The weight-byte scratch of the context must hold this layer's N x K image.  Growing it is safe between
+  // forwards only (synchronise first: a forward of another layer may still be reading the old one).
+  const size_t b8_need = static_cast<size_t>(N) * K;
+  if (ctx->b8_bytes < b8_need) {
+    if (cudaDeviceSynchronize() != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK) {
+      cudaFree(ctx->b8);
+      ctx->bytes -= ctx->b8_bytes;
+      ctx->b8_bytes = 0;
+      st = dev_alloc(&ctx->b8, b8_need, &ctx->bytes);
+      if (st == W4A4_OK) ctx->b8_bytes = b8_need;
+    }
+  }
   int* d_bad = nullptr;
-  st = dev_alloc(&d_bad, 1, nullptr);
+  if (st == W4A4_OK) st = dev_alloc(&d_bad, 1, nullptr);
   if (st == W4A4_OK && cudaMemset(d_bad, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
 
   for (int ei = 0; st == W4A4_OK && ei < d->num_experts; ++ei) {
@@ -481,11 +506,7 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
     cudaFree(l2_own);
     if (st != W4A4_OK) break;
 
-    if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, kBK / 2, kBN,
-                   CU_TENSOR_MAP_SWIZZLE_NONE))
-      st = W4A4_ERR_CUDA;
-    if (st == W4A4_OK &&
-        !encode_2d(ctx->encode, &e.tmSW, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, e.wscale, N, G, static_cast<uint64_t>(N) * 4,
+    if (!encode_2d(ctx->encode, &e.tmSW, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, e.wscale, N, G, static_cast<uint64_t>(N) * 4,
                    kBN, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
       st = W4A4_ERR_CUDA;
     if (st == W4A4_OK && r > 0 &&
