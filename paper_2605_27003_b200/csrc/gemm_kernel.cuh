@@ -25,12 +25,17 @@
 //                 (first slot of a tile).  One barrier round trip per stage, not per group: a single
 //                 thread needs ~300 cycles per wait/issue/commit cycle, more than one group's MMA time.
 //   warp 2        TMEM allocation / release.
-//   warps 4-11    epilogue: TMEM -> registers (accumulator-fragment shape: 4 rows x 16 channels per
-//                 thread), * sw[g,n] * s[m,g] into FP32 accumulators, finally + bias, BF16.
+//   warps 4-19    epilogue: TMEM -> registers with the 32x32b shape (a thread reads its own TMEM lane, i.e. one
+//                 token row; by far the fastest of the load shapes: ~830 B/clk/SM against ~250 for the
+//                 16x256b accumulator-fragment shape), * sw[g,n] * s[m,g] into 32 FP32 accumulators per thread
+//                 (one row x 32 output channels), finally + bias, BF16.  Sixteen warps, four per scheduler,
+//                 so that TMEM and shared-memory latencies of one warp hide behind the arithmetic of others.
 //
 // The epilogue's FP32 work (one multiply and one fused multiply-add per partial sum, all with distinct
-// register operands) is what bounds this kernel, not the tensor core; its loop is therefore written one
-// stage (two groups) per iteration with all ring bookkeeping kept incremental.
+// register operands) and the shared-memory port (operand tiles written by TMA and read by the tensor core,
+// plus the broadcast loads of the weight scales) are what bound this kernel, not the tensor core; the
+// epilogue loop is therefore written one stage (two groups) per iteration with all ring bookkeeping kept
+// incremental.
 //
 // Every wait on an mbarrier is bounded: after kWaitLimitNs without progress (or as soon as another
 // CTA has reported an error) the role leaves its loop, the CTA records a code in *err and exits
@@ -52,9 +57,11 @@ constexpr int kS8Stages = 6;        // operand ring: A and B tiles of one stage,
 constexpr int kScaleStages = 12;   // ring of scale blocks (2 groups x (kBN weight scales + kBM activation scales));
                                    // deeper than the TMA producer can ever run ahead of the epilogue, so it needs no barriers
 constexpr int kTmemSlots = 2;       // TMEM slots of 2 x kBN columns: one per stage in flight
-constexpr int kGemmThreads = 384;
-constexpr int kEpiWarp0 = 4, kEpiWarps = 8;
-constexpr int kRegsControl = 56, kRegsEpilogue = 216;   // setmaxnreg budgets per role (4 x 32 x 56 + 8 x 32 x 216 <= 64 K)
+constexpr int kGemmThreads = 640;
+constexpr int kEpiWarp0 = 4, kEpiWarps = 16;
+constexpr int kEpiCols = kBN / (kEpiWarps / 4);   // output channels per epilogue thread (32)
+constexpr int kRegsControl = 40, kRegsEpilogue = 104;   // setmaxnreg budgets per role: 4 x 32 x 40 + 16 x 32 x 104 fits the
+                                                        // 640 x 96 registers the CTA is launched with
 
 constexpr uint32_t kS8ATile = kBM * kBK;             // 16 KiB
 constexpr uint32_t kS8BTile = kBN * kBK;             // 16 KiB
@@ -141,44 +148,29 @@ struct GemmParams {
   int dbg_m0, dbg_n0;
 };
 
-// Output-channel order inside every 64-column block of a tile.  The epilogue reads TMEM with the
-// accumulator-fragment shape (16 lanes x 256 bits), where a thread (r = lane / 4, q = lane % 4) sees
-// columns 8 j + 2 q + e, j = 0..7, e = 0..1.  The packed weights (and the low-rank factor) are laid out
-// at pack time so that those 16 columns are the 16 consecutive output channels 16 q .. 16 q + 15:
-// column 8 j + 2 q + e holds channel 16 q + 4 ((j / 2) xor (q / 2)) + 2 (j % 2) + e.  Every thread then
-// reads its 16 weight scales with four 128-bit shared loads and stores 32 contiguous bytes per output
-// row; the xor makes the four addresses of each of those loads (q = 0..3, 64 bytes apart) fall into
-// different 16-byte bank groups, which a plain "16 q + 2 j + e" order would not.
-__host__ __device__ constexpr int tile_column_to_channel(int c) {
-  return 16 * ((c >> 1) & 3) + 4 * (((c >> 4) & 3) ^ ((c >> 2) & 1)) + 2 * ((c >> 3) & 1) + (c & 1);
-}
-
-// Rescales one fragment (16 TMEM lanes x 64 columns: two rows x 16 channels per thread) of a group's
-// partial sums P (integers held in FP32) into the FP32 accumulators:  acc += P * sw[channel] * sa[row].
-//   v     the fragment as loaded by tmem_ld_16x256b_x8
-//   w     the thread's 16 weight scales, channel order
-//   sa_t  activation scales of the thread's two rows (r and r + 8 of the 16-lane half)
-//   acc   [0..8): first row, [8..16): second row
-//   w[i]  holds the thread's channels 4 (i xor swap) .. + 3 (see tile_column_to_channel), swap = q / 2
+// Rescales one fragment (32 token rows x 16 columns: one row x 16 channels per thread) of a group's partial
+// sums P (integers held in FP32) into the FP32 accumulators:  acc += P * sw[channel] * sa[row].
+//   v     the fragment as loaded by tmem_ld_32x32b_x16: v[c] is column c of the thread's row
+//   swp   the 16 weight scales of those columns in shared memory (the same for every lane: broadcast loads)
+//   sa    activation scale of the thread's row
+//   acc   8 accumulator pairs, pair k = columns 2 k, 2 k + 1
 template <bool DEBUG>
-__device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[32], const float4 (&w)[4], float sa_t0,
-                                                 float sa_t1, float2* acc, int32_t* dbg_row0, int32_t* dbg_row1,
-                                                 int swap = 0) {
-  const float2 s0 = make_float2(sa_t0, sa_t0), s1 = make_float2(sa_t1, sa_t1);
+__device__ __forceinline__ void rescale_fragment(const uint32_t (&v)[16], const float4* swp, float sa, float2* acc,
+                                                 int32_t* dbg_row) {
+  const float2 s2 = make_float2(sa, sa);
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float2 wj = (j & 1) ? make_float2(w[j >> 1].z, w[j >> 1].w) : make_float2(w[j >> 1].x, w[j >> 1].y);
-    const float2 p0 = make_float2(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]));
-    const float2 p1 = make_float2(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-    acc[j] = __ffma2_rn(__fmul2_rn(p0, wj), s0, acc[j]);
-    acc[8 + j] = __ffma2_rn(__fmul2_rn(p1, wj), s1, acc[8 + j]);
+  for (int i = 0; i < 4; ++i) {
+    const float4 w = swp[i];
+    const float2 p0 = make_float2(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]));
+    const float2 p1 = make_float2(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+    acc[2 * i] = __ffma2_rn(__fmul2_rn(p0, make_float2(w.x, w.y)), s2, acc[2 * i]);
+    acc[2 * i + 1] = __ffma2_rn(__fmul2_rn(p1, make_float2(w.z, w.w)), s2, acc[2 * i + 1]);
     if (DEBUG) {
-      if (dbg_row0 != nullptr) {
-        const int o = 4 * ((j >> 1) ^ swap) + 2 * (j & 1);  // channel offset of columns (j, 0), (j, 1)
-        dbg_row0[o] = static_cast<int32_t>(p0.x);
-        dbg_row0[o + 1] = static_cast<int32_t>(p0.y);
-        dbg_row1[o] = static_cast<int32_t>(p1.x);
-        dbg_row1[o + 1] = static_cast<int32_t>(p1.y);
+      if (dbg_row != nullptr) {
+        dbg_row[4 * i] = static_cast<int32_t>(p0.x);
+        dbg_row[4 * i + 1] = static_cast<int32_t>(p0.y);
+        dbg_row[4 * i + 2] = static_cast<int32_t>(p1.x);
+        dbg_row[4 * i + 3] = static_cast<int32_t>(p1.y);
       }
     }
   }
@@ -343,45 +335,39 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     set_max_regs_inc<kRegsEpilogue>();
     if (live) {
       // ------------------------------------------------------------------ epilogue warps
-      // Warp ew owns TMEM lanes 32 * (ew % 4) .. +31 (token rows) and the 64-column block ew / 4.  A
-      // thread (r = lane / 4, q = lane % 4) owns rows r, r + 8, r + 16, r + 24 of that quarter and the 16
-      // consecutive output channels 16 q .. 16 q + 15 of the block (see tile_column_to_channel).
-      // Software pipeline over 16-lane fragments: while one fragment is being rescaled the next TMEM
-      // load (and, at stage boundaries, the barrier wait in front of it) is already in flight.
+      // Warp ew owns TMEM lanes 32 * (ew % 4) .. +31 (token rows) and the 32-column block ew / 4; a thread owns
+      // one row (its lane) and the block's 32 output channels.  Four epilogue warps per scheduler hide one
+      // another's TMEM and shared-memory latencies.  Software pipeline over fragments of 16 columns: while one
+      // fragment is being rescaled the next TMEM load (and, at stage boundaries, the barrier wait in front of
+      // it) is already in flight.
       const int ew = warp - kEpiWarp0;
       const int quarter = ew & 3, colblk = ew >> 2;
-      const int fr = lane >> 2, fq = lane & 3;
-      const int swap = fq >> 1;  // see tile_column_to_channel
-      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colblk;
-      constexpr uint32_t kHalf = 16u << 16;  // second 16-lane half of the quarter
-      // Per scale stage: sw[2][kBN] then sa[2][kBM] floats.  The thread's 16 weight scales start at
-      // float 64 colblk + 16 q, its four activation scales at float 2 kBN + 32 quarter + r + 8 t.
-      const float* sw_thread = reinterpret_cast<const float*>(smem + (scale_base - smem_base)) + 64 * colblk + 16 * fq;
-      const float* sa_thread = reinterpret_cast<const float*>(smem + (scale_base - smem_base)) + 2 * kBN + 32 * quarter + fr;
+      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + kEpiCols * colblk;
+      // Per scale stage: sw[2][kBN] then sa[2][kBM] floats.  The warp's weight scales start at float
+      // kEpiCols colblk, the thread's activation scale is float 2 kBN + 32 quarter + lane.
+      const float* sw_warp = reinterpret_cast<const float*>(smem + (scale_base - smem_base)) + kEpiCols * colblk;
+      const float* sa_thread = reinterpret_cast<const float*>(smem + (scale_base - smem_base)) + 2 * kBN + 32 * quarter + lane;
       Ring<kTmemSlots> tm;
       Ring<kScaleStages> sc;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
-        const int row0 = m0 + 32 * quarter + fr;  // the thread's rows are row0 + 8 t, t = 0..3
-        const int ch0 = n0 + 64 * colblk + 16 * fq;
+        const int row = m0 + 32 * quarter + lane;
+        const int ch0 = n0 + kEpiCols * colblk;
         const bool dbg_tile = DEBUG && p.dbg_P != nullptr && m0 == p.dbg_m0 && n0 == p.dbg_n0;
-        float2 acc[32];  // [t][j]: row row0 + 8 t, channels ch0 + 2 j, ch0 + 2 j + 1
-        uint32_t vA[32], vB[32];
+        float2 acc[16];  // pair k: channels ch0 + 2 k, ch0 + 2 k + 1
+        uint32_t vA[16], vB[16];
         // First slot of the tile.
         ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
         if (!ok) break;
         tc_fence_after_sync();
-        tmem_ld_16x256b_x8(t_lane + tm.slot * 2 * kBN, vA);
+        tmem_ld_32x32b_x16(t_lane + tm.slot * 2 * kBN, vA);
         tmem_wait_ld();
         if (n_lr_stages > 0) {
           // The low-rank product T L2 (FP32) seeds the accumulators.
-          tmem_ld_16x256b_x8(t_lane + kHalf + tm.slot * 2 * kBN, vB);
+          tmem_ld_32x32b_x16(t_lane + 16 + tm.slot * 2 * kBN, vB);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            acc[j] = make_float2(__uint_as_float(vA[4 * j]), __uint_as_float(vA[4 * j + 1]));
-            acc[8 + j] = make_float2(__uint_as_float(vA[4 * j + 2]), __uint_as_float(vA[4 * j + 3]));
-          }
+          for (int k = 0; k < 8; ++k) acc[k] = make_float2(__uint_as_float(vA[2 * k]), __uint_as_float(vA[2 * k + 1]));
           tmem_wait_ld();
           tc_fence_before_sync();
           __syncwarp();
@@ -390,73 +376,52 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
           if (!ok) break;
           tc_fence_after_sync();
-          tmem_ld_16x256b_x8(t_lane + tm.slot * 2 * kBN, vA);
+          tmem_ld_32x32b_x16(t_lane + tm.slot * 2 * kBN, vA);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            acc[16 + j] = make_float2(__uint_as_float(vB[4 * j]), __uint_as_float(vB[4 * j + 1]));
-            acc[24 + j] = make_float2(__uint_as_float(vB[4 * j + 2]), __uint_as_float(vB[4 * j + 3]));
-          }
+          for (int k = 0; k < 8; ++k) acc[8 + k] = make_float2(__uint_as_float(vB[2 * k]), __uint_as_float(vB[2 * k + 1]));
           tmem_wait_ld();
         } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[j] = make_float2(0.0f, 0.0f);
+          for (int j = 0; j < 16; ++j) acc[j] = make_float2(0.0f, 0.0f);
         }
         // Invariant at the top of each iteration: the stage's TMEM slot has been waited for and vA
-        // holds the first 16-lane fragment of its first group.
-        float2 (&acc_lo)[16] = *reinterpret_cast<float2(*)[16]>(&acc[0]);   // rows row0, row0 + 8
-        float2 (&acc_hi)[16] = *reinterpret_cast<float2(*)[16]>(&acc[16]);  // rows row0 + 16, row0 + 24
+        // holds the first 16-column fragment of its first group.
+        float2 (&acc_lo)[8] = *reinterpret_cast<float2(*)[8]>(&acc[0]);  // channels ch0 .. ch0 + 15
+        float2 (&acc_hi)[8] = *reinterpret_cast<float2(*)[8]>(&acc[8]);  // channels ch0 + 16 .. ch0 + 31
         for (int st = 0; st < n_int_stages; ++st) {
           const int g0 = 2 * st;
           const bool two = g0 + 1 < G;
           const bool last_stage = st + 1 == n_int_stages;
           const uint32_t t_grp = t_lane + tm.slot * 2 * kBN;
-          tmem_ld_16x256b_x8_before(t_grp + kHalf, vB, vA[0]);
+          tmem_ld_32x32b_x16_before(t_grp + 16, vB, vA[0]);
           // The stage's scales landed before the MMA that produced this slot was even issued (they ride
           // on the operand tiles' mbarrier), so they can be read without a wait of their own.
-          const float4* swp = reinterpret_cast<const float4*>(sw_thread + sc.slot * (kScaleStageBytes / 4));
+          const float4* swp = reinterpret_cast<const float4*>(sw_warp + sc.slot * (kScaleStageBytes / 4));
           const float* sap = sa_thread + sc.slot * (kScaleStageBytes / 4);
-          float2 sa[4];  // .x: group g0, .y: group g0 + 1
-#pragma unroll
-          for (int t = 0; t < 4; ++t) sa[t] = make_float2(sap[8 * t], sap[kBM + 8 * t]);
-          float4 w[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) w[i] = swp[i ^ swap];
-          int32_t *d0 = nullptr, *d1 = nullptr, *d2 = nullptr, *d3 = nullptr;
+          const float sa0 = sap[0], sa1 = sap[kBM];  // first / second group of the stage
+          int32_t* d0 = nullptr;
           if (DEBUG) {
-            if (dbg_tile) {
-              const size_t rs = static_cast<size_t>(8) * G * kBN;
-              d0 = p.dbg_P + (static_cast<size_t>(32 * quarter + fr) * G + g0) * kBN + 64 * colblk + 16 * fq;
-              d1 = d0 + rs;
-              d2 = d1 + rs;
-              d3 = d2 + rs;
-            }
+            if (dbg_tile) d0 = p.dbg_P + (static_cast<size_t>(32 * quarter + lane) * G + g0) * kBN + kEpiCols * colblk;
           }
           // ---- group g0
-          rescale_fragment<DEBUG>(vA, w, sa[0].x, sa[1].x, acc, d0, d1, swap);
+          rescale_fragment<DEBUG>(vA, swp, sa0, acc, d0);
           tmem_wait_ld_after(acc_lo);
           if (two) {
-            tmem_ld_16x256b_x8_before(t_grp + kBN, vA, vB[0]);
+            tmem_ld_32x32b_x16_before(t_grp + kBN, vA, vB[0]);
           } else {
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
           }
-          rescale_fragment<DEBUG>(vB, w, sa[2].x, sa[3].x, acc + 16, d2, d3, swap);
+          rescale_fragment<DEBUG>(vB, swp + 4, sa0, acc + 8, DEBUG && d0 ? d0 + 16 : nullptr);
           if (two) {
             // ---- group g0 + 1
             tmem_wait_ld_after(acc_hi);
-            tmem_ld_16x256b_x8_before(t_grp + kBN + kHalf, vB, vA[0]);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) w[i] = swp[kBN / 4 + (i ^ swap)];
+            tmem_ld_32x32b_x16_before(t_grp + kBN + 16, vB, vA[0]);
             if (DEBUG) {
-              if (dbg_tile) {
-                d0 += kBN;
-                d1 += kBN;
-                d2 += kBN;
-                d3 += kBN;
-              }
+              if (dbg_tile) d0 += kBN;
             }
-            rescale_fragment<DEBUG>(vA, w, sa[0].y, sa[1].y, acc, d0, d1, swap);
+            rescale_fragment<DEBUG>(vA, swp + kBN / 4, sa1, acc, d0);
             tmem_wait_ld_after(acc_lo);
             // The whole slot is in registers: hand it back to the MMA warp.
             tc_fence_before_sync();
@@ -468,43 +433,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
             if (!ok) break;
             tc_fence_after_sync();
-            tmem_ld_16x256b_x8_before(t_lane + tm.slot * 2 * kBN, vA, vB[0]);
+            tmem_ld_32x32b_x16_before(t_lane + tm.slot * 2 * kBN, vA, vB[0]);
           }
-          if (two) rescale_fragment<DEBUG>(vB, w, sa[2].y, sa[3].y, acc + 16, d2, d3, swap);
+          if (two) rescale_fragment<DEBUG>(vB, swp + kBN / 4 + 4, sa1, acc + 8, DEBUG && d0 ? d0 + 16 : nullptr);
           if (!last_stage) tmem_wait_ld_after(acc_hi);
           sc.advance();
         }
         if (!ok) break;
-        {
-          float4 bv[4];
+        if (row < p.M) {
+          // The thread's channels are contiguous bytes of its output row.
+          uint4* yrow = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch0);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            bv[i] = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const int rw = row0 + 8 * t;
-            if (rw < p.M) {
-              uint4* yrow = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(rw) * p.N + ch0);
-#pragma unroll
-              for (int i = 0; i < 2; ++i) {  // 8 channels per 16-byte store
-                // acc[8 t + j] holds channels 4 ((j / 2) xor swap) + 2 (j % 2) + {0, 1}: undo the swap here.
-                const float2 x0 = acc[8 * t + 4 * i], x1 = acc[8 * t + 4 * i + 1], x2 = acc[8 * t + 4 * i + 2],
-                             x3 = acc[8 * t + 4 * i + 3];
-                const float2 a0 = swap ? x2 : x0, a1 = swap ? x3 : x1, a2 = swap ? x0 : x2, a3 = swap ? x1 : x3;
-                const float4 b0 = bv[2 * i], b1 = bv[2 * i + 1];
-                __nv_bfloat162 o0 = __floats2bfloat162_rn(a0.x + b0.x, a0.y + b0.y);
-                __nv_bfloat162 o1 = __floats2bfloat162_rn(a1.x + b0.z, a1.y + b0.w);
-                __nv_bfloat162 o2 = __floats2bfloat162_rn(a2.x + b1.x, a2.y + b1.y);
-                __nv_bfloat162 o3 = __floats2bfloat162_rn(a3.x + b1.z, a3.y + b1.w);
-                uint4 o;
-                o.x = *reinterpret_cast<uint32_t*>(&o0);
-                o.y = *reinterpret_cast<uint32_t*>(&o1);
-                o.z = *reinterpret_cast<uint32_t*>(&o2);
-                o.w = *reinterpret_cast<uint32_t*>(&o3);
-                yrow[i] = o;
-              }
+          for (int i = 0; i < kEpiCols / 8; ++i) {  // 8 channels per 16-byte store
+            float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+            if (p.bias) {
+              b0 = __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + 2 * i);
+              b1 = __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + 2 * i + 1);
             }
+            const float2 a0 = acc[4 * i], a1 = acc[4 * i + 1], a2 = acc[4 * i + 2], a3 = acc[4 * i + 3];
+            __nv_bfloat162 o0 = __floats2bfloat162_rn(a0.x + b0.x, a0.y + b0.y);
+            __nv_bfloat162 o1 = __floats2bfloat162_rn(a1.x + b0.z, a1.y + b0.w);
+            __nv_bfloat162 o2 = __floats2bfloat162_rn(a2.x + b1.x, a2.y + b1.y);
+            __nv_bfloat162 o3 = __floats2bfloat162_rn(a3.x + b1.z, a3.y + b1.w);
+            uint4 o;
+            o.x = *reinterpret_cast<uint32_t*>(&o0);
+            o.y = *reinterpret_cast<uint32_t*>(&o1);
+            o.z = *reinterpret_cast<uint32_t*>(&o2);
+            o.w = *reinterpret_cast<uint32_t*>(&o3);
+            yrow[i] = o;
           }
         }
       }

@@ -45,20 +45,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Non-blocking probe of a phase (try_wait may suspend the thread for a while when the phase is still open).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
 
 // Makes generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem() {
@@ -94,18 +80,6 @@ __device__ __forceinline__ void tc_fence_before_sync() {
 __device__ __forceinline__ void tc_fence_after_sync() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem];  one thread issues for the whole CTA.
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 // kind::f8f6f4 with 8-bit operands: same shared-memory layout and K = 32 per instruction as kind::i8.
 __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                         uint32_t accumulate) {
@@ -135,21 +109,31 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// 32 lanes x 32 columns of 32-bit: thread i of the warp receives lane (base_lane + i), columns c .. c+31.
-__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&v)[32]) {
+// TMEM -> registers, shape 32x32b: thread i of the warp reads TMEM lane (base lane + i), 16 consecutive 32-bit
+// columns starting at the base column; v[c] is column c.  The load is asynchronous until tcgen05.wait::ld.
+//
+// The "_before" / "_after" variants carry scheduling pins for software pipelining.  A TMEM load writes its
+// registers at some point before the wait, so (1) it must not be moved above the last read of the buffer it
+// overwrites: `pin` is a register the caller still reads from that buffer, tied as an in/out operand; and
+// (2) arithmetic the caller wants to overlap with the load must not sink below the wait: the wait takes the
+// accumulators that arithmetic produces as in/out operands.
+__device__ __forceinline__ void tmem_ld_32x32b_x16_before(uint32_t taddr, uint32_t (&v)[16], uint32_t& pin) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%17];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "+r"(pin)
       : "r"(taddr)
       : "memory");
 }
-
-// 32 lanes x 16 columns of 32-bit.
+__device__ __forceinline__ void tmem_wait_ld_after(float2 (&a)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+f"(a[0].x), "+f"(a[0].y), "+f"(a[1].x), "+f"(a[1].y), "+f"(a[2].x), "+f"(a[2].y), "+f"(a[3].x),
+                 "+f"(a[3].y), "+f"(a[4].x), "+f"(a[4].y), "+f"(a[5].x), "+f"(a[5].y), "+f"(a[6].x), "+f"(a[6].y),
+                 "+f"(a[7].x), "+f"(a[7].y)
+               :
+               : "memory");
+}
 __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -160,49 +144,7 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&v)
       : "memory");
 }
 
-// 16 lanes x (8 repetitions of 256 bits): the accumulator-fragment shape.  With r = laneid / 4 and
-// q = laneid % 4, register 4 j + 2 t + e of a thread holds TMEM lane (base_lane + r + 8 t), column
-// (base_col + 8 j + 2 q + e),  j = 0..7, t = 0..1, e = 0..1.
-__device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
 
-// Scheduling pins.  The compiler is free to move register-only arithmetic across the (volatile)
-// TMEM load and wait instructions, which would serialise "load the next fragment" and "rescale the
-// current one".  `pin` (a register the following arithmetic reads) makes that arithmetic stay below
-// the load; tmem_wait_ld_after() takes the arithmetic's results as operands so that the wait stays
-// below it.  Neither adds an instruction.
-__device__ __forceinline__ void tmem_ld_16x256b_x8_before(uint32_t taddr, uint32_t (&v)[32], uint32_t& pin) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "+r"(pin)
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld_after(float2 (&a)[16]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+f"(a[0].x), "+f"(a[0].y), "+f"(a[1].x), "+f"(a[1].y), "+f"(a[2].x), "+f"(a[2].y), "+f"(a[3].x),
-                 "+f"(a[3].y), "+f"(a[4].x), "+f"(a[4].y), "+f"(a[5].x), "+f"(a[5].y), "+f"(a[6].x), "+f"(a[6].y),
-                 "+f"(a[7].x), "+f"(a[7].y), "+f"(a[8].x), "+f"(a[8].y), "+f"(a[9].x), "+f"(a[9].y), "+f"(a[10].x),
-                 "+f"(a[10].y), "+f"(a[11].x), "+f"(a[11].y), "+f"(a[12].x), "+f"(a[12].y), "+f"(a[13].x),
-                 "+f"(a[13].y), "+f"(a[14].x), "+f"(a[14].y), "+f"(a[15].x), "+f"(a[15].y)
-               :
-               : "memory");
-}
 
 // Shared-memory operand descriptor, K-major tile with the 128-byte swizzle: rows of 128 bytes,
 // 8-row swizzle atoms of 1024 bytes stacked along M/N (stride-byte-offset 1024), tile base aligned

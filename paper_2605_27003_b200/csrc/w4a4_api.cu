@@ -22,15 +22,15 @@ __global__ void reciprocal_kernel(const float* __restrict__ lam, float* __restri
   if (k < K) out[k] = __fdiv_rn(1.0f, lam[k]);
 }
 
-// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed as code + 8 (the weights' format at rest), rows
-// in the tile order of tile_column_to_channel (see gemm_kernel.cuh); byte j of a row holds K offsets 2 j (low
-// nibble) and 2 j + 1 (high nibble).  One thread builds one 16-byte chunk (32 consecutive K).
+// Residual codes [K, N] (one per byte) -> [N, K/2] nibble-packed as code + 8 (the weights' format at rest);
+// byte j of a row holds K offsets 2 j (low nibble) and 2 j + 1 (high nibble).  One thread builds one
+// 16-byte chunk (32 consecutive K of one output channel).
 __global__ void pack_weight_kernel(const int8_t* __restrict__ q, uint8_t* __restrict__ out, int K, int N,
                                    int* __restrict__ bad) {
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;  // packed row = position in the tile
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;  // output channel = packed row
   const int c = blockIdx.y;
   if (n >= N) return;
-  const int ch = (n & ~63) + tile_column_to_channel(n & 63);  // output channel stored at that position
+  const int ch = n;
   uint32_t w[4] = {0, 0, 0, 0};
   bool oob = false;
   for (int o = 0; o < 32; ++o) {
@@ -66,14 +66,13 @@ __global__ void l1_fragment_kernel(const uint16_t* __restrict__ L1, uint2* __res
                         static_cast<uint32_t>(v[2]) | (static_cast<uint32_t>(v[3]) << 16));
 }
 
-// L2 [r, N] BF16 -> [N, 2r]: the transposed factor twice, matching the [T_hi | T_lo] split of T,
-// rows in the same tile order as the packed weights.
+// L2 [r, N] BF16 -> [N, 2r]: the transposed factor twice, matching the [T_hi | T_lo] split of T.
 __global__ void l2_dup_kernel(const uint16_t* __restrict__ L2, uint16_t* __restrict__ out, int r, int N) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(N) * 2 * r) return;
   const int c = idx % (2 * r);
   const int n = idx / (2 * r);
-  const int ch = (n & ~63) + tile_column_to_channel(n & 63);
+  const int ch = n;
   out[idx] = L2[static_cast<size_t>(c % r) * N + ch];
 }
 
