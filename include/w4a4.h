@@ -13,6 +13,10 @@
  * column) (Eq. 6), and L1 (K x r), L2 (r x N) the BF16 low-rank pair (Eq. 6).  rho is fetched on the
  * device from a table indexed by (expert, layer, timestep bin) (Sec. III-C, last paragraph).
  *
+ * sm_100a has no 4-bit integer tensor-core instruction.  The 4-bit codes (integers -8 .. 7) are fed to the
+ * tensor core as E4M3 bytes, which represent them exactly; products and 64-term group sums are exact in the
+ * FP32 accumulator, so Eq. 7's integer partial sums come out bit for bit.
+ *
  * Every step runs in hand-written CUDA kernels; there is no CPU fallback.  All entry points return
  * a status code, never throw and never abort.  Unless stated otherwise pointers are DEVICE pointers
  * owned by the caller, 16-byte aligned, and only read/written during the call (asynchronously, on
@@ -67,13 +71,16 @@ typedef struct {
 
 /* Creates a context on `device` whose workspace fits M <= max_M tokens, K <= max_K, r <= max_r.
  * One context serves one stream at a time (calls on it reuse the same workspace in stream order).
- * Sec. III (whole forward) -- the workspace holds Q_A(Xh), its scales and Xh*L1 between the two kernels. */
+ * Sec. III (whole forward) -- the workspace holds Q_A(Xh) (one byte per code), its scales and Xh*L1 between
+ * the kernels, and the 8-bit image of the running layer's weights (N x K bytes, sized by w4a4_pack_weights
+ * for the largest layer packed on the context). */
 w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_ctx_t* out);
 void w4a4_ctx_destroy(w4a4_ctx_t ctx);
 
 /* Copies and repacks one layer's constants (Eq. 5-6) into the library's own device layout:
- * reciprocal smoothing vector, nibble-packed K-interleaved residual codes, scales, low-rank factors
- * in tensor-core fragment order, bias.  Synchronous; allocates device memory owned by the handle. */
+ * reciprocal smoothing vector, nibble-packed residual codes (4 bits per weight at rest), scales, low-rank
+ * factors in tensor-core order, bias.  Synchronous; allocates device memory owned by the handle, and grows
+ * the context's weight-image scratch if this layer is the largest so far (it synchronises the device first). */
 w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* desc, w4a4_handle_t* out);
 void w4a4_destroy(w4a4_handle_t h);
 
@@ -82,7 +89,8 @@ void w4a4_destroy(w4a4_handle_t h);
  *   X   device BF16 [M, K] row-major (leading dimension K), 16-byte aligned
  *   Y   device BF16 [M, N] row-major, 16-byte aligned
  *   clip_table  device FP32 [num_experts, num_layers, num_bins], values in [1e-4, 1]
- *   stream      a cudaStream_t (as void*); two kernels are enqueued, no host synchronisation.
+ *   stream      a cudaStream_t (as void*); three kernels are enqueued (activation quantization, expansion of
+ *               the layer's 4-bit weights to bytes, GEMM), no host synchronisation.
  * M may be 0 (nothing is launched).  Errors: INVALID_ARG, SHAPE (M > max_M), CUDA. */
 w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
                                   const float* clip_table, void* Y, void* stream);
