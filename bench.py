@@ -310,7 +310,7 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                     for b, alpha in ((0, 0.7), (1, 1.0)):
                         tq, tg = time_layer(w4, layer, xs, [b] * n_x, 0, clip, Y, M, args.steps, max(3, args.warmup), stream)
                         ops = 2.0 * M * K * N
-                        qb = M * (2.5625 * K + 2.0 * r)
+                        qb = M * (3.0625 * K + 4.0 * r)
                         rows.append(dict(M=M, K=K, N=N, r=r, outlier_fraction=frac, alpha=alpha, quantize_ms=tq, gemm_ms=tg,
                                          layer_tops=ops / ((tq + tg) * 1e-3) / 1e12, gemm_tops=ops / (tg * 1e-3) / 1e12,
                                          gemm_frac=ops / (tg * 1e-3) / 1e12 / int8_peak,
@@ -332,12 +332,58 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                           best_point=best, gpu_launches=3 * args.steps * len(rows))), flush=True)
 
 
+def run_clip_search(args, w4, dev, local_rank, rank, peaks):
+    """Clipping-ratio search (Eq. 10) at the attention-projection shape: six candidates, two calibration samples
+    per search; every candidate runs the real forward with the squared error fused into the GEMM epilogue."""
+    if rank != 0:
+        return
+    shape = gen.CONFIG_SHAPES["attn_proj"]
+    M, K, N, r = shape["M"], shape["K"], shape["N"], shape["r"]
+    cands = [0.5, 0.6, 0.7, 0.8, 0.9, 1.0]
+    n_samples = 2
+    lay = gen.make_layer_direct(K, N, r, seed=7000, device=dev)
+    idx = gen.outlier_channels(K, 0.01, 7001)
+    xs = [gen.make_activations(M, K, sigma=gen.sigma_for_bin(3), outlier_idx=idx, outlier_gain=50.0, seed=7002 + i, device=dev)
+          for i in range(n_samples)]
+    ys = [gen.reference_output(x, lay) for x in xs]
+    ctx = w4.Context(local_rank, M, K, r)
+    layer = w4.Layer(ctx, [lay], num_bins=8)
+    table = torch.ones((1, 1, 8), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(1, min(args.warmup, 2))):
+        w4.w4a4_clip_search(layer.ptr, xs, ys, M, 0, 3, cands, table)
+    searches = max(1, min(args.steps, 5))
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(searches):
+        best, errs = w4.w4a4_clip_search(layer.ptr, xs, ys, M, 0, 3, cands, table)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / searches
+    forwards = len(cands) * n_samples
+    ctx.check()
+    print(json.dumps(dict(
+        metric=METRIC, value=2.0 * M * K * N * forwards / (ms * 1e-3) / 1e12, unit=UNIT, n_gpus=1, steps=searches,
+        warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e4m3",
+        data="synthetic",
+        config=dict(workload="clip_search", M=M, K=K, N=N, r=r, candidates=cands, samples=n_samples,
+                    l2="inputs larger than L2: activations and reference outputs of %.0f MB each" % (M * K * 2 / 1e6)),
+        ms_per_forward=ms / forwards, best_candidate=cands[best], objective=errs,
+        gpu_launches=(2 * forwards + 2) * searches, clocks=clocks)), flush=True)
+    layer.close()
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep"])
+    ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search"])
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -376,6 +422,9 @@ def main():
         return
     if args.workload == "sweep":
         run_sweep(args, w4, dev, local_rank, rank, peaks)
+        return
+    if args.workload == "clip_search":
+        run_clip_search(args, w4, dev, local_rank, rank, peaks)
         return
     n_buf = 4
     w = workload_inputs(args.workload, dev, n_buf)

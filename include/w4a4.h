@@ -115,6 +115,27 @@ w4a4_status_t w4a4_quantize_activations(w4a4_handle_t h, const void* X, int M, i
                                         const float* clip_table, void* stream);
 w4a4_status_t w4a4_gemm_from_workspace(w4a4_handle_t h, int M, int expert_id, void* Y, void* stream);
 
+/* Timestep-wise clipping-ratio search for one (expert, layer, timestep bin), Sec. III-C, Eq. 8-10:
+ *     rho* = argmin over rho in R of  sum over calibration samples t in the bin of  || Y(t) - Y_hat(t; rho) ||_2^2
+ * Y(t) is the full-precision layer output supplied by the caller, Y_hat(t; rho) the output of this quantized
+ * layer (Eq. 11) with ratio rho, rounded to BF16 as the forward stores it.  Every candidate runs the real
+ * forward kernels; the GEMM epilogue accumulates the squared error instead of storing Y_hat (FP32 inside a
+ * warp and tile, FP64 across them).  The winning ratio (the first one on ties) is written into
+ * clip_table[(expert_id * num_layers + layer_id) * num_bins + timestep_bin]; no other entry is touched.
+ *   X_samples     host array of num_samples DEVICE pointers, each BF16 [M, K] (calibration activations of the bin)
+ *   Yref_samples  host array of num_samples DEVICE pointers, each BF16 [M, N] (full-precision outputs)
+ *   candidates    HOST array of num_candidates ratios in [1e-4, 1]  (1 <= num_candidates <= 256)
+ *   clip_table    device FP32 table as in w4a4_linear_forward (read-modify-write of one entry)
+ *   errors_out    HOST array of num_candidates doubles (the objective per candidate) or NULL
+ *   best_out      HOST int (index of the winner) or NULL
+ * A calibration-time call: it allocates a few hundred bytes of device scratch, enqueues
+ * num_samples x num_candidates forwards on `stream` and synchronises the stream before returning.
+ * Errors: INVALID_ARG (NULL / misaligned pointers, candidate out of range, M < 1), SHAPE (M > max_M), ALLOC, CUDA. */
+w4a4_status_t w4a4_clip_search(w4a4_handle_t h, const void* const* X_samples, const void* const* Yref_samples,
+                               int num_samples, int M, int expert_id, int timestep_bin, const float* candidates,
+                               int num_candidates, float* clip_table, double* errors_out, int* best_out,
+                               void* stream);
+
 /* Parity taps (tests only; same kernels, extra stores).
  * w4a4_debug_quantize: runs the activation kernel and decodes its outputs to plain layouts:
  *   codes  device int8 [M, K] (logical 4-bit codes, Eq. 3), scales device FP32 [M, K/64] (Eq. 9),

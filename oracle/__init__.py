@@ -165,3 +165,34 @@ def forward_noquant(X, lam, L1, L2, R, bias):
                                         _p(R, np.float64), _p(bias, np.float64), M, K, N, r, _p(Y, np.float64))
     assert rc == 0
     return Y
+
+
+def bf16_bits_to_f64(bits):
+    """BF16 bit patterns -> the values they denote, as FP64 (exact)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def clip_search(X_samples_bits, Yref_samples_bits, lam, candidates, L1_bits, L2_bits, qw, sw, bias):
+    """Timestep-wise clipping-ratio search for one (layer, bin), Sec. III-C, Eq. 10.
+
+    For every candidate ratio rho the objective is the sum, over the calibration samples of the bin, of the
+    squared Euclidean distance between the full-precision layer output Y (given, BF16) and the output of the
+    quantized layer with that ratio (Eq. 11, rounded to BF16 as the layer stores it), accumulated in FP64.
+    Returns (index of the smallest objective -- the first one on ties --, list of objectives).
+    """
+    errs = []
+    for rho in candidates:
+        e = 0.0
+        for Xb, Yb in zip(X_samples_bits, Yref_samples_bits):
+            Xb = _as(Xb, np.uint16)
+            out = forward_rows(Xb, np.arange(Xb.shape[0], dtype=np.int32), lam, float(np.float32(rho)), L1_bits, L2_bits,
+                               qw, sw, bias)
+            d = bf16_bits_to_f64(Yb) - bf16_bits_to_f64(out["Ybf16"])
+            e += float(np.sum(d * d))
+        errs.append(e)
+    best = 0
+    for i in range(1, len(errs)):
+        if errs[i] < errs[best]:
+            best = i
+    return best, errs

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_ALLOC", 4
 EXPORTED_SYMBOLS = (
     "w4a4_ctx_create", "w4a4_ctx_destroy", "w4a4_pack_weights", "w4a4_destroy", "w4a4_linear_forward",
     "w4a4_ctx_enable_host_io", "w4a4_linear_forward_host", "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
-    "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
+    "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
 
@@ -71,6 +71,9 @@ def _lib():
         lib.w4a4_debug_quantize.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.w4a4_debug_partials.argtypes = [vp, vp, ci, ci, ci, vp, vp, ci, ci, vp, vp]
         lib.w4a4_quantize_noalloc.argtypes = [vp, ci, ci, vp, vp, ci, vp, vp, vp]
+        lib.w4a4_clip_search.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ci, ci, ci, ci,
+                                         ctypes.POINTER(ctypes.c_float), ci, vp, ctypes.POINTER(ctypes.c_double),
+                                         ctypes.POINTER(ci), vp]
         lib.w4a4_tile_shape.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
         lib.w4a4_tile_shape.restype = None
         lib.w4a4_query_status.argtypes = [vp]
@@ -206,6 +209,20 @@ def w4a4_quantize_noalloc(X, M, K, lam, clip_table, clip_index, codes, scales, s
     """Context-free activation quantization into caller buffers; the library's built-in scratch is used."""
     _check(_lib().w4a4_quantize_noalloc(_ptr(X), M, K, _ptr(lam), _ptr(clip_table), clip_index, _ptr(codes),
                                         _ptr(scales), _stream(stream)), "w4a4_quantize_noalloc")
+
+
+def w4a4_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_bin, candidates, clip_table, stream=None):
+    """Eq. 10 on the device: returns (index of the best candidate, list of the candidates' squared errors) and
+    writes the winning ratio into the clip table entry of (expert, layer, bin)."""
+    n_s, n_c = len(X_samples), len(candidates)
+    xs = (ctypes.c_void_p * n_s)(*[_ptr(x) for x in X_samples])
+    ys = (ctypes.c_void_p * n_s)(*[_ptr(y) for y in Yref_samples])
+    cand = (ctypes.c_float * n_c)(*[float(c) for c in candidates])
+    errs = (ctypes.c_double * n_c)()
+    best = ctypes.c_int(-1)
+    _check(_lib().w4a4_clip_search(handle, xs, ys, n_s, M, expert_id, timestep_bin, cand, n_c, _ptr(clip_table), errs,
+                                   ctypes.byref(best), _stream(stream)), "w4a4_clip_search")
+    return int(best.value), [float(e) for e in errs]
 
 
 def w4a4_query_status(ctx) -> int:

@@ -146,6 +146,10 @@ struct GemmParams {
   int* err;
   int32_t* dbg_P;       // debug tap: [kBM, G, kBN] or nullptr
   int dbg_m0, dbg_n0;
+  // Clip-ratio search (Eq. 10): when yref is set, Y is not stored; the squared distance between the layer's
+  // BF16 output and yref is accumulated into *sq_err instead.
+  const uint16_t* yref; // [M, N] BF16 or nullptr
+  double* sq_err;
 };
 
 // Rescales one fragment (32 token rows x 16 columns: one row x 16 channels per thread) of a group's partial
@@ -440,7 +444,37 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           sc.advance();
         }
         if (!ok) break;
-        if (row < p.M) {
+        if (p.yref != nullptr) {
+          // Eq. 10's objective: || Y_ref - Y_hat ||^2 over the tile, with Y_hat rounded to BF16 exactly as the
+          // forward would store it.  FP32 within the thread and the warp, FP64 across warps and tiles.
+          float e = 0.0f;
+          if (row < p.M) {
+            const uint4* yr = reinterpret_cast<const uint4*>(p.yref + static_cast<size_t>(row) * p.N + ch0);
+#pragma unroll
+            for (int i = 0; i < kEpiCols / 8; ++i) {
+              float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+              if (p.bias) {
+                b0 = __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + 2 * i);
+                b1 = __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + 2 * i + 1);
+              }
+              const uint4 ref = __ldg(yr + i);
+              const float2 a0 = acc[4 * i], a1 = acc[4 * i + 1], a2 = acc[4 * i + 2], a3 = acc[4 * i + 3];
+              const float yh[8] = {a0.x + b0.x, a0.y + b0.y, a1.x + b0.z, a1.y + b0.w,
+                                   a2.x + b1.x, a2.y + b1.y, a3.x + b1.z, a3.y + b1.w};
+              const uint32_t rw[4] = {ref.x, ref.y, ref.z, ref.w};
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                const float y_hat = __bfloat162float(__float2bfloat16_rn(yh[c]));
+                const float y_ref = __uint_as_float((c & 1) ? (rw[c >> 1] & 0xffff0000u) : (rw[c >> 1] << 16));
+                const float d = y_ref - y_hat;
+                e = fmaf(d, d, e);
+              }
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+          if (lane == 0) atomicAdd(p.sq_err, static_cast<double>(e));
+        } else if (row < p.M) {
           // The thread's channels are contiguous bytes of its output row.
           uint4* yrow = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch0);
 #pragma unroll

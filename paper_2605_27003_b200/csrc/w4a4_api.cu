@@ -76,6 +76,19 @@ __global__ void l2_dup_kernel(const uint16_t* __restrict__ L2, uint16_t* __restr
   out[idx] = L2[static_cast<size_t>(c % r) * N + ch];
 }
 
+// Eq. 10: index of the smallest accumulated error (the first one on ties); the winning ratio goes into the
+// clip table entry of (expert, layer, bin).
+__global__ void clip_argmin_kernel(const double* __restrict__ err, const float* __restrict__ cand, int n,
+                                   float* __restrict__ table_entry, int* __restrict__ best) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  int b = 0;
+  for (int i = 1; i < n; ++i) {
+    if (err[i] < err[b]) b = i;
+  }
+  *table_entry = cand[b];
+  *best = b;
+}
+
 // Test-only decoders of the activation kernel's outputs.
 __global__ void decode_codes_kernel(const uint8_t* __restrict__ e4m3, int8_t* __restrict__ codes, int M, int K) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -231,12 +244,15 @@ w4a4_status_t check_forward_args(w4a4_handle_t h, const void* X, int M, int expe
   return W4A4_OK;
 }
 
-w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_id, int bin, const float* clip_table,
-                              cudaStream_t stream) {
+// Index of (expert, this layer, bin) in a clip table (Sec. III-C: one ratio per expert, layer and timestep bin).
+int clip_table_index(const w4a4_layer* h, int expert_id, int bin) { return (expert_id * h->L + h->layer_id) * h->B + bin; }
+
+// Kernel 1 with the ratio read from clip_table[clip_index].
+w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expert_id, const float* clip_table,
+                                 int clip_index, cudaStream_t stream) {
   if (M == 0) return W4A4_OK;
   w4a4_ctx* ctx = h->ctx;
   const ExpertData& e = h->experts[expert_id];
-  const int clip_index = (expert_id * h->L + h->layer_id) * h->B + bin;
   const int rows_per_cta = kQuantRows * quantize_warps(h->r);
   const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
@@ -254,8 +270,17 @@ w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
 
+w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_id, int bin, const float* clip_table,
+                              cudaStream_t stream) {
+  return launch_quantize_at(h, X, M, expert_id, clip_table, clip_table_index(h, expert_id, bin), stream);
+}
+
+// Kernel 2 (preceded by the expansion of the expert's 4-bit weights unless `expand` is false, i.e. the
+// context's byte image already holds them).  With yref set, the squared distance to yref is accumulated into
+// *sq_err instead of storing Y.
 w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream, int32_t* dbg_P,
-                          int dbg_m0, int dbg_n0) {
+                          int dbg_m0, int dbg_n0, const void* yref = nullptr, double* sq_err = nullptr,
+                          bool expand = true) {
   if (M == 0) return W4A4_OK;
   w4a4_ctx* ctx = h->ctx;
   const ExpertData& e = h->experts[expert_id];
@@ -272,6 +297,8 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   p.dbg_P = dbg_P;
   p.dbg_m0 = dbg_m0;
   p.dbg_n0 = dbg_n0;
+  p.yref = static_cast<const uint16_t*>(yref);
+  p.sq_err = sq_err;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
   // The context's weight-byte scratch may have been reallocated (a larger layer packed since): re-aim the map.
@@ -281,9 +308,11 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
       return W4A4_ERR_CUDA;
     h->tmB_base = ctx->b8;
   }
-  const size_t chunks = static_cast<size_t>(h->N) * h->K / 32;
-  expand_weight_kernel<<<static_cast<unsigned>((chunks + 255) / 256), 256, 0, stream>>>(
-      reinterpret_cast<const uint4*>(e.bpacked), reinterpret_cast<uint4*>(ctx->b8), chunks);
+  if (expand) {
+    const size_t chunks = static_cast<size_t>(h->N) * h->K / 32;
+    expand_weight_kernel<<<static_cast<unsigned>((chunks + 255) / 256), 256, 0, stream>>>(
+        reinterpret_cast<const uint4*>(e.bpacked), reinterpret_cast<uint4*>(ctx->b8), chunks);
+  }
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : h->tmB;
   if (dbg_P) {
@@ -554,6 +583,65 @@ w4a4_status_t w4a4_gemm_from_workspace(w4a4_handle_t h, int M, int expert_id, vo
   if (M > 0 && (!Y || !aligned16(Y))) return W4A4_ERR_INVALID_ARG;
   DeviceGuard guard(h->ctx->device);
   return launch_gemm(h, M, expert_id, Y, static_cast<cudaStream_t>(stream), nullptr, 0, 0);
+}
+
+w4a4_status_t w4a4_clip_search(w4a4_handle_t h, const void* const* X_samples, const void* const* Yref_samples,
+                               int num_samples, int M, int expert_id, int timestep_bin, const float* candidates,
+                               int num_candidates, float* clip_table, double* errors_out, int* best_out,
+                               void* stream) {
+  if (!h || !h->ctx) return W4A4_ERR_INVALID_ARG;
+  if (num_samples < 1 || num_candidates < 1 || num_candidates > 256 || M < 1) return W4A4_ERR_INVALID_ARG;
+  if (!X_samples || !Yref_samples || !candidates || !clip_table) return W4A4_ERR_INVALID_ARG;
+  for (int c = 0; c < num_candidates; ++c) {
+    if (!(candidates[c] >= 1e-4f && candidates[c] <= 1.0f)) return W4A4_ERR_INVALID_ARG;
+  }
+  for (int s = 0; s < num_samples; ++s) {
+    w4a4_status_t st = check_forward_args(h, X_samples[s], M, expert_id, timestep_bin, clip_table, true);
+    if (st != W4A4_OK) return st;
+    if (!Yref_samples[s] || !aligned16(Yref_samples[s])) return W4A4_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(h->ctx->device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+  cudaStream_t st_ = static_cast<cudaStream_t>(stream);
+  double* d_err = nullptr;
+  float* d_cand = nullptr;
+  int* d_best = nullptr;
+  w4a4_status_t st = dev_alloc(&d_err, static_cast<size_t>(num_candidates), nullptr);
+  if (st == W4A4_OK) st = dev_alloc(&d_cand, static_cast<size_t>(num_candidates), nullptr);
+  if (st == W4A4_OK) st = dev_alloc(&d_best, 1, nullptr);
+  if (st == W4A4_OK &&
+      (cudaMemsetAsync(d_err, 0, sizeof(double) * num_candidates, st_) != cudaSuccess ||
+       cudaMemcpyAsync(d_cand, candidates, sizeof(float) * num_candidates, cudaMemcpyHostToDevice, st_) != cudaSuccess))
+    st = W4A4_ERR_CUDA;
+  // Every candidate runs the real forward (kernel 1 with that ratio, kernel 2 on the same weight image, which
+  // is expanded once) and leaves only its squared error behind.
+  bool expanded = false;
+  for (int s = 0; st == W4A4_OK && s < num_samples; ++s) {
+    for (int c = 0; st == W4A4_OK && c < num_candidates; ++c) {
+      st = launch_quantize_at(h, X_samples[s], M, expert_id, d_cand, c, st_);
+      if (st == W4A4_OK)
+        st = launch_gemm(h, M, expert_id, nullptr, st_, nullptr, 0, 0, Yref_samples[s], d_err + c, !expanded);
+      expanded = true;
+    }
+  }
+  int best = 0;
+  if (st == W4A4_OK) {
+    clip_argmin_kernel<<<1, 32, 0, st_>>>(d_err, d_cand, num_candidates,
+                                          clip_table + clip_table_index(h, expert_id, timestep_bin), d_best);
+    if (cudaGetLastError() != cudaSuccess) st = W4A4_ERR_CUDA;
+  }
+  if (st == W4A4_OK && errors_out &&
+      cudaMemcpyAsync(errors_out, d_err, sizeof(double) * num_candidates, cudaMemcpyDeviceToHost, st_) != cudaSuccess)
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && cudaMemcpyAsync(&best, d_best, sizeof(int), cudaMemcpyDeviceToHost, st_) != cudaSuccess)
+    st = W4A4_ERR_CUDA;
+  if (cudaStreamSynchronize(st_) != cudaSuccess && st == W4A4_OK) st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && best_out) *best_out = best;
+  cudaFree(d_err);
+  cudaFree(d_cand);
+  cudaFree(d_best);
+  if (st != W4A4_OK) cudaGetLastError();
+  return st;
 }
 
 w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,

@@ -196,6 +196,28 @@ def make_layer_direct(K: int, N: int, r: int, *, seed: int = 0, device="cpu", wi
     return LayerInputs(K, N, r, lam, L1, L2, q, scale, bias)
 
 
+def reference_output(x: torch.Tensor, layer: LayerInputs) -> torch.Tensor:
+    """The full-precision layer output Y = X W + b that a calibration run would record (Eq. 10's target), BF16.
+
+    W is the layer's original weight when the recipe kept it, else the weight its quantized pieces stand for,
+    diag(1/lam) (L1 L2 + codes * scale).  FP64 on the CPU, FP32 on a GPU (tooling, not part of the method)."""
+    dev = x.device
+    wide = torch.float64 if dev.type == "cpu" else torch.float32
+    if layer.W is not None:
+        W = layer.W.to(dev, wide)
+    else:
+        G = layer.K // 64
+        deq = layer.qweight.to(dev, wide).view(G, 64, layer.N) * layer.wscale.to(dev, wide).view(G, 1, layer.N)
+        W = deq.view(layer.K, layer.N)
+        if layer.r > 0:
+            W = W + layer.L1.to(dev, wide) @ layer.L2.to(dev, wide)
+        W = W / layer.lam.to(dev, wide).view(-1, 1)
+    y = x.to(wide) @ W
+    if layer.bias is not None:
+        y = y + layer.bias.to(dev, wide)
+    return y.to(torch.bfloat16)
+
+
 def sigma_for_bin(bin_index: int, sigma0: float = 2.0, decay: float = 0.8) -> float:
     """Activation spread per timestep bin: large at early (high-noise) bins, shrinking later."""
     return sigma0 * (decay ** bin_index)
