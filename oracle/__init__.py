@@ -196,3 +196,62 @@ def clip_search(X_samples_bits, Yref_samples_bits, lam, candidates, L1_bits, L2_
         if errs[i] < errs[best]:
             best = i
     return best, errs
+
+
+# ----------------------------------------------------------------------------- MXFP4 variant
+MX_BLOCK = 32
+E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def e2m1_values(codes):
+    """E2M1 codes (bit 3 = sign, bits 0-2 = magnitude index) -> the values they denote."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    v = E2M1_VALUES[codes & 7]
+    return np.where(codes & 8, -v, v)
+
+
+def e2m1_rne_sat(v: float) -> int:
+    lib = _load()
+    lib.oracle_e2m1_rne_sat.restype = ctypes.c_uint8
+    lib.oracle_e2m1_rne_sat.argtypes = [ctypes.c_float]
+    return int(lib.oracle_e2m1_rne_sat(ctypes.c_float(v)))
+
+
+def mx_quantize(X_bits, lam, rho):
+    """MXFP4 activation quantization (OCP MX v1.0 conversion with the clip threshold of Eq. 8 as block maximum).
+    -> codes uint8 [M, K] (E2M1), exps uint8 [M, K/32] (E8M0)."""
+    X_bits = _as(X_bits, np.uint16)
+    lam = _as(lam, np.float32)
+    M, K = X_bits.shape
+    codes = np.empty((M, K), np.uint8)
+    exps = np.empty((M, K // MX_BLOCK), np.uint8)
+    rc = _load().oracle_mx_quantize(_p(X_bits, np.uint16), _p(lam, np.float32), ctypes.c_float(rho), M, K,
+                                    _p(codes, np.uint8), _p(exps, np.uint8))
+    assert rc == 0
+    return codes, exps
+
+
+def mx_forward_rows(X_bits, rows, lam, rho, L1_bits, L2_bits, wcodes, wexps, bias):
+    """Whole MXFP4 layer on the chosen rows.  Returns dict(codes, exps, T, Y64, Ybf16) indexed by position in rows."""
+    X_bits = _as(X_bits, np.uint16)
+    rows = _as(rows, np.int32)
+    lam = _as(lam, np.float32)
+    wcodes = _as(wcodes, np.uint8)
+    wexps = _as(wexps, np.uint8)
+    bias = _as(bias, np.float32)
+    M, K = X_bits.shape
+    N = wcodes.shape[1]
+    r = 0 if L1_bits is None else L1_bits.shape[1]
+    L1_bits = _as(L1_bits, np.uint16)
+    L2_bits = _as(L2_bits, np.uint16)
+    n = rows.shape[0]
+    out = dict(codes=np.empty((n, K), np.uint8), exps=np.empty((n, K // MX_BLOCK), np.uint8),
+               T=np.empty((n, r), np.float32) if r > 0 else None,
+               Y64=np.empty((n, N), np.float64), Ybf16=np.empty((n, N), np.uint16))
+    rc = _load().oracle_mx_forward_rows(_p(X_bits, np.uint16), _p(rows, np.int32), n, K, N, r, _p(lam, np.float32),
+                                        ctypes.c_float(rho), _p(L1_bits, np.uint16), _p(L2_bits, np.uint16),
+                                        _p(wcodes, np.uint8), _p(wexps, np.uint8), _p(bias, np.float32),
+                                        _p(out["codes"], np.uint8), _p(out["exps"], np.uint8), _p(out["T"], np.float32),
+                                        _p(out["Y64"], np.float64), _p(out["Ybf16"], np.uint16))
+    assert rc == 0
+    return out

@@ -32,6 +32,8 @@
 // two's complement codes, q_max = 7 for the scale and [-8, 7] for the clip, ties to even, group 64,
 // multiplication by a reciprocal in place of the division inside Eq. 3, bias added at the end.
 //
+// The second half of the file holds the MXFP4 variant of the layer (its own header comment).
+//
 // Parity status: every function below is pinned by tests that do not come from this file
 // (on-grid round trips, tie cases, saturation, brute-force dot products, the r = 0 and
 // "quantization disabled" reductions to a plain FP64 matrix product).  The paper prints no worked
@@ -263,5 +265,146 @@ int oracle_forward_noquant(const double* X, const double* lambda, const double* 
 
 // BF16 conversion exposed for its own pin (compared against an independent implementation).
 uint16_t oracle_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+
+}  // extern "C"
+
+// =====================================================================================================
+// MXFP4 variant of the same layer (the data format the paper's Table 1 says its 4-bit runs used, and the
+// "native FP4/MXFP4 tensor operations" its Sec. IV-D asks for).  Element and scale formats and the
+// conversion rule are those of the OCP Microscaling Formats (MX) specification v1.0:
+//
+//   block          32 consecutive input channels of one token (activations) / of one output column (weights)
+//   scale          E8M0: one byte e, value 2^(e - 127)
+//   element        E2M1: sign, 2 exponent bits, 1 mantissa bit: +-{0, 0.5, 1, 1.5, 2, 3, 4, 6}
+//   conversion     shared exponent = floor(log2(block maximum)) - 2 (2 = exponent of the largest E2M1 binade),
+//                  element = round-to-nearest-even of value / 2^shared onto the E2M1 grid, saturating at +-6
+//
+// The paper's clipping ratio enters exactly where Eq. 8 puts it: the block maximum is replaced by the clip
+// threshold rho * max|xh| before the shared exponent is taken.
+//
+//   xh[m,k]   = f32(X[m,k]) * (1.0f / lambda[k])                      as in the INT4 path (Eq. 5)
+//   u         = rho * max_{k in block} |xh[m,k]|                      FP32 multiply (Eq. 8)
+//   e[m,b]    = max(exponent field of u - 2, 0)                       (u == 0: e = 0, all elements 0;
+//                                                                      the exponent field of a subnormal u is 0)
+//   a[m,k]    = E2M1_RNE_sat( xh[m,k] * 2^(127 - e[m,b]) )            exact power-of-two scaling, then rounding
+//   Y[m,n]    = sum_b 2^(e[m,b]-127) 2^(ew[b,n]-127) sum_{k in b} a[m,k] w[k,n]  +  T L2  +  b     (FP64)
+//
+// T is the same low-rank intermediate as in the INT4 path.
+// =====================================================================================================
+namespace {
+
+constexpr int kMxBlock = 32;
+const float kE2M1Value[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+// Round to nearest E2M1 value, ties to the code with an even mantissa bit, saturate at 6.  Returns the 4-bit code
+// (bit 3 = sign, taken from v even when the magnitude rounds to zero).
+inline uint8_t e2m1_rne_sat(float v) {
+  const uint8_t sign = std::signbit(v) ? 8u : 0u;
+  const float a = std::fabs(v);
+  int idx = 7;
+  for (int i = 0; i < 7; ++i) {
+    const float lo = kE2M1Value[i], hi = kE2M1Value[i + 1];
+    if (a < hi) {
+      const float mid = 0.5f * (lo + hi);  // exact
+      if (a < mid) idx = i;
+      else if (a > mid) idx = i + 1;
+      else idx = (i % 2 == 0) ? i : i + 1;  // tie: the code whose last bit is 0
+      break;
+    }
+  }
+  return static_cast<uint8_t>(sign | idx);
+}
+
+inline double e2m1_value(uint8_t code) {
+  const double v = kE2M1Value[code & 7];
+  return (code & 8) ? -v : v;
+}
+
+inline uint32_t f32_bits(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, sizeof(u));
+  return u;
+}
+
+// One row: codes[K] (one E2M1 code per byte), exps[K/32] (E8M0 bytes).
+void mx_quantize_row(const uint16_t* x, const float* rl, float rho, int K, uint8_t* codes, uint8_t* exps) {
+  for (int b = 0; b < K / kMxBlock; ++b) {
+    float xh[kMxBlock];
+    float a = 0.0f;
+    for (int i = 0; i < kMxBlock; ++i) {
+      xh[i] = smooth(x[b * kMxBlock + i], rl[b * kMxBlock + i]);
+      const float t = std::fabs(xh[i]);
+      if (t > a) a = t;
+    }
+    const float u = rho * a;
+    const int field = static_cast<int>((f32_bits(u) >> 23) & 0xffu);
+    const int e = field > 2 ? field - 2 : 0;
+    exps[b] = static_cast<uint8_t>(e);
+    const float inv = std::ldexp(1.0f, 127 - e);  // 2^(127 - e), a normal FP32 number for every e in [0, 252]
+    for (int i = 0; i < kMxBlock; ++i) {
+      codes[b * kMxBlock + i] = (a > 0.0f) ? e2m1_rne_sat(xh[i] * inv) : 0;
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+// MXFP4 activation quantization of every row.  codes: M x K, exps: M x K/32.
+int oracle_mx_quantize(const uint16_t* X, const float* lambda, float rho, int M, int K, uint8_t* codes, uint8_t* exps) {
+  if (K <= 0 || K % kMxBlock != 0 || M < 0) return 1;
+  std::vector<float> rl;
+  reciprocal_lambda(lambda, K, rl);
+  for (int m = 0; m < M; ++m) {
+    mx_quantize_row(X + static_cast<size_t>(m) * K, rl.data(), rho, K, codes + static_cast<size_t>(m) * K,
+                    exps + static_cast<size_t>(m) * (K / kMxBlock));
+  }
+  return 0;
+}
+
+// The E2M1 rounding on its own, for its pins.
+uint8_t oracle_e2m1_rne_sat(float v) { return e2m1_rne_sat(v); }
+
+// The whole MXFP4 layer for a chosen set of rows.  wcodes: K x N E2M1 codes (one per byte), wexps: K/32 x N E8M0.
+// Any of codes, exps, T, Ybf16 may be null.
+int oracle_mx_forward_rows(const uint16_t* X, const int* rows, int num_rows, int K, int N, int r, const float* lambda,
+                           float rho, const uint16_t* L1, const uint16_t* L2, const uint8_t* wcodes,
+                           const uint8_t* wexps, const float* bias, uint8_t* codes, uint8_t* exps, float* T,
+                           double* Y64, uint16_t* Ybf16) {
+  if (K <= 0 || K % kMxBlock != 0 || N <= 0 || r < 0) return 1;
+  const int B = K / kMxBlock;
+  std::vector<float> rl;
+  reciprocal_lambda(lambda, K, rl);
+  std::vector<uint8_t> crow(static_cast<size_t>(K)), erow(static_cast<size_t>(B));
+  std::vector<float> trow(static_cast<size_t>(r > 0 ? r : 1));
+  for (int i = 0; i < num_rows; ++i) {
+    const uint16_t* x = X + static_cast<size_t>(rows[i]) * K;
+    mx_quantize_row(x, rl.data(), rho, K, crow.data(), erow.data());
+    if (r > 0) lowrank_down_row(x, rl.data(), L1, K, r, trow.data());
+    for (int n = 0; n < N; ++n) {
+      double y = 0.0;
+      for (int b = 0; b < B; ++b) {
+        double dot = 0.0;  // multiples of 0.25, at most 32 * 36: exact
+        for (int j = 0; j < kMxBlock; ++j) {
+          const int k = b * kMxBlock + j;
+          dot += e2m1_value(crow[k]) * e2m1_value(wcodes[static_cast<size_t>(k) * N + n]);
+        }
+        y += dot * std::ldexp(1.0, static_cast<int>(erow[b]) - 127) *
+             std::ldexp(1.0, static_cast<int>(wexps[static_cast<size_t>(b) * N + n]) - 127);
+      }
+      for (int j = 0; j < r; ++j) {
+        y += static_cast<double>(trow[j]) * static_cast<double>(bf16_to_f32(L2[static_cast<size_t>(j) * N + n]));
+      }
+      if (bias) y += static_cast<double>(bias[n]);
+      if (Y64) Y64[static_cast<size_t>(i) * N + n] = y;
+      if (Ybf16) Ybf16[static_cast<size_t>(i) * N + n] = f32_to_bf16_rne(static_cast<float>(y));
+    }
+    if (codes) std::memcpy(codes + static_cast<size_t>(i) * K, crow.data(), static_cast<size_t>(K));
+    if (exps) std::memcpy(exps + static_cast<size_t>(i) * B, erow.data(), static_cast<size_t>(B));
+    if (T && r > 0) std::memcpy(T + static_cast<size_t>(i) * r, trow.data(), sizeof(float) * r);
+  }
+  return 0;
+}
 
 }  // extern "C"

@@ -196,6 +196,92 @@ def make_layer_direct(K: int, N: int, r: int, *, seed: int = 0, device="cpu", wi
     return LayerInputs(K, N, r, lam, L1, L2, q, scale, bias)
 
 
+# ----------------------------------------------------------------------------- MXFP4 variant of the layer constants
+MX_BLOCK = 32
+_E2M1_GRID = (0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0)
+
+
+@dataclass
+class MxLayerInputs:
+    """Constants of one MXFP4-quantized linear (OCP MX v1.0: E2M1 elements, one E8M0 scale per 32 input channels)."""
+
+    K: int
+    N: int
+    r: int
+    lam: torch.Tensor  # [K] float32
+    L1: Optional[torch.Tensor]  # [K, r] bfloat16
+    L2: Optional[torch.Tensor]  # [r, N] bfloat16
+    wcodes: torch.Tensor  # [K, N] uint8: E2M1 code (bit 3 sign, bits 0-2 magnitude index)
+    wexps: torch.Tensor  # [K/32, N] uint8: E8M0 exponent, scale = 2^(e - 127)
+    bias: Optional[torch.Tensor]  # [N] float32
+    W: Optional[torch.Tensor] = None  # [K, N] float64 original weight (SVD recipe only)
+
+    def to(self, device) -> "MxLayerInputs":
+        def mv(x):
+            return None if x is None else x.to(device)
+
+        return MxLayerInputs(self.K, self.N, self.r, mv(self.lam), mv(self.L1), mv(self.L2), mv(self.wcodes),
+                             mv(self.wexps), mv(self.bias), mv(self.W))
+
+
+def mx_dequantize(codes: torch.Tensor, exps: torch.Tensor) -> torch.Tensor:
+    """[K, N] E2M1 codes + [K/32, N] E8M0 exponents -> float64 values."""
+    grid = torch.tensor(_E2M1_GRID, dtype=torch.float64, device=codes.device)
+    v = grid[(codes & 7).long()]
+    v = torch.where((codes & 8) != 0, -v, v)
+    K, N = codes.shape
+    scale = torch.pow(torch.tensor(2.0, dtype=torch.float64, device=codes.device), exps.to(torch.float64) - 127.0)
+    return (v.view(K // MX_BLOCK, MX_BLOCK, N) * scale[:, None, :]).view(K, N)
+
+
+def _round_residual_mx(R: torch.Tensor):
+    """Residual [K, N] float64 -> MXFP4 per (32-row block, column), the MX specification's conversion:
+    shared exponent floor(log2(block max)) - 2, elements rounded to the nearest E2M1 value (ties to the even
+    code), saturating at 6."""
+    K, N = R.shape
+    B = K // MX_BLOCK
+    Rb = R.reshape(B, MX_BLOCK, N)
+    amax = Rb.abs().amax(dim=1)
+    e = torch.floor(torch.log2(torch.clamp(amax, min=2.0 ** -120))) - 2.0
+    e = torch.where(amax > 0, e, torch.full_like(e, -127.0)).clamp_(-127.0, 125.0)
+    v = (Rb / torch.pow(torch.tensor(2.0, dtype=torch.float64, device=R.device), e)[:, None, :]).abs().clamp_(max=6.0)
+    grid = torch.tensor(_E2M1_GRID, dtype=torch.float64, device=R.device)
+    idx = torch.zeros_like(v, dtype=torch.int64)
+    for i in range(7):
+        lo, hi = _E2M1_GRID[i], _E2M1_GRID[i + 1]
+        mid = 0.5 * (lo + hi)
+        up = (v > mid) | ((v == mid) & (i % 2 == 1))  # ties go to the even code
+        idx = torch.where((v >= lo) & (v < hi) & up, torch.full_like(idx, i + 1), idx)
+        idx = torch.where((v >= lo) & (v < hi) & ~up, torch.full_like(idx, i), idx)
+    idx = torch.where(v >= 6.0, torch.full_like(idx, 7), idx)
+    codes = (idx + 8 * (Rb < 0).long()).to(torch.uint8).reshape(K, N)
+    del grid
+    return codes, (e + 127.0).to(torch.uint8)
+
+
+def make_layer_mx_svd(K: int, N: int, r: int, x_calib: torch.Tensor, *, seed: int = 0, bias_std: Optional[float] = None,
+                      device="cpu") -> MxLayerInputs:
+    """The SVD recipe of make_layer_svd with the residual rounded to MXFP4 instead of INT4."""
+    base = make_layer_svd(K, N, r, x_calib, seed=seed, bias_std=bias_std, device=device)
+    codes, exps = _round_residual_mx(base.R)
+    return MxLayerInputs(K, N, r, base.lam, base.L1, base.L2, codes, exps, base.bias, W=base.W)
+
+
+def make_layer_mx_direct(K: int, N: int, r: int, *, seed: int = 0, device="cpu", with_bias: bool = True) -> MxLayerInputs:
+    """MXFP4 constants drawn directly: codes uniform over the 16 E2M1 patterns, exponents uniform in [-9, -6] + 127;
+    lam, L1, L2, bias as in make_layer_direct."""
+    g = _gen(seed, device)
+    codes = torch.randint(0, 16, (K, N), generator=g, device=device, dtype=torch.uint8)
+    exps = torch.randint(118, 122, (K // MX_BLOCK, N), generator=g, device=device, dtype=torch.uint8)
+    lam = torch.exp(0.5 * torch.randn(K, generator=g, device=device, dtype=torch.float32))
+    L1 = L2 = None
+    if r > 0:
+        L1 = (0.05 * torch.randn(K, r, generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
+        L2 = (0.05 * torch.randn(r, N, generator=g, device=device, dtype=torch.float32)).to(torch.bfloat16)
+    bias = 0.01 * torch.randn(N, generator=g, device=device, dtype=torch.float32) if with_bias else None
+    return MxLayerInputs(K, N, r, lam, L1, L2, codes, exps, bias)
+
+
 def reference_output(x: torch.Tensor, layer: LayerInputs) -> torch.Tensor:
     """The full-precision layer output Y = X W + b that a calibration run would record (Eq. 10's target), BF16.
 
