@@ -170,6 +170,50 @@ void w4a4_tile_shape(int* tile_m, int* tile_n);
 w4a4_status_t w4a4_quantize_noalloc(const void* X, int M, int K, const float* lambda, const float* clip_table,
                                     int clip_index, int8_t* codes, float* scales, void* stream);
 
+/* ---- MXFP4 variant of the same layer -------------------------------------------------------------------------
+ * The caption of the paper's Table 1 states that all its 4-bit runs use the MXFP4 data format, and Sec. IV-D asks
+ * for "native FP4/MXFP4 tensor operations".  This variant computes Eq. 11 with both 4-bit operands in MXFP4 as
+ * the OCP Microscaling Formats specification v1.0 defines it: E2M1 elements (+-{0, 0.5, 1, 1.5, 2, 3, 4, 6}), one
+ * E8M0 scale (a byte e, value 2^(e-127)) per block of 32 consecutive input channels, conversion by shared exponent
+ * floor(log2(block maximum)) - 2 and round-to-nearest-even with saturation.  The clipping ratio of Eq. 8-9 scales the
+ * block maximum before the shared exponent is taken (threshold = rho * max|Xh|).  Smoothing (Eq. 5), the BF16
+ * low-rank branch (Eq. 6-7), the (expert, layer, bin) clip table and the bias are as in the INT4 entry points.
+ * The block scales are applied inside the tensor core (tcgen05.mma kind::mxf4.block_scale), FP32 accumulation.
+ * K must be a multiple of 256, N of 128; r in {0, 16, 32, 64}.  A context serves both variants. */
+typedef struct w4a4_mx_layer* w4a4_mx_handle_t;
+
+typedef struct {
+  int K, N, r;
+  int num_experts, num_bins, num_layers, layer_id;
+  int pointers_on_device;
+  const uint8_t* const* wcodes; /* [E] -> K x N row-major, one E2M1 code per byte: bit 3 sign, bits 0-2 magnitude index */
+  const uint8_t* const* wexps;  /* [E] -> (K/32) x N row-major E8M0 bytes (0xFF, the NaN encoding, is rejected) */
+  const float* const* lambda;   /* [E] -> K FP32, > 0 */
+  const uint16_t* const* L1;    /* [E] -> K x r BF16 bit patterns (ignored if r == 0) */
+  const uint16_t* const* L2;    /* [E] -> r x N BF16 bit patterns (ignored if r == 0) */
+  const float* const* bias;     /* [E] -> N FP32; the array or an entry may be NULL */
+} w4a4_mx_weight_desc_t;
+
+/* Copies and repacks one layer's MXFP4 constants (two codes per byte, scale bytes in the tensor core's atom
+ * layout).  Synchronous; allocates device memory owned by the handle (and, once per context, the activation
+ * scale workspace).  Errors: SHAPE, INVALID_ARG (also: a code above 15, a 0xFF scale byte), ALLOC, CUDA. */
+w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* desc, w4a4_mx_handle_t* out);
+void w4a4_mx_destroy(w4a4_mx_handle_t h);
+size_t w4a4_mx_handle_bytes(w4a4_mx_handle_t h);
+
+/* Eq. 11 in MXFP4: arguments, layouts, ownership and errors exactly as w4a4_linear_forward.  Two kernels are
+ * enqueued on `stream`; no host synchronisation. */
+w4a4_status_t w4a4_mx_linear_forward(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                     const float* clip_table, void* Y, void* stream);
+/* Its two halves, for per-kernel timing. */
+w4a4_status_t w4a4_mx_quantize_activations(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                           const float* clip_table, void* stream);
+w4a4_status_t w4a4_mx_gemm_from_workspace(w4a4_mx_handle_t h, int M, int expert_id, void* Y, void* stream);
+/* Parity tap: runs the activation kernel and decodes its outputs: codes device uint8 [M, K] (E2M1 codes),
+ * exps device uint8 [M, K/32] (E8M0), T device FP32 [M, r] or NULL. */
+w4a4_status_t w4a4_mx_debug_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                     const float* clip_table, uint8_t* codes, uint8_t* exps, float* T, void* stream);
+
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
  * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
 w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);

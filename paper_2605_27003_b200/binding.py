@@ -23,7 +23,9 @@ STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_ALLOC", 4
 EXPORTED_SYMBOLS = (
     "w4a4_ctx_create", "w4a4_ctx_destroy", "w4a4_pack_weights", "w4a4_destroy", "w4a4_linear_forward",
     "w4a4_ctx_enable_host_io", "w4a4_linear_forward_host", "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
-    "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
+    "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search",
+    "w4a4_mx_pack_weights", "w4a4_mx_destroy", "w4a4_mx_handle_bytes", "w4a4_mx_linear_forward",
+    "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
 
@@ -39,6 +41,17 @@ class WeightDesc(ctypes.Structure):
         ("num_experts", ctypes.c_int), ("num_bins", ctypes.c_int), ("num_layers", ctypes.c_int),
         ("layer_id", ctypes.c_int), ("pointers_on_device", ctypes.c_int),
         ("qweight", ctypes.POINTER(ctypes.c_void_p)), ("wscale", ctypes.POINTER(ctypes.c_void_p)),
+        ("lambda_", ctypes.POINTER(ctypes.c_void_p)), ("L1", ctypes.POINTER(ctypes.c_void_p)),
+        ("L2", ctypes.POINTER(ctypes.c_void_p)), ("bias", ctypes.POINTER(ctypes.c_void_p)),
+    ]
+
+
+class MxWeightDesc(ctypes.Structure):
+    _fields_ = [
+        ("K", ctypes.c_int), ("N", ctypes.c_int), ("r", ctypes.c_int),
+        ("num_experts", ctypes.c_int), ("num_bins", ctypes.c_int), ("num_layers", ctypes.c_int),
+        ("layer_id", ctypes.c_int), ("pointers_on_device", ctypes.c_int),
+        ("wcodes", ctypes.POINTER(ctypes.c_void_p)), ("wexps", ctypes.POINTER(ctypes.c_void_p)),
         ("lambda_", ctypes.POINTER(ctypes.c_void_p)), ("L1", ctypes.POINTER(ctypes.c_void_p)),
         ("L2", ctypes.POINTER(ctypes.c_void_p)), ("bias", ctypes.POINTER(ctypes.c_void_p)),
     ]
@@ -74,6 +87,15 @@ def _lib():
         lib.w4a4_clip_search.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ci, ci, ci, ci,
                                          ctypes.POINTER(ctypes.c_float), ci, vp, ctypes.POINTER(ctypes.c_double),
                                          ctypes.POINTER(ci), vp]
+        lib.w4a4_mx_pack_weights.argtypes = [vp, ctypes.POINTER(MxWeightDesc), ctypes.POINTER(vp)]
+        lib.w4a4_mx_destroy.argtypes = [vp]
+        lib.w4a4_mx_destroy.restype = None
+        lib.w4a4_mx_handle_bytes.argtypes = [vp]
+        lib.w4a4_mx_handle_bytes.restype = ctypes.c_size_t
+        lib.w4a4_mx_linear_forward.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
+        lib.w4a4_mx_quantize_activations.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        lib.w4a4_mx_gemm_from_workspace.argtypes = [vp, ci, ci, vp, vp]
+        lib.w4a4_mx_debug_quantize.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.w4a4_tile_shape.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
         lib.w4a4_tile_shape.restype = None
         lib.w4a4_query_status.argtypes = [vp]
@@ -225,6 +247,71 @@ def w4a4_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_bin
     return int(best.value), [float(e) for e in errs]
 
 
+# ----------------------------------------------------------------------------- MXFP4 variant
+def w4a4_mx_pack_weights(ctx, *, K: int, N: int, r: int, num_bins: int, num_layers: int, layer_id: int,
+                         wcodes: Sequence[torch.Tensor], wexps: Sequence[torch.Tensor], lam: Sequence[torch.Tensor],
+                         L1: Optional[Sequence[torch.Tensor]], L2: Optional[Sequence[torch.Tensor]],
+                         bias: Optional[Sequence[Optional[torch.Tensor]]]) -> ctypes.c_void_p:
+    """One tensor per expert in every list; all on the host or all on one CUDA device, contiguous."""
+    E = len(wcodes)
+    on_dev = wcodes[0].is_cuda
+    keep = []
+
+    def arr(ts, dtype, shape):
+        if ts is None:
+            return None
+        a = (ctypes.c_void_p * E)()
+        for i, t in enumerate(ts):
+            if t is None:
+                a[i] = None
+                continue
+            assert t.dtype == dtype and tuple(t.shape) == shape and t.is_contiguous() and t.is_cuda == on_dev, \
+                (t.dtype, tuple(t.shape), shape)
+            keep.append(t)
+            a[i] = t.data_ptr()
+        return a
+
+    d = MxWeightDesc(K=K, N=N, r=r, num_experts=E, num_bins=num_bins, num_layers=num_layers, layer_id=layer_id,
+                     pointers_on_device=int(on_dev))
+    d.wcodes = arr(wcodes, torch.uint8, (K, N))
+    d.wexps = arr(wexps, torch.uint8, (K // 32, N))
+    d.lambda_ = arr(lam, torch.float32, (K,))
+    d.L1 = arr(L1, torch.bfloat16, (K, r)) if r > 0 else None
+    d.L2 = arr(L2, torch.bfloat16, (r, N)) if r > 0 else None
+    d.bias = arr(bias, torch.float32, (N,)) if bias is not None else None
+    out = ctypes.c_void_p()
+    _check(_lib().w4a4_mx_pack_weights(ctx, ctypes.byref(d), ctypes.byref(out)), "w4a4_mx_pack_weights")
+    return out
+
+
+def w4a4_mx_destroy(handle):
+    _lib().w4a4_mx_destroy(handle)
+
+
+def w4a4_mx_handle_bytes(handle) -> int:
+    return int(_lib().w4a4_mx_handle_bytes(handle))
+
+
+def w4a4_mx_linear_forward(handle, X, M, expert_id, timestep_bin, clip_table, Y, stream=None):
+    _check(_lib().w4a4_mx_linear_forward(handle, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table), _ptr(Y),
+                                         _stream(stream)), "w4a4_mx_linear_forward")
+
+
+def w4a4_mx_quantize_activations(handle, X, M, expert_id, timestep_bin, clip_table, stream=None):
+    _check(_lib().w4a4_mx_quantize_activations(handle, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table),
+                                               _stream(stream)), "w4a4_mx_quantize_activations")
+
+
+def w4a4_mx_gemm_from_workspace(handle, M, expert_id, Y, stream=None):
+    _check(_lib().w4a4_mx_gemm_from_workspace(handle, M, expert_id, _ptr(Y), _stream(stream)),
+           "w4a4_mx_gemm_from_workspace")
+
+
+def w4a4_mx_debug_quantize(handle, X, M, expert_id, timestep_bin, clip_table, codes, exps, T=None, stream=None):
+    _check(_lib().w4a4_mx_debug_quantize(handle, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table), _ptr(codes),
+                                         _ptr(exps), _ptr(T), _stream(stream)), "w4a4_mx_debug_quantize")
+
+
 def w4a4_query_status(ctx) -> int:
     return int(_lib().w4a4_query_status(ctx))
 
@@ -288,6 +375,42 @@ class Layer:
     def close(self):
         if self.ptr is not None:
             w4a4_destroy(self.ptr)
+            self.ptr = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class MxLayer:
+    """Owns a w4a4_mx_handle_t built from one MxLayerInputs-like object per expert."""
+
+    def __init__(self, ctx: Context, experts, *, num_bins: int, num_layers: int = 1, layer_id: int = 0):
+        e0 = experts[0]
+        self.ctx, self.K, self.N, self.r, self.E = ctx, e0.K, e0.N, e0.r, len(experts)
+        has_bias = any(e.bias is not None for e in experts)
+        self.ptr = w4a4_mx_pack_weights(
+            ctx.ptr, K=e0.K, N=e0.N, r=e0.r, num_bins=num_bins, num_layers=num_layers, layer_id=layer_id,
+            wcodes=[e.wcodes.contiguous() for e in experts], wexps=[e.wexps.contiguous() for e in experts],
+            lam=[e.lam.contiguous() for e in experts],
+            L1=[e.L1.contiguous() for e in experts] if e0.r > 0 else None,
+            L2=[e.L2.contiguous() for e in experts] if e0.r > 0 else None,
+            bias=[None if e.bias is None else e.bias.contiguous() for e in experts] if has_bias else None)
+
+    def forward(self, X: torch.Tensor, expert_id: int, timestep_bin: int, clip_table: torch.Tensor,
+                Y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        assert X.dtype == torch.bfloat16 and X.is_cuda and X.is_contiguous() and X.shape[1] == self.K
+        M = X.shape[0]
+        if Y is None:
+            Y = torch.empty(M, self.N, dtype=torch.bfloat16, device=X.device)
+        w4a4_mx_linear_forward(self.ptr, X, M, expert_id, timestep_bin, clip_table, Y, stream)
+        return Y
+
+    def close(self):
+        if self.ptr is not None:
+            w4a4_mx_destroy(self.ptr)
             self.ptr = None
 
     def __del__(self):  # pragma: no cover

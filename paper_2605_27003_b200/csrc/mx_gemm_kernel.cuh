@@ -1,0 +1,318 @@
+// Kernel 2 of the MXFP4 variant: block-scaled FP4 GEMM + low-rank up-projection + bias + BF16 store.
+//
+//   Y[m,n] = sum_b 2^(ea[m,b]-127) 2^(ew[b,n]-127) sum_{k in block b} a[m,k] w[k,n]  +  sum_j T[m,j] L2[j,n]  +  b[n]
+//
+// a, w are E2M1 elements, ea / ew the E8M0 exponents of their 32-element blocks along K (OCP MX v1.0, the data
+// format the paper's Table 1 names).  tcgen05.mma kind::mxf4.block_scale applies both block scales inside the
+// tensor core and accumulates in FP32, so -- unlike the INT4 kernel -- nothing is rescaled on the CUDA cores and
+// the whole K extent accumulates into one TMEM tile; the epilogue runs once per output tile.
+//
+// Persistent kernel, one CTA per SM, 128 x 128 output tiles, column tile fastest.  Warp roles:
+//   warp 0      producer (one lane): per stage of 256 K elements one TMA each for the packed A and B tiles
+//               (128 rows x 128 bytes, 128-byte swizzle) and one bulk copy each for their scale bytes (1 KiB:
+//               two 512-byte atoms, the layout the tensor core wants); the BF16 low-rank operands T and L2
+//               go through the same ring first.
+//   warp 1      MMA issuer (one lane): per stage four tcgen05.cp (scale atoms, shared memory -> TMEM: 32 lanes x
+//               128 bits, replicated to the four lane quarters) and four tcgen05.mma kind::mxf4 (K = 64 each,
+//               two scale blocks per row, selected by the scale-factor id 0 / 2 inside the 4-byte TMEM column);
+//               kind::f16 for [T_hi | T_lo] [L2 | L2]^T into the same accumulator first.  tcgen05.cp and
+//               tcgen05.mma of one thread execute in issue order, so one TMEM scale region serves every stage.
+//   warp 2      TMEM allocation / release.
+//   warps 4-7   epilogue: TMEM (32x32b loads, a token row per thread) + bias -> BF16 -> global.  Two accumulator
+//               buffers in TMEM, so the epilogue of a tile overlaps the MMAs of the next.
+//
+// Every wait is bounded exactly as in gemm_kernel.cuh (whose Ring / bounded_wait helpers are used here).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "gemm_kernel.cuh"
+#include "ptx.cuh"
+
+namespace w4a4 {
+
+constexpr int kMxBK = 256;                       // K elements per stage = 128 bytes per operand row
+constexpr int kMxStages = 6;
+constexpr int kMxThreads = 256;
+constexpr int kMxEpiWarp0 = 4, kMxEpiWarps = 4;
+constexpr uint32_t kMxOpTile = kBM * 128;        // 16 KiB (A and B tiles alike: kBM == kBN == 128 rows)
+constexpr uint32_t kMxSfTile = 2 * 512;          // scale bytes of 128 rows x 8 blocks: two atoms
+constexpr uint32_t kMxStageBytes = 2 * kMxOpTile + 2 * kMxSfTile;
+constexpr uint32_t kMxNumBarriers = 2 * kMxStages + 4;
+constexpr uint32_t kMxSmemBytes = 1024 + kMxStages * kMxStageBytes + kMxNumBarriers * 8 + 16;
+constexpr uint32_t kMxTmemSfA = 256, kMxTmemSfB = 264;   // columns: accumulators 0..255, then 8 + 8 scale columns
+static_assert(kBM == 128 && kBN == 128, "the scale-factor atoms and the TMEM layout assume 128 x 128 tiles");
+
+struct MxGemmParams {
+  const float* bias;     // [N] or nullptr
+  uint16_t* Y;           // [M, N] BF16
+  const uint8_t* sfa;    // activation scale atoms: [ceil(M/128)][K/128][512]
+  const uint8_t* sfb;    // weight scale atoms:     [N/128][K/128][512]
+  int M, N, K, r;
+  int tiles_m, tiles_n;
+  int* err;
+};
+
+// Shared-memory descriptor of one scale atom (32 rows x 16 bytes, rows contiguous): K-major, no swizzle, 8-row
+// core matrices 128 bytes apart.
+__device__ __forceinline__ uint64_t mx_sf_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu);
+  d |= static_cast<uint64_t>(1u) << 16;
+  d |= static_cast<uint64_t>((128u >> 4) & 0x3FFFu) << 32;
+  d |= static_cast<uint64_t>(1u) << 46;
+  return d;
+}
+__device__ __forceinline__ void tmem_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// Instruction descriptor of kind::mxf4 (block-scaled): E2M1 x E2M1, E8M0 scales, K-major operands, K = 64.
+__host__ __device__ constexpr uint32_t mx_idesc(uint32_t M, uint32_t N, uint32_t a_sf_id, uint32_t b_sf_id) {
+  return (b_sf_id << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24) | (a_sf_id << 29);
+}
+__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t tsfa,
+                                          uint32_t tsfb, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+      : "memory");
+}
+// Plain (untiled) bulk copy global -> shared, completion on an mbarrier.  Both addresses 16-byte aligned,
+// size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__global__ void __launch_bounds__(kMxThreads, 1)
+mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL2, const MxGemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kMxStages * kMxStageBytes;
+  const uint32_t bar_full = bar_base;
+  const uint32_t bar_empty = bar_full + 8 * kMxStages;
+  const uint32_t bar_acc_full = bar_empty + 8 * kMxStages;
+  const uint32_t bar_acc_empty = bar_acc_full + 16;
+  const uint32_t misc_off = (bar_acc_empty + 16) - smem_base;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_k_stages = p.K / kMxBK;
+  const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
+  const int atoms_k = p.K / 128;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const WaitEnv env{p.err, s_abort};
+
+  if (threadIdx.x == 0) {
+    *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
+    for (int i = 0; i < kMxStages; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_acc_full + 8 * i, 1);
+      mbar_init(bar_acc_empty + 8 * i, kMxEpiWarps);
+    }
+    mbar_fence_init();
+    fence_proxy_async_smem();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    if (p.r > 0) {
+      tma_prefetch_desc(&tmT);
+      tma_prefetch_desc(&tmL2);
+    }
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+    tc_fence_before_sync();
+  }
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const bool live = (*s_abort == 0);
+
+  if (live && warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ producer
+    Ring<kMxStages> rg;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+      const int m0 = tm * kBM, n0 = tn * kBN;
+      for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
+        ok = bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait);
+        if (!ok) break;
+        const uint32_t full = bar_full + 8 * rg.slot;
+        const uint32_t dst = smem_base + rg.slot * kMxStageBytes;
+        if (st < n_lr_stages) {
+          mbar_arrive_expect_tx(full, 2 * kMxOpTile);
+          tma_load_2d(dst, &tmT, full, st * 64, m0);
+          tma_load_2d(dst + kMxOpTile, &tmL2, full, st * 64, n0);
+        } else {
+          const int ks = st - n_lr_stages;
+          mbar_arrive_expect_tx(full, kMxStageBytes);
+          tma_load_2d(dst, &tmA, full, ks * 128, m0);
+          tma_load_2d(dst + kMxOpTile, &tmB, full, ks * 128, n0);
+          bulk_load(dst + 2 * kMxOpTile, p.sfa + (static_cast<size_t>(tm) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
+          bulk_load(dst + 2 * kMxOpTile + kMxSfTile, p.sfb + (static_cast<size_t>(tn) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
+        }
+        rg.advance();
+      }
+    }
+  } else if (live && warp == 1 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
+    Ring<kMxStages> rg;
+    Ring<2> ab;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      ok = bounded_wait<64>(bar_acc_empty + 8 * ab.slot, ab.parity ^ 1u, env, kErrMmaWait);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t d = tmem_base + ab.slot * kBN;
+      uint32_t accumulate = 0;
+      for (int st = 0; ok && st < n_lr_stages + n_k_stages; ++st) {
+        ok = bounded_wait<64>(bar_full + 8 * rg.slot, rg.parity, env, kErrMmaWait);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a = smem_base + rg.slot * kMxStageBytes, b = a + kMxOpTile;
+        if (st < n_lr_stages) {
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            umma_f16(d, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_bf16, accumulate);
+            accumulate = 1;
+          }
+        } else {
+          const uint32_t sf = a + 2 * kMxOpTile;
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            tmem_cp_32x128b_warpx4(tmem_base + kMxTmemSfA + 4 * t, mx_sf_desc(sf + 512 * t));
+            tmem_cp_32x128b_warpx4(tmem_base + kMxTmemSfB + 4 * t, mx_sf_desc(sf + kMxSfTile + 512 * t));
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {  // bytes [32 j, 32 j + 32) of every row: scale blocks 2 j, 2 j + 1
+            const uint32_t id = 2u * (j & 1);
+            umma_mxf4(d, umma_desc_k_sw128(a, 32 * j), umma_desc_k_sw128(b, 32 * j), mx_idesc(kBM, kBN, id, id),
+                      (tmem_base + kMxTmemSfA + 4 * (j >> 1)) | (id << 30), (tmem_base + kMxTmemSfB + 4 * (j >> 1)) | (id << 30),
+                      accumulate);
+            accumulate = 1;
+          }
+        }
+        umma_commit(bar_empty + 8 * rg.slot);
+        rg.advance();
+      }
+      if (!ok) break;
+      umma_commit(bar_acc_full + 8 * ab.slot);
+      ab.advance();
+    }
+  } else if (live && warp >= kMxEpiWarp0) {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp - kMxEpiWarp0;
+    Ring<2> ab;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+      const int row = m0 + 32 * quarter + lane;
+      ok = bounded_wait(bar_acc_full + 8 * ab.slot, ab.parity, env, kErrEpilogueWait);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + ab.slot * kBN;
+#pragma unroll 2
+      for (int c = 0; c < kBN / 16; ++c) {
+        uint32_t v[16];
+        tmem_ld_32x32b_x16(t_row + 16 * c, v);
+        tmem_wait_ld();
+        if (c == kBN / 16 - 1) {
+          // The whole accumulator is in registers or on its way out: hand the buffer back to the MMA warp.
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_acc_empty + 8 * ab.slot);
+        }
+        if (row < p.M) {
+          const int ch = n0 + 16 * c;
+          uint4 o[2];
+          uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(__uint_as_float(v[4 * i]) + b4.x, __uint_as_float(v[4 * i + 1]) + b4.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(__uint_as_float(v[4 * i + 2]) + b4.z, __uint_as_float(v[4 * i + 3]) + b4.w);
+            ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
+            ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
+          }
+          uint4* y = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch);
+          y[0] = o[0];
+          y[1] = o[1];
+        }
+      }
+      ab.advance();
+    }
+  }
+
+  // ---------------------------------------------------------------------- common tail
+  tc_fence_before_sync();
+  __syncthreads();
+  if (*s_abort) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 2) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Weight pack kernels of the MXFP4 variant (run once per layer).
+// codes [K, N] (one E2M1 code per byte) -> [N, K/2], two codes per byte, even K in the low nibble.
+__global__ void mx_pack_weight_kernel(const uint8_t* __restrict__ codes, uint8_t* __restrict__ out, int K, int N,
+                                      int* __restrict__ bad) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int c = blockIdx.y;  // chunk of 32 consecutive K
+  if (n >= N) return;
+  uint32_t w[4] = {0, 0, 0, 0};
+  bool oob = false;
+  for (int o = 0; o < 32; ++o) {
+    const uint32_t v = codes[static_cast<size_t>(32 * c + o) * N + n];
+    oob |= v > 15u;
+    w[o >> 3] |= (v & 15u) << (4 * (o & 7));
+  }
+  if (oob) atomicOr(bad, 1);
+  *reinterpret_cast<uint4*>(out + static_cast<size_t>(n) * (K >> 1) + 16 * c) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+// exps [K/32, N] (E8M0 bytes) -> scale atoms [N/128][K/128][512].
+__global__ void mx_pack_wscale_kernel(const uint8_t* __restrict__ exps, uint8_t* __restrict__ out, int K, int N,
+                                      int* __restrict__ bad) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int B = K / 32;
+  if (idx >= static_cast<size_t>(B) * N) return;
+  const int n = idx % N, b = idx / N;
+  const uint8_t e = exps[idx];
+  if (e == 0xFF) atomicOr(bad, 1);  // E8M0's NaN encoding
+  out[(static_cast<size_t>(n >> 7) * (K / 128) + (b >> 2)) * 512 + (n & 31) * 16 + ((n & 127) >> 5) * 4 + (b & 3)] = e;
+}
+// Test-only decoders of the MXFP4 activation kernel's outputs.
+__global__ void mx_decode_codes_kernel(const uint8_t* __restrict__ packed, uint8_t* __restrict__ codes, int M, int K) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(M) * K) return;
+  const uint8_t b = packed[idx >> 1];
+  codes[idx] = (idx & 1) ? (b >> 4) : (b & 15);
+}
+__global__ void mx_decode_exps_kernel(const uint8_t* __restrict__ atoms, int atoms_k, uint8_t* __restrict__ exps, int M, int B) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(M) * B) return;
+  const int b = idx % B;
+  const int m = idx / B;
+  exps[idx] = atoms[(static_cast<size_t>(m >> 7) * atoms_k + (b >> 2)) * 512 + (m & 31) * 16 + ((m & 127) >> 5) * 4 + (b & 3)];
+}
+
+}  // namespace w4a4

@@ -16,10 +16,14 @@
 // not care about order), so the lane's 16 channels are used as-is as A-fragment slots and the L1
 // fragments are laid out at pack time to match (see l1_fragment_channel()).
 //
-// Code output, two formats (template parameter BYTES):
-//   BYTES = true   one E4M3 byte per code, row-major [M, K]: the tensor-core operand of kernel 2 as it is
-//                  (fp8_codes.cuh), fetched by TMA straight into the swizzled operand tile;
-//   BYTES = false  nibble-packed, half the bytes, for callers that want the compact form.
+// Code output, three formats (template parameter FORMAT):
+//   kCodesE4M3    one E4M3 byte per code, row-major [M, K]: the tensor-core operand of kernel 2 as it is
+//                 (fp8_codes.cuh), fetched by TMA straight into the swizzled operand tile;
+//   kCodesPacked  nibble-packed INT4, half the bytes, for callers that want the compact form;
+//   kCodesMxfp4   the MXFP4 variant of the layer (OCP MX v1.0: E2M1 elements, one E8M0 scale per 32 channels,
+//                 shared exponent floor(log2(rho * block maximum)) - 2): two codes per byte, row-major
+//                 [M, K/2], and the scale bytes in the 512-byte atoms the block-scaled tensor-core
+//                 instruction wants in TMEM (see mx_gemm_kernel.cuh).
 // Packed activation layout: per row, per 32 consecutive channels
 // [32c, 32c+32) one 16-byte chunk of four 32-bit words; word w, byte b holds channel 32c + 4w + b in
 // its LOW nibble and channel 32c + 16 + 4w + b in its HIGH nibble (two's complement nibbles).  With
@@ -35,6 +39,7 @@
 
 namespace w4a4 {
 
+constexpr int kCodesPacked = 0, kCodesE4M3 = 1, kCodesMxfp4 = 2;
 constexpr int kQuantRows = 16;      // token rows per CTA
 // Warps per CTA (16 rows each).  Small CTAs spread evenly over the 148 SMs; the widest rank shares its
 // larger L1 fragments among more warps.
@@ -151,7 +156,45 @@ __device__ __forceinline__ uint2 quantize16(const float* xh, float is) {
   return make_uint2(w0 ^ 0x88888888u, w1 ^ 0x88888888u);  // offset-binary -> two's complement nibbles
 }
 
-template <int R, int WARPS, bool BYTES>
+// Eight FP32 values -> eight E2M1 codes (round to nearest even, saturating at +-6), element 0 in the lowest nibble.
+__device__ __forceinline__ uint32_t e2m1x8(const float* v) {
+  uint32_t r;
+  asm("{\n"
+      ".reg .b8 t0, t1, t2, t3;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n"
+      "mov.b32 %0, {t0, t1, t2, t3};\n"
+      "}"
+      : "=r"(r)
+      : "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]));
+  return r;
+}
+
+// MXFP4 conversion of the lane's 16 values of one row; they all lie in one 32-channel block, whose other half the
+// neighbouring lane holds.  Returns the E8M0 exponent byte; packed codes in lo (elements 0..7) and hi (8..15).
+__device__ __forceinline__ uint32_t mxfp4_block16(const float* xh, float rho, uint32_t& lo, uint32_t& hi) {
+  float a0 = fmaxf(fabsf(xh[0]), fabsf(xh[1])), a1 = fmaxf(fabsf(xh[2]), fabsf(xh[3]));
+#pragma unroll
+  for (int e = 4; e < 16; e += 2) {
+    a0 = fmaxf(a0, fabsf(xh[e]));
+    a1 = fmaxf(a1, fabsf(xh[e + 1]));
+  }
+  float a = fmaxf(a0, a1);
+  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+  const uint32_t field = (__float_as_uint(__fmul_rn(rho, a)) >> 23) & 0xffu;   // exponent of the clip threshold (Eq. 8)
+  const uint32_t ex = field > 2u ? field - 2u : 0u;                            // minus the exponent of E2M1's top binade
+  const float inv = __uint_as_float((254u - ex) << 23);                        // 2^(127 - ex): exact scaling
+  float v[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) v[e] = __fmul_rn(xh[e], inv);
+  lo = e2m1x8(v);
+  hi = e2m1x8(v + 8);
+  return ex;
+}
+
+template <int R, int WARPS, int FORMAT>
 __global__ void __launch_bounds__(32 * WARPS)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
@@ -237,13 +280,36 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     smooth8(cb0, l0, l1, xhB);
     smooth8(cb1, l4, l5, xhB + 8);
 
+    if constexpr (FORMAT == kCodesMxfp4) {
+      // `scales` is the scale-byte workspace here: per 128-row block and per 4 scale blocks (128 channels) one
+      // 512-byte atom, byte (row % 32) * 16 + (row % 128 / 32) * 4 + (scale block % 4); scales_ld = atoms per row block.
+      uint32_t loA, hiA, loB, hiB;
+      const uint32_t exA = mxfp4_block16(xhA, rho, loA, hiA), exB = mxfp4_block16(xhB, rho, loB, hiB);
+      uint8_t* ca = codes + static_cast<size_t>(rowA) * (K >> 1) + 32 * g + (coff >> 1);
+      uint8_t* cb = codes + static_cast<size_t>(rowB) * (K >> 1) + 32 * g + (coff >> 1);
+      if (okA) {
+        *reinterpret_cast<uint32_t*>(ca) = loA;
+        *reinterpret_cast<uint32_t*>(ca + 8) = hiA;
+      }
+      if (okB) {
+        *reinterpret_cast<uint32_t*>(cb) = loB;
+        *reinterpret_cast<uint32_t*>(cb + 8) = hiB;
+      }
+      if ((qj & 1) == 0) {
+        uint8_t* sf = reinterpret_cast<uint8_t*>(scales);
+        const int sb = 2 * g + (qj >> 1);  // scale block of this lane's channels
+        const size_t atom_col = static_cast<size_t>(sb >> 2) * 512 + (sb & 3);
+        if (okA) sf[(static_cast<size_t>(rowA >> 7) * scales_ld) * 512 + atom_col + (rowA & 31) * 16 + ((rowA & 127) >> 5) * 4] = static_cast<uint8_t>(exA);
+        if (okB) sf[(static_cast<size_t>(rowB >> 7) * scales_ld) * 512 + atom_col + (rowB & 31) * 16 + ((rowB & 127) >> 5) * 4] = static_cast<uint8_t>(exB);
+      }
+    } else {
     // Even lanes of the quad derive row A's scale, odd lanes row B's; one shuffle shares the reciprocals.
     const float aA = quad_absmax16(xhA), aB = quad_absmax16(xhB);
     float s_mine, is_mine;
     group_scale(rho, (qj & 1) ? aB : aA, s_mine, is_mine);
     const float is_other = __shfl_xor_sync(0xffffffffu, is_mine, 1);
     const float isA = (qj & 1) ? is_other : is_mine, isB = (qj & 1) ? is_mine : is_other;
-    if constexpr (BYTES) {
+    if constexpr (FORMAT == kCodesE4M3) {
       const uint4 bA = quantize16_bytes(xhA, isA);
       const uint4 bB = quantize16_bytes(xhB, isB);
       uint8_t* ca = codes + static_cast<size_t>(rowA) * K + 64 * g + coff;
@@ -266,6 +332,7 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     // Scales are stored group-major ([G][scales_ld]): kernel 2 fetches a (2 groups x 128 rows) block by TMA.
     if (qj == 0 && okA) scales[static_cast<size_t>(g) * scales_ld + rowA] = s_mine;
     if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = s_mine;
+    }
 
     if constexpr (NT > 0) {
       // Fragment storage: [i][n-tile pair][lane] as uint4 = (b0, b1) of n-tile 2p, (b0, b1) of n-tile 2p + 1.

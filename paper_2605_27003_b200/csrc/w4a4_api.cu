@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "gemm_kernel.cuh"
+#include "host_common.h"
 #include "quantize_kernel.cuh"
 
 namespace w4a4 {
@@ -118,32 +119,6 @@ __global__ void decode_t_kernel(const uint16_t* __restrict__ thl, float* __restr
 using namespace w4a4;
 
 // ------------------------------------------------------------------------------------ host objects
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-struct w4a4_ctx {
-  int device = 0;
-  int max_M = 0, max_K = 0, max_r = 0;
-  uint8_t* codes = nullptr;   // [max_M, K] activation codes, one E4M3 byte each (pitch K of the running layer)
-  float* scales = nullptr;    // [K/64, scales_ld] group-major activation scales
-  int scales_ld = 0;          // max_M rounded up to a multiple of 4 (16-byte rows for TMA)
-  uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
-  uint8_t* b8 = nullptr;      // [N, K] E4M3 image of the running layer's weight codes (rewritten by every forward)
-  size_t b8_bytes = 0;        // grows to the largest N x K packed on this context
-  int* d_err = nullptr;       // device error word
-  size_t bytes = 0;
-  int num_sms = 0;
-  EncodeTiledFn encode = nullptr;
-  // Host-buffer forward (w4a4_linear_forward_host): staging buffers, copy streams and events.
-  int host_chunk_rows = 0, host_max_N = 0;
-  uint16_t* hx[2] = {nullptr, nullptr};  // device staging of an activation chunk (double buffered)
-  uint16_t* hy[2] = {nullptr, nullptr};  // device staging of an output chunk
-  cudaStream_t s_h2d = nullptr, s_compute = nullptr, s_d2h = nullptr;
-  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
-  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
-};
-
 struct ExpertData {
   uint8_t* bpacked = nullptr;  // [N, K/2]
   float* wscale = nullptr;     // [G, N]
@@ -165,46 +140,6 @@ struct w4a4_layer {
 
 namespace {
 
-struct DeviceGuard {
-  int prev = -1;
-  bool ok = true;
-  explicit DeviceGuard(int dev) {
-    if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
-    if (ok && prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-  }
-  ~DeviceGuard() {
-    int cur = -1;
-    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
-  }
-};
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-template <typename T>
-w4a4_status_t dev_alloc(T** p, size_t count, size_t* tally) {
-  *p = nullptr;
-  if (count == 0) return W4A4_OK;
-  void* q = nullptr;
-  if (cudaMalloc(&q, count * sizeof(T)) != cudaSuccess) {
-    cudaGetLastError();
-    return W4A4_ERR_ALLOC;
-  }
-  *p = static_cast<T*>(q);
-  if (tally) *tally += count * sizeof(T);
-  return W4A4_OK;
-}
-
-bool encode_2d(EncodeTiledFn fn, CUtensorMap* tm, CUtensorMapDataType dt, size_t elem, void* base, uint64_t inner,
-               uint64_t outer, uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle sw) {
-  const cuuint64_t dims[2] = {inner, outer};
-  const cuuint64_t strides[1] = {pitch_bytes};
-  const cuuint32_t box[2] = {box_inner, box_outer};
-  const cuuint32_t es[2] = {1, 1};
-  (void)elem;
-  return fn(tm, dt, 2, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 void free_expert(ExpertData& e) {
   cudaFree(e.bpacked);
   cudaFree(e.wscale);
@@ -215,20 +150,6 @@ void free_expert(ExpertData& e) {
   e = ExpertData();
 }
 
-// Brings `count` elements at `src` (host or device) into a fresh device staging buffer when needed.
-template <typename T>
-w4a4_status_t stage_in(const T* src, size_t count, bool on_device, const T** dev, T** owned) {
-  *owned = nullptr;
-  if (on_device) {
-    *dev = src;
-    return W4A4_OK;
-  }
-  w4a4_status_t st = dev_alloc(owned, count, nullptr);
-  if (st != W4A4_OK) return st;
-  if (cudaMemcpy(*owned, src, count * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return W4A4_ERR_CUDA;
-  *dev = *owned;
-  return W4A4_OK;
-}
 
 w4a4_status_t check_forward_args(w4a4_handle_t h, const void* X, int M, int expert_id, int bin,
                                  const float* clip_table, bool need_x) {
@@ -257,7 +178,7 @@ w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expe
   const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define W4A4_LAUNCH_Q(R)                                                                                         \
-  quantize_kernel<R, quantize_warps(R), true><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
+  quantize_kernel<R, quantize_warps(R), kCodesE4M3><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
                                                  ctx->scales, ctx->scales_ld, ctx->t_hilo)
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
@@ -390,7 +311,7 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
       cudaMemset(ctx->t_hilo, 0, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8) * sizeof(uint16_t)) != cudaSuccess)
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) {
-    cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesE4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          static_cast<int>(quantize_smem_bytes(64)));
     cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
@@ -412,6 +333,7 @@ void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
   DeviceGuard guard(ctx->device);
   cudaFree(ctx->codes);
   cudaFree(ctx->b8);
+  cudaFree(ctx->mx_sfa);
   cudaFree(ctx->scales);
   cudaFree(ctx->t_hilo);
   cudaFree(ctx->d_err);
@@ -781,3 +703,5 @@ w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx) {
 }
 
 }  // extern "C"
+
+#include "w4a4_mx_api.cuh"

@@ -1,0 +1,285 @@
+// C-ABI entry points of the MXFP4 variant of the layer (included at the end of w4a4_api.cu, whose set-up
+// kernels and host helpers it shares).  Same structure as the INT4 path: pack once, then two kernels per forward.
+#pragma once
+
+#include "mx_gemm_kernel.cuh"
+
+struct MxExpertData {
+  uint8_t* bpacked = nullptr;  // [N, K/2] two E2M1 codes per byte
+  uint8_t* sfb = nullptr;      // weight scale atoms [N/128][K/128][512]
+  float* rlam = nullptr;       // [K]
+  uint2* l1frag = nullptr;
+  uint16_t* l2dup = nullptr;   // [N, 2r]
+  float* bias = nullptr;       // [N] or null
+  CUtensorMap tmB, tmL2;
+};
+
+struct w4a4_mx_layer {
+  w4a4_ctx* ctx = nullptr;
+  int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0;
+  std::vector<MxExpertData> experts;
+  CUtensorMap tmA, tmT;
+  size_t bytes = 0;
+};
+
+namespace {
+
+void mx_free_expert(MxExpertData& e) {
+  cudaFree(e.bpacked);
+  cudaFree(e.sfb);
+  cudaFree(e.rlam);
+  cudaFree(e.l1frag);
+  cudaFree(e.l2dup);
+  cudaFree(e.bias);
+  e = MxExpertData();
+}
+
+size_t mx_sfa_bytes(int max_M, int K) { return static_cast<size_t>((max_M + 127) / 128) * (K / 128) * 512; }
+
+w4a4_status_t mx_check_forward_args(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int bin,
+                                    const float* clip_table, bool need_x) {
+  if (!h || !h->ctx) return W4A4_ERR_INVALID_ARG;
+  if (M < 0 || expert_id < 0 || expert_id >= h->E) return W4A4_ERR_INVALID_ARG;
+  if (M > h->ctx->max_M) return W4A4_ERR_SHAPE;
+  if (need_x) {
+    if (bin < 0 || bin >= h->B) return W4A4_ERR_INVALID_ARG;
+    if (M > 0 && (!X || !aligned16(X))) return W4A4_ERR_INVALID_ARG;
+    if (!clip_table) return W4A4_ERR_INVALID_ARG;
+  }
+  return W4A4_OK;
+}
+
+w4a4_status_t mx_launch_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int bin, const float* clip_table,
+                                 cudaStream_t stream) {
+  if (M == 0) return W4A4_OK;
+  w4a4_ctx* ctx = h->ctx;
+  const MxExpertData& e = h->experts[expert_id];
+  const int clip_index = (expert_id * h->L + h->layer_id) * h->B + bin;
+  const int rows_per_cta = kQuantRows * quantize_warps(h->r);
+  const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
+  const uint16_t* x = static_cast<const uint16_t*>(X);
+  float* sf = reinterpret_cast<float*>(ctx->mx_sfa);
+#define W4A4_LAUNCH_MXQ(R)                                                                                             \
+  quantize_kernel<R, quantize_warps(R), kCodesMxfp4><<<grid, block, quantize_smem_bytes(R), stream>>>(                 \
+      x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, sf, h->K / 128, ctx->t_hilo)
+  switch (h->r) {
+    case 0: W4A4_LAUNCH_MXQ(0); break;
+    case 16: W4A4_LAUNCH_MXQ(16); break;
+    case 32: W4A4_LAUNCH_MXQ(32); break;
+    case 64: W4A4_LAUNCH_MXQ(64); break;
+    default: return W4A4_ERR_SHAPE;
+  }
+#undef W4A4_LAUNCH_MXQ
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream) {
+  if (M == 0) return W4A4_OK;
+  w4a4_ctx* ctx = h->ctx;
+  const MxExpertData& e = h->experts[expert_id];
+  MxGemmParams p;
+  p.bias = e.bias;
+  p.Y = static_cast<uint16_t*>(Y);
+  p.sfa = ctx->mx_sfa;
+  p.sfb = e.sfb;
+  p.M = M;
+  p.N = h->N;
+  p.K = h->K;
+  p.r = h->r;
+  p.tiles_m = (M + kBM - 1) / kBM;
+  p.tiles_n = h->N / kBN;
+  p.err = ctx->d_err;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
+  const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;  // unused when r == 0
+  const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
+  mx_gemm_kernel<<<grid, block, kMxSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+void w4a4_mx_destroy(w4a4_mx_handle_t h) {
+  if (!h) return;
+  if (h->ctx) {
+    DeviceGuard guard(h->ctx->device);
+    for (auto& e : h->experts) mx_free_expert(e);
+  }
+  delete h;
+}
+
+size_t w4a4_mx_handle_bytes(w4a4_mx_handle_t h) { return h ? h->bytes : 0; }
+
+w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* d, w4a4_mx_handle_t* out) {
+  if (!out) return W4A4_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !d) return W4A4_ERR_INVALID_ARG;
+  if (d->K <= 0 || d->K % kMxBK != 0 || d->N <= 0 || d->N % kBN != 0) return W4A4_ERR_SHAPE;
+  if (!(d->r == 0 || d->r == 16 || d->r == 32 || d->r == 64)) return W4A4_ERR_SHAPE;
+  if (d->K > ctx->max_K || d->r > ctx->max_r) return W4A4_ERR_SHAPE;
+  if (d->num_experts < 1 || d->num_bins < 1 || d->num_layers < 1 || d->layer_id < 0 || d->layer_id >= d->num_layers)
+    return W4A4_ERR_INVALID_ARG;
+  if (!d->wcodes || !d->wexps || !d->lambda || (d->r > 0 && (!d->L1 || !d->L2))) return W4A4_ERR_INVALID_ARG;
+  for (int e = 0; e < d->num_experts; ++e) {
+    if (!d->wcodes[e] || !d->wexps[e] || !d->lambda[e] || (d->r > 0 && (!d->L1[e] || !d->L2[e]))) return W4A4_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+
+  w4a4_mx_layer* h = new (std::nothrow) w4a4_mx_layer();
+  if (!h) return W4A4_ERR_ALLOC;
+  h->ctx = ctx;
+  h->K = d->K;
+  h->N = d->N;
+  h->r = d->r;
+  h->E = d->num_experts;
+  h->B = d->num_bins;
+  h->L = d->num_layers;
+  h->layer_id = d->layer_id;
+  h->experts.resize(d->num_experts);
+  const int K = d->K, N = d->N, r = d->r, G = K / 64;
+  const bool dev = d->pointers_on_device != 0;
+  w4a4_status_t st = W4A4_OK;
+
+  // The activation scale atoms live in the context (zero-filled once: rows past M of the last row block are
+  // read by the tensor core and must not hold E8M0's NaN byte).
+  if (!ctx->mx_sfa) {
+    const size_t nb = mx_sfa_bytes(ctx->max_M, ctx->max_K);
+    st = dev_alloc(&ctx->mx_sfa, nb, &ctx->bytes);
+    if (st == W4A4_OK && cudaMemset(ctx->mx_sfa, 0, nb) != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK)
+      cudaFuncSetAttribute(mx_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMxSmemBytes));
+    if (st == W4A4_OK)
+      cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesMxfp4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(quantize_smem_bytes(64)));
+  }
+  int* d_bad = nullptr;
+  if (st == W4A4_OK) st = dev_alloc(&d_bad, 1, nullptr);
+  if (st == W4A4_OK && cudaMemset(d_bad, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
+
+  for (int ei = 0; st == W4A4_OK && ei < d->num_experts; ++ei) {
+    MxExpertData& e = h->experts[ei];
+    st = dev_alloc(&e.bpacked, static_cast<size_t>(N) * (K / 2), &h->bytes);
+    if (st == W4A4_OK) st = dev_alloc(&e.sfb, static_cast<size_t>(N / 128) * (K / 128) * 512, &h->bytes);
+    if (st == W4A4_OK) st = dev_alloc(&e.rlam, static_cast<size_t>(K), &h->bytes);
+    if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l1frag, static_cast<size_t>(G) * 4 * (r / 8) * 32, &h->bytes);
+    if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l2dup, static_cast<size_t>(N) * 2 * r, &h->bytes);
+    const float* bias_src = d->bias ? d->bias[ei] : nullptr;
+    if (st == W4A4_OK && bias_src) st = dev_alloc(&e.bias, static_cast<size_t>(N), &h->bytes);
+    if (st != W4A4_OK) break;
+    const cudaMemcpyKind kind = dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    if (bias_src && cudaMemcpy(e.bias, bias_src, sizeof(float) * N, kind) != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st != W4A4_OK) break;
+
+    const uint8_t *c_dev = nullptr, *x_dev = nullptr;
+    uint8_t *c_own = nullptr, *x_own = nullptr;
+    const float* lam_dev = nullptr;
+    float* lam_own = nullptr;
+    const uint16_t *l1_dev = nullptr, *l2_dev = nullptr;
+    uint16_t *l1_own = nullptr, *l2_own = nullptr;
+    st = stage_in(d->wcodes[ei], static_cast<size_t>(K) * N, dev, &c_dev, &c_own);
+    if (st == W4A4_OK) st = stage_in(d->wexps[ei], static_cast<size_t>(K / 32) * N, dev, &x_dev, &x_own);
+    if (st == W4A4_OK) st = stage_in(d->lambda[ei], static_cast<size_t>(K), dev, &lam_dev, &lam_own);
+    if (st == W4A4_OK && r > 0) st = stage_in(d->L1[ei], static_cast<size_t>(K) * r, dev, &l1_dev, &l1_own);
+    if (st == W4A4_OK && r > 0) st = stage_in(d->L2[ei], static_cast<size_t>(r) * N, dev, &l2_dev, &l2_own);
+    if (st == W4A4_OK) {
+      reciprocal_kernel<<<(K + 255) / 256, 256>>>(lam_dev, e.rlam, K);
+      mx_pack_weight_kernel<<<dim3((N + 127) / 128, K / 32), 128>>>(c_dev, e.bpacked, K, N, d_bad);
+      const size_t ns = static_cast<size_t>(K / 32) * N;
+      mx_pack_wscale_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256>>>(x_dev, e.sfb, K, N, d_bad);
+      if (r > 0) {
+        const size_t nf = static_cast<size_t>(G) * 4 * (r / 8) * 32;
+        l1_fragment_kernel<<<static_cast<unsigned>((nf + 255) / 256), 256>>>(l1_dev, e.l1frag, K, r);
+        const size_t nl = static_cast<size_t>(N) * 2 * r;
+        l2_dup_kernel<<<static_cast<unsigned>((nl + 255) / 256), 256>>>(l2_dev, e.l2dup, r, N);
+      }
+      if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) st = W4A4_ERR_CUDA;
+    }
+    cudaFree(c_own);
+    cudaFree(x_own);
+    cudaFree(lam_own);
+    cudaFree(l1_own);
+    cudaFree(l2_own);
+    if (st != W4A4_OK) break;
+    if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, 128, kBN,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+      st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK && r > 0 &&
+        !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kBN,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+      st = W4A4_ERR_CUDA;
+  }
+  if (st == W4A4_OK) {
+    int bad = 0;
+    if (cudaMemcpy(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) st = W4A4_ERR_CUDA;
+    else if (bad) st = W4A4_ERR_INVALID_ARG;  // a code above 15 or the NaN scale byte
+  }
+  cudaFree(d_bad);
+  if (st == W4A4_OK &&
+      !encode_2d(ctx->encode, &h->tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->codes, K / 2, ctx->max_M, K / 2, 128, kBM,
+                 CU_TENSOR_MAP_SWIZZLE_128B))
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && r > 0 &&
+      !encode_2d(ctx->encode, &h->tmT, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo, 2 * r, ctx->max_M, 4 * r, 64,
+                 kBM, CU_TENSOR_MAP_SWIZZLE_128B))
+    st = W4A4_ERR_CUDA;
+  if (st != W4A4_OK) {
+    cudaGetLastError();
+    w4a4_mx_destroy(h);
+    return st;
+  }
+  *out = h;
+  return W4A4_OK;
+}
+
+w4a4_status_t w4a4_mx_quantize_activations(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                           const float* clip_table, void* stream) {
+  w4a4_status_t st = mx_check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  DeviceGuard guard(h->ctx->device);
+  return mx_launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, static_cast<cudaStream_t>(stream));
+}
+
+w4a4_status_t w4a4_mx_gemm_from_workspace(w4a4_mx_handle_t h, int M, int expert_id, void* Y, void* stream) {
+  w4a4_status_t st = mx_check_forward_args(h, nullptr, M, expert_id, 0, nullptr, false);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!Y || !aligned16(Y))) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(h->ctx->device);
+  return mx_launch_gemm(h, M, expert_id, Y, static_cast<cudaStream_t>(stream));
+}
+
+w4a4_status_t w4a4_mx_linear_forward(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                     const float* clip_table, void* Y, void* stream) {
+  w4a4_status_t st = mx_check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!Y || !aligned16(Y))) return W4A4_ERR_INVALID_ARG;
+  DeviceGuard guard(h->ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = mx_launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
+  if (st != W4A4_OK) return st;
+  return mx_launch_gemm(h, M, expert_id, Y, s);
+}
+
+w4a4_status_t w4a4_mx_debug_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
+                                     const float* clip_table, uint8_t* codes, uint8_t* exps, float* T, void* stream) {
+  w4a4_status_t st = mx_check_forward_args(h, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  if (M > 0 && (!codes || !exps)) return W4A4_ERR_INVALID_ARG;
+  if (M == 0) return W4A4_OK;
+  DeviceGuard guard(h->ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = mx_launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
+  if (st != W4A4_OK) return st;
+  const size_t nc = static_cast<size_t>(M) * h->K, ns = static_cast<size_t>(M) * (h->K / 32);
+  mx_decode_codes_kernel<<<static_cast<unsigned>((nc + 255) / 256), 256, 0, s>>>(h->ctx->codes, codes, M, h->K);
+  mx_decode_exps_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256, 0, s>>>(h->ctx->mx_sfa, h->K / 128, exps, M, h->K / 32);
+  if (T && h->r > 0) {
+    const size_t nt = static_cast<size_t>(M) * h->r;
+    decode_t_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, s>>>(h->ctx->t_hilo, T, M, h->r);
+  }
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -103,7 +103,7 @@ extern "C" w4a4_status_t w4a4_quantize_noalloc(const void* X, int M, int K, cons
   // Every scratch byte that is read below is written first by this same call: nothing has to start at zero.
   noalloc_reciprocal_kernel<<<(K + 255) / 256, 256, 0, s>>>(lambda, rlam, K);
   constexpr int kWarps = w4a4::quantize_warps(0);
-  w4a4::quantize_kernel<0, kWarps, false><<<(M + w4a4::kQuantRows * kWarps - 1) / (w4a4::kQuantRows * kWarps), 32 * kWarps,
+  w4a4::quantize_kernel<0, kWarps, w4a4::kCodesPacked><<<(M + w4a4::kQuantRows * kWarps - 1) / (w4a4::kQuantRows * kWarps), 32 * kWarps,
                                      w4a4::quantize_smem_bytes(0), s>>>(
       static_cast<const uint16_t*>(X), M, K, rlam, clip_table, clip_index, nullptr, ws_codes, ws_scales, ld, nullptr);
   const size_t nc = static_cast<size_t>(M) * K, ns = static_cast<size_t>(M) * G;
