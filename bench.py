@@ -332,6 +332,74 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                           best_point=best, gpu_launches=3 * args.steps * len(rows))), flush=True)
 
 
+def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
+    """The MXFP4 variant of the layer (E2M1 elements, E8M0 block scales applied inside the tensor core) on the
+    shape of one of the single-layer workloads: `--workload mxfp4_attn_proj | mxfp4_ffn_up | mxfp4_ffn_down`."""
+    if rank != 0:
+        return
+    name = args.workload[len("mxfp4_"):]
+    shp = gen.CONFIG_SHAPES[name]
+    M, K, N, r = shp["M"], shp["K"], shp["N"], shp["r"]
+    num_bins, n_buf = 8, 4
+    dist = "gelu" if name == "ffn_down" else "normal"
+    gain = 80.0 if name == "ffn_down" else 50.0
+    idx = gen.outlier_channels(K, 0.01, 2)
+    sig = (lambda b: 1.0) if dist == "gelu" else gen.sigma_for_bin
+    lay = gen.make_layer_mx_direct(K, N, r, seed=2001, device=dev)
+    bins = [b % num_bins for b in range(n_buf)]
+    xs = [gen.make_activations(M, K, sigma=sig(b), outlier_idx=idx, outlier_gain=gain, dist=dist, seed=2002 + i, device=dev)
+          for i, b in enumerate(bins)]
+    clip = gen.make_clip_table(1, 1, num_bins, [(0.6, 1.0)], seed=2).to(dev)
+    ctx = w4.Context(local_rank, M, K, r)
+    layer = w4.MxLayer(ctx, [lay], num_bins=num_bins)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+    for i in range(max(3, args.warmup)):
+        w4.w4a4_mx_linear_forward(layer.ptr, xs[i % n_buf], M, 0, bins[i % n_buf], clip, Y, stream)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        w4.w4a4_mx_linear_forward(layer.ptr, xs[i % n_buf], M, 0, bins[i % n_buf], clip, Y, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(min(args.steps, 50))]
+    for i, e in enumerate(ev):
+        e[0].record(stream)
+        w4.w4a4_mx_quantize_activations(layer.ptr, xs[i % n_buf], M, 0, bins[i % n_buf], clip, stream)
+        e[1].record(stream)
+        w4.w4a4_mx_gemm_from_workspace(layer.ptr, M, 0, Y, stream)
+        e[2].record(stream)
+    torch.cuda.synchronize()
+    ctx.check()
+    tq = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    tg = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    ops = 2.0 * M * K * N
+    fp4_peak = 4.0 * peaks["bf16_sustained"]  # dense FP4 = 4 x dense BF16 (nominal ratio 9 / 2.25)
+    gemm_tops = ops / (tg * 1e-3) / 1e12
+    q_bytes = M * (2.0 * K + K / 2.0 + K / 32.0 + 4.0 * r)  # X read, packed codes, scale bytes, T hi | lo
+    print(json.dumps(dict(
+        metric=METRIC, value=ops / (ms * 1e-3) / 1e12, unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e2m1 x e8m0 (mxfp4)",
+        data="synthetic",
+        config=dict(workload=args.workload, M=M, K=K, N=N, r=r, block=32, experts=1, bins=num_bins,
+                    l2="inputs larger than L2: 4 rotating activation buffers of %.0f MB" % (M * K * 2 / 1e6)),
+        roofline=dict(bound="tensor", achieved=gemm_tops, peak=fp4_peak, unit="TOP/s", frac=gemm_tops / fp4_peak,
+                      traffic=None, kernel="mx_gemm_kernel", ms=tg,
+                      peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 4 "
+                                  "(nominal FP4:BF16 ratio)", frac_of_nominal_9000=gemm_tops / 9000.0),
+        roofline_quantize=dict(bound="hbm", achieved=q_bytes / (tq * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                               frac=q_bytes / (tq * 1e-3) / 1e9 / peaks["hbm_gbs"], kernel="quantize_kernel (MXFP4 format)",
+                               ms=tq, algorithmic_bytes=q_bytes, peak_source=peaks["source"]),
+        kernel_ms=dict(quantize_mean=tq, gemm_mean=tg), e2e=None, gpu_launches=2 * args.steps, clocks=clocks)), flush=True)
+    layer.close()
+    ctx.close()
+
+
 def run_clip_search(args, w4, dev, local_rank, rank, peaks):
     """Clipping-ratio search (Eq. 10) at the attention-projection shape: six candidates, two calibration samples
     per search; every candidate runs the real forward with the squared error fused into the GEMM epilogue."""
@@ -383,7 +451,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search"])
+    ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search", "mxfp4_attn_proj", "mxfp4_ffn_up",
+                                                            "mxfp4_ffn_down"])
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -422,6 +491,9 @@ def main():
         return
     if args.workload == "sweep":
         run_sweep(args, w4, dev, local_rank, rank, peaks)
+        return
+    if args.workload.startswith("mxfp4_"):
+        run_mxfp4(args, w4, dev, local_rank, rank, peaks)
         return
     if args.workload == "clip_search":
         run_clip_search(args, w4, dev, local_rank, rank, peaks)
