@@ -7,19 +7,22 @@
 // tensor core and accumulates in FP32, so -- unlike the INT4 kernel -- nothing is rescaled on the CUDA cores and
 // the whole K extent accumulates into one TMEM tile; the epilogue runs once per output tile.
 //
-// Persistent kernel, one CTA per SM, 128 x 128 output tiles, column tile fastest.  Warp roles:
-//   warp 0      producer (one lane): per stage of 256 K elements one TMA each for the packed A and B tiles
-//               (128 rows x 128 bytes, 128-byte swizzle) and one bulk copy each for their scale bytes (1 KiB:
-//               two 512-byte atoms, the layout the tensor core wants); the BF16 low-rank operands T and L2
-//               go through the same ring first.
-//   warp 1      MMA issuer (one lane): per stage four tcgen05.cp (scale atoms, shared memory -> TMEM: 32 lanes x
-//               128 bits, replicated to the four lane quarters) and four tcgen05.mma kind::mxf4 (K = 64 each,
-//               two scale blocks per row, selected by the scale-factor id 0 / 2 inside the 4-byte TMEM column);
-//               kind::f16 for [T_hi | T_lo] [L2 | L2]^T into the same accumulator first.  tcgen05.cp and
-//               tcgen05.mma of one thread execute in issue order, so one TMEM scale region serves every stage.
+// Persistent kernel, one CTA per SM, 128 x 256 output tiles, column tile fastest.  At the FP4 rate the tensor
+// core consumes operands faster than L2 and the shared-memory port deliver them, so the tile is as wide as TMEM
+// allows (operand bytes per MAC fall by a quarter against 128 x 128).  Warp roles:
+//   warp 0      producer (one lane): per stage of 256 K elements one TMA each for the packed A tile (128 rows x
+//               128 bytes) and B tile (256 rows x 128 bytes), 128-byte swizzle, and bulk copies for their scale
+//               bytes (1 KiB per 128 rows: two 512-byte atoms, the layout the tensor core wants); the BF16
+//               low-rank operands T and L2 go through the same ring first.
+//   warp 1      MMA issuer (one lane): per stage six tcgen05.cp (scale atoms, shared memory -> TMEM: 32 lanes x
+//               128 bits, replicated to the four lane quarters) and four tcgen05.mma kind::mxf4 (128 x 256, K = 64
+//               each: two scale blocks per row, selected by the scale-factor id 0 / 2 inside the 4-byte TMEM
+//               column); kind::f16 for [T_hi | T_lo] [L2 | L2]^T into the same accumulator first.  tcgen05.cp
+//               and tcgen05.mma of one thread execute in issue order, so one TMEM scale region serves every stage.
 //   warp 2      TMEM allocation / release.
-//   warps 4-7   epilogue: TMEM (32x32b loads, a token row per thread) + bias -> BF16 -> global.  Two accumulator
-//               buffers in TMEM, so the epilogue of a tile overlaps the MMAs of the next.
+//   warps 4-11  epilogue: TMEM (32x32b loads, a token row per thread, 128 columns per warp) + bias -> BF16 ->
+//               global.  One accumulator (256 columns) plus the scale columns fill TMEM, so the MMA warp waits
+//               for the epilogue to drain it (the loads only: ~2 % of a tile's time) before the next tile.
 //
 // Every wait is bounded exactly as in gemm_kernel.cuh (whose Ring / bounded_wait helpers are used here).
 #pragma once
@@ -32,17 +35,20 @@
 
 namespace w4a4 {
 
+constexpr int kMxBN = 256;                       // output tile columns
 constexpr int kMxBK = 256;                       // K elements per stage = 128 bytes per operand row
-constexpr int kMxStages = 6;
-constexpr int kMxThreads = 256;
-constexpr int kMxEpiWarp0 = 4, kMxEpiWarps = 4;
-constexpr uint32_t kMxOpTile = kBM * 128;        // 16 KiB (A and B tiles alike: kBM == kBN == 128 rows)
+constexpr int kMxStages = 4;
+constexpr int kMxThreads = 384;
+constexpr int kMxEpiWarp0 = 4, kMxEpiWarps = 8;
+constexpr uint32_t kMxATile = kBM * 128;         // 16 KiB
+constexpr uint32_t kMxBTile = kMxBN * 128;       // 32 KiB
 constexpr uint32_t kMxSfTile = 2 * 512;          // scale bytes of 128 rows x 8 blocks: two atoms
-constexpr uint32_t kMxStageBytes = 2 * kMxOpTile + 2 * kMxSfTile;
-constexpr uint32_t kMxNumBarriers = 2 * kMxStages + 4;
+constexpr uint32_t kMxStageBytes = kMxATile + kMxBTile + 3 * kMxSfTile;   // A, B, scales of A and of both halves of B
+constexpr uint32_t kMxNumBarriers = 2 * kMxStages + 2;
 constexpr uint32_t kMxSmemBytes = 1024 + kMxStages * kMxStageBytes + kMxNumBarriers * 8 + 16;
-constexpr uint32_t kMxTmemSfA = 256, kMxTmemSfB = 264;   // columns: accumulators 0..255, then 8 + 8 scale columns
-static_assert(kBM == 128 && kBN == 128, "the scale-factor atoms and the TMEM layout assume 128 x 128 tiles");
+constexpr uint32_t kMxTmemSfA = 256, kMxTmemSfB = 264;   // columns: accumulator 0..255, then 8 + 16 scale columns
+static_assert(kBM == 128, "the scale-factor atoms and the TMEM layout assume 128-row tiles");
+static_assert(kMxStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned");
 
 struct MxGemmParams {
   const float* bias;     // [N] or nullptr
@@ -100,8 +106,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t bar_full = bar_base;
   const uint32_t bar_empty = bar_full + 8 * kMxStages;
   const uint32_t bar_acc_full = bar_empty + 8 * kMxStages;
-  const uint32_t bar_acc_empty = bar_acc_full + 16;
-  const uint32_t misc_off = (bar_acc_empty + 16) - smem_base;
+  const uint32_t bar_acc_empty = bar_acc_full + 8;
+  const uint32_t misc_off = (bar_acc_empty + 8) - smem_base;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
 
@@ -118,10 +124,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(bar_full + 8 * i, 1);
       mbar_init(bar_empty + 8 * i, 1);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_acc_full + 8 * i, 1);
-      mbar_init(bar_acc_empty + 8 * i, kMxEpiWarps);
-    }
+    mbar_init(bar_acc_full, 1);
+    mbar_init(bar_acc_empty, kMxEpiWarps);
     mbar_fence_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmA);
@@ -141,50 +145,55 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t tmem_base = *tmem_slot;
   const bool live = (*s_abort == 0);
 
+  // Shared-memory stage: A tile | B tile (256 rows) | scale atoms of A | of B rows 0..127 | of B rows 128..255.
   if (live && warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ producer
     Ring<kMxStages> rg;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
       const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
-      const int m0 = tm * kBM, n0 = tn * kBN;
+      const int m0 = tm * kBM, n0 = tn * kMxBN;
+      const bool upper = n0 + 128 < p.N;  // does the tile's second 128-column half exist?
       for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
         ok = bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait);
         if (!ok) break;
         const uint32_t full = bar_full + 8 * rg.slot;
         const uint32_t dst = smem_base + rg.slot * kMxStageBytes;
         if (st < n_lr_stages) {
-          mbar_arrive_expect_tx(full, 2 * kMxOpTile);
+          mbar_arrive_expect_tx(full, kMxATile + kMxBTile);
           tma_load_2d(dst, &tmT, full, st * 64, m0);
-          tma_load_2d(dst + kMxOpTile, &tmL2, full, st * 64, n0);
+          tma_load_2d(dst + kMxATile, &tmL2, full, st * 64, n0);  // rows past N arrive as zeros
         } else {
           const int ks = st - n_lr_stages;
-          mbar_arrive_expect_tx(full, kMxStageBytes);
+          const uint32_t sf = dst + kMxATile + kMxBTile;
+          mbar_arrive_expect_tx(full, kMxATile + kMxBTile + (upper ? 3u : 2u) * kMxSfTile);
           tma_load_2d(dst, &tmA, full, ks * 128, m0);
-          tma_load_2d(dst + kMxOpTile, &tmB, full, ks * 128, n0);
-          bulk_load(dst + 2 * kMxOpTile, p.sfa + (static_cast<size_t>(tm) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
-          bulk_load(dst + 2 * kMxOpTile + kMxSfTile, p.sfb + (static_cast<size_t>(tn) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
+          tma_load_2d(dst + kMxATile, &tmB, full, ks * 128, n0);
+          bulk_load(sf, p.sfa + (static_cast<size_t>(tm) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
+          bulk_load(sf + kMxSfTile, p.sfb + (static_cast<size_t>(2 * tn) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
+          if (upper)
+            bulk_load(sf + 2 * kMxSfTile, p.sfb + (static_cast<size_t>(2 * tn + 1) * atoms_k + 2 * ks) * 512, kMxSfTile, full);
         }
         rg.advance();
       }
     }
   } else if (live && warp == 1 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
+    constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kMxBN);
     Ring<kMxStages> rg;
-    Ring<2> ab;
+    Ring<1> ab;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-      ok = bounded_wait<64>(bar_acc_empty + 8 * ab.slot, ab.parity ^ 1u, env, kErrMmaWait);
+      ok = bounded_wait<64>(bar_acc_empty, ab.parity ^ 1u, env, kErrMmaWait);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t d = tmem_base + ab.slot * kBN;
+      const uint32_t d = tmem_base;
       uint32_t accumulate = 0;
       for (int st = 0; ok && st < n_lr_stages + n_k_stages; ++st) {
         ok = bounded_wait<64>(bar_full + 8 * rg.slot, rg.parity, env, kErrMmaWait);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t a = smem_base + rg.slot * kMxStageBytes, b = a + kMxOpTile;
+        const uint32_t a = smem_base + rg.slot * kMxStageBytes, b = a + kMxATile;
         if (st < n_lr_stages) {
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk) {
@@ -192,17 +201,20 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             accumulate = 1;
           }
         } else {
-          const uint32_t sf = a + 2 * kMxOpTile;
+          // TMEM scale columns: A: 4 per K atom (one per 32 rows); B: 8 per K atom (256 rows).  The columns of
+          // a missing upper half keep whatever they held: they scale zero operands into columns never stored.
+          const uint32_t sf = b + kMxBTile;
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             tmem_cp_32x128b_warpx4(tmem_base + kMxTmemSfA + 4 * t, mx_sf_desc(sf + 512 * t));
-            tmem_cp_32x128b_warpx4(tmem_base + kMxTmemSfB + 4 * t, mx_sf_desc(sf + kMxSfTile + 512 * t));
+            tmem_cp_32x128b_warpx4(tmem_base + kMxTmemSfB + 8 * t, mx_sf_desc(sf + kMxSfTile + 512 * t));
+            tmem_cp_32x128b_warpx4(tmem_base + kMxTmemSfB + 8 * t + 4, mx_sf_desc(sf + 2 * kMxSfTile + 512 * t));
           }
 #pragma unroll
           for (int j = 0; j < 4; ++j) {  // bytes [32 j, 32 j + 32) of every row: scale blocks 2 j, 2 j + 1
             const uint32_t id = 2u * (j & 1);
-            umma_mxf4(d, umma_desc_k_sw128(a, 32 * j), umma_desc_k_sw128(b, 32 * j), mx_idesc(kBM, kBN, id, id),
-                      (tmem_base + kMxTmemSfA + 4 * (j >> 1)) | (id << 30), (tmem_base + kMxTmemSfB + 4 * (j >> 1)) | (id << 30),
+            umma_mxf4(d, umma_desc_k_sw128(a, 32 * j), umma_desc_k_sw128(b, 32 * j), mx_idesc(kBM, kMxBN, id, id),
+                      (tmem_base + kMxTmemSfA + 4 * (j >> 1)) | (id << 30), (tmem_base + kMxTmemSfB + 8 * (j >> 1)) | (id << 30),
                       accumulate);
             accumulate = 1;
           }
@@ -211,47 +223,55 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         rg.advance();
       }
       if (!ok) break;
-      umma_commit(bar_acc_full + 8 * ab.slot);
+      umma_commit(bar_acc_full);
       ab.advance();
     }
   } else if (live && warp >= kMxEpiWarp0) {
     // ------------------------------------------------------------------ epilogue
-    const int quarter = warp - kMxEpiWarp0;
-    Ring<2> ab;
+    // Warp ew: TMEM lanes 32 * (ew % 4) .. + 31 (token rows), columns 128 * (ew / 4) .. + 127.  The accumulator is
+    // read in two halves of 64 columns; the buffer goes back to the MMA warp as soon as the second half is in
+    // registers, before it is converted and stored.
+    const int ew = warp - kMxEpiWarp0;
+    const int quarter = ew & 3, half = ew >> 2;
+    Ring<1> ab;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-      const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+      const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kMxBN;
       const int row = m0 + 32 * quarter + lane;
-      ok = bounded_wait(bar_acc_full + 8 * ab.slot, ab.parity, env, kErrEpilogueWait);
+      ok = bounded_wait(bar_acc_full, ab.parity, env, kErrEpilogueWait);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + ab.slot * kBN;
-#pragma unroll 2
-      for (int c = 0; c < kBN / 16; ++c) {
-        uint32_t v[16];
-        tmem_ld_32x32b_x16(t_row + 16 * c, v);
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 128 * half;
+#pragma unroll
+      for (int part = 0; part < 2; ++part) {
+        uint32_t v[4][16];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x16(t_row + 64 * part + 16 * c, v[c]);
         tmem_wait_ld();
-        if (c == kBN / 16 - 1) {
-          // The whole accumulator is in registers or on its way out: hand the buffer back to the MMA warp.
+        if (part == 1) {
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_acc_empty + 8 * ab.slot);
+          if (lane == 0) mbar_arrive(bar_acc_empty);
         }
-        if (row < p.M) {
-          const int ch = n0 + 16 * c;
-          uint4 o[2];
-          uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+        const int ch0 = n0 + 128 * half + 64 * part;
+        if (row < p.M && ch0 < p.N) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-            __nv_bfloat162 lo = __floats2bfloat162_rn(__uint_as_float(v[4 * i]) + b4.x, __uint_as_float(v[4 * i + 1]) + b4.y);
-            __nv_bfloat162 hi = __floats2bfloat162_rn(__uint_as_float(v[4 * i + 2]) + b4.z, __uint_as_float(v[4 * i + 3]) + b4.w);
-            ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
-            ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
+          for (int c = 0; c < 4; ++c) {
+            const int ch = ch0 + 16 * c;
+            uint4 o[2];
+            uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+              __nv_bfloat162 lo = __floats2bfloat162_rn(__uint_as_float(v[c][4 * i]) + b4.x, __uint_as_float(v[c][4 * i + 1]) + b4.y);
+              __nv_bfloat162 hi = __floats2bfloat162_rn(__uint_as_float(v[c][4 * i + 2]) + b4.z, __uint_as_float(v[c][4 * i + 3]) + b4.w);
+              ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
+              ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
+            }
+            uint4* y = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch);
+            y[0] = o[0];
+            y[1] = o[1];
           }
-          uint4* y = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch);
-          y[0] = o[0];
-          y[1] = o[1];
         }
       }
       ab.advance();

@@ -87,7 +87,7 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   p.K = h->K;
   p.r = h->r;
   p.tiles_m = (M + kBM - 1) / kBM;
-  p.tiles_n = h->N / kBN;
+  p.tiles_n = (h->N + kMxBN - 1) / kMxBN;
   p.err = ctx->d_err;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
@@ -203,11 +203,11 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     cudaFree(l1_own);
     cudaFree(l2_own);
     if (st != W4A4_OK) break;
-    if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, 128, kBN,
+    if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, 128, kMxBN,
                    CU_TENSOR_MAP_SWIZZLE_128B))
       st = W4A4_ERR_CUDA;
     if (st == W4A4_OK && r > 0 &&
-        !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kBN,
+        !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kMxBN,
                    CU_TENSOR_MAP_SWIZZLE_128B))
       st = W4A4_ERR_CUDA;
   }
