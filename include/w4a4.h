@@ -209,6 +209,13 @@ w4a4_status_t w4a4_mx_linear_forward(w4a4_mx_handle_t h, const void* X, int M, i
 w4a4_status_t w4a4_mx_quantize_activations(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
                                            const float* clip_table, void* stream);
 w4a4_status_t w4a4_mx_gemm_from_workspace(w4a4_mx_handle_t h, int M, int expert_id, void* Y, void* stream);
+/* Clipping-ratio search (Eq. 8-10) for the MXFP4 variant: arguments, behaviour and errors exactly as
+ * w4a4_clip_search.  Because the shared exponent is a floor of log2(rho * block maximum), candidates act only
+ * through the blocks whose threshold they move across a power of two. */
+w4a4_status_t w4a4_mx_clip_search(w4a4_mx_handle_t h, const void* const* X_samples, const void* const* Yref_samples,
+                                  int num_samples, int M, int expert_id, int timestep_bin, const float* candidates,
+                                  int num_candidates, float* clip_table, double* errors_out, int* best_out,
+                                  void* stream);
 /* Parity tap: runs the activation kernel and decodes its outputs: codes device uint8 [M, K] (E2M1 codes),
  * exps device uint8 [M, K/32] (E8M0), T device FP32 [M, r] or NULL. */
 w4a4_status_t w4a4_mx_debug_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,

@@ -255,3 +255,22 @@ def mx_forward_rows(X_bits, rows, lam, rho, L1_bits, L2_bits, wcodes, wexps, bia
                                         _p(out["Y64"], np.float64), _p(out["Ybf16"], np.uint16))
     assert rc == 0
     return out
+
+
+def mx_clip_search(X_samples_bits, Yref_samples_bits, lam, candidates, L1_bits, L2_bits, wcodes, wexps, bias):
+    """Eq. 10 for the MXFP4 variant: as clip_search, with mx_forward_rows as the quantized layer."""
+    errs = []
+    for rho in candidates:
+        e = 0.0
+        for Xb, Yb in zip(X_samples_bits, Yref_samples_bits):
+            Xb = _as(Xb, np.uint16)
+            out = mx_forward_rows(Xb, np.arange(Xb.shape[0], dtype=np.int32), lam, float(np.float32(rho)), L1_bits,
+                                  L2_bits, wcodes, wexps, bias)
+            d = bf16_bits_to_f64(Yb) - bf16_bits_to_f64(out["Ybf16"])
+            e += float(np.sum(d * d))
+        errs.append(e)
+    best = 0
+    for i in range(1, len(errs)):
+        if errs[i] < errs[best]:
+            best = i
+    return best, errs

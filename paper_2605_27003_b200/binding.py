@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "w4a4_ctx_enable_host_io", "w4a4_linear_forward_host", "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
     "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search",
     "w4a4_mx_pack_weights", "w4a4_mx_destroy", "w4a4_mx_handle_bytes", "w4a4_mx_linear_forward",
-    "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
+    "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_mx_clip_search", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
 
@@ -96,6 +96,7 @@ def _lib():
         lib.w4a4_mx_quantize_activations.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         lib.w4a4_mx_gemm_from_workspace.argtypes = [vp, ci, ci, vp, vp]
         lib.w4a4_mx_debug_quantize.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.w4a4_mx_clip_search.argtypes = lib.w4a4_clip_search.argtypes
         lib.w4a4_tile_shape.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
         lib.w4a4_tile_shape.restype = None
         lib.w4a4_query_status.argtypes = [vp]
@@ -233,18 +234,25 @@ def w4a4_quantize_noalloc(X, M, K, lam, clip_table, clip_index, codes, scales, s
                                         _ptr(scales), _stream(stream)), "w4a4_quantize_noalloc")
 
 
-def w4a4_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_bin, candidates, clip_table, stream=None):
+def w4a4_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_bin, candidates, clip_table, stream=None,
+                     *, mx: bool = False):
     """Eq. 10 on the device: returns (index of the best candidate, list of the candidates' squared errors) and
-    writes the winning ratio into the clip table entry of (expert, layer, bin)."""
+    writes the winning ratio into the clip table entry of (expert, layer, bin).  mx=True: MXFP4 handle."""
     n_s, n_c = len(X_samples), len(candidates)
     xs = (ctypes.c_void_p * n_s)(*[_ptr(x) for x in X_samples])
     ys = (ctypes.c_void_p * n_s)(*[_ptr(y) for y in Yref_samples])
     cand = (ctypes.c_float * n_c)(*[float(c) for c in candidates])
     errs = (ctypes.c_double * n_c)()
     best = ctypes.c_int(-1)
-    _check(_lib().w4a4_clip_search(handle, xs, ys, n_s, M, expert_id, timestep_bin, cand, n_c, _ptr(clip_table), errs,
-                                   ctypes.byref(best), _stream(stream)), "w4a4_clip_search")
+    fn, name = (_lib().w4a4_mx_clip_search, "w4a4_mx_clip_search") if mx else (_lib().w4a4_clip_search, "w4a4_clip_search")
+    _check(fn(handle, xs, ys, n_s, M, expert_id, timestep_bin, cand, n_c, _ptr(clip_table), errs, ctypes.byref(best),
+              _stream(stream)), name)
     return int(best.value), [float(e) for e in errs]
+
+
+def w4a4_mx_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_bin, candidates, clip_table, stream=None):
+    return w4a4_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_bin, candidates, clip_table, stream,
+                            mx=True)
 
 
 # ----------------------------------------------------------------------------- MXFP4 variant

@@ -58,6 +58,10 @@ struct MxGemmParams {
   int M, N, K, r;
   int tiles_m, tiles_n;
   int* err;
+  // Clip-ratio search (Eq. 10): when yref is set, Y is not stored; the squared distance between the layer's
+  // BF16 output and yref is accumulated into *sq_err instead.
+  const uint16_t* yref;  // [M, N] BF16 or nullptr
+  double* sq_err;
 };
 
 // Shared-memory descriptor of one scale atom (32 rows x 16 bytes, rows contiguous): K-major, no swizzle, 8-row
@@ -254,7 +258,33 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (lane == 0) mbar_arrive(bar_acc_empty);
         }
         const int ch0 = n0 + 128 * half + 64 * part;
-        if (row < p.M && ch0 < p.N) {
+        if (p.yref != nullptr) {
+          // Eq. 10's objective over this thread's 64 outputs, Y_hat rounded to BF16 as the forward stores it.
+          float e = 0.0f;
+          if (row < p.M && ch0 < p.N) {
+            const uint4* yr = reinterpret_cast<const uint4*>(p.yref + static_cast<size_t>(row) * p.N + ch0);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                const uint4 ref = __ldg(yr + 2 * c + h);
+                const uint32_t rw[4] = {ref.x, ref.y, ref.z, ref.w};
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const int col = 8 * h + i;
+                  const float b = p.bias ? __ldg(p.bias + ch0 + 16 * c + col) : 0.0f;
+                  const float y_hat = __bfloat162float(__float2bfloat16_rn(__uint_as_float(v[c][col]) + b));
+                  const float y_ref = __uint_as_float((i & 1) ? (rw[i >> 1] & 0xffff0000u) : (rw[i >> 1] << 16));
+                  const float d = y_ref - y_hat;
+                  e = fmaf(d, d, e);
+                }
+              }
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+          if (lane == 0) atomicAdd(p.sq_err, static_cast<double>(e));
+        } else if (row < p.M && ch0 < p.N) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const int ch = ch0 + 16 * c;

@@ -49,12 +49,11 @@ w4a4_status_t mx_check_forward_args(w4a4_mx_handle_t h, const void* X, int M, in
   return W4A4_OK;
 }
 
-w4a4_status_t mx_launch_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int bin, const float* clip_table,
-                                 cudaStream_t stream) {
+w4a4_status_t mx_launch_quantize_at(w4a4_mx_handle_t h, const void* X, int M, int expert_id, const float* clip_table,
+                                    int clip_index, cudaStream_t stream) {
   if (M == 0) return W4A4_OK;
   w4a4_ctx* ctx = h->ctx;
   const MxExpertData& e = h->experts[expert_id];
-  const int clip_index = (expert_id * h->L + h->layer_id) * h->B + bin;
   const int rows_per_cta = kQuantRows * quantize_warps(h->r);
   const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
@@ -73,7 +72,13 @@ w4a4_status_t mx_launch_quantize(w4a4_mx_handle_t h, const void* X, int M, int e
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
 
-w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream) {
+w4a4_status_t mx_launch_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int bin, const float* clip_table,
+                                 cudaStream_t stream) {
+  return mx_launch_quantize_at(h, X, M, expert_id, clip_table, (expert_id * h->L + h->layer_id) * h->B + bin, stream);
+}
+
+w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream,
+                             const void* yref = nullptr, double* sq_err = nullptr) {
   if (M == 0) return W4A4_OK;
   w4a4_ctx* ctx = h->ctx;
   const MxExpertData& e = h->experts[expert_id];
@@ -89,6 +94,8 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   p.tiles_m = (M + kBM - 1) / kBM;
   p.tiles_n = (h->N + kMxBN - 1) / kMxBN;
   p.err = ctx->d_err;
+  p.yref = static_cast<const uint16_t*>(yref);
+  p.sq_err = sq_err;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;  // unused when r == 0
@@ -260,6 +267,60 @@ w4a4_status_t w4a4_mx_linear_forward(w4a4_mx_handle_t h, const void* X, int M, i
   st = mx_launch_quantize(h, X, M, expert_id, timestep_bin, clip_table, s);
   if (st != W4A4_OK) return st;
   return mx_launch_gemm(h, M, expert_id, Y, s);
+}
+
+w4a4_status_t w4a4_mx_clip_search(w4a4_mx_handle_t h, const void* const* X_samples, const void* const* Yref_samples,
+                                  int num_samples, int M, int expert_id, int timestep_bin, const float* candidates,
+                                  int num_candidates, float* clip_table, double* errors_out, int* best_out,
+                                  void* stream) {
+  if (!h || !h->ctx) return W4A4_ERR_INVALID_ARG;
+  if (num_samples < 1 || num_candidates < 1 || num_candidates > 256 || M < 1) return W4A4_ERR_INVALID_ARG;
+  if (!X_samples || !Yref_samples || !candidates || !clip_table) return W4A4_ERR_INVALID_ARG;
+  for (int c = 0; c < num_candidates; ++c) {
+    if (!(candidates[c] >= 1e-4f && candidates[c] <= 1.0f)) return W4A4_ERR_INVALID_ARG;
+  }
+  for (int s = 0; s < num_samples; ++s) {
+    w4a4_status_t st = mx_check_forward_args(h, X_samples[s], M, expert_id, timestep_bin, clip_table, true);
+    if (st != W4A4_OK) return st;
+    if (!Yref_samples[s] || !aligned16(Yref_samples[s])) return W4A4_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(h->ctx->device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+  cudaStream_t st_ = static_cast<cudaStream_t>(stream);
+  double* d_err = nullptr;
+  float* d_cand = nullptr;
+  int* d_best = nullptr;
+  w4a4_status_t st = dev_alloc(&d_err, static_cast<size_t>(num_candidates), nullptr);
+  if (st == W4A4_OK) st = dev_alloc(&d_cand, static_cast<size_t>(num_candidates), nullptr);
+  if (st == W4A4_OK) st = dev_alloc(&d_best, 1, nullptr);
+  if (st == W4A4_OK &&
+      (cudaMemsetAsync(d_err, 0, sizeof(double) * num_candidates, st_) != cudaSuccess ||
+       cudaMemcpyAsync(d_cand, candidates, sizeof(float) * num_candidates, cudaMemcpyHostToDevice, st_) != cudaSuccess))
+    st = W4A4_ERR_CUDA;
+  for (int s = 0; st == W4A4_OK && s < num_samples; ++s) {
+    for (int c = 0; st == W4A4_OK && c < num_candidates; ++c) {
+      st = mx_launch_quantize_at(h, X_samples[s], M, expert_id, d_cand, c, st_);
+      if (st == W4A4_OK) st = mx_launch_gemm(h, M, expert_id, nullptr, st_, Yref_samples[s], d_err + c);
+    }
+  }
+  int best = 0;
+  if (st == W4A4_OK) {
+    clip_argmin_kernel<<<1, 32, 0, st_>>>(d_err, d_cand, num_candidates,
+                                          clip_table + (expert_id * h->L + h->layer_id) * h->B + timestep_bin, d_best);
+    if (cudaGetLastError() != cudaSuccess) st = W4A4_ERR_CUDA;
+  }
+  if (st == W4A4_OK && errors_out &&
+      cudaMemcpyAsync(errors_out, d_err, sizeof(double) * num_candidates, cudaMemcpyDeviceToHost, st_) != cudaSuccess)
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && cudaMemcpyAsync(&best, d_best, sizeof(int), cudaMemcpyDeviceToHost, st_) != cudaSuccess)
+    st = W4A4_ERR_CUDA;
+  if (cudaStreamSynchronize(st_) != cudaSuccess && st == W4A4_OK) st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && best_out) *best_out = best;
+  cudaFree(d_err);
+  cudaFree(d_cand);
+  cudaFree(d_best);
+  if (st != W4A4_OK) cudaGetLastError();
+  return st;
 }
 
 w4a4_status_t w4a4_mx_debug_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,

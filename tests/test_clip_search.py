@@ -166,3 +166,53 @@ def test_clip_search_rejects_bad_arguments():
     assert table.item() == 1.0
     L.close()
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- MXFP4 variant
+def test_mx_search_picks_the_exact_ratio_on_grid_data():
+    # Activations that MXFP4 represents exactly at rho = 1 (block maximum 6 * 2^k), exact weights: Y_ref is the FP64
+    # product of the raw inputs; rho = 1 reproduces it bit for bit, rho <= 0.5 lowers every shared exponent by one
+    # and clips the block maxima (6 -> 12 saturates).
+    rng = np.random.default_rng(4)
+    M, K, N = 6, 128, 8
+    grid = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    xa = rng.choice(grid, size=(M, K)) * rng.choice([-1.0, 1.0], size=(M, K))
+    xa[:, ::32] = 6.0
+    x = torch.tensor(xa, dtype=torch.float32).to(torch.bfloat16)
+    wcodes = rng.integers(0, 16, size=(K, N)).astype(np.uint8)
+    wexps = rng.integers(122, 126, size=(K // 32, N)).astype(np.uint8)
+    W = gen.mx_dequantize(torch.tensor(wcodes), torch.tensor(wexps)).numpy()
+    yref = bits(torch.tensor(xa @ W, dtype=torch.float64).to(torch.bfloat16))
+    cands = [0.4, 0.5, 0.8, 1.0]
+    best, errs = oracle.mx_clip_search([bits(x)], [yref], np.ones(K, np.float32), cands, None, None, wcodes, wexps, None)
+    assert errs[3] == 0.0 and errs[2] == 0.0        # 0.8 * 6 = 4.8 stays in the binade of 4: same exponent, same result
+    assert errs[0] > 0.0 and errs[1] > 0.0           # 0.5 * 6 = 3 and 0.4 * 6 = 2.4 drop a binade: the 6s saturate
+    assert best == 2                                 # the first of the tied minima
+
+
+@pytest.mark.gpu
+def test_mx_clip_search_parity():
+    w4 = _gpu_modules()
+    dev = "cuda:0"
+    M, K, N, r = 200, 512, 384, 16
+    cands = [0.45, 0.55, 0.7, 0.85, 1.0]
+    idx = gen.outlier_channels(K, 0, 3, count=6)
+    xs = [gen.make_activations(M, K, outlier_idx=idx, outlier_gain=40.0, seed=30 + s) for s in range(2)]
+    layer = gen.make_layer_mx_svd(K, N, r, xs[0], seed=31, bias_std=0.01)
+    yrefs = [gen.reference_output(x, layer) for x in xs]
+    want_best, want_errs = oracle.mx_clip_search([bits(x) for x in xs], [bits(y) for y in yrefs], layer.lam.numpy(), cands,
+                                                 bits(layer.L1), bits(layer.L2), layer.wcodes.numpy(), layer.wexps.numpy(),
+                                                 layer.bias.numpy())
+    ctx = w4.Context(0, M, K, r)
+    L = w4.MxLayer(ctx, [layer.to(dev)], num_bins=2)
+    table = torch.full((1, 1, 2), 0.123, dtype=torch.float32, device=dev)
+    best, errs = w4.w4a4_mx_clip_search(L.ptr, [x.to(dev) for x in xs], [y.to(dev) for y in yrefs], M, 0, 1, cands, table)
+    ctx.check()
+    assert np.allclose(errs, want_errs, rtol=2e-3, atol=0.0), (errs, want_errs)
+    order = np.argsort(want_errs)
+    if want_errs[order[1]] > want_errs[order[0]] * (1.0 + 5e-3):
+        assert best == want_best
+    t = table.cpu()
+    assert t[0, 0, 1].item() == np.float32(cands[best]) and t[0, 0, 0].item() == np.float32(0.123)
+    L.close()
+    ctx.close()
