@@ -20,6 +20,7 @@ struct w4a4_ctx {
   uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
   uint8_t* b8 = nullptr;      // [N, K] E4M3 image of the running layer's weight codes (rewritten by every forward)
   size_t b8_bytes = 0;        // grows to the largest N x K packed on this context
+  float* t_partial = nullptr; // [kMaxKSplits, min(max_M, kKSplitMaxRows), max_r] FP32 partial sums of T when kernel 1 splits K
   uint8_t* mx_sfa = nullptr;  // MXFP4 variant: activation scale atoms [ceil(max_M/128)][max_K/128][512] (allocated on first use)
   int* d_err = nullptr;       // device error word
   size_t bytes = 0;

@@ -16,6 +16,11 @@
 // not care about order), so the lane's 16 channels are used as-is as A-fragment slots and the L1
 // fragments are laid out at pack time to match (see l1_fragment_channel()).
 //
+// K split (gridDim.y > 1): with few token rows there are too few 16-row warps to fill the machine, so the K groups
+// are divided among gridDim.y CTAs per row block.  Codes and scales of different groups are independent; the
+// partial sums of T go to an FP32 scratch [split][M][r] and t_reduce_kernel adds them in split order and writes
+// the BF16 high | low pair.
+//
 // Code output, three formats (template parameter FORMAT):
 //   kCodesE4M3    one E4M3 byte per code, row-major [M, K]: the tensor-core operand of kernel 2 as it is
 //                 (fp8_codes.cuh), fetched by TMA straight into the swizzled operand tile;
@@ -199,7 +204,7 @@ __global__ void __launch_bounds__(32 * WARPS)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
                 uint8_t* __restrict__ codes, float* __restrict__ scales, int scales_ld,
-                uint16_t* __restrict__ t_hilo) {
+                uint16_t* __restrict__ t_hilo, float* __restrict__ t_partial) {
   constexpr int NT = R / 8;                          // n-tiles of the m16n8k16 MMA
   constexpr int kFragBytes = 4 * NT * 32 * 8;        // L1 fragments of one group (4 KiB at r = 32)
   constexpr int kFragChunks = kFragBytes / 16;
@@ -253,13 +258,17 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(rlam + 64 * gg + 4 * threadIdx.x) : "memory");
     }
   };
+  // This CTA's share of the groups (all of them unless the launch splits K).
+  const int g_per_split = (G + gridDim.y - 1) / gridDim.y;
+  const int g_begin = blockIdx.y * g_per_split;
+  const int g_end = min(G, g_begin + g_per_split);
 #pragma unroll
   for (int d = 0; d < kStages - 1; ++d) {
-    if (d < G) issue(d, d);
+    if (g_begin + d < g_end) issue(g_begin + d, d);
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
   int stage = 0;
-  for (int g = 0; g < G; ++g) {
+  for (int g = g_begin; g < g_end; ++g) {
     // This thread's copies for group g have landed; after the barrier so have everyone's, and every warp
     // has finished group g - 1, whose ring slot the prefetch below overwrites.
     asm volatile("cp.async.wait_group %0;" ::"n"(kStages - 2) : "memory");
@@ -267,7 +276,7 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     {
       int pstage = stage + kStages - 1;
       if (pstage >= kStages) pstage -= kStages;
-      if (g + kStages - 1 < G) issue(g + kStages - 1, pstage);
+      if (g + kStages - 1 < g_end) issue(g + kStages - 1, pstage);
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const uint4* slot = &xring[warp][stage][0][lane];
@@ -356,8 +365,9 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
   }
 
   if constexpr (NT > 0) {
-    // Each warp owns its 16 rows over all of K: T is complete in its accumulators.  Store it as a BF16
-    // high part and the BF16 rounding of the remainder ([T_hi | T_lo], two values per 32-bit store).
+    // Each warp owns its 16 rows over all of K (or over its split of K): T, or its partial sum, is complete in
+    // the accumulators.  Unsplit: store it as a BF16 high part and the BF16 rounding of the remainder
+    // ([T_hi | T_lo], two values per 32-bit store).  Split: store the FP32 partial sums for t_reduce_kernel.
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int c = 8 * nt + 2 * qj;
@@ -366,6 +376,10 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
         const int row = h ? rowB : rowA;
         if (row < M) {
           const float t0 = acc[nt][2 * h], t1 = acc[nt][2 * h + 1];
+          if (gridDim.y > 1) {
+            *reinterpret_cast<float2*>(t_partial + (static_cast<size_t>(blockIdx.y) * M + row) * R + c) = make_float2(t0, t1);
+            continue;
+          }
           const __nv_bfloat16 h0 = __float2bfloat16_rn(t0), h1 = __float2bfloat16_rn(t1);
           const uint32_t hi = pack_bf16x2(__bfloat162float(h0), __bfloat162float(h1));
           const uint32_t lo = pack_bf16x2(t0 - __bfloat162float(h0), t1 - __bfloat162float(h1));
@@ -376,6 +390,33 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
       }
     }
   }
+}
+
+// Sum of the K splits' partial T (in split order), written as the BF16 high | low pair kernel 2 reads.
+static __global__ void t_reduce_kernel(const float* __restrict__ t_partial, int splits, int M, int r, uint16_t* __restrict__ t_hilo) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(M) * r) return;
+  float t = 0.0f;
+  for (int s = 0; s < splits; ++s) t += t_partial[static_cast<size_t>(s) * M * r + idx];
+  const size_t row = idx / r;
+  const int c = static_cast<int>(idx % r);
+  const __nv_bfloat16 hi = __float2bfloat16_rn(t);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(t - __bfloat162float(hi));
+  t_hilo[row * 2 * r + c] = *reinterpret_cast<const uint16_t*>(&hi);
+  t_hilo[row * 2 * r + r + c] = *reinterpret_cast<const uint16_t*>(&lo);
+}
+
+// Number of K splits for a launch of `row_ctas` row blocks over G groups on a device with `sms` SMs: enough CTAs
+// for about three per SM, at most kMaxKSplits, and only while the partial sums of T fit the scratch
+// (M <= kKSplitMaxRows).
+constexpr int kMaxKSplits = 8;
+constexpr int kKSplitMaxRows = 8192;
+inline int quantize_k_splits(int row_ctas, int G, int M, int sms) {
+  if (M > kKSplitMaxRows || row_ctas >= 2 * sms) return 1;
+  int s = (3 * sms + row_ctas - 1) / row_ctas;
+  if (s > kMaxKSplits) s = kMaxKSplits;
+  if (s > G) s = G;
+  return s < 1 ? 1 : s;
 }
 
 }  // namespace w4a4

@@ -175,11 +175,13 @@ w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expe
   w4a4_ctx* ctx = h->ctx;
   const ExpertData& e = h->experts[expert_id];
   const int rows_per_cta = kQuantRows * quantize_warps(h->r);
-  const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
+  const int row_ctas = (M + rows_per_cta - 1) / rows_per_cta;
+  const int splits = quantize_k_splits(row_ctas, h->K / 64, M, ctx->num_sms);
+  const dim3 grid(row_ctas, splits), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define W4A4_LAUNCH_Q(R)                                                                                         \
   quantize_kernel<R, quantize_warps(R), kCodesE4M3><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
-                                                 ctx->scales, ctx->scales_ld, ctx->t_hilo)
+                                                 ctx->scales, ctx->scales_ld, ctx->t_hilo, ctx->t_partial)
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
     case 16: W4A4_LAUNCH_Q(16); break;
@@ -188,6 +190,10 @@ w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expe
     default: return W4A4_ERR_SHAPE;
   }
 #undef W4A4_LAUNCH_Q
+  if (splits > 1 && h->r > 0) {
+    const size_t nt = static_cast<size_t>(M) * h->r;
+    t_reduce_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, stream>>>(ctx->t_partial, splits, M, h->r, ctx->t_hilo);
+  }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
 
@@ -303,6 +309,9 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(ctx->scales_ld) * (max_K / 64), &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->scales, 0, sizeof(float) * ctx->scales_ld * (max_K / 64)) != cudaSuccess) st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) st = dev_alloc(&ctx->t_hilo, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8), &ctx->bytes);
+  if (st == W4A4_OK && max_r > 0)
+    st = dev_alloc(&ctx->t_partial,
+                   static_cast<size_t>(kMaxKSplits) * (max_M < kKSplitMaxRows ? max_M : kKSplitMaxRows) * max_r, &ctx->bytes);
   if (st == W4A4_OK) st = dev_alloc(&ctx->d_err, 1, &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->d_err, 0, sizeof(int)) != cudaSuccess) st = W4A4_ERR_CUDA;
   // The workspace is read by TMA for rows up to max_M even when fewer are valid: start it defined.
@@ -334,6 +343,7 @@ void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
   cudaFree(ctx->codes);
   cudaFree(ctx->b8);
   cudaFree(ctx->mx_sfa);
+  cudaFree(ctx->t_partial);
   cudaFree(ctx->scales);
   cudaFree(ctx->t_hilo);
   cudaFree(ctx->d_err);

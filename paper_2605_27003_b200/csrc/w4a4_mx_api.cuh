@@ -55,12 +55,14 @@ w4a4_status_t mx_launch_quantize_at(w4a4_mx_handle_t h, const void* X, int M, in
   w4a4_ctx* ctx = h->ctx;
   const MxExpertData& e = h->experts[expert_id];
   const int rows_per_cta = kQuantRows * quantize_warps(h->r);
-  const dim3 grid((M + rows_per_cta - 1) / rows_per_cta), block(32 * quantize_warps(h->r));
+  const int row_ctas = (M + rows_per_cta - 1) / rows_per_cta;
+  const int splits = quantize_k_splits(row_ctas, h->K / 64, M, ctx->num_sms);
+  const dim3 grid(row_ctas, splits), block(32 * quantize_warps(h->r));
   const uint16_t* x = static_cast<const uint16_t*>(X);
   float* sf = reinterpret_cast<float*>(ctx->mx_sfa);
 #define W4A4_LAUNCH_MXQ(R)                                                                                             \
   quantize_kernel<R, quantize_warps(R), kCodesMxfp4><<<grid, block, quantize_smem_bytes(R), stream>>>(                 \
-      x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, sf, h->K / 128, ctx->t_hilo)
+      x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, sf, h->K / 128, ctx->t_hilo, ctx->t_partial)
   switch (h->r) {
     case 0: W4A4_LAUNCH_MXQ(0); break;
     case 16: W4A4_LAUNCH_MXQ(16); break;
@@ -69,6 +71,10 @@ w4a4_status_t mx_launch_quantize_at(w4a4_mx_handle_t h, const void* X, int M, in
     default: return W4A4_ERR_SHAPE;
   }
 #undef W4A4_LAUNCH_MXQ
+  if (splits > 1 && h->r > 0) {
+    const size_t nt = static_cast<size_t>(M) * h->r;
+    t_reduce_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, stream>>>(ctx->t_partial, splits, M, h->r, ctx->t_hilo);
+  }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
 
