@@ -453,6 +453,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search", "mxfp4_attn_proj", "mxfp4_ffn_up",
                                                             "mxfp4_ffn_down"])
+    ap.add_argument("--chunk-rows", type=int, default=4096, help="token rows per chunk of the host-buffer forward (e2e)")
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -542,7 +543,7 @@ def main():
     e2e_steps = max(1, min(args.e2e_steps, args.steps))
     xh = [torch.empty(M, K, dtype=torch.bfloat16).pin_memory().copy_(w["xs"][i]) for i in range(2)]
     yh = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
-    chunk_rows = min(M, 4096)
+    chunk_rows = min(M, args.chunk_rows)
     w4.w4a4_ctx_enable_host_io(ctx.ptr, chunk_rows, N)
 
     def e2e_step(i):

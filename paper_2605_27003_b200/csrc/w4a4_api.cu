@@ -648,7 +648,8 @@ w4a4_status_t w4a4_linear_forward_host(w4a4_handle_t h, const void* X_host, int 
     if (ok && i >= 2) ok = cudaStreamWaitEvent(ctx->s_compute, ctx->ev_out[b], 0) == cudaSuccess;  // staging Y[b] drained
     if (!ok) break;
     st = launch_quantize(h, ctx->hx[b], rows, expert_id, timestep_bin, clip_table, ctx->s_compute);
-    if (st == W4A4_OK) st = launch_gemm(h, rows, expert_id, ctx->hy[b], ctx->s_compute, nullptr, 0, 0);
+    // The weight byte image is the same for every chunk: expand it with the first one only.
+    if (st == W4A4_OK) st = launch_gemm(h, rows, expert_id, ctx->hy[b], ctx->s_compute, nullptr, 0, 0, nullptr, nullptr, i == 0);
     if (st != W4A4_OK) return st;
     ok = cudaEventRecord(ctx->ev_done[b], ctx->s_compute) == cudaSuccess &&
          cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_done[b], 0) == cudaSuccess &&
