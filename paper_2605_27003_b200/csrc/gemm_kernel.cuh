@@ -53,7 +53,7 @@ namespace w4a4 {
 constexpr int kBM = 128;            // output tile rows (tokens)
 constexpr int kBN = 128;            // output tile columns (output channels)
 constexpr int kBK = 128;            // K codes per pipeline stage = 2 quantization groups
-constexpr int kS8Stages = 6;        // operand ring: A and B tiles of one stage, one byte per code, tensor-core ready
+constexpr int kOpStages = 6;        // operand ring: A and B tiles of one stage, one byte per code, tensor-core ready
 constexpr int kScaleStages = 12;   // ring of scale blocks (2 groups x (kBN weight scales + kBM activation scales));
                                    // deeper than the TMA producer can ever run ahead of the epilogue, so it needs no barriers
 constexpr int kTmemSlots = 2;       // TMEM slots of 2 x kBN columns: one per stage in flight
@@ -63,12 +63,12 @@ constexpr int kEpiCols = kBN / (kEpiWarps / 4);   // output channels per epilogu
 constexpr int kRegsControl = 40, kRegsEpilogue = 104;   // setmaxnreg budgets per role: 4 x 32 x 40 + 16 x 32 x 104 fits the
                                                         // 640 x 96 registers the CTA is launched with
 
-constexpr uint32_t kS8ATile = kBM * kBK;             // 16 KiB
-constexpr uint32_t kS8BTile = kBN * kBK;             // 16 KiB
-constexpr uint32_t kS8StageBytes = kS8ATile + kS8BTile;
+constexpr uint32_t kOpATile = kBM * kBK;             // 16 KiB
+constexpr uint32_t kOpBTile = kBN * kBK;             // 16 KiB
+constexpr uint32_t kOpStageBytes = kOpATile + kOpBTile;
 constexpr uint32_t kScaleStageBytes = 2 * (kBN + kBM) * 4;   // 2 KiB: sw[2][kBN] then sa[2][kBM]
-constexpr uint32_t kNumBarriers = 2 * kS8Stages + 2 * kTmemSlots;
-constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kS8Stages * kS8StageBytes +
+constexpr uint32_t kNumBarriers = 2 * kOpStages + 2 * kTmemSlots;
+constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kOpStages * kOpStageBytes +
                                     kScaleStages * kScaleStageBytes + kNumBarriers * 8 + 16;
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;     // 2 s
@@ -202,12 +202,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t s8_base = smem_base;
-  const uint32_t scale_base = s8_base + kS8Stages * kS8StageBytes;
+  const uint32_t op_base = smem_base;
+  const uint32_t scale_base = op_base + kOpStages * kOpStageBytes;
   const uint32_t bar_base = scale_base + kScaleStages * kScaleStageBytes;
-  const uint32_t bar_s8_full = bar_base;
-  const uint32_t bar_s8_empty = bar_s8_full + 8 * kS8Stages;
-  const uint32_t bar_tmem_full = bar_s8_empty + 8 * kS8Stages;
+  const uint32_t bar_op_full = bar_base;
+  const uint32_t bar_op_empty = bar_op_full + 8 * kOpStages;
+  const uint32_t bar_tmem_full = bar_op_empty + 8 * kOpStages;
   const uint32_t bar_tmem_empty = bar_tmem_full + 8 * kTmemSlots;
   const uint32_t misc_off = (bar_tmem_empty + 8 * kTmemSlots) - smem_base;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
@@ -222,9 +222,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
-    for (int i = 0; i < kS8Stages; ++i) {
-      mbar_init(bar_s8_full + 8 * i, 1);
-      mbar_init(bar_s8_empty + 8 * i, 1);
+    for (int i = 0; i < kOpStages; ++i) {
+      mbar_init(bar_op_full + 8 * i, 1);
+      mbar_init(bar_op_empty + 8 * i, 1);
     }
     for (int i = 0; i < kTmemSlots; ++i) {
       mbar_init(bar_tmem_full + 8 * i, 1);
@@ -259,55 +259,55 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // ------------------------------------------------------------------ TMA producer
       // Slots of the operand ring in the order the MMA warp consumes them: per tile the low-rank stages
       // (T and the duplicated L2 factor, BF16) first, then the code stages with their scales.
-      Ring<kS8Stages> s8;
+      Ring<kOpStages> op;
       Ring<kScaleStages> sc;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
         for (int st = 0; st < n_lr_stages + n_int_stages; ++st) {
-          ok = bounded_wait<128>(bar_s8_empty + 8 * s8.slot, s8.parity ^ 1u, env, kErrProducerWait);
+          ok = bounded_wait<128>(bar_op_empty + 8 * op.slot, op.parity ^ 1u, env, kErrProducerWait);
           if (!ok) break;
-          const uint32_t full = bar_s8_full + 8 * s8.slot;
-          const uint32_t dst = s8_base + s8.slot * kS8StageBytes;
+          const uint32_t full = bar_op_full + 8 * op.slot;
+          const uint32_t dst = op_base + op.slot * kOpStageBytes;
           if (st < n_lr_stages) {
-            mbar_arrive_expect_tx(full, kS8StageBytes);
+            mbar_arrive_expect_tx(full, kOpStageBytes);
             tma_load_2d(dst, &tmT, full, st * 64, m0);
-            tma_load_2d(dst + kS8ATile, &tmL2, full, st * 64, n0);
+            tma_load_2d(dst + kOpATile, &tmL2, full, st * 64, n0);
           } else {
             const int ks = st - n_lr_stages;
             const uint32_t sdst = scale_base + sc.slot * kScaleStageBytes;
-            mbar_arrive_expect_tx(full, kS8StageBytes + kScaleStageBytes);
+            mbar_arrive_expect_tx(full, kOpStageBytes + kScaleStageBytes);
             tma_load_2d(dst, &tmA, full, ks * kBK, m0);
-            tma_load_2d(dst + kS8ATile, &tmB, full, ks * kBK, n0);
+            tma_load_2d(dst + kOpATile, &tmB, full, ks * kBK, n0);
             tma_load_2d(sdst, &tmSW, full, n0, 2 * ks);
             tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * ks);
             sc.advance();
           }
-          s8.advance();
+          op.advance();
         }
       }
     } else if (live && warp == 1 && lane == 0) {
       // ------------------------------------------------------------------ MMA issuer
       constexpr uint32_t idesc_f8 = umma_idesc(1, 0, kBM, kBN);
       constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
-      Ring<kS8Stages> s8;
+      Ring<kOpStages> op;
       Ring<kTmemSlots> tm;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         if (n_lr_stages > 0) {
           ok = bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait);
           for (int l = 0; ok && l < n_lr_stages; ++l) {
-            ok = bounded_wait<64>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
+            ok = bounded_wait<64>(bar_op_full + 8 * op.slot, op.parity, env, kErrMmaWait);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t a = s8_base + s8.slot * kS8StageBytes, b = a + kS8ATile;
+            const uint32_t a = op_base + op.slot * kOpStageBytes, b = a + kOpATile;
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
               umma_f16(tmem_base + tm.slot * 2 * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk),
                        idesc_bf16, (l > 0 || kk > 0) ? 1u : 0u);
             }
-            umma_commit(bar_s8_empty + 8 * s8.slot);
-            s8.advance();
+            umma_commit(bar_op_empty + 8 * op.slot);
+            op.advance();
           }
           if (!ok) break;
           umma_commit(bar_tmem_full + 8 * tm.slot);
@@ -315,10 +315,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int st = 0; ok && st < n_int_stages; ++st) {
           ok = bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait) &&
-               bounded_wait<64>(bar_s8_full + 8 * s8.slot, s8.parity, env, kErrMmaWait);
+               bounded_wait<64>(bar_op_full + 8 * op.slot, op.parity, env, kErrMmaWait);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t a = s8_base + s8.slot * kS8StageBytes, b = a + kS8ATile;
+          const uint32_t a = op_base + op.slot * kOpStageBytes, b = a + kOpATile;
           const uint32_t d = tmem_base + tm.slot * 2 * kBN;
           const int groups = (2 * st + 1 < G) ? 2 : 1;
 #pragma unroll
@@ -328,9 +328,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                       kk & 1);
             }
           }
-          umma_commit(bar_s8_empty + 8 * s8.slot);
+          umma_commit(bar_op_empty + 8 * op.slot);
           umma_commit(bar_tmem_full + 8 * tm.slot);
-          s8.advance();
+          op.advance();
           tm.advance();
         }
       }

@@ -1,5 +1,7 @@
-// C-ABI entry points of libw4a4: context / handle management, weight repacking and the launches of
-// the two forward kernels.  Host code only does argument checks, descriptor set-up and launches.
+// C-ABI entry points of libw4a4: context / handle management, weight repacking and the launches of the
+// forward kernels (activation quantization, weight expansion, GEMM) and of the clipping-ratio search; the MXFP4
+// variant's entry points are in w4a4_mx_api.cuh, included at the end.  Host code only does argument checks,
+// descriptor set-up and launches.
 #include "../../include/w4a4.h"
 
 #include <cuda.h>
