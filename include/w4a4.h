@@ -42,6 +42,13 @@ typedef enum {
   W4A4_ERR_TIMEOUT = 6      /* a kernel gave up on a bounded wait and returned early (see w4a4_query_status) */
 } w4a4_status_t;
 
+/* Activation fused into the output of a layer (no counterpart in the paper's equations; it is the producer-side
+ * fusion for the FFN, whose second linear consumes GELU of the first one's output: applying it in the GEMM's
+ * epilogue saves the element-wise pass over the 13824-wide hidden activations).  GELU_TANH is
+ * 0.5 y (1 + tanh(sqrt(2/pi) (y + 0.044715 y^3))) evaluated in FP32 on y = Eq. 11's value before the BF16 rounding. */
+#define W4A4_ACT_NONE 0
+#define W4A4_ACT_GELU_TANH 1
+
 typedef struct w4a4_ctx* w4a4_ctx_t;      /* per-stream workspace: activation codes, scales, low-rank intermediate */
 typedef struct w4a4_layer* w4a4_handle_t; /* one layer position: packed constants of all its experts */
 
@@ -61,6 +68,7 @@ typedef struct {
   int num_layers;  /* layers per expert in the clip table */
   int layer_id;    /* this layer's index into the clip table */
   int pointers_on_device;
+  int output_activation; /* W4A4_ACT_NONE, or W4A4_ACT_GELU_TANH: the layer returns GELU(Y) (see below) */
   const int8_t* const* qweight;  /* [E] -> K x N row-major, one code per byte, values in [-8, 7] */
   const float* const* wscale;    /* [E] -> (K/64) x N row-major FP32 */
   const float* const* lambda;    /* [E] -> K FP32, > 0 (diagonal of the smoothing matrix D_l) */
@@ -186,6 +194,7 @@ typedef struct {
   int K, N, r;
   int num_experts, num_bins, num_layers, layer_id;
   int pointers_on_device;
+  int output_activation; /* W4A4_ACT_NONE or W4A4_ACT_GELU_TANH, as in w4a4_weight_desc_t */
   const uint8_t* const* wcodes; /* [E] -> K x N row-major, one E2M1 code per byte: bit 3 sign, bits 0-2 magnitude index */
   const uint8_t* const* wexps;  /* [E] -> (K/32) x N row-major E8M0 bytes (0xFF, the NaN encoding, is rejected) */
   const float* const* lambda;   /* [E] -> K FP32, > 0 */

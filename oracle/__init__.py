@@ -274,3 +274,10 @@ def mx_clip_search(X_samples_bits, Yref_samples_bits, lam, candidates, L1_bits, 
         if errs[i] < errs[best]:
             best = i
     return best, errs
+
+
+def gelu_tanh(y):
+    """GELU in its tanh form, 0.5 y (1 + tanh(sqrt(2/pi) (y + 0.044715 y^3))), on FP64 values: the output
+    activation a layer can be asked to fuse (the FFN's nonlinearity; not part of the paper's equations)."""
+    y = np.asarray(y, dtype=np.float64)
+    return 0.5 * y * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (y + 0.044715 * y ** 3)))

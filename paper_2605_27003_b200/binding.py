@@ -15,6 +15,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libw4a4.so")
 
+ACT_NONE, ACT_GELU_TANH = 0, 1
 W4A4_OK = 0
 STATUS_NAMES = {0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_SHAPE", 3: "ERR_ALLOC", 4: "ERR_CUDA", 5: "ERR_ARCH",
                 6: "ERR_TIMEOUT"}
@@ -39,7 +40,7 @@ class WeightDesc(ctypes.Structure):
     _fields_ = [
         ("K", ctypes.c_int), ("N", ctypes.c_int), ("r", ctypes.c_int), ("group", ctypes.c_int),
         ("num_experts", ctypes.c_int), ("num_bins", ctypes.c_int), ("num_layers", ctypes.c_int),
-        ("layer_id", ctypes.c_int), ("pointers_on_device", ctypes.c_int),
+        ("layer_id", ctypes.c_int), ("pointers_on_device", ctypes.c_int), ("output_activation", ctypes.c_int),
         ("qweight", ctypes.POINTER(ctypes.c_void_p)), ("wscale", ctypes.POINTER(ctypes.c_void_p)),
         ("lambda_", ctypes.POINTER(ctypes.c_void_p)), ("L1", ctypes.POINTER(ctypes.c_void_p)),
         ("L2", ctypes.POINTER(ctypes.c_void_p)), ("bias", ctypes.POINTER(ctypes.c_void_p)),
@@ -50,7 +51,7 @@ class MxWeightDesc(ctypes.Structure):
     _fields_ = [
         ("K", ctypes.c_int), ("N", ctypes.c_int), ("r", ctypes.c_int),
         ("num_experts", ctypes.c_int), ("num_bins", ctypes.c_int), ("num_layers", ctypes.c_int),
-        ("layer_id", ctypes.c_int), ("pointers_on_device", ctypes.c_int),
+        ("layer_id", ctypes.c_int), ("pointers_on_device", ctypes.c_int), ("output_activation", ctypes.c_int),
         ("wcodes", ctypes.POINTER(ctypes.c_void_p)), ("wexps", ctypes.POINTER(ctypes.c_void_p)),
         ("lambda_", ctypes.POINTER(ctypes.c_void_p)), ("L1", ctypes.POINTER(ctypes.c_void_p)),
         ("L2", ctypes.POINTER(ctypes.c_void_p)), ("bias", ctypes.POINTER(ctypes.c_void_p)),
@@ -153,7 +154,7 @@ def w4a4_pack_weights(ctx, *, K: int, N: int, r: int, num_bins: int, num_layers:
                       qweight: Sequence[torch.Tensor], wscale: Sequence[torch.Tensor],
                       lam: Sequence[torch.Tensor], L1: Optional[Sequence[torch.Tensor]],
                       L2: Optional[Sequence[torch.Tensor]], bias: Optional[Sequence[Optional[torch.Tensor]]],
-                      group: int = 64) -> ctypes.c_void_p:
+                      group: int = 64, output_activation: int = 0) -> ctypes.c_void_p:
     """One tensor per expert in every list; all on the host or all on one CUDA device, contiguous."""
     E = len(qweight)
     on_dev = qweight[0].is_cuda
@@ -175,7 +176,7 @@ def w4a4_pack_weights(ctx, *, K: int, N: int, r: int, num_bins: int, num_layers:
 
     G = K // group
     d = WeightDesc(K=K, N=N, r=r, group=group, num_experts=E, num_bins=num_bins, num_layers=num_layers,
-                   layer_id=layer_id, pointers_on_device=int(on_dev))
+                   layer_id=layer_id, pointers_on_device=int(on_dev), output_activation=output_activation)
     d.qweight = arr(qweight, torch.int8, (K, N))
     d.wscale = arr(wscale, torch.float32, (G, N))
     d.lambda_ = arr(lam, torch.float32, (K,))
@@ -259,7 +260,7 @@ def w4a4_mx_clip_search(handle, X_samples, Yref_samples, M, expert_id, timestep_
 def w4a4_mx_pack_weights(ctx, *, K: int, N: int, r: int, num_bins: int, num_layers: int, layer_id: int,
                          wcodes: Sequence[torch.Tensor], wexps: Sequence[torch.Tensor], lam: Sequence[torch.Tensor],
                          L1: Optional[Sequence[torch.Tensor]], L2: Optional[Sequence[torch.Tensor]],
-                         bias: Optional[Sequence[Optional[torch.Tensor]]]) -> ctypes.c_void_p:
+                         bias: Optional[Sequence[Optional[torch.Tensor]]], output_activation: int = 0) -> ctypes.c_void_p:
     """One tensor per expert in every list; all on the host or all on one CUDA device, contiguous."""
     E = len(wcodes)
     on_dev = wcodes[0].is_cuda
@@ -280,7 +281,7 @@ def w4a4_mx_pack_weights(ctx, *, K: int, N: int, r: int, num_bins: int, num_laye
         return a
 
     d = MxWeightDesc(K=K, N=N, r=r, num_experts=E, num_bins=num_bins, num_layers=num_layers, layer_id=layer_id,
-                     pointers_on_device=int(on_dev))
+                     pointers_on_device=int(on_dev), output_activation=output_activation)
     d.wcodes = arr(wcodes, torch.uint8, (K, N))
     d.wexps = arr(wexps, torch.uint8, (K // 32, N))
     d.lambda_ = arr(lam, torch.float32, (K,))
@@ -359,7 +360,8 @@ class Context:
 class Layer:
     """Owns a w4a4_handle_t built from one LayerInputs-like object per expert."""
 
-    def __init__(self, ctx: Context, experts, *, num_bins: int, num_layers: int = 1, layer_id: int = 0):
+    def __init__(self, ctx: Context, experts, *, num_bins: int, num_layers: int = 1, layer_id: int = 0,
+                 output_activation: int = 0):
         e0 = experts[0]
         self.ctx, self.K, self.N, self.r, self.E = ctx, e0.K, e0.N, e0.r, len(experts)
         has_bias = any(e.bias is not None for e in experts)
@@ -369,7 +371,8 @@ class Layer:
             lam=[e.lam.contiguous() for e in experts],
             L1=[e.L1.contiguous() for e in experts] if e0.r > 0 else None,
             L2=[e.L2.contiguous() for e in experts] if e0.r > 0 else None,
-            bias=[None if e.bias is None else e.bias.contiguous() for e in experts] if has_bias else None)
+            bias=[None if e.bias is None else e.bias.contiguous() for e in experts] if has_bias else None,
+            output_activation=output_activation)
 
     def forward(self, X: torch.Tensor, expert_id: int, timestep_bin: int, clip_table: torch.Tensor,
                 Y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
@@ -395,7 +398,8 @@ class Layer:
 class MxLayer:
     """Owns a w4a4_mx_handle_t built from one MxLayerInputs-like object per expert."""
 
-    def __init__(self, ctx: Context, experts, *, num_bins: int, num_layers: int = 1, layer_id: int = 0):
+    def __init__(self, ctx: Context, experts, *, num_bins: int, num_layers: int = 1, layer_id: int = 0,
+                 output_activation: int = 0):
         e0 = experts[0]
         self.ctx, self.K, self.N, self.r, self.E = ctx, e0.K, e0.N, e0.r, len(experts)
         has_bias = any(e.bias is not None for e in experts)
@@ -405,7 +409,8 @@ class MxLayer:
             lam=[e.lam.contiguous() for e in experts],
             L1=[e.L1.contiguous() for e in experts] if e0.r > 0 else None,
             L2=[e.L2.contiguous() for e in experts] if e0.r > 0 else None,
-            bias=[None if e.bias is None else e.bias.contiguous() for e in experts] if has_bias else None)
+            bias=[None if e.bias is None else e.bias.contiguous() for e in experts] if has_bias else None,
+            output_activation=output_activation)
 
     def forward(self, X: torch.Tensor, expert_id: int, timestep_bin: int, clip_table: torch.Tensor,
                 Y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

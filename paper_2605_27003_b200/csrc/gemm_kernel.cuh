@@ -138,6 +138,15 @@ __device__ __forceinline__ void set_max_regs_dec() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
+// Output activation of the layer (W4A4_ACT_*), applied in FP32 before the BF16 rounding.
+__device__ __forceinline__ float apply_activation(float y, int act) {
+  if (act == 1) {
+    const float u = 0.7978845608028654f * (y + 0.044715f * y * y * y);
+    return 0.5f * y * (1.0f + tanhf(u));
+  }
+  return y;
+}
+
 struct GemmParams {
   const float* bias;    // [N] or nullptr
   uint16_t* Y;          // [M, N] BF16
@@ -150,6 +159,7 @@ struct GemmParams {
   // BF16 output and yref is accumulated into *sq_err instead.
   const uint16_t* yref; // [M, N] BF16 or nullptr
   double* sq_err;
+  int act;              // output activation: 0 none, 1 GELU (tanh form)
 };
 
 // Rescales one fragment (32 token rows x 16 columns: one row x 16 channels per thread) of a group's partial
@@ -464,7 +474,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               const uint32_t rw[4] = {ref.x, ref.y, ref.z, ref.w};
 #pragma unroll
               for (int c = 0; c < 8; ++c) {
-                const float y_hat = __bfloat162float(__float2bfloat16_rn(yh[c]));
+                const float y_hat = __bfloat162float(__float2bfloat16_rn(apply_activation(yh[c], p.act)));
                 const float y_ref = __uint_as_float((c & 1) ? (rw[c >> 1] & 0xffff0000u) : (rw[c >> 1] << 16));
                 const float d = y_ref - y_hat;
                 e = fmaf(d, d, e);
@@ -485,10 +495,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               b1 = __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + 2 * i + 1);
             }
             const float2 a0 = acc[4 * i], a1 = acc[4 * i + 1], a2 = acc[4 * i + 2], a3 = acc[4 * i + 3];
-            __nv_bfloat162 o0 = __floats2bfloat162_rn(a0.x + b0.x, a0.y + b0.y);
-            __nv_bfloat162 o1 = __floats2bfloat162_rn(a1.x + b0.z, a1.y + b0.w);
-            __nv_bfloat162 o2 = __floats2bfloat162_rn(a2.x + b1.x, a2.y + b1.y);
-            __nv_bfloat162 o3 = __floats2bfloat162_rn(a3.x + b1.z, a3.y + b1.w);
+            const int act = p.act;
+            __nv_bfloat162 o0 = __floats2bfloat162_rn(apply_activation(a0.x + b0.x, act), apply_activation(a0.y + b0.y, act));
+            __nv_bfloat162 o1 = __floats2bfloat162_rn(apply_activation(a1.x + b0.z, act), apply_activation(a1.y + b0.w, act));
+            __nv_bfloat162 o2 = __floats2bfloat162_rn(apply_activation(a2.x + b1.x, act), apply_activation(a2.y + b1.y, act));
+            __nv_bfloat162 o3 = __floats2bfloat162_rn(apply_activation(a3.x + b1.z, act), apply_activation(a3.y + b1.w, act));
             uint4 o;
             o.x = *reinterpret_cast<uint32_t*>(&o0);
             o.y = *reinterpret_cast<uint32_t*>(&o1);

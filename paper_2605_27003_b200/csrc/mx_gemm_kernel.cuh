@@ -62,6 +62,7 @@ struct MxGemmParams {
   // BF16 output and yref is accumulated into *sq_err instead.
   const uint16_t* yref;  // [M, N] BF16 or nullptr
   double* sq_err;
+  int act;              // output activation: 0 none, 1 GELU (tanh form)
 };
 
 // Shared-memory descriptor of one scale atom (32 rows x 16 bytes, rows contiguous): K-major, no swizzle, 8-row
@@ -273,7 +274,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int i = 0; i < 8; ++i) {
                   const int col = 8 * h + i;
                   const float b = p.bias ? __ldg(p.bias + ch0 + 16 * c + col) : 0.0f;
-                  const float y_hat = __bfloat162float(__float2bfloat16_rn(__uint_as_float(v[c][col]) + b));
+                  const float y_hat = __bfloat162float(__float2bfloat16_rn(apply_activation(__uint_as_float(v[c][col]) + b, p.act)));
                   const float y_ref = __uint_as_float((i & 1) ? (rw[i >> 1] & 0xffff0000u) : (rw[i >> 1] << 16));
                   const float d = y_ref - y_hat;
                   e = fmaf(d, d, e);
@@ -293,8 +294,10 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-              __nv_bfloat162 lo = __floats2bfloat162_rn(__uint_as_float(v[c][4 * i]) + b4.x, __uint_as_float(v[c][4 * i + 1]) + b4.y);
-              __nv_bfloat162 hi = __floats2bfloat162_rn(__uint_as_float(v[c][4 * i + 2]) + b4.z, __uint_as_float(v[c][4 * i + 3]) + b4.w);
+              __nv_bfloat162 lo = __floats2bfloat162_rn(apply_activation(__uint_as_float(v[c][4 * i]) + b4.x, p.act),
+                                                        apply_activation(__uint_as_float(v[c][4 * i + 1]) + b4.y, p.act));
+              __nv_bfloat162 hi = __floats2bfloat162_rn(apply_activation(__uint_as_float(v[c][4 * i + 2]) + b4.z, p.act),
+                                                        apply_activation(__uint_as_float(v[c][4 * i + 3]) + b4.w, p.act));
               ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
               ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
             }

@@ -133,7 +133,7 @@ struct ExpertData {
 
 struct w4a4_layer {
   w4a4_ctx* ctx = nullptr;
-  int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0;
+  int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0, act = 0;
   std::vector<ExpertData> experts;
   CUtensorMap tmA, tmSA, tmT, tmB;
   const uint8_t* tmB_base = nullptr;  // the context's weight-byte scratch this handle's tmB was encoded for
@@ -228,6 +228,7 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   p.dbg_n0 = dbg_n0;
   p.yref = static_cast<const uint16_t*>(yref);
   p.sq_err = sq_err;
+  p.act = h->act;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
   // The context's weight-byte scratch may have been reallocated (a larger layer packed since): re-aim the map.
@@ -386,6 +387,7 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
   if (d->num_experts < 1 || d->num_bins < 1 || d->num_layers < 1 || d->layer_id < 0 || d->layer_id >= d->num_layers)
     return W4A4_ERR_INVALID_ARG;
   if (!d->qweight || !d->wscale || !d->lambda || (d->r > 0 && (!d->L1 || !d->L2))) return W4A4_ERR_INVALID_ARG;
+  if (d->output_activation != W4A4_ACT_NONE && d->output_activation != W4A4_ACT_GELU_TANH) return W4A4_ERR_INVALID_ARG;
   for (int e = 0; e < d->num_experts; ++e) {
     if (!d->qweight[e] || !d->wscale[e] || !d->lambda[e] || (d->r > 0 && (!d->L1[e] || !d->L2[e])))
       return W4A4_ERR_INVALID_ARG;
@@ -403,6 +405,7 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
   h->B = d->num_bins;
   h->L = d->num_layers;
   h->layer_id = d->layer_id;
+  h->act = d->output_activation;
   h->experts.resize(d->num_experts);
   const int K = d->K, N = d->N, r = d->r, G = K / 64;
   const bool dev = d->pointers_on_device != 0;

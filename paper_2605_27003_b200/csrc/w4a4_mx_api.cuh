@@ -16,7 +16,7 @@ struct MxExpertData {
 
 struct w4a4_mx_layer {
   w4a4_ctx* ctx = nullptr;
-  int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0;
+  int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0, act = 0;
   std::vector<MxExpertData> experts;
   CUtensorMap tmA, tmT;
   size_t bytes = 0;
@@ -102,6 +102,7 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   p.err = ctx->d_err;
   p.yref = static_cast<const uint16_t*>(yref);
   p.sq_err = sq_err;
+  p.act = h->act;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;  // unused when r == 0
@@ -135,6 +136,7 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
   if (d->num_experts < 1 || d->num_bins < 1 || d->num_layers < 1 || d->layer_id < 0 || d->layer_id >= d->num_layers)
     return W4A4_ERR_INVALID_ARG;
   if (!d->wcodes || !d->wexps || !d->lambda || (d->r > 0 && (!d->L1 || !d->L2))) return W4A4_ERR_INVALID_ARG;
+  if (d->output_activation != W4A4_ACT_NONE && d->output_activation != W4A4_ACT_GELU_TANH) return W4A4_ERR_INVALID_ARG;
   for (int e = 0; e < d->num_experts; ++e) {
     if (!d->wcodes[e] || !d->wexps[e] || !d->lambda[e] || (d->r > 0 && (!d->L1[e] || !d->L2[e]))) return W4A4_ERR_INVALID_ARG;
   }
@@ -151,6 +153,7 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
   h->B = d->num_bins;
   h->L = d->num_layers;
   h->layer_id = d->layer_id;
+  h->act = d->output_activation;
   h->experts.resize(d->num_experts);
   const int K = d->K, N = d->N, r = d->r, G = K / 64;
   const bool dev = d->pointers_on_device != 0;
