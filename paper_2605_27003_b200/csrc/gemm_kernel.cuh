@@ -495,11 +495,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               b1 = __ldg(reinterpret_cast<const float4*>(p.bias + ch0) + 2 * i + 1);
             }
             const float2 a0 = acc[4 * i], a1 = acc[4 * i + 1], a2 = acc[4 * i + 2], a3 = acc[4 * i + 3];
-            const int act = p.act;
-            __nv_bfloat162 o0 = __floats2bfloat162_rn(apply_activation(a0.x + b0.x, act), apply_activation(a0.y + b0.y, act));
-            __nv_bfloat162 o1 = __floats2bfloat162_rn(apply_activation(a1.x + b0.z, act), apply_activation(a1.y + b0.w, act));
-            __nv_bfloat162 o2 = __floats2bfloat162_rn(apply_activation(a2.x + b1.x, act), apply_activation(a2.y + b1.y, act));
-            __nv_bfloat162 o3 = __floats2bfloat162_rn(apply_activation(a3.x + b1.z, act), apply_activation(a3.y + b1.w, act));
+            float y[8] = {a0.x + b0.x, a0.y + b0.y, a1.x + b0.z, a1.y + b0.w, a2.x + b1.x, a2.y + b1.y, a3.x + b1.z, a3.y + b1.w};
+            if (p.act != 0) {  // uniform over the grid
+#pragma unroll
+              for (int c = 0; c < 8; ++c) y[c] = apply_activation(y[c], p.act);
+            }
+            __nv_bfloat162 o0 = __floats2bfloat162_rn(y[0], y[1]);
+            __nv_bfloat162 o1 = __floats2bfloat162_rn(y[2], y[3]);
+            __nv_bfloat162 o2 = __floats2bfloat162_rn(y[4], y[5]);
+            __nv_bfloat162 o3 = __floats2bfloat162_rn(y[6], y[7]);
             uint4 o;
             o.x = *reinterpret_cast<uint32_t*>(&o0);
             o.y = *reinterpret_cast<uint32_t*>(&o1);

@@ -20,9 +20,10 @@
 //               column); kind::f16 for [T_hi | T_lo] [L2 | L2]^T into the same accumulator first.  tcgen05.cp
 //               and tcgen05.mma of one thread execute in issue order, so one TMEM scale region serves every stage.
 //   warp 2      TMEM allocation / release.
-//   warps 4-11  epilogue: TMEM (32x32b loads, a token row per thread, 128 columns per warp) + bias -> BF16 ->
+//   warps 4-19  epilogue: TMEM (32x32b loads, a token row per thread, 64 columns per warp) + bias -> BF16 ->
 //               global.  One accumulator (256 columns) plus the scale columns fill TMEM, so the MMA warp waits
-//               for the epilogue to drain it (the loads only: ~2 % of a tile's time) before the next tile.
+//               for the epilogue to drain it before the next tile: sixteen warps pull the whole accumulator into
+//               registers at once and hand it back before they convert and store.
 //
 // Every wait is bounded exactly as in gemm_kernel.cuh (whose Ring / bounded_wait helpers are used here).
 #pragma once
@@ -38,8 +39,8 @@ namespace w4a4 {
 constexpr int kMxBN = 256;                       // output tile columns
 constexpr int kMxBK = 256;                       // K elements per stage = 128 bytes per operand row
 constexpr int kMxStages = 4;
-constexpr int kMxThreads = 384;
-constexpr int kMxEpiWarp0 = 4, kMxEpiWarps = 8;
+constexpr int kMxThreads = 640;
+constexpr int kMxEpiWarp0 = 4, kMxEpiWarps = 16;
 constexpr uint32_t kMxATile = kBM * 128;         // 16 KiB
 constexpr uint32_t kMxBTile = kMxBN * 128;       // 32 KiB
 constexpr uint32_t kMxSfTile = 2 * 512;          // scale bytes of 128 rows x 8 blocks: two atoms
@@ -233,11 +234,10 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (live && warp >= kMxEpiWarp0) {
     // ------------------------------------------------------------------ epilogue
-    // Warp ew: TMEM lanes 32 * (ew % 4) .. + 31 (token rows), columns 128 * (ew / 4) .. + 127.  The accumulator is
-    // read in two halves of 64 columns; the buffer goes back to the MMA warp as soon as the second half is in
-    // registers, before it is converted and stored.
+    // Warp ew: TMEM lanes 32 * (ew % 4) .. + 31 (token rows), columns 64 * (ew / 4) .. + 63.  The buffer goes back to
+    // the MMA warp as soon as the warp's part of it is in registers, before it is converted and stored.
     const int ew = warp - kMxEpiWarp0;
-    const int quarter = ew & 3, half = ew >> 2;
+    const int quarter = ew & 3, colblk = ew >> 2;
     Ring<1> ab;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
@@ -246,65 +246,66 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ok = bounded_wait(bar_acc_full, ab.parity, env, kErrEpilogueWait);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 128 * half;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colblk;
+      uint32_t v[4][16];
 #pragma unroll
-      for (int part = 0; part < 2; ++part) {
-        uint32_t v[4][16];
+      for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x16(t_row + 16 * c, v[c]);
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty);
+      const int ch0 = n0 + 64 * colblk;
+      if (p.yref != nullptr) {
+        // Eq. 10's objective over this thread's 64 outputs, Y_hat rounded to BF16 as the forward stores it.
+        float e = 0.0f;
+        if (row < p.M && ch0 < p.N) {
+          const uint4* yr = reinterpret_cast<const uint4*>(p.yref + static_cast<size_t>(row) * p.N + ch0);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x16(t_row + 64 * part + 16 * c, v[c]);
-        tmem_wait_ld();
-        if (part == 1) {
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_acc_empty);
-        }
-        const int ch0 = n0 + 128 * half + 64 * part;
-        if (p.yref != nullptr) {
-          // Eq. 10's objective over this thread's 64 outputs, Y_hat rounded to BF16 as the forward stores it.
-          float e = 0.0f;
-          if (row < p.M && ch0 < p.N) {
-            const uint4* yr = reinterpret_cast<const uint4*>(p.yref + static_cast<size_t>(row) * p.N + ch0);
+          for (int c = 0; c < 4; ++c) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int h = 0; h < 2; ++h) {
+              const uint4 ref = __ldg(yr + 2 * c + h);
+              const uint32_t rw[4] = {ref.x, ref.y, ref.z, ref.w};
 #pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                const uint4 ref = __ldg(yr + 2 * c + h);
-                const uint32_t rw[4] = {ref.x, ref.y, ref.z, ref.w};
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  const int col = 8 * h + i;
-                  const float b = p.bias ? __ldg(p.bias + ch0 + 16 * c + col) : 0.0f;
-                  const float y_hat = __bfloat162float(__float2bfloat16_rn(apply_activation(__uint_as_float(v[c][col]) + b, p.act)));
-                  const float y_ref = __uint_as_float((i & 1) ? (rw[i >> 1] & 0xffff0000u) : (rw[i >> 1] << 16));
-                  const float d = y_ref - y_hat;
-                  e = fmaf(d, d, e);
-                }
+              for (int i = 0; i < 8; ++i) {
+                const int col = 8 * h + i;
+                const float b = p.bias ? __ldg(p.bias + ch0 + 16 * c + col) : 0.0f;
+                const float y_hat = __bfloat162float(__float2bfloat16_rn(apply_activation(__uint_as_float(v[c][col]) + b, p.act)));
+                const float y_ref = __uint_as_float((i & 1) ? (rw[i >> 1] & 0xffff0000u) : (rw[i >> 1] << 16));
+                const float d = y_ref - y_hat;
+                e = fmaf(d, d, e);
               }
             }
           }
+        }
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-          if (lane == 0) atomicAdd(p.sq_err, static_cast<double>(e));
-        } else if (row < p.M && ch0 < p.N) {
+        for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+        if (lane == 0) atomicAdd(p.sq_err, static_cast<double>(e));
+      } else if (row < p.M && ch0 < p.N) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const int ch = ch0 + 16 * c;
-            uint4 o[2];
-            uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+        for (int c = 0; c < 4; ++c) {
+          const int ch = ch0 + 16 * c;
+          uint4 o[2];
+          uint32_t* ow = reinterpret_cast<uint32_t*>(o);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-              __nv_bfloat162 lo = __floats2bfloat162_rn(apply_activation(__uint_as_float(v[c][4 * i]) + b4.x, p.act),
-                                                        apply_activation(__uint_as_float(v[c][4 * i + 1]) + b4.y, p.act));
-              __nv_bfloat162 hi = __floats2bfloat162_rn(apply_activation(__uint_as_float(v[c][4 * i + 2]) + b4.z, p.act),
-                                                        apply_activation(__uint_as_float(v[c][4 * i + 3]) + b4.w, p.act));
-              ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
-              ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
+          for (int i = 0; i < 4; ++i) {
+            const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float y0 = __uint_as_float(v[c][4 * i]) + b4.x, y1 = __uint_as_float(v[c][4 * i + 1]) + b4.y;
+            float y2 = __uint_as_float(v[c][4 * i + 2]) + b4.z, y3 = __uint_as_float(v[c][4 * i + 3]) + b4.w;
+            if (p.act != 0) {  // uniform over the grid: the plain layer pays one predicate per four outputs
+              y0 = apply_activation(y0, p.act);
+              y1 = apply_activation(y1, p.act);
+              y2 = apply_activation(y2, p.act);
+              y3 = apply_activation(y3, p.act);
             }
-            uint4* y = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch);
-            y[0] = o[0];
-            y[1] = o[1];
+            __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(y2, y3);
+            ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
+            ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
           }
+          uint4* y = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch);
+          y[0] = o[0];
+          y[1] = o[1];
         }
       }
       ab.advance();

@@ -167,6 +167,7 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     if (st == W4A4_OK && cudaMemset(ctx->mx_sfa, 0, nb) != cudaSuccess) st = W4A4_ERR_CUDA;
     if (st == W4A4_OK)
       cudaFuncSetAttribute(mx_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMxSmemBytes));
+
     if (st == W4A4_OK)
       cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesMxfp4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            static_cast<int>(quantize_smem_bytes(64)));
