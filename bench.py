@@ -400,6 +400,28 @@ def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
     ctx.close()
 
 
+def mxfp4_context(w4, ctx, w, clip, Y, stream, iters: int = 20):
+    """The same layer shape through the MXFP4 variant (E2M1 elements, E8M0 block scales applied inside the tensor
+    core), timed on the buffers of the main run: a different quantizer, reported for context, never part of `value`."""
+    M, K, N, r = w["M"], w["K"], w["N"], w["r"]
+    lay = w4.MxLayer(ctx, [gen.make_layer_mx_direct(K, N, r, seed=2001, device=Y.device)], num_bins=w["num_bins"])
+    xs, bins = w["xs"], w["bins"]
+    for i in range(3):
+        w4.w4a4_mx_linear_forward(lay.ptr, xs[i % len(xs)], M, 0, bins[i % len(xs)], clip, Y, stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(iters):
+        w4.w4a4_mx_linear_forward(lay.ptr, xs[i % len(xs)], M, 0, bins[i % len(xs)], clip, Y, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ctx.check()
+    ms = e0.elapsed_time(e1) / iters
+    lay.close()
+    return dict(value=2.0 * M * K * N / (ms * 1e-3) / 1e12, unit=UNIT, ms_per_step=ms, steps=iters,
+                note="MXFP4 variant of the same layer shape (w4a4_mx_linear_forward): a different quantizer, for context only")
+
+
 def run_clip_search(args, w4, dev, local_rank, rank, peaks):
     """Clipping-ratio search (Eq. 10) at the attention-projection shape: six candidates, two calibration samples
     per search; every candidate runs the real forward with the squared error fused into the GEMM epilogue."""
@@ -592,6 +614,8 @@ def main():
                      path="w4a4_linear_forward_host: pinned host X -> %d-row chunks over 3 streams -> pinned host Y"
                           % chunk_rows),
             gpu_launches=3 * args.steps, clocks=clocks)
+        if args.workload != "tiny":
+            line["mxfp4_variant"] = mxfp4_context(w4, ctx, w, clip, Y, stream)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(w)
         print(json.dumps(line), flush=True)
