@@ -223,7 +223,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;  // provably warp-uniform
   const int G = p.K >> 6;
   const int n_int_stages = (G + 1) >> 1;
   const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
@@ -258,8 +258,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
-  const bool live = (*s_abort == 0);
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+  const bool live = __all_sync(0xffffffffu, *s_abort == 0);
 
   // Per tile the TMEM slots are used by: [one slot for the low-rank product, if r > 0] followed by
   // one slot per K stage (two groups, 128 columns each).

@@ -66,6 +66,21 @@ struct MxGemmParams {
   int act;              // output activation: 0 none, 1 GELU (tanh form)
 };
 
+// One lane of a converged warp.  The MMA warp runs its loop with all lanes (waits included) and only predicates
+// the tcgen05 instructions on this: everything they take as operands then stays warp-uniform for the compiler,
+// which keeps descriptors and addresses in uniform registers instead of converting them per instruction.
+__device__ __forceinline__ bool elect_one_lane() {
+  uint32_t pred;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "elect.sync _|p, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // Shared-memory descriptor of one scale atom (32 rows x 16 bytes, rows contiguous): K-major, no swizzle, 8-row
 // core matrices 128 bytes apart.
 __device__ __forceinline__ uint64_t mx_sf_desc(uint32_t smem_addr) {
@@ -117,7 +132,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;  // provably warp-uniform
   const int n_k_stages = p.K / kMxBK;
   const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
   const int atoms_k = p.K / 128;
@@ -148,8 +163,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
-  const bool live = (*s_abort == 0);
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+  const bool live = __all_sync(0xffffffffu, *s_abort == 0);
 
   // Shared-memory stage: A tile | B tile (256 rows) | scale atoms of A | of B rows 0..127 | of B rows 128..255.
   if (live && warp == 0 && lane == 0) {
@@ -183,30 +198,30 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         rg.advance();
       }
     }
-  } else if (live && warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (live && warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (all lanes loop, one issues)
     constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kMxBN);
+    const bool issuer = elect_one_lane();
     Ring<kMxStages> rg;
     Ring<1> ab;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-      ok = bounded_wait<64>(bar_acc_empty, ab.parity ^ 1u, env, kErrMmaWait);
+      ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_acc_empty, ab.parity ^ 1u, env, kErrMmaWait));
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t d = tmem_base;
       uint32_t accumulate = 0;
       for (int st = 0; ok && st < n_lr_stages + n_k_stages; ++st) {
-        ok = bounded_wait<64>(bar_full + 8 * rg.slot, rg.parity, env, kErrMmaWait);
+        ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_full + 8 * rg.slot, rg.parity, env, kErrMmaWait));
         if (!ok) break;
-        tc_fence_after_sync();
         const uint32_t a = smem_base + rg.slot * kMxStageBytes, b = a + kMxATile;
         if (st < n_lr_stages) {
+          if (issuer) {
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            umma_f16(d, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_bf16, accumulate);
-            accumulate = 1;
+            for (int kk = 0; kk < 4; ++kk)
+              umma_f16(d, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_bf16, kk > 0 ? 1u : accumulate);
           }
-        } else {
+        } else if (issuer) {
           // TMEM scale columns: A: 4 per K atom (one per 32 rows); B: 8 per K atom (256 rows).  The columns of
           // a missing upper half keep whatever they held: they scale zero operands into columns never stored.
           const uint32_t sf = b + kMxBTile;
@@ -221,15 +236,15 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t id = 2u * (j & 1);
             umma_mxf4(d, umma_desc_k_sw128(a, 32 * j), umma_desc_k_sw128(b, 32 * j), mx_idesc(kBM, kMxBN, id, id),
                       (tmem_base + kMxTmemSfA + 4 * (j >> 1)) | (id << 30), (tmem_base + kMxTmemSfB + 8 * (j >> 1)) | (id << 30),
-                      accumulate);
-            accumulate = 1;
+                      j > 0 ? 1u : accumulate);
           }
         }
-        umma_commit(bar_empty + 8 * rg.slot);
+        accumulate = 1;
+        if (issuer) umma_commit(bar_empty + 8 * rg.slot);
         rg.advance();
       }
       if (!ok) break;
-      umma_commit(bar_acc_full);
+      if (issuer) umma_commit(bar_acc_full);
       ab.advance();
     }
   } else if (live && warp >= kMxEpiWarp0) {
@@ -323,6 +338,323 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 2) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// The same GEMM on pairs of CTAs (a thread-block cluster of two, tcgen05 cta_group::2).  mx_gemm_kernel is bound
+// by the bytes that come from L2 into shared memory.  With cta_group::2 one MMA spans both SMs of the pair: a
+// 256 x 256 x 64 product whose A rows 0..127 / 128..255 and whose B rows (output columns) 0..127 / 128..255 lie in
+// the shared memory of CTA 0 / CTA 1, at the same offsets, and whose accumulator rows land in the TMEM of the CTA
+// that holds the A rows.  Each CTA therefore fetches its own A tile and only HALF of the B tile: 35 KB per stage
+// instead of 51 KB for the same 128 x 256 outputs per CTA, and the ring is six stages deep instead of four.
+//
+// CTA 0 (the leader) issues every tcgen05.cp and tcgen05.mma for the pair.  Cross-CTA signalling:
+//   full[s]    (leader)   both CTAs' TMA loads of stage s report their bytes here (cta_group::2 loads may name a
+//                         barrier of the neighbour); the leader's producer posts the expected total;
+//   empty[s]   (both)     the leader commits its MMAs onto its own barrier and onto the neighbour's;
+//   acc_full   (both)     likewise;
+//   acc_empty  (leader)   all 32 epilogue warps of the pair have pulled their part of the accumulator.
+// Scale factors: every CTA needs the A scales of its own rows and the B scales of all 256 columns in its own TMEM;
+// tcgen05.cp.cta_group::2 copies them from each CTA's own shared memory.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// 2D tiled load into this CTA's shared memory whose byte count is reported to `bar_cluster_addr`, a barrier of
+// this CTA or of the other CTA of the pair.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst_smem, const CUtensorMap* tm, uint32_t bar_cluster_addr, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_cp2_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void umma2_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t tsfa,
+                                           uint32_t tsfb, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+      : "memory");
+}
+__device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier at `cluster_addr` (this CTA's or the neighbour's) once the pair's MMAs issued so far are done.
+__device__ __forceinline__ void umma2_commit(uint32_t cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+constexpr int kMx2Stages = 6;
+constexpr uint32_t kMx2BHalf = kMxBTile / 2;                                  // 16 KiB: this CTA's 128 rows of B
+constexpr uint32_t kMx2StageBytes = kMxATile + kMx2BHalf + 3 * kMxSfTile;      // 35 KiB
+constexpr uint32_t kMx2NumBarriers = 2 * kMx2Stages + 2;
+constexpr uint32_t kMx2SmemBytes = 1024 + kMx2Stages * kMx2StageBytes + kMx2NumBarriers * 8 + 16;
+static_assert(kMx2StageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned");
+
+__global__ void __launch_bounds__(kMxThreads, 1)
+mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBhalf,
+                const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL2half,
+                const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB, const MxGemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kMx2Stages * kMx2StageBytes;
+  const uint32_t bar_full = bar_base;
+  const uint32_t bar_empty = bar_full + 8 * kMx2Stages;
+  const uint32_t bar_acc_full = bar_empty + 8 * kMx2Stages;
+  const uint32_t bar_acc_empty = bar_acc_full + 8;
+  const uint32_t misc_off = (bar_acc_empty + 8) - smem_base;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
+
+  const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;  // provably warp-uniform
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int n_k_stages = p.K / kMxBK;
+  const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
+  const int num_items = ((p.tiles_m + 1) / 2) * p.tiles_n;
+  const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+  const WaitEnv env{p.err, s_abort};
+
+  if (threadIdx.x == 0) {
+    *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
+    for (int i = 0; i < kMx2Stages; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    mbar_init(bar_acc_full, 1);
+    mbar_init(bar_acc_empty, 2 * kMxEpiWarps);
+    mbar_fence_init();
+    fence_proxy_async_smem();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmBhalf);
+    tma_prefetch_desc(&tmSFA);
+    tma_prefetch_desc(&tmSFB);
+    if (p.r > 0) {
+      tma_prefetch_desc(&tmT);
+      tma_prefetch_desc(&tmL2half);
+    }
+  }
+  if (warp == 2) {
+    tmem_alloc2(smem_u32(tmem_slot), 512);
+    tc_fence_before_sync();
+  }
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers and TMEM exist before anything crosses over
+  tc_fence_after_sync();
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+  const bool live = __all_sync(0xffffffffu, *s_abort == 0);
+
+  // Shared-memory stage: A tile | this CTA's half of B | scale atoms of A | of B columns 0..127 | of B columns 128..255.
+  if (live && warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ producer (both CTAs)
+    // Rows and columns past the matrices (an odd count of row tiles; N = 128 mod 256) are filled with zeros by the
+    // TMA unit and still count their bytes, so every stage reports the same total.
+    Ring<kMx2Stages> rg;
+    bool ok = true;
+    for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
+      const int tm = 2 * (item / p.tiles_n) + static_cast<int>(rank), tn = item % p.tiles_n;
+      const int m0 = tm * kBM, n0 = tn * kMxBN;
+      for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
+        ok = bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait);
+        if (!ok) break;
+        const uint32_t full = map_to_cta(bar_full + 8 * rg.slot, 0);
+        const uint32_t dst = smem_base + rg.slot * kMx2StageBytes;
+        if (st < n_lr_stages) {
+          if (leader) mbar_arrive_expect_tx(bar_full + 8 * rg.slot, 2 * (kMxATile + kMx2BHalf));
+          tma2_load_2d(dst, &tmT, full, st * 64, m0);
+          tma2_load_2d(dst + kMxATile, &tmL2half, full, st * 64, n0 + 128 * static_cast<int>(rank));
+        } else {
+          const int ks = st - n_lr_stages;
+          const uint32_t sf = dst + kMxATile + kMx2BHalf;
+          if (leader) mbar_arrive_expect_tx(bar_full + 8 * rg.slot, 2 * kMx2StageBytes);
+          tma2_load_2d(dst, &tmA, full, ks * 128, m0);
+          tma2_load_2d(dst + kMxATile, &tmBhalf, full, ks * 128, n0 + 128 * static_cast<int>(rank));
+          tma2_load_2d(sf, &tmSFA, full, ks * 256, tm);
+          tma2_load_2d(sf + kMxSfTile, &tmSFB, full, ks * 256, 2 * tn);
+          tma2_load_2d(sf + 2 * kMxSfTile, &tmSFB, full, ks * 256, 2 * tn + 1);
+        }
+        rg.advance();
+      }
+    }
+  } else if (live && warp == 1 && leader) {
+    // ------------------------------------------------------------------ MMA issuer (CTA 0, for the pair)
+    constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, 2 * kBM, kMxBN);
+    const bool issuer = elect_one_lane();
+    const uint32_t peer_empty = map_to_cta(bar_empty, 1), peer_acc_full = map_to_cta(bar_acc_full, 1);
+    Ring<kMx2Stages> rg;
+    Ring<1> ab;
+    bool ok = true;
+    for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
+      ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_acc_empty, ab.parity ^ 1u, env, kErrMmaWait));
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t d = tmem_base;
+      uint32_t accumulate = 0;
+      for (int st = 0; ok && st < n_lr_stages + n_k_stages; ++st) {
+        ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_full + 8 * rg.slot, rg.parity, env, kErrMmaWait));
+        if (!ok) break;
+        const uint32_t a = smem_base + rg.slot * kMx2StageBytes, b = a + kMxATile;
+        if (st < n_lr_stages) {
+          if (issuer) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma2_f16(d, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_bf16, kk > 0 ? 1u : accumulate);
+          }
+        } else if (issuer) {
+          const uint32_t sf = b + kMx2BHalf;
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            tmem_cp2_32x128b_warpx4(tmem_base + kMxTmemSfA + 4 * t, mx_sf_desc(sf + 512 * t));
+            tmem_cp2_32x128b_warpx4(tmem_base + kMxTmemSfB + 8 * t, mx_sf_desc(sf + kMxSfTile + 512 * t));
+            tmem_cp2_32x128b_warpx4(tmem_base + kMxTmemSfB + 8 * t + 4, mx_sf_desc(sf + 2 * kMxSfTile + 512 * t));
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t id = 2u * (j & 1);
+            umma2_mxf4(d, umma_desc_k_sw128(a, 32 * j), umma_desc_k_sw128(b, 32 * j), mx_idesc(2 * kBM, kMxBN, id, id),
+                       (tmem_base + kMxTmemSfA + 4 * (j >> 1)) | (id << 30), (tmem_base + kMxTmemSfB + 8 * (j >> 1)) | (id << 30),
+                       j > 0 ? 1u : accumulate);
+          }
+        }
+        accumulate = 1;
+        if (issuer) {
+          umma2_commit(bar_empty + 8 * rg.slot);
+          umma2_commit(peer_empty + 8 * rg.slot);
+        }
+        rg.advance();
+      }
+      if (!ok) break;
+      if (issuer) {
+        umma2_commit(bar_acc_full);
+        umma2_commit(peer_acc_full);
+      }
+      ab.advance();
+    }
+  } else if (live && warp >= kMxEpiWarp0) {
+    // ------------------------------------------------------------------ epilogue (both CTAs, own rows)
+    const int ew = warp - kMxEpiWarp0;
+    const int quarter = ew & 3, colblk = ew >> 2;
+    const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
+    Ring<1> ab;
+    bool ok = true;
+    for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
+      const int m0 = (2 * (item / p.tiles_n) + static_cast<int>(rank)) * kBM, n0 = (item % p.tiles_n) * kMxBN;
+      const int row = m0 + 32 * quarter + lane;
+      ok = bounded_wait(bar_acc_full, ab.parity, env, kErrEpilogueWait);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + 64 * colblk;
+      uint32_t v[4][16];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x16(t_row + 16 * c, v[c]);
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(acc_empty_leader);
+      const int ch0 = n0 + 64 * colblk;
+      if (p.yref != nullptr) {
+        float e = 0.0f;
+        if (row < p.M && ch0 < p.N) {
+          const uint4* yr = reinterpret_cast<const uint4*>(p.yref + static_cast<size_t>(row) * p.N + ch0);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const uint4 ref = __ldg(yr + 2 * c + h);
+              const uint32_t rw[4] = {ref.x, ref.y, ref.z, ref.w};
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int col = 8 * h + i;
+                const float b = p.bias ? __ldg(p.bias + ch0 + 16 * c + col) : 0.0f;
+                const float y_hat = __bfloat162float(__float2bfloat16_rn(apply_activation(__uint_as_float(v[c][col]) + b, p.act)));
+                const float y_ref = __uint_as_float((i & 1) ? (rw[i >> 1] & 0xffff0000u) : (rw[i >> 1] << 16));
+                const float d = y_ref - y_hat;
+                e = fmaf(d, d, e);
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+        if (lane == 0) atomicAdd(p.sq_err, static_cast<double>(e));
+      } else if (row < p.M && ch0 < p.N) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int ch = ch0 + 16 * c;
+          uint4 o[2];
+          uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float4 b4 = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float y0 = __uint_as_float(v[c][4 * i]) + b4.x, y1 = __uint_as_float(v[c][4 * i + 1]) + b4.y;
+            float y2 = __uint_as_float(v[c][4 * i + 2]) + b4.z, y3 = __uint_as_float(v[c][4 * i + 3]) + b4.w;
+            if (p.act != 0) {
+              y0 = apply_activation(y0, p.act);
+              y1 = apply_activation(y1, p.act);
+              y2 = apply_activation(y2, p.act);
+              y3 = apply_activation(y3, p.act);
+            }
+            __nv_bfloat162 lo = __floats2bfloat162_rn(y0, y1);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(y2, y3);
+            ow[2 * i] = *reinterpret_cast<uint32_t*>(&lo);
+            ow[2 * i + 1] = *reinterpret_cast<uint32_t*>(&hi);
+          }
+          uint4* y = reinterpret_cast<uint4*>(p.Y + static_cast<size_t>(row) * p.N + ch);
+          y[0] = o[0];
+          y[1] = o[1];
+        }
+      }
+      ab.advance();
+    }
+  }
+
+  // ---------------------------------------------------------------------- common tail
+  tc_fence_before_sync();
+  __syncthreads();
+  if (*s_abort) {
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  cluster_sync_all();  // nothing may still be in flight towards a CTA that is about to leave
+  if (warp == 2) {
+    tc_fence_after_sync();
+    tmem_dealloc2(tmem_base, 512);
   }
 }
 

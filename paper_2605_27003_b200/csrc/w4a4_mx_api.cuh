@@ -12,6 +12,8 @@ struct MxExpertData {
   uint16_t* l2dup = nullptr;   // [N, 2r]
   float* bias = nullptr;       // [N] or null
   CUtensorMap tmB, tmL2;
+  CUtensorMap tmBhalf, tmL2half;   // 128-row boxes: what one CTA of a pair fetches (mx_gemm2_kernel)
+  CUtensorMap tmSFB;               // scale atoms as 32-bit words: [N/128] rows of K words, boxes of 1 KiB
 };
 
 struct w4a4_mx_layer {
@@ -19,6 +21,7 @@ struct w4a4_mx_layer {
   int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0, act = 0;
   std::vector<MxExpertData> experts;
   CUtensorMap tmA, tmT;
+  CUtensorMap tmSFA;               // activation scale atoms as 32-bit words: [max_M/128] rows of K words
   size_t bytes = 0;
 };
 
@@ -107,6 +110,33 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;  // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
+  // CTA pairs (cta_group::2) need at least two row tiles and an even number of CTAs.
+  static const bool pair_allowed = [] {
+    const char* v = std::getenv("W4A4_MX_GEMM");
+    return !(v && std::strcmp(v, "single") == 0);
+  }();
+  if (pair_allowed && p.tiles_m >= 2 && ctx->num_sms >= 2) {
+    const int items = ((p.tiles_m + 1) / 2) * p.tiles_n;
+    const int ctas = 2 * items < ctx->num_sms ? 2 * items : (ctx->num_sms & ~1);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctas);
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = kMx2SmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const CUtensorMap& tmL2h = h->r > 0 ? e.tmL2half : e.tmBhalf;
+    if (cudaLaunchKernelEx(&cfg, mx_gemm2_kernel, h->tmA, e.tmBhalf, tmT, tmL2h, h->tmSFA, e.tmSFB, p) != cudaSuccess) {
+      cudaGetLastError();
+      return W4A4_ERR_CUDA;
+    }
+    return W4A4_OK;
+  }
   mx_gemm_kernel<<<grid, block, kMxSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
@@ -167,6 +197,8 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     if (st == W4A4_OK && cudaMemset(ctx->mx_sfa, 0, nb) != cudaSuccess) st = W4A4_ERR_CUDA;
     if (st == W4A4_OK)
       cudaFuncSetAttribute(mx_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMxSmemBytes));
+    if (st == W4A4_OK)
+      cudaFuncSetAttribute(mx_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMx2SmemBytes));
 
     if (st == W4A4_OK)
       cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesMxfp4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -223,6 +255,18 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     if (!encode_2d(ctx->encode, &e.tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, 128, kMxBN,
                    CU_TENSOR_MAP_SWIZZLE_128B))
       st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK &&
+        !encode_2d(ctx->encode, &e.tmBhalf, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, e.bpacked, K / 2, N, K / 2, 128, kMxBN / 2,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+      st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK &&
+        !encode_2d(ctx->encode, &e.tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, e.sfb, K, N / 128, 4 * static_cast<uint64_t>(K), 256,
+                   1, CU_TENSOR_MAP_SWIZZLE_NONE))
+      st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK && r > 0 &&
+        !encode_2d(ctx->encode, &e.tmL2half, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kMxBN / 2,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+      st = W4A4_ERR_CUDA;
     if (st == W4A4_OK && r > 0 &&
         !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kMxBN,
                    CU_TENSOR_MAP_SWIZZLE_128B))
@@ -237,6 +281,10 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
   if (st == W4A4_OK &&
       !encode_2d(ctx->encode, &h->tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->codes, K / 2, ctx->max_M, K / 2, 128, kBM,
                  CU_TENSOR_MAP_SWIZZLE_128B))
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK &&
+      !encode_2d(ctx->encode, &h->tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, ctx->mx_sfa, K, (ctx->max_M + 127) / 128,
+                 4 * static_cast<uint64_t>(K), 256, 1, CU_TENSOR_MAP_SWIZZLE_NONE))
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK && r > 0 &&
       !encode_2d(ctx->encode, &h->tmT, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo, 2 * r, ctx->max_M, 4 * r, 64,
