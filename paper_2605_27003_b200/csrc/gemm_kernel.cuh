@@ -118,6 +118,19 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, cons
 
 // Position in a ring of N mbarrier pairs: slot index and the parity of the phase a consumer waits
 // for (a producer waits for parity ^ 1).  Advanced incrementally: no division in the hot loops.
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one_lane() {
+  uint32_t pred;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "elect.sync _|p, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 template <int N>
 struct Ring {
   uint32_t slot = 0, parity = 0;
@@ -265,8 +278,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   // one slot per K stage (two groups, 128 columns each).
   if (warp < kEpiWarp0) {
     set_max_regs_dec<kRegsControl>();
-    if (live && warp == 0 && lane == 0) {
+    if (live && warp == 0) {
       // ------------------------------------------------------------------ TMA producer
+      // All lanes run the loop (waits included) and one elected lane issues: what the TMA and tcgen05
+      // instructions take as operands then stays warp-uniform for the compiler, which keeps it in uniform
+      // registers instead of converting per instruction.
+      const bool issuer = elect_one_lane();
       // Slots of the operand ring in the order the MMA warp consumes them: per tile the low-rank stages
       // (T and the duplicated L2 factor, BF16) first, then the code stages with their scales.
       Ring<kOpStages> op;
@@ -275,71 +292,80 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
         for (int st = 0; st < n_lr_stages + n_int_stages; ++st) {
-          ok = bounded_wait<128>(bar_op_empty + 8 * op.slot, op.parity ^ 1u, env, kErrProducerWait);
+          ok = __all_sync(0xffffffffu, bounded_wait<128>(bar_op_empty + 8 * op.slot, op.parity ^ 1u, env, kErrProducerWait));
           if (!ok) break;
           const uint32_t full = bar_op_full + 8 * op.slot;
           const uint32_t dst = op_base + op.slot * kOpStageBytes;
           if (st < n_lr_stages) {
-            mbar_arrive_expect_tx(full, kOpStageBytes);
-            tma_load_2d(dst, &tmT, full, st * 64, m0);
-            tma_load_2d(dst + kOpATile, &tmL2, full, st * 64, n0);
+            if (issuer) {
+              mbar_arrive_expect_tx(full, kOpStageBytes);
+              tma_load_2d(dst, &tmT, full, st * 64, m0);
+              tma_load_2d(dst + kOpATile, &tmL2, full, st * 64, n0);
+            }
           } else {
             const int ks = st - n_lr_stages;
             const uint32_t sdst = scale_base + sc.slot * kScaleStageBytes;
-            mbar_arrive_expect_tx(full, kOpStageBytes + kScaleStageBytes);
-            tma_load_2d(dst, &tmA, full, ks * kBK, m0);
-            tma_load_2d(dst + kOpATile, &tmB, full, ks * kBK, n0);
-            tma_load_2d(sdst, &tmSW, full, n0, 2 * ks);
-            tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * ks);
+            if (issuer) {
+              mbar_arrive_expect_tx(full, kOpStageBytes + kScaleStageBytes);
+              tma_load_2d(dst, &tmA, full, ks * kBK, m0);
+              tma_load_2d(dst + kOpATile, &tmB, full, ks * kBK, n0);
+              tma_load_2d(sdst, &tmSW, full, n0, 2 * ks);
+              tma_load_2d(sdst + 2 * kBN * 4, &tmSA, full, m0, 2 * ks);
+            }
             sc.advance();
           }
           op.advance();
         }
       }
-    } else if (live && warp == 1 && lane == 0) {
-      // ------------------------------------------------------------------ MMA issuer
+    } else if (live && warp == 1) {
+      // ------------------------------------------------------------------ MMA issuer (all lanes loop, one issues)
       constexpr uint32_t idesc_f8 = umma_idesc(1, 0, kBM, kBN);
       constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
+      const bool issuer = elect_one_lane();
       Ring<kOpStages> op;
       Ring<kTmemSlots> tm;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         if (n_lr_stages > 0) {
-          ok = bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait);
+          ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait));
           for (int l = 0; ok && l < n_lr_stages; ++l) {
-            ok = bounded_wait<64>(bar_op_full + 8 * op.slot, op.parity, env, kErrMmaWait);
+            ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_op_full + 8 * op.slot, op.parity, env, kErrMmaWait));
             if (!ok) break;
             tc_fence_after_sync();
             const uint32_t a = op_base + op.slot * kOpStageBytes, b = a + kOpATile;
+            if (issuer) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-              umma_f16(tmem_base + tm.slot * 2 * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk),
-                       idesc_bf16, (l > 0 || kk > 0) ? 1u : 0u);
+              for (int kk = 0; kk < 4; ++kk) {
+                umma_f16(tmem_base + tm.slot * 2 * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk),
+                         idesc_bf16, (l > 0 || kk > 0) ? 1u : 0u);
+              }
+              umma_commit(bar_op_empty + 8 * op.slot);
             }
-            umma_commit(bar_op_empty + 8 * op.slot);
             op.advance();
           }
           if (!ok) break;
-          umma_commit(bar_tmem_full + 8 * tm.slot);
+          if (issuer) umma_commit(bar_tmem_full + 8 * tm.slot);
           tm.advance();
         }
         for (int st = 0; ok && st < n_int_stages; ++st) {
-          ok = bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait) &&
-               bounded_wait<64>(bar_op_full + 8 * op.slot, op.parity, env, kErrMmaWait);
+          ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait) &&
+                                           bounded_wait<64>(bar_op_full + 8 * op.slot, op.parity, env, kErrMmaWait));
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t a = op_base + op.slot * kOpStageBytes, b = a + kOpATile;
           const uint32_t d = tmem_base + tm.slot * 2 * kBN;
           const int groups = (2 * st + 1 < G) ? 2 : 1;
+          if (issuer) {
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {  // bytes [32 kk, 32 kk + 32) of every row: group kk / 2, K half kk % 2
-            if (kk < 2 * groups) {
-              umma_f8(d + (kk >> 1) * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_f8,
-                      kk & 1);
+            for (int kk = 0; kk < 4; ++kk) {  // bytes [32 kk, 32 kk + 32) of every row: group kk / 2, K half kk % 2
+              if (kk < 2 * groups) {
+                umma_f8(d + (kk >> 1) * kBN, umma_desc_k_sw128(a, 32 * kk), umma_desc_k_sw128(b, 32 * kk), idesc_f8,
+                        kk & 1);
+              }
             }
+            umma_commit(bar_op_empty + 8 * op.slot);
+            umma_commit(bar_tmem_full + 8 * tm.slot);
           }
-          umma_commit(bar_op_empty + 8 * op.slot);
-          umma_commit(bar_tmem_full + 8 * tm.slot);
           op.advance();
           tm.advance();
         }
@@ -372,7 +398,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float2 acc[16];  // pair k: channels ch0 + 2 k, ch0 + 2 k + 1
         uint32_t vA[16], vB[16];
         // First slot of the tile.
-        ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
+        ok = __all_sync(0xffffffffu, bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait));
         if (!ok) break;
         tc_fence_after_sync();
         tmem_ld_32x32b_x16(t_lane + tm.slot * 2 * kBN, vA);
@@ -387,7 +413,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
           tm.advance();
-          ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
+          ok = __all_sync(0xffffffffu, bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait));
           if (!ok) break;
           tc_fence_after_sync();
           tmem_ld_32x32b_x16(t_lane + tm.slot * 2 * kBN, vA);
@@ -444,7 +470,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           tm.advance();
           if (!last_stage) {
-            ok = bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait);
+            ok = __all_sync(0xffffffffu, bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait));
             if (!ok) break;
             tc_fence_after_sync();
             tmem_ld_32x32b_x16_before(t_lane + tm.slot * 2 * kBN, vA, vB[0]);

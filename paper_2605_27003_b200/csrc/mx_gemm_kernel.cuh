@@ -68,18 +68,8 @@ struct MxGemmParams {
 
 // One lane of a converged warp.  The MMA warp runs its loop with all lanes (waits included) and only predicates
 // the tcgen05 instructions on this: everything they take as operands then stays warp-uniform for the compiler,
-// which keeps descriptors and addresses in uniform registers instead of converting them per instruction.
-__device__ __forceinline__ bool elect_one_lane() {
-  uint32_t pred;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "elect.sync _|p, 0xffffffff;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(pred));
-  return pred != 0;
-}
+// which keeps descriptors and addresses in uniform registers instead of converting them per instruction
+// (elect_one_lane() comes from gemm_kernel.cuh).
 
 // Shared-memory descriptor of one scale atom (32 rows x 16 bytes, rows contiguous): K-major, no swizzle, 8-row
 // core matrices 128 bytes apart.
@@ -167,8 +157,9 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const bool live = __all_sync(0xffffffffu, *s_abort == 0);
 
   // Shared-memory stage: A tile | B tile (256 rows) | scale atoms of A | of B rows 0..127 | of B rows 128..255.
-  if (live && warp == 0 && lane == 0) {
-    // ------------------------------------------------------------------ producer
+  if (live && warp == 0) {
+    // ------------------------------------------------------------------ producer (all lanes loop, one issues)
+    const bool issuer = elect_one_lane();
     Ring<kMxStages> rg;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
@@ -176,15 +167,17 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = tm * kBM, n0 = tn * kMxBN;
       const bool upper = n0 + 128 < p.N;  // does the tile's second 128-column half exist?
       for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
-        ok = bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait);
+        ok = __all_sync(0xffffffffu, bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait));
         if (!ok) break;
         const uint32_t full = bar_full + 8 * rg.slot;
         const uint32_t dst = smem_base + rg.slot * kMxStageBytes;
         if (st < n_lr_stages) {
-          mbar_arrive_expect_tx(full, kMxATile + kMxBTile);
-          tma_load_2d(dst, &tmT, full, st * 64, m0);
-          tma_load_2d(dst + kMxATile, &tmL2, full, st * 64, n0);  // rows past N arrive as zeros
-        } else {
+          if (issuer) {
+            mbar_arrive_expect_tx(full, kMxATile + kMxBTile);
+            tma_load_2d(dst, &tmT, full, st * 64, m0);
+            tma_load_2d(dst + kMxATile, &tmL2, full, st * 64, n0);  // rows past N arrive as zeros
+          }
+        } else if (issuer) {
           const int ks = st - n_lr_stages;
           const uint32_t sf = dst + kMxATile + kMxBTile;
           mbar_arrive_expect_tx(full, kMxATile + kMxBTile + (upper ? 3u : 2u) * kMxSfTile);
@@ -371,8 +364,11 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Relaxed on purpose: the arrive only hands TMEM columns back (tcgen05.wait::ld has completed the reads, the
+// tcgen05 fence orders them); a release at cluster scope would also wait for the warp's earlier global stores
+// (the previous tile's outputs) to become visible, which cost about 1200 clocks per tile.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // 2D tiled load into this CTA's shared memory whose byte count is reported to `bar_cluster_addr`, a barrier of
 // this CTA or of the other CTA of the pair.
@@ -480,25 +476,29 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const bool live = __all_sync(0xffffffffu, *s_abort == 0);
 
   // Shared-memory stage: A tile | this CTA's half of B | scale atoms of A | of B columns 0..127 | of B columns 128..255.
-  if (live && warp == 0 && lane == 0) {
-    // ------------------------------------------------------------------ producer (both CTAs)
+  if (live && warp == 0) {
+    // ------------------------------------------------------------------ producer (both CTAs; all lanes loop, one issues)
     // Rows and columns past the matrices (an odd count of row tiles; N = 128 mod 256) are filled with zeros by the
     // TMA unit and still count their bytes, so every stage reports the same total.
+    const bool issuer = elect_one_lane();
+    const uint32_t full0 = map_to_cta(bar_full, 0);
     Ring<kMx2Stages> rg;
     bool ok = true;
     for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
       const int tm = 2 * (item / p.tiles_n) + static_cast<int>(rank), tn = item % p.tiles_n;
       const int m0 = tm * kBM, n0 = tn * kMxBN;
       for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
-        ok = bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait);
+        ok = __all_sync(0xffffffffu, bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait));
         if (!ok) break;
-        const uint32_t full = map_to_cta(bar_full + 8 * rg.slot, 0);
+        const uint32_t full = full0 + 8 * rg.slot;
         const uint32_t dst = smem_base + rg.slot * kMx2StageBytes;
         if (st < n_lr_stages) {
-          if (leader) mbar_arrive_expect_tx(bar_full + 8 * rg.slot, 2 * (kMxATile + kMx2BHalf));
-          tma2_load_2d(dst, &tmT, full, st * 64, m0);
-          tma2_load_2d(dst + kMxATile, &tmL2half, full, st * 64, n0 + 128 * static_cast<int>(rank));
-        } else {
+          if (issuer) {
+            if (leader) mbar_arrive_expect_tx(bar_full + 8 * rg.slot, 2 * (kMxATile + kMx2BHalf));
+            tma2_load_2d(dst, &tmT, full, st * 64, m0);
+            tma2_load_2d(dst + kMxATile, &tmL2half, full, st * 64, n0 + 128 * static_cast<int>(rank));
+          }
+        } else if (issuer) {
           const int ks = st - n_lr_stages;
           const uint32_t sf = dst + kMxATile + kMx2BHalf;
           if (leader) mbar_arrive_expect_tx(bar_full + 8 * rg.slot, 2 * kMx2StageBytes);
