@@ -62,6 +62,10 @@ constexpr int kEpiWarp0 = 4, kEpiWarps = 16;
 constexpr int kEpiCols = kBN / (kEpiWarps / 4);   // output channels per epilogue thread (32)
 constexpr int kRegsControl = 40, kRegsEpilogue = 104;   // setmaxnreg budgets per role: 4 x 32 x 40 + 16 x 32 x 104 fits the
                                                         // 640 x 96 registers the CTA is launched with
+// setmaxnreg.inc blocks until the CTA's own allocation (threads x the compiled register count, which the launch
+// bound fixes at 96) has that many registers free: a budget above it never returns.
+static_assert(kEpiWarp0 * 32 * kRegsControl + kEpiWarps * 32 * kRegsEpilogue <= kGemmThreads * 96,
+              "setmaxnreg budgets exceed the registers the CTA is launched with");
 
 constexpr uint32_t kOpATile = kBM * kBK;             // 16 KiB
 constexpr uint32_t kOpBTile = kBN * kBK;             // 16 KiB
