@@ -389,7 +389,7 @@ def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
         config=dict(workload=args.workload, M=M, K=K, N=N, r=r, block=32, experts=1, bins=num_bins,
                     l2="inputs larger than L2: 4 rotating activation buffers of %.0f MB" % (M * K * 2 / 1e6)),
         roofline=dict(bound="tensor", achieved=gemm_tops, peak=fp4_peak, unit="TOP/s", frac=gemm_tops / fp4_peak,
-                      traffic=None, kernel="mx_gemm_kernel", ms=tg,
+                      traffic=None, kernel="mx_gemm2_kernel (CTA pairs; mx_gemm_kernel when M <= 128)", ms=tg,
                       peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 4 "
                                   "(nominal FP4:BF16 ratio)", frac_of_nominal_9000=gemm_tops / 9000.0),
         roofline_quantize=dict(bound="hbm", achieved=q_bytes / (tq * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",

@@ -230,6 +230,22 @@ w4a4_status_t w4a4_mx_clip_search(w4a4_mx_handle_t h, const void* const* X_sampl
 w4a4_status_t w4a4_mx_debug_quantize(w4a4_mx_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
                                      const float* clip_table, uint8_t* codes, uint8_t* exps, float* T, void* stream);
 
+/* Two consecutive layers of the MXFP4 variant in one call (Sec. III: the FFN, whose second linear reads the
+ * activation of the first; Eq. 7 and Eq. 8-9 for both).  `up` runs as w4a4_mx_linear_forward does, except that the
+ * epilogue of its GEMM applies bias and output activation, rounds to BF16 and then does the work of `down`'s
+ * activation kernel on the result (smoothing by `down`'s lambda, MXFP4 codes and block exponents with `down`'s clip
+ * ratio, the low-rank projection onto `down`'s L1) into a second workspace of the context; `down`'s GEMM reads it
+ * from there and writes Y.  The intermediate activation [M, up.N] is never stored.  The result equals
+ * w4a4_mx_linear_forward(up) followed by w4a4_mx_linear_forward(down) except for the summation order of T.
+ *   X  device BF16 [M, up.K], 16-byte aligned;  Y  device BF16 [M, down.N], 16-byte aligned;  both handles on the
+ *   same context with up.N == down.K; expert_id, timestep_bin, clip_table as for the single layer (each layer
+ *   reads its own entry).  M > 128 (else W4A4_ERR_SHAPE).  Asynchronous on `stream`; errors as the single layer. */
+w4a4_status_t w4a4_mx_ffn_forward(w4a4_mx_handle_t up, w4a4_mx_handle_t down, const void* X, int M, int expert_id,
+                                  int timestep_bin, const float* clip_table, void* Y, void* stream);
+/* Parity tap: decodes what the last w4a4_mx_ffn_forward left for `down` in the second workspace: codes device
+ * uint8 [M, down.K], exps device uint8 [M, down.K/32], T device FP32 [M, down.r] or NULL. */
+w4a4_status_t w4a4_mx_debug_fused_input(w4a4_mx_handle_t down, int M, uint8_t* codes, uint8_t* exps, float* T, void* stream);
+
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
  * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
 w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);

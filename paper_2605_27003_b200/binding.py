@@ -26,7 +26,8 @@ EXPORTED_SYMBOLS = (
     "w4a4_ctx_enable_host_io", "w4a4_linear_forward_host", "w4a4_quantize_activations", "w4a4_gemm_from_workspace", "w4a4_debug_quantize", "w4a4_debug_partials",
     "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search",
     "w4a4_mx_pack_weights", "w4a4_mx_destroy", "w4a4_mx_handle_bytes", "w4a4_mx_linear_forward",
-    "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_mx_clip_search", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
+    "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_mx_clip_search",
+    "w4a4_mx_ffn_forward", "w4a4_mx_debug_fused_input", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
 
@@ -97,6 +98,8 @@ def _lib():
         lib.w4a4_mx_quantize_activations.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         lib.w4a4_mx_gemm_from_workspace.argtypes = [vp, ci, ci, vp, vp]
         lib.w4a4_mx_debug_quantize.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.w4a4_mx_ffn_forward.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, vp]
+        lib.w4a4_mx_debug_fused_input.argtypes = [vp, ci, vp, vp, vp, vp]
         lib.w4a4_mx_clip_search.argtypes = lib.w4a4_clip_search.argtypes
         lib.w4a4_tile_shape.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
         lib.w4a4_tile_shape.restype = None
@@ -319,6 +322,16 @@ def w4a4_mx_gemm_from_workspace(handle, M, expert_id, Y, stream=None):
 def w4a4_mx_debug_quantize(handle, X, M, expert_id, timestep_bin, clip_table, codes, exps, T=None, stream=None):
     _check(_lib().w4a4_mx_debug_quantize(handle, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table), _ptr(codes),
                                          _ptr(exps), _ptr(T), _stream(stream)), "w4a4_mx_debug_quantize")
+
+
+def w4a4_mx_ffn_forward(up, down, X, M, expert_id, timestep_bin, clip_table, Y, stream=None):
+    _check(_lib().w4a4_mx_ffn_forward(up, down, _ptr(X), M, expert_id, timestep_bin, _ptr(clip_table), _ptr(Y),
+                                      _stream(stream)), "w4a4_mx_ffn_forward")
+
+
+def w4a4_mx_debug_fused_input(down, M, codes, exps, T=None, stream=None):
+    _check(_lib().w4a4_mx_debug_fused_input(down, M, _ptr(codes), _ptr(exps), _ptr(T), _stream(stream)),
+           "w4a4_mx_debug_fused_input")
 
 
 def w4a4_query_status(ctx) -> int:

@@ -22,6 +22,12 @@ struct w4a4_ctx {
   size_t b8_bytes = 0;        // grows to the largest N x K packed on this context
   float* t_partial = nullptr; // [kMaxKSplits, min(max_M, kKSplitMaxRows), max_r] FP32 partial sums of T when kernel 1 splits K
   uint8_t* mx_sfa = nullptr;  // MXFP4 variant: activation scale atoms [ceil(max_M/128)][max_K/128][512] (allocated on first use)
+  // MXFP4 variant, fused FFN (allocated with mx_sfa): the second workspace a producing GEMM's epilogue quantizes
+  // the next layer's input into, while the first still holds its own operands.
+  uint8_t* mx_codes2 = nullptr;   // [max_M, max_K / 2]
+  uint8_t* mx_sfa2 = nullptr;     // scale atoms, as mx_sfa
+  float* mx_t32 = nullptr;        // [max_M, max_r] FP32 accumulators of the next layer's T
+  uint16_t* t_hilo2 = nullptr;    // [max_M, 2 max_r] BF16 high | low of the same
   int* d_err = nullptr;       // device error word
   size_t bytes = 0;
   int num_sms = 0;

@@ -33,6 +33,7 @@
 
 #include "gemm_kernel.cuh"
 #include "ptx.cuh"
+#include "quantize_kernel.cuh"
 
 namespace w4a4 {
 
@@ -421,19 +422,88 @@ constexpr uint32_t kMx2NumBarriers = 2 * kMx2Stages + 2;
 constexpr uint32_t kMx2SmemBytes = 1024 + kMx2Stages * kMx2StageBytes + kMx2NumBarriers * 8 + 16;
 static_assert(kMx2StageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligned");
 
+// ---- Fused form (FUSE = true): the epilogue does not store the layer's output but quantizes it for the NEXT layer
+// (Sec. III: the FFN's second linear reads GELU of the first): y -> BF16 -> x_hat = y / lambda' -> MXFP4 codes and
+// block exponents straight into the next layer's workspace, exactly what kernel 1 would produce from the stored
+// output, and the next layer's low-rank projection T' = bf16(x_hat) L1' (Eq. 7) on the tensor core: the epilogue
+// leaves bf16(x_hat) of the tile in shared memory as a K-major operand, a fourth control warp multiplies it by the
+// matching 256 rows of L1' (tcgen05.mma kind::f16, M = 256 over the pair, N = r') into a small TMEM accumulator
+// that stays resident while the cluster walks the column tiles of one row pair (items are dealt to clusters in
+// contiguous runs for that), and is added into an FP32 [M, r'] array when the row pair ends.
+// Shared memory: four stages instead of six, the 64 KiB x_hat tile, 16 KiB for the L1' tile.
+// Barriers: xh_full (leader; 32 epilogue warps: "x_hat tile written"), xh_empty (both; committed after the T MMAs:
+// x_hat and L1' tiles may be overwritten), l1_full (leader; TMA bytes of both CTAs' L1' halves), t_full[2] (both;
+// committed after the last T MMA of a row pair), t_empty[2] (leader; 8 warps: "T buffer read").
+constexpr int kMx2FuseStages = 4;
+constexpr uint32_t kMx2XhBytes = 4 * kMxATile;       // 128 rows x 256 channels BF16: four K slices of 64 channels
+constexpr uint32_t kMx2L1SliceBytes = 4096;           // up to 32 rows (r' / 2 <= 32) x 128 bytes
+constexpr uint32_t kMx2FuseBarriers = 2 * kMx2FuseStages + 2 + 7;
+constexpr uint32_t kMx2FuseSmemBytes = 1024 + kMx2FuseStages * kMx2StageBytes + kMx2XhBytes + 4 * kMx2L1SliceBytes +
+                                       kMx2FuseBarriers * 8 + 16;
+static_assert(kMx2FuseSmemBytes <= 232448, "shared memory budget of one CTA");
+constexpr uint32_t kMxTmemT = 320;                    // two T buffers of 64 columns: 320..447
+
+struct MxNextParams {
+  const float* rlam;     // next layer's reciprocal smoothing factors [N]
+  const float* rho;      // the next layer's clip ratio (one float on the device)
+  uint8_t* codes;        // next layer's packed E2M1 codes [M, N/2]
+  uint8_t* sfa;          // next layer's activation scale atoms [ceil(M/128)][N/128][512]
+  float* t32;            // next layer's T accumulators [M, r2] FP32, zero before the launch
+  int r2;                // next layer's rank: 0, 16, 32 or 64
+};
+
+// MXFP4 conversion of 32 consecutive channels held by one thread (the same arithmetic as kernel 1's
+// mxfp4_block16, without the shuffle): returns the E8M0 exponent byte, packed codes in w[0..3].
+__device__ __forceinline__ uint32_t mxfp4_block32(const uint32_t (&lo)[16], const uint32_t (&hi)[16], float rho, uint4& w) {
+  float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+  for (int e = 0; e < 16; e += 2) {
+    a0 = fmaxf(a0, fmaxf(fabsf(__uint_as_float(lo[e])), fabsf(__uint_as_float(hi[e]))));
+    a1 = fmaxf(a1, fmaxf(fabsf(__uint_as_float(lo[e + 1])), fabsf(__uint_as_float(hi[e + 1]))));
+  }
+  const float a = fmaxf(a0, a1);
+  const uint32_t field = (__float_as_uint(__fmul_rn(rho, a)) >> 23) & 0xffu;
+  const uint32_t ex = field > 2u ? field - 2u : 0u;
+  const float inv = __uint_as_float((254u - ex) << 23);
+  float t[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) t[e] = __fmul_rn(__uint_as_float(lo[e]), inv);
+  w.x = e2m1x8(t);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) t[e] = __fmul_rn(__uint_as_float(lo[8 + e]), inv);
+  w.y = e2m1x8(t);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) t[e] = __fmul_rn(__uint_as_float(hi[e]), inv);
+  w.z = e2m1x8(t);
+#pragma unroll
+  for (int e = 0; e < 8; ++e) t[e] = __fmul_rn(__uint_as_float(hi[8 + e]), inv);
+  w.w = e2m1x8(t);
+  return ex;
+}
+
+template <bool FUSE>
 __global__ void __launch_bounds__(kMxThreads, 1)
 mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmBhalf,
                 const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL2half,
-                const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB, const MxGemmParams p) {
+                const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
+                const __grid_constant__ CUtensorMap tmL1T, const MxGemmParams p, const MxNextParams nx) {
+  constexpr int STAGES = FUSE ? kMx2FuseStages : kMx2Stages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kMx2Stages * kMx2StageBytes;
+  const uint32_t xh_base = smem_base + STAGES * kMx2StageBytes;          // FUSE only: x_hat tile, then the L1' tile
+  const uint32_t l1_base = xh_base + kMx2XhBytes;
+  const uint32_t bar_base = FUSE ? l1_base + 4 * kMx2L1SliceBytes : xh_base;
   const uint32_t bar_full = bar_base;
-  const uint32_t bar_empty = bar_full + 8 * kMx2Stages;
-  const uint32_t bar_acc_full = bar_empty + 8 * kMx2Stages;
+  const uint32_t bar_empty = bar_full + 8 * STAGES;
+  const uint32_t bar_acc_full = bar_empty + 8 * STAGES;
   const uint32_t bar_acc_empty = bar_acc_full + 8;
-  const uint32_t misc_off = (bar_acc_empty + 8) - smem_base;
+  const uint32_t bar_xh_full = bar_acc_empty + 8;      // the next seven exist only when FUSE
+  const uint32_t bar_xh_empty = bar_xh_full + 8;
+  const uint32_t bar_l1_full = bar_xh_empty + 8;
+  const uint32_t bar_t_full = bar_l1_full + 8;          // [2]
+  const uint32_t bar_t_empty = bar_t_full + 16;         // [2]
+  const uint32_t misc_off = (FUSE ? bar_t_empty + 16 : bar_acc_empty + 8) - smem_base;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + misc_off);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + misc_off + 4);
 
@@ -445,15 +515,31 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int num_items = ((p.tiles_m + 1) / 2) * p.tiles_n;
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
   const WaitEnv env{p.err, s_abort};
+  // Items of this cluster: interleaved over the clusters, or (FUSE) one contiguous run, so that the column tiles of
+  // a row pair follow one another and the next layer's T can stay in TMEM between them.
+  const int items_per_cluster = (num_items + num_clusters - 1) / num_clusters;
+  const int item_begin = FUSE ? cluster_id * items_per_cluster : cluster_id;
+  const int item_step = FUSE ? 1 : num_clusters;
+  const int item_end = FUSE ? (item_begin + items_per_cluster < num_items ? item_begin + items_per_cluster : num_items) : num_items;
 
   if (threadIdx.x == 0) {
     *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
-    for (int i = 0; i < kMx2Stages; ++i) {
+    for (int i = 0; i < STAGES; ++i) {
       mbar_init(bar_full + 8 * i, 1);
       mbar_init(bar_empty + 8 * i, 1);
     }
     mbar_init(bar_acc_full, 1);
     mbar_init(bar_acc_empty, 2 * kMxEpiWarps);
+    if (FUSE) {
+      mbar_init(bar_xh_full, 2 * kMxEpiWarps);
+      mbar_init(bar_xh_empty, 1);
+      mbar_init(bar_l1_full, 1);
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(bar_t_full + 8 * i, 1);
+        mbar_init(bar_t_empty + 8 * i, 8);
+      }
+      tma_prefetch_desc(&tmL1T);
+    }
     mbar_fence_init();
     fence_proxy_async_smem();
     tma_prefetch_desc(&tmA);
@@ -482,9 +568,9 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // TMA unit and still count their bytes, so every stage reports the same total.
     const bool issuer = elect_one_lane();
     const uint32_t full0 = map_to_cta(bar_full, 0);
-    Ring<kMx2Stages> rg;
+    Ring<STAGES> rg;
     bool ok = true;
-    for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
+    for (int item = item_begin; ok && item < item_end; item += item_step) {
       const int tm = 2 * (item / p.tiles_n) + static_cast<int>(rank), tn = item % p.tiles_n;
       const int m0 = tm * kBM, n0 = tn * kMxBN;
       for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
@@ -516,10 +602,10 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, 2 * kBM, kMxBN);
     const bool issuer = elect_one_lane();
     const uint32_t peer_empty = map_to_cta(bar_empty, 1), peer_acc_full = map_to_cta(bar_acc_full, 1);
-    Ring<kMx2Stages> rg;
+    Ring<STAGES> rg;
     Ring<1> ab;
     bool ok = true;
-    for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
+    for (int item = item_begin; ok && item < item_end; item += item_step) {
       ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_acc_empty, ab.parity ^ 1u, env, kErrMmaWait));
       if (!ok) break;
       tc_fence_after_sync();
@@ -565,14 +651,72 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       ab.advance();
     }
+  } else if (FUSE && live && warp == 3 && nx.r2 > 0) {
+    // ------------------------------------------------------------------ next layer's T = bf16(x_hat) L1' (FUSE)
+    // Both CTAs fetch their half of the L1' rows that match the item's 256 channels; CTA 0 issues the MMAs.
+    const bool issuer = elect_one_lane();
+    const uint32_t idesc_t = umma_idesc(1, 1, 2 * kBM, static_cast<uint32_t>(nx.r2));
+    const uint32_t l1_full0 = map_to_cta(bar_l1_full, 0);
+    const uint32_t peer_xh_empty = map_to_cta(bar_xh_empty, 1), peer_t_full = map_to_cta(bar_t_full, 1);
+    const int l1_rows = nx.r2 / 2;
+    uint32_t k = 0, tb = 0, uses0 = 0, uses1 = 0;
+    bool ok = true;
+    for (int item = item_begin; ok && item < item_end; item += item_step, ++k) {
+      // The x_hat and L1' tiles are free once the T MMAs of the previous item have completed.
+      ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_xh_empty, (k & 1u) ^ 1u, env, kErrMmaWait));
+      if (!ok) break;
+      const int n0 = (item % p.tiles_n) * kMxBN;
+      if (issuer) {
+        if (leader) mbar_arrive_expect_tx(bar_l1_full, 2u * 4u * static_cast<uint32_t>(l1_rows) * 128u);
+#pragma unroll
+        for (int sl = 0; sl < 4; ++sl)
+          tma2_load_2d(l1_base + sl * kMx2L1SliceBytes, &tmL1T, l1_full0, n0 + 64 * sl, static_cast<int>(rank) * l1_rows);
+      }
+      if (leader) {
+        ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_xh_full, k & 1u, env, kErrMmaWait) &&
+                                         bounded_wait<64>(bar_l1_full, k & 1u, env, kErrMmaWait));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int pm = item / p.tiles_n;
+        const bool first = item == item_begin || (item - 1) / p.tiles_n != pm;
+        const bool last = item + 1 == item_end || (item + 1) / p.tiles_n != pm;
+        if (first) {  // the buffer's previous row pair must have been read out
+          const uint32_t uses = tb ? uses1 : uses0;
+          ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_t_empty + 8 * tb, (uses & 1u) ^ 1u, env, kErrMmaWait));
+          if (!ok) break;
+          tc_fence_after_sync();
+        }
+        if (issuer) {
+          const uint32_t d = tmem_base + kMxTmemT + 64 * tb;
+#pragma unroll
+          for (int sl = 0; sl < 4; ++sl) {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma2_f16(d, umma_desc_k_sw128(xh_base + sl * kMxATile, 32 * kk), umma_desc_k_sw128(l1_base + sl * kMx2L1SliceBytes, 32 * kk),
+                        idesc_t, (first && sl == 0 && kk == 0) ? 0u : 1u);
+          }
+          umma2_commit(bar_xh_empty);
+          umma2_commit(peer_xh_empty);
+          if (last) {
+            umma2_commit(bar_t_full + 8 * tb);
+            umma2_commit(peer_t_full + 8 * tb);
+          }
+        }
+        if (last) {
+          if (tb) ++uses1; else ++uses0;
+          tb ^= 1u;
+        }
+      }
+    }
   } else if (live && warp >= kMxEpiWarp0) {
     // ------------------------------------------------------------------ epilogue (both CTAs, own rows)
     const int ew = warp - kMxEpiWarp0;
     const int quarter = ew & 3, colblk = ew >> 2;
     const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
     Ring<1> ab;
+    uint32_t kq = 0, tb = 0, t_uses0 = 0, t_uses1 = 0;   // FUSE: items done, T buffer, drains per buffer
     bool ok = true;
-    for (int item = cluster_id; ok && item < num_items; item += num_clusters) {
+    for (int item = item_begin; ok && item < item_end; item += item_step) {
       const int m0 = (2 * (item / p.tiles_n) + static_cast<int>(rank)) * kBM, n0 = (item % p.tiles_n) * kMxBN;
       const int row = m0 + 32 * quarter + lane;
       ok = bounded_wait(bar_acc_full, ab.parity, env, kErrEpilogueWait);
@@ -587,7 +731,94 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(acc_empty_leader);
       const int ch0 = n0 + 64 * colblk;
-      if (p.yref != nullptr) {
+      if (FUSE) {
+        // The layer's output never reaches memory: bias, activation and BF16 rounding as the plain epilogue would
+        // apply them, then the next layer's kernel 1 on the thread's 64 channels (two MX blocks).
+        const bool with_t = nx.r2 > 0;
+        if (with_t) {  // the previous item's T MMAs have read the x_hat tile
+          ok = __all_sync(0xffffffffu, bounded_wait(bar_xh_empty, (kq & 1u) ^ 1u, env, kErrEpilogueWait));
+          if (!ok) break;
+        }
+        const bool row_ok = row < p.M, ch_ok = ch0 < p.N;
+        const int rr = 32 * quarter + lane;
+        const uint32_t xrow = xh_base + colblk * kMxATile + (rr >> 3) * 1024 + (rr & 7) * 128;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int ch = ch0 + 16 * c;
+          uint32_t xw[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f), l4 = b4;
+            if (ch_ok) {
+              if (p.bias) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i);
+              l4 = __ldg(reinterpret_cast<const float4*>(nx.rlam + ch) + i);
+            }
+            const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
+            float xh[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float y = __uint_as_float(v[c][4 * i + e]) + bb[e];
+              if (p.act != 0) y = apply_activation(y, p.act);
+              const float yb = __bfloat162float(__float2bfloat16_rn(y));   // what the plain epilogue would store
+              xh[e] = ch_ok ? __fmul_rn(yb, ll[e]) : 0.0f;                  // smoothing, as kernel 1 does it
+              v[c][4 * i + e] = __float_as_uint(xh[e]);
+            }
+            xw[2 * i] = pack_bf16x2(xh[0], xh[1]);
+            xw[2 * i + 1] = pack_bf16x2(xh[2], xh[3]);
+          }
+          if (with_t) {  // 128-byte swizzle of a K-major operand row: 16-byte chunk j sits at j ^ (row % 8)
+            const uint32_t j0 = static_cast<uint32_t>(2 * c), sw = static_cast<uint32_t>(rr & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + ((j0 ^ sw) << 4)), "r"(xw[0]), "r"(xw[1]), "r"(xw[2]), "r"(xw[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + (((j0 + 1) ^ sw) << 4)), "r"(xw[4]), "r"(xw[5]), "r"(xw[6]), "r"(xw[7]) : "memory");
+          }
+        }
+        if (with_t) {
+          fence_proxy_async_smem();   // generic-proxy stores -> visible to the tensor core's reads
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(map_to_cta(bar_xh_full, 0));
+        }
+        if (row_ok && ch_ok) {
+          const float rho2 = __ldg(nx.rho);
+          uint4 w0, w1;
+          const uint32_t ex0 = mxfp4_block32(v[0], v[1], rho2, w0);
+          const uint32_t ex1 = mxfp4_block32(v[2], v[3], rho2, w1);
+          uint4* cdst = reinterpret_cast<uint4*>(nx.codes + static_cast<size_t>(row) * (p.N >> 1) + (ch0 >> 1));
+          cdst[0] = w0;
+          cdst[1] = w1;
+          const int sb = ch0 >> 5;   // even: the two exponent bytes are neighbours inside the atom
+          uint8_t* sdst = nx.sfa + (static_cast<size_t>(row >> 7) * (p.N >> 7) + (sb >> 2)) * 512 + (row & 31) * 16 +
+                          ((row & 127) >> 5) * 4 + (sb & 3);
+          *reinterpret_cast<uint16_t*>(sdst) = static_cast<uint16_t>(ex0 | (ex1 << 8));
+        }
+        if (with_t) {
+          const int pm = item / p.tiles_n;
+          const bool last = item + item_step >= item_end || (item + item_step) / p.tiles_n != pm;
+          if (last) {   // the row pair's T is complete after this item's MMAs: add it to the FP32 array
+            const uint32_t uses = tb ? t_uses1 : t_uses0;
+            ok = __all_sync(0xffffffffu, bounded_wait(bar_t_full + 8 * tb, uses & 1u, env, kErrEpilogueWait));
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (colblk == 0) {
+              const uint32_t t_src = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + kMxTmemT + 64 * tb;
+              for (int cc = 0; cc < nx.r2 / 16; ++cc) {
+                uint32_t tv[16];
+                tmem_ld_32x32b_x16(t_src + 16 * cc, tv);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) atomicAdd(nx.t32 + static_cast<size_t>(row) * nx.r2 + 16 * cc + j, __uint_as_float(tv[j]));
+                }
+              }
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive_remote(map_to_cta(bar_t_empty + 8 * tb, 0));
+            }
+            if (tb) ++t_uses1; else ++t_uses0;
+            tb ^= 1u;
+          }
+        }
+        ++kq;
+      } else if (p.yref != nullptr) {
         float e = 0.0f;
         if (row < p.M && ch0 < p.N) {
           const uint4* yr = reinterpret_cast<const uint4*>(p.yref + static_cast<size_t>(row) * p.N + ch0);
@@ -659,6 +890,13 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 // Weight pack kernels of the MXFP4 variant (run once per layer).
+// L1 [K, r] BF16 -> L1 transposed [r, K]: the K-major B operand of the fused producer's T MMA.
+__global__ void mx_transpose_l1_kernel(const uint16_t* __restrict__ l1, uint16_t* __restrict__ out, int K, int r) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(K) * r) return;
+  const int k = static_cast<int>(idx / r), c = static_cast<int>(idx % r);
+  out[static_cast<size_t>(c) * K + k] = l1[idx];
+}
 // codes [K, N] (one E2M1 code per byte) -> [N, K/2], two codes per byte, even K in the low nibble.
 __global__ void mx_pack_weight_kernel(const uint8_t* __restrict__ codes, uint8_t* __restrict__ out, int K, int N,
                                       int* __restrict__ bad) {

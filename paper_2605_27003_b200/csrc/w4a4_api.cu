@@ -347,6 +347,10 @@ void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
   cudaFree(ctx->codes);
   cudaFree(ctx->b8);
   cudaFree(ctx->mx_sfa);
+  cudaFree(ctx->mx_codes2);
+  cudaFree(ctx->mx_sfa2);
+  cudaFree(ctx->mx_t32);
+  cudaFree(ctx->t_hilo2);
   cudaFree(ctx->t_partial);
   cudaFree(ctx->scales);
   cudaFree(ctx->t_hilo);

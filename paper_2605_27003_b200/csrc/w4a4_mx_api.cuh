@@ -14,6 +14,8 @@ struct MxExpertData {
   CUtensorMap tmB, tmL2;
   CUtensorMap tmBhalf, tmL2half;   // 128-row boxes: what one CTA of a pair fetches (mx_gemm2_kernel)
   CUtensorMap tmSFB;               // scale atoms as 32-bit words: [N/128] rows of K words, boxes of 1 KiB
+  uint16_t* l1t = nullptr;         // L1 transposed, BF16 [r, K]: B operand of the fused producer's T MMA
+  CUtensorMap tmL1T;               // boxes of 64 channels x r/2 rows
 };
 
 struct w4a4_mx_layer {
@@ -22,6 +24,7 @@ struct w4a4_mx_layer {
   std::vector<MxExpertData> experts;
   CUtensorMap tmA, tmT;
   CUtensorMap tmSFA;               // activation scale atoms as 32-bit words: [max_M/128] rows of K words
+  CUtensorMap tmA2, tmT2, tmSFA2;  // the same three on the context's second workspace (input written by a fused producer)
   size_t bytes = 0;
 };
 
@@ -34,6 +37,7 @@ void mx_free_expert(MxExpertData& e) {
   cudaFree(e.l1frag);
   cudaFree(e.l2dup);
   cudaFree(e.bias);
+  cudaFree(e.l1t);
   e = MxExpertData();
 }
 
@@ -86,15 +90,18 @@ w4a4_status_t mx_launch_quantize(w4a4_mx_handle_t h, const void* X, int M, int e
   return mx_launch_quantize_at(h, X, M, expert_id, clip_table, (expert_id * h->L + h->layer_id) * h->B + bin, stream);
 }
 
+// `second_ws`: the layer's input (codes, scale atoms, T) lies in the context's second workspace.  `next` / `next_e`:
+// fused form, the epilogue quantizes the output for that layer into the second workspace instead of storing Y.
 w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream,
-                             const void* yref = nullptr, double* sq_err = nullptr) {
+                             const void* yref = nullptr, double* sq_err = nullptr, bool second_ws = false,
+                             w4a4_mx_handle_t next = nullptr, const float* next_rho = nullptr) {
   if (M == 0) return W4A4_OK;
   w4a4_ctx* ctx = h->ctx;
   const MxExpertData& e = h->experts[expert_id];
   MxGemmParams p;
   p.bias = e.bias;
   p.Y = static_cast<uint16_t*>(Y);
-  p.sfa = ctx->mx_sfa;
+  p.sfa = second_ws ? ctx->mx_sfa2 : ctx->mx_sfa;
   p.sfb = e.sfb;
   p.M = M;
   p.N = h->N;
@@ -108,7 +115,9 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   p.act = h->act;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
-  const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;  // unused when r == 0
+  const CUtensorMap& tmA = second_ws ? h->tmA2 : h->tmA;
+  const CUtensorMap& tmSFA = second_ws ? h->tmSFA2 : h->tmSFA;
+  const CUtensorMap& tmT = h->r > 0 ? (second_ws ? h->tmT2 : h->tmT) : tmA;  // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
   // CTA pairs (cta_group::2) need at least two row tiles and an even number of CTAs.
   static const bool pair_allowed = [] {
@@ -131,13 +140,30 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const CUtensorMap& tmL2h = h->r > 0 ? e.tmL2half : e.tmBhalf;
-    if (cudaLaunchKernelEx(&cfg, mx_gemm2_kernel, h->tmA, e.tmBhalf, tmT, tmL2h, h->tmSFA, e.tmSFB, p) != cudaSuccess) {
+    MxNextParams nx = {};
+    cudaError_t le;
+    if (next) {
+      const MxExpertData& ne = next->experts[expert_id];
+      nx.rlam = ne.rlam;
+      nx.rho = next_rho;
+      nx.codes = ctx->mx_codes2;
+      nx.sfa = ctx->mx_sfa2;
+      nx.t32 = ctx->mx_t32;
+      nx.r2 = next->r;
+      cfg.dynamicSmemBytes = kMx2FuseSmemBytes;
+      const CUtensorMap& tmL1T = next->r > 0 ? ne.tmL1T : e.tmBhalf;
+      le = cudaLaunchKernelEx(&cfg, mx_gemm2_kernel<true>, tmA, e.tmBhalf, tmT, tmL2h, tmSFA, e.tmSFB, tmL1T, p, nx);
+    } else {
+      le = cudaLaunchKernelEx(&cfg, mx_gemm2_kernel<false>, tmA, e.tmBhalf, tmT, tmL2h, tmSFA, e.tmSFB, e.tmBhalf, p, nx);
+    }
+    if (le != cudaSuccess) {
       cudaGetLastError();
       return W4A4_ERR_CUDA;
     }
     return W4A4_OK;
   }
-  mx_gemm_kernel<<<grid, block, kMxSmemBytes, stream>>>(h->tmA, e.tmB, tmT, tmL2, p);
+  if (next) return W4A4_ERR_SHAPE;   // the fused form runs on CTA pairs only
+  mx_gemm_kernel<<<grid, block, kMxSmemBytes, stream>>>(tmA, e.tmB, tmT, tmL2, p);
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
 
@@ -198,7 +224,19 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     if (st == W4A4_OK)
       cudaFuncSetAttribute(mx_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMxSmemBytes));
     if (st == W4A4_OK)
-      cudaFuncSetAttribute(mx_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMx2SmemBytes));
+      cudaFuncSetAttribute(mx_gemm2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMx2SmemBytes));
+    if (st == W4A4_OK)
+      cudaFuncSetAttribute(mx_gemm2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMx2FuseSmemBytes));
+    // Second workspace of the fused FFN.
+    const size_t codes2 = static_cast<size_t>(ctx->max_M) * (ctx->max_K / 2);
+    const int rr = ctx->max_r > 0 ? ctx->max_r : 8;
+    if (st == W4A4_OK) st = dev_alloc(&ctx->mx_codes2, codes2, &ctx->bytes);
+    if (st == W4A4_OK && cudaMemset(ctx->mx_codes2, 0, codes2) != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK) st = dev_alloc(&ctx->mx_sfa2, nb, &ctx->bytes);
+    if (st == W4A4_OK && cudaMemset(ctx->mx_sfa2, 0, nb) != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK) st = dev_alloc(&ctx->mx_t32, static_cast<size_t>(ctx->max_M) * rr, &ctx->bytes);
+    if (st == W4A4_OK) st = dev_alloc(&ctx->t_hilo2, static_cast<size_t>(ctx->max_M) * 2 * rr, &ctx->bytes);
+    if (st == W4A4_OK && cudaMemset(ctx->t_hilo2, 0, sizeof(uint16_t) * ctx->max_M * 2 * rr) != cudaSuccess) st = W4A4_ERR_CUDA;
 
     if (st == W4A4_OK)
       cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesMxfp4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -215,6 +253,7 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     if (st == W4A4_OK) st = dev_alloc(&e.rlam, static_cast<size_t>(K), &h->bytes);
     if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l1frag, static_cast<size_t>(G) * 4 * (r / 8) * 32, &h->bytes);
     if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l2dup, static_cast<size_t>(N) * 2 * r, &h->bytes);
+    if (st == W4A4_OK && r > 0) st = dev_alloc(&e.l1t, static_cast<size_t>(r) * K, &h->bytes);
     const float* bias_src = d->bias ? d->bias[ei] : nullptr;
     if (st == W4A4_OK && bias_src) st = dev_alloc(&e.bias, static_cast<size_t>(N), &h->bytes);
     if (st != W4A4_OK) break;
@@ -243,6 +282,8 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
         l1_fragment_kernel<<<static_cast<unsigned>((nf + 255) / 256), 256>>>(l1_dev, e.l1frag, K, r);
         const size_t nl = static_cast<size_t>(N) * 2 * r;
         l2_dup_kernel<<<static_cast<unsigned>((nl + 255) / 256), 256>>>(l2_dev, e.l2dup, r, N);
+        const size_t nt = static_cast<size_t>(K) * r;
+        mx_transpose_l1_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256>>>(l1_dev, e.l1t, K, r);
       }
       if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) st = W4A4_ERR_CUDA;
     }
@@ -262,6 +303,10 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
     if (st == W4A4_OK &&
         !encode_2d(ctx->encode, &e.tmSFB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, e.sfb, K, N / 128, 4 * static_cast<uint64_t>(K), 256,
                    1, CU_TENSOR_MAP_SWIZZLE_NONE))
+      st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK && r > 0 &&
+        !encode_2d(ctx->encode, &e.tmL1T, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l1t, K, r, 2 * static_cast<uint64_t>(K), 64, r / 2,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
       st = W4A4_ERR_CUDA;
     if (st == W4A4_OK && r > 0 &&
         !encode_2d(ctx->encode, &e.tmL2half, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kMxBN / 2,
@@ -285,6 +330,18 @@ w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* 
   if (st == W4A4_OK &&
       !encode_2d(ctx->encode, &h->tmSFA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, ctx->mx_sfa, K, (ctx->max_M + 127) / 128,
                  4 * static_cast<uint64_t>(K), 256, 1, CU_TENSOR_MAP_SWIZZLE_NONE))
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK &&
+      !encode_2d(ctx->encode, &h->tmA2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->mx_codes2, K / 2, ctx->max_M, K / 2, 128, kBM,
+                 CU_TENSOR_MAP_SWIZZLE_128B))
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK &&
+      !encode_2d(ctx->encode, &h->tmSFA2, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, ctx->mx_sfa2, K, (ctx->max_M + 127) / 128,
+                 4 * static_cast<uint64_t>(K), 256, 1, CU_TENSOR_MAP_SWIZZLE_NONE))
+    st = W4A4_ERR_CUDA;
+  if (st == W4A4_OK && r > 0 &&
+      !encode_2d(ctx->encode, &h->tmT2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo2, 2 * r, ctx->max_M, 4 * r, 64,
+                 kBM, CU_TENSOR_MAP_SWIZZLE_128B))
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK && r > 0 &&
       !encode_2d(ctx->encode, &h->tmT, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo, 2 * r, ctx->max_M, 4 * r, 64,
@@ -397,6 +454,56 @@ w4a4_status_t w4a4_mx_debug_quantize(w4a4_mx_handle_t h, const void* X, int M, i
   if (T && h->r > 0) {
     const size_t nt = static_cast<size_t>(M) * h->r;
     decode_t_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, s>>>(h->ctx->t_hilo, T, M, h->r);
+  }
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+// Fused pair of layers (Sec. III, the FFN): `up` runs as usual except that its GEMM's epilogue applies bias and
+// activation, rounds to BF16 and quantizes the result for `down` (codes, block exponents, the low-rank projection T)
+// straight into the context's second workspace; `down`'s GEMM then reads its operands from there.  The hidden
+// activation never reaches memory and `down`'s activation kernel does not run.
+w4a4_status_t w4a4_mx_ffn_forward(w4a4_mx_handle_t up, w4a4_mx_handle_t down, const void* X, int M, int expert_id,
+                                  int timestep_bin, const float* clip_table, void* Y, void* stream) {
+  w4a4_status_t st = mx_check_forward_args(up, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  st = mx_check_forward_args(down, X, M, expert_id, timestep_bin, clip_table, true);
+  if (st != W4A4_OK) return st;
+  if (up->ctx != down->ctx || up->N != down->K) return W4A4_ERR_SHAPE;
+  if (M > 0 && (!Y || !aligned16(Y))) return W4A4_ERR_INVALID_ARG;
+  if (M == 0) return W4A4_OK;
+  if (M <= kBM) return W4A4_ERR_SHAPE;   // the fused epilogue exists in the CTA-pair kernel only (two row tiles)
+  w4a4_ctx* ctx = up->ctx;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = mx_launch_quantize(up, X, M, expert_id, timestep_bin, clip_table, s);
+  if (st != W4A4_OK) return st;
+  if (down->r > 0 &&
+      cudaMemsetAsync(ctx->mx_t32, 0, sizeof(float) * static_cast<size_t>(M) * down->r, s) != cudaSuccess)
+    return W4A4_ERR_CUDA;
+  const float* rho2 = clip_table + (static_cast<size_t>(expert_id) * down->L + down->layer_id) * down->B + timestep_bin;
+  st = mx_launch_gemm(up, M, expert_id, nullptr, s, nullptr, nullptr, false, down, rho2);
+  if (st != W4A4_OK) return st;
+  if (down->r > 0) {
+    const size_t nt = static_cast<size_t>(M) * down->r;
+    t_reduce_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, s>>>(ctx->mx_t32, 1, M, down->r, ctx->t_hilo2);
+    if (cudaGetLastError() != cudaSuccess) return W4A4_ERR_CUDA;
+  }
+  return mx_launch_gemm(down, M, expert_id, Y, s, nullptr, nullptr, true);
+}
+
+// Parity tap of the fused form: decodes what the last w4a4_mx_ffn_forward left in the second workspace for `down`.
+w4a4_status_t w4a4_mx_debug_fused_input(w4a4_mx_handle_t down, int M, uint8_t* codes, uint8_t* exps, float* T, void* stream) {
+  if (!down || !down->ctx || M < 0 || M > down->ctx->max_M) return W4A4_ERR_INVALID_ARG;
+  if (M > 0 && (!codes || !exps)) return W4A4_ERR_INVALID_ARG;
+  if (M == 0) return W4A4_OK;
+  DeviceGuard guard(down->ctx->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t nc = static_cast<size_t>(M) * down->K, ns = static_cast<size_t>(M) * (down->K / 32);
+  mx_decode_codes_kernel<<<static_cast<unsigned>((nc + 255) / 256), 256, 0, s>>>(down->ctx->mx_codes2, codes, M, down->K);
+  mx_decode_exps_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256, 0, s>>>(down->ctx->mx_sfa2, down->K / 128, exps, M, down->K / 32);
+  if (T && down->r > 0) {
+    const size_t nt = static_cast<size_t>(M) * down->r;
+    decode_t_kernel<<<static_cast<unsigned>((nt + 255) / 256), 256, 0, s>>>(down->ctx->t_hilo2, T, M, down->r);
   }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
