@@ -400,6 +400,75 @@ def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
     ctx.close()
 
 
+def run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks):
+    """The FFN of the MXFP4 variant, 5120 -> 13824 (GELU) -> 5120 at M = 32760: the fused call (the up-projection's
+    epilogue quantizes for the down-projection; the hidden activation never reaches memory) against the same two
+    layers as two calls (`--workload mxfp4_ffn`)."""
+    if rank != 0:
+        return
+    up_s, dn_s = gen.CONFIG_SHAPES["ffn_up"], gen.CONFIG_SHAPES["ffn_down"]
+    M, K, H, N, r = up_s["M"], up_s["K"], up_s["N"], dn_s["N"], up_s["r"]
+    num_bins, n_buf = 8, 4
+    idx = gen.outlier_channels(K, 0.01, 2)
+    up = gen.make_layer_mx_direct(K, H, r, seed=2101, device=dev)
+    down = gen.make_layer_mx_direct(H, N, r, seed=2102, device=dev)
+    bins = [b % num_bins for b in range(n_buf)]
+    xs = [gen.make_activations(M, K, sigma=gen.sigma_for_bin(b), outlier_idx=idx, outlier_gain=50.0, seed=2103 + i, device=dev)
+          for i, b in enumerate(bins)]
+    clip = gen.make_clip_table(1, 2, num_bins, [(0.6, 1.0)], seed=2).to(dev)
+    ctx = w4.Context(local_rank, M, max(K, H), r)
+    l_up = w4.MxLayer(ctx, [up], num_bins=num_bins, num_layers=2, layer_id=0, output_activation=w4.ACT_GELU_TANH)
+    l_dn = w4.MxLayer(ctx, [down], num_bins=num_bins, num_layers=2, layer_id=1)
+    hidden = torch.empty(M, H, dtype=torch.bfloat16, device=dev)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def fused(i):
+        w4.w4a4_mx_ffn_forward(l_up.ptr, l_dn.ptr, xs[i % n_buf], M, 0, bins[i % n_buf], clip, Y, stream)
+
+    def two_calls(i):
+        w4.w4a4_mx_linear_forward(l_up.ptr, xs[i % n_buf], M, 0, bins[i % n_buf], clip, hidden, stream)
+        w4.w4a4_mx_linear_forward(l_dn.ptr, hidden, M, 0, bins[i % n_buf], clip, Y, stream)
+
+    def timed(fn):
+        for i in range(max(3, args.warmup)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    ms_two = timed(two_calls)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms = timed(fused)
+    clocks = sampler.stop()
+    ctx.check()
+    ops = 2.0 * M * K * H + 2.0 * M * H * N
+    fp4_peak = 4.0 * peaks["bf16_sustained"]
+    print(json.dumps(dict(
+        metric=METRIC, value=ops / (ms * 1e-3) / 1e12, unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e2m1 x e8m0 (mxfp4)",
+        data="synthetic",
+        config=dict(workload=args.workload, M=M, K=K, hidden=H, N=N, r=r, block=32, activation="gelu_tanh",
+                    l2="inputs larger than L2: 4 rotating activation buffers of %.0f MB" % (M * K * 2 / 1e6)),
+        roofline=dict(bound="tensor", achieved=ops / (ms * 1e-3) / 1e12, peak=fp4_peak, unit="TOP/s",
+                      frac=ops / (ms * 1e-3) / 1e12 / fp4_peak, traffic=None,
+                      kernel="whole fused call: quantize, mx_gemm2_kernel<fused epilogue>, T finish, mx_gemm2_kernel",
+                      peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 4 "
+                                  "(nominal FP4:BF16 ratio)"),
+        two_calls=dict(ms_per_step=ms_two, value=ops / (ms_two * 1e-3) / 1e12, unit=UNIT,
+                       note="same layers as w4a4_mx_linear_forward twice (hidden activation stored and re-read)"),
+        e2e=None, gpu_launches=5 * args.steps, clocks=clocks)), flush=True)
+    l_up.close()
+    l_dn.close()
+    ctx.close()
+
+
 def mxfp4_context(w4, ctx, w, clip, Y, stream, iters: int = 20):
     """The same layer shape through the MXFP4 variant (E2M1 elements, E8M0 block scales applied inside the tensor
     core), timed on the buffers of the main run: a different quantizer, reported for context, never part of `value`."""
@@ -474,7 +543,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search", "mxfp4_attn_proj", "mxfp4_ffn_up",
-                                                            "mxfp4_ffn_down"])
+                                                            "mxfp4_ffn_down", "mxfp4_ffn"])
     ap.add_argument("--chunk-rows", type=int, default=4096, help="token rows per chunk of the host-buffer forward (e2e)")
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
@@ -514,6 +583,9 @@ def main():
         return
     if args.workload == "sweep":
         run_sweep(args, w4, dev, local_rank, rank, peaks)
+        return
+    if args.workload == "mxfp4_ffn":
+        run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks)
         return
     if args.workload.startswith("mxfp4_"):
         run_mxfp4(args, w4, dev, local_rank, rank, peaks)

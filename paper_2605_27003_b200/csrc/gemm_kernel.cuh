@@ -156,10 +156,20 @@ __device__ __forceinline__ void set_max_regs_dec() {
 }
 
 // Output activation of the layer (W4A4_ACT_*), applied in FP32 before the BF16 rounding.
+// GELU, tanh form: 0.5 y (1 + tanh u) with u = sqrt(2/pi) (y + 0.044715 y^3) equals y * sigmoid(2 u) =
+// y / (1 + exp(-2 u)); written that way it needs one ex2 and one reciprocal (both accurate to about 2^-22) instead
+// of a full-precision tanh, and has no cancellation for negative y.
 __device__ __forceinline__ float apply_activation(float y, int act) {
   if (act == 1) {
-    const float u = 0.7978845608028654f * (y + 0.044715f * y * y * y);
-    return 0.5f * y * (1.0f + tanhf(u));
+    const float y2 = y * y;
+    // -2 u log2(e) = y (c1 + c3 y^2)
+    const float t = y * fmaf(y2, -2.0f * 0.7978845608028654f * 0.044715f * 1.4426950408889634f,
+                             -2.0f * 0.7978845608028654f * 1.4426950408889634f);
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
+    float rcp;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(1.0f + e));
+    return y * rcp;
   }
   return y;
 }

@@ -65,6 +65,7 @@ struct MxGemmParams {
   const uint16_t* yref;  // [M, N] BF16 or nullptr
   double* sq_err;
   int act;              // output activation: 0 none, 1 GELU (tanh form)
+  int run;              // CTA-pair kernel: consecutive column tiles of a row pair that one cluster takes at a time
 };
 
 // One lane of a converged warp.  The MMA warp runs its loop with all lanes (waits included) and only predicates
@@ -428,8 +429,8 @@ static_assert(kMx2StageBytes % 1024 == 0, "operand tiles must stay 1024-byte ali
 // output, and the next layer's low-rank projection T' = bf16(x_hat) L1' (Eq. 7) on the tensor core: the epilogue
 // leaves bf16(x_hat) of the tile in shared memory as a K-major operand, a fourth control warp multiplies it by the
 // matching 256 rows of L1' (tcgen05.mma kind::f16, M = 256 over the pair, N = r') into a small TMEM accumulator
-// that stays resident while the cluster walks the column tiles of one row pair (items are dealt to clusters in
-// contiguous runs for that), and is added into an FP32 [M, r'] array when the row pair ends.
+// that stays resident while the cluster walks a run of column tiles of one row pair (work is dealt to clusters in
+// such runs), and is added into an FP32 [M, r'] array when the run ends.
 // Shared memory: four stages instead of six, the 64 KiB x_hat tile, 16 KiB for the L1' tile.
 // Barriers: xh_full (leader; 32 epilogue warps: "x_hat tile written"), xh_empty (both; committed after the T MMAs:
 // x_hat and L1' tiles may be overwritten), l1_full (leader; TMA bytes of both CTAs' L1' halves), t_full[2] (both;
@@ -512,16 +513,14 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const bool leader = rank == 0;
   const int n_k_stages = p.K / kMxBK;
   const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
-  const int num_items = ((p.tiles_m + 1) / 2) * p.tiles_n;
+  // Work is dealt to the clusters in runs of p.run consecutive column tiles of one row pair (run = 1: plain
+  // interleaving).  The fused form uses longer runs so that the next layer's T can stay in TMEM over a run; short
+  // enough that the clusters running at the same time still share their A rows in L2.
+  const int run = p.run;
+  const int runs_per_pair = (p.tiles_n + run - 1) / run;
+  const int num_runs = ((p.tiles_m + 1) / 2) * runs_per_pair;
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
   const WaitEnv env{p.err, s_abort};
-  // Items of this cluster: interleaved over the clusters, or (FUSE) one contiguous run, so that the column tiles of
-  // a row pair follow one another and the next layer's T can stay in TMEM between them.
-  const int items_per_cluster = (num_items + num_clusters - 1) / num_clusters;
-  const int item_begin = FUSE ? cluster_id * items_per_cluster : cluster_id;
-  const int item_step = FUSE ? 1 : num_clusters;
-  const int item_end = FUSE ? (item_begin + items_per_cluster < num_items ? item_begin + items_per_cluster : num_items) : num_items;
-
   if (threadIdx.x == 0) {
     *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
     for (int i = 0; i < STAGES; ++i) {
@@ -570,8 +569,9 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t full0 = map_to_cta(bar_full, 0);
     Ring<STAGES> rg;
     bool ok = true;
-    for (int item = item_begin; ok && item < item_end; item += item_step) {
-      const int tm = 2 * (item / p.tiles_n) + static_cast<int>(rank), tn = item % p.tiles_n;
+    for (int q = cluster_id; ok && q < num_runs; q += num_clusters)
+    for (int tn = (q % runs_per_pair) * run, tn1 = min(tn + run, p.tiles_n); ok && tn < tn1; ++tn) {
+      const int tm = 2 * (q / runs_per_pair) + static_cast<int>(rank);
       const int m0 = tm * kBM, n0 = tn * kMxBN;
       for (int st = 0; st < n_lr_stages + n_k_stages; ++st) {
         ok = __all_sync(0xffffffffu, bounded_wait<128>(bar_empty + 8 * rg.slot, rg.parity ^ 1u, env, kErrProducerWait));
@@ -605,7 +605,8 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     Ring<STAGES> rg;
     Ring<1> ab;
     bool ok = true;
-    for (int item = item_begin; ok && item < item_end; item += item_step) {
+    for (int q = cluster_id; ok && q < num_runs; q += num_clusters)
+    for (int tn = (q % runs_per_pair) * run, tn1 = min(tn + run, p.tiles_n); ok && tn < tn1; ++tn) {
       ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_acc_empty, ab.parity ^ 1u, env, kErrMmaWait));
       if (!ok) break;
       tc_fence_after_sync();
@@ -659,27 +660,27 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t l1_full0 = map_to_cta(bar_l1_full, 0);
     const uint32_t peer_xh_empty = map_to_cta(bar_xh_empty, 1), peer_t_full = map_to_cta(bar_t_full, 1);
     const int l1_rows = nx.r2 / 2;
+    const uint32_t l1_pitch = l1_rows * 128 < 1024 ? 1024u : static_cast<uint32_t>(l1_rows) * 128u;   // whole swizzle atoms
     uint32_t k = 0, tb = 0, uses0 = 0, uses1 = 0;
     bool ok = true;
-    for (int item = item_begin; ok && item < item_end; item += item_step, ++k) {
+    for (int q = cluster_id; ok && q < num_runs; q += num_clusters)
+    for (int tn0 = (q % runs_per_pair) * run, tn = tn0, tn1 = min(tn0 + run, p.tiles_n); ok && tn < tn1; ++tn, ++k) {
       // The x_hat and L1' tiles are free once the T MMAs of the previous item have completed.
       ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_xh_empty, (k & 1u) ^ 1u, env, kErrMmaWait));
       if (!ok) break;
-      const int n0 = (item % p.tiles_n) * kMxBN;
+      const int n0 = tn * kMxBN;
       if (issuer) {
         if (leader) mbar_arrive_expect_tx(bar_l1_full, 2u * 4u * static_cast<uint32_t>(l1_rows) * 128u);
 #pragma unroll
         for (int sl = 0; sl < 4; ++sl)
-          tma2_load_2d(l1_base + sl * kMx2L1SliceBytes, &tmL1T, l1_full0, n0 + 64 * sl, static_cast<int>(rank) * l1_rows);
+          tma2_load_2d(l1_base + sl * l1_pitch, &tmL1T, l1_full0, n0 + 64 * sl, static_cast<int>(rank) * l1_rows);
       }
       if (leader) {
         ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_xh_full, k & 1u, env, kErrMmaWait) &&
                                          bounded_wait<64>(bar_l1_full, k & 1u, env, kErrMmaWait));
         if (!ok) break;
         tc_fence_after_sync();
-        const int pm = item / p.tiles_n;
-        const bool first = item == item_begin || (item - 1) / p.tiles_n != pm;
-        const bool last = item + 1 == item_end || (item + 1) / p.tiles_n != pm;
+        const bool first = tn == tn0, last = tn + 1 == tn1;
         if (first) {  // the buffer's previous row pair must have been read out
           const uint32_t uses = tb ? uses1 : uses0;
           ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_t_empty + 8 * tb, (uses & 1u) ^ 1u, env, kErrMmaWait));
@@ -692,7 +693,7 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           for (int sl = 0; sl < 4; ++sl) {
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              umma2_f16(d, umma_desc_k_sw128(xh_base + sl * kMxATile, 32 * kk), umma_desc_k_sw128(l1_base + sl * kMx2L1SliceBytes, 32 * kk),
+              umma2_f16(d, umma_desc_k_sw128(xh_base + sl * kMxATile, 32 * kk), umma_desc_k_sw128(l1_base + sl * l1_pitch, 32 * kk),
                         idesc_t, (first && sl == 0 && kk == 0) ? 0u : 1u);
           }
           umma2_commit(bar_xh_empty);
@@ -716,9 +717,26 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     Ring<1> ab;
     uint32_t kq = 0, tb = 0, t_uses0 = 0, t_uses1 = 0;   // FUSE: items done, T buffer, drains per buffer
     bool ok = true;
-    for (int item = item_begin; ok && item < item_end; item += item_step) {
-      const int m0 = (2 * (item / p.tiles_n) + static_cast<int>(rank)) * kBM, n0 = (item % p.tiles_n) * kMxBN;
+    for (int q = cluster_id; ok && q < num_runs; q += num_clusters)
+    for (int tn = (q % runs_per_pair) * run, tn1 = min(tn + run, p.tiles_n); ok && tn < tn1; ++tn) {
+      const int m0 = (2 * (q / runs_per_pair) + static_cast<int>(rank)) * kBM, n0 = tn * kMxBN;
       const int row = m0 + 32 * quarter + lane;
+      // FUSE: the warp's 64 bias values and 64 reciprocal smoothing factors of the next layer go into a table of its
+      // own in shared memory (the half of the L1' area that ranks up to 32 leave free) while the tile is still
+      // being accumulated; from global memory each of them would be a long-latency load in front of its use.
+      const bool use_tab = FUSE && nx.r2 <= 32;
+      const uint32_t tab = l1_base + 8192 + static_cast<uint32_t>(ew) * 512;
+      if (use_tab) {
+        const int chq = n0 + 64 * colblk + 4 * (lane & 15);
+        float4 t4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (chq < p.N) {
+          if (lane >= 16) t4 = __ldg(reinterpret_cast<const float4*>(nx.rlam + chq));
+          else if (p.bias) t4 = __ldg(reinterpret_cast<const float4*>(p.bias + chq));
+        }
+        __syncwarp();   // the previous item's reads of the table are done
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(tab + 16 * lane), "f"(t4.x), "f"(t4.y), "f"(t4.z), "f"(t4.w) : "memory");
+        __syncwarp();
+      }
       ok = bounded_wait(bar_acc_full, ab.parity, env, kErrEpilogueWait);
       if (!ok) break;
       tc_fence_after_sync();
@@ -749,7 +767,10 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f), l4 = b4;
-            if (ch_ok) {
+            if (use_tab) {
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(b4.x), "=f"(b4.y), "=f"(b4.z), "=f"(b4.w) : "r"(tab + 64 * c + 16 * i));
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(l4.x), "=f"(l4.y), "=f"(l4.z), "=f"(l4.w) : "r"(tab + 256 + 64 * c + 16 * i));
+            } else if (ch_ok) {
               if (p.bias) b4 = __ldg(reinterpret_cast<const float4*>(p.bias + ch) + i);
               l4 = __ldg(reinterpret_cast<const float4*>(nx.rlam + ch) + i);
             }
@@ -791,9 +812,8 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           *reinterpret_cast<uint16_t*>(sdst) = static_cast<uint16_t>(ex0 | (ex1 << 8));
         }
         if (with_t) {
-          const int pm = item / p.tiles_n;
-          const bool last = item + item_step >= item_end || (item + item_step) / p.tiles_n != pm;
-          if (last) {   // the row pair's T is complete after this item's MMAs: add it to the FP32 array
+          const bool last = tn + 1 == tn1;
+          if (last) {   // the run's T is complete after this item's MMAs: add it to the FP32 array
             const uint32_t uses = tb ? t_uses1 : t_uses0;
             ok = __all_sync(0xffffffffu, bounded_wait(bar_t_full + 8 * tb, uses & 1u, env, kErrEpilogueWait));
             if (!ok) break;

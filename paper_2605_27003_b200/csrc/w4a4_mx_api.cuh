@@ -113,6 +113,9 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   p.yref = static_cast<const uint16_t*>(yref);
   p.sq_err = sq_err;
   p.act = h->act;
+  // Runs of column tiles per cluster: 1 = interleave; the fused form takes six at a time (T stays in TMEM over a
+  // run, and the 74 clusters of a wave then cover about a dozen row pairs whose A rows they share in L2).
+  p.run = next ? (p.tiles_n < 6 ? p.tiles_n : 6) : 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kMxThreads);
   const CUtensorMap& tmA = second_ws ? h->tmA2 : h->tmA;
@@ -125,8 +128,8 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
     return !(v && std::strcmp(v, "single") == 0);
   }();
   if (pair_allowed && p.tiles_m >= 2 && ctx->num_sms >= 2) {
-    const int items = ((p.tiles_m + 1) / 2) * p.tiles_n;
-    const int ctas = 2 * items < ctx->num_sms ? 2 * items : (ctx->num_sms & ~1);
+    const int runs = ((p.tiles_m + 1) / 2) * ((p.tiles_n + p.run - 1) / p.run);
+    const int ctas = 2 * runs < ctx->num_sms ? 2 * runs : (ctx->num_sms & ~1);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctas);
     cfg.blockDim = block;
