@@ -7,14 +7,19 @@
 // tensor core and accumulates in FP32, so -- unlike the INT4 kernel -- nothing is rescaled on the CUDA cores and
 // the whole K extent accumulates into one TMEM tile; the epilogue runs once per output tile.
 //
+// Three kernels in this file: mx_gemm_kernel (one CTA per 128 x 256 tile; described next), mx_gemm2_kernel<false>
+// (the default: a cluster of two CTAs per 256 x 256 tile, tcgen05 cta_group::2) and mx_gemm2_kernel<true> (the same
+// with an epilogue that, instead of storing Y, quantizes it for the next layer); the latter two are described in
+// front of their definition.
+//
 // Persistent kernel, one CTA per SM, 128 x 256 output tiles, column tile fastest.  At the FP4 rate the tensor
 // core consumes operands faster than L2 and the shared-memory port deliver them, so the tile is as wide as TMEM
 // allows (operand bytes per MAC fall by a quarter against 128 x 128).  Warp roles:
-//   warp 0      producer (one lane): per stage of 256 K elements one TMA each for the packed A tile (128 rows x
+//   warp 0      producer (all lanes loop, one elected lane issues): per stage of 256 K elements one TMA each for the packed A tile (128 rows x
 //               128 bytes) and B tile (256 rows x 128 bytes), 128-byte swizzle, and bulk copies for their scale
 //               bytes (1 KiB per 128 rows: two 512-byte atoms, the layout the tensor core wants); the BF16
 //               low-rank operands T and L2 go through the same ring first.
-//   warp 1      MMA issuer (one lane): per stage six tcgen05.cp (scale atoms, shared memory -> TMEM: 32 lanes x
+//   warp 1      MMA issuer (all lanes loop, one elected lane issues): per stage six tcgen05.cp (scale atoms, shared memory -> TMEM: 32 lanes x
 //               128 bits, replicated to the four lane quarters) and four tcgen05.mma kind::mxf4 (128 x 256, K = 64
 //               each: two scale blocks per row, selected by the scale-factor id 0 / 2 inside the 4-byte TMEM
 //               column); kind::f16 for [T_hi | T_lo] [L2 | L2]^T into the same accumulator first.  tcgen05.cp
