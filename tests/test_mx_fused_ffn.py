@@ -84,6 +84,49 @@ def test_fused_ffn_many_tiles():
     run_fused_case(2048 + 77, 512, 2048, 512, 32, 32, 1, 0.85, 0.9, True, seed=5)
 
 
+def test_fused_ffn_full_size_sampled_rows():
+    """The bench's configuration (M = 32760, 5120 -> 13824 -> 5120, r = 32, GELU): sampled token rows of the second
+    layer's input and output against the oracle."""
+    import paper_2605_27003_b200 as w4
+    up_s, dn_s = gen.CONFIG_SHAPES["ffn_up"], gen.CONFIG_SHAPES["ffn_down"]
+    M, K, H, N, r = up_s["M"], up_s["K"], up_s["N"], dn_s["N"], up_s["r"]
+    x = gen.make_activations(M, K, sigma=gen.sigma_for_bin(2), outlier_idx=gen.outlier_channels(K, 0.01, 7),
+                             outlier_gain=50.0, seed=41, device=DEV)
+    up = gen.make_layer_mx_direct(K, H, r, seed=42)
+    down = gen.make_layer_mx_direct(H, N, r, seed=43)
+    clip = gen.make_clip_table(1, 2, 8, [(0.6, 1.0)], seed=6)
+    clip_d = clip.to(DEV)
+    ctx = w4.Context(0, M, max(K, H), r)
+    Lup = w4.MxLayer(ctx, [up.to(DEV)], num_bins=8, num_layers=2, layer_id=0, output_activation=1)
+    Ldn = w4.MxLayer(ctx, [down.to(DEV)], num_bins=8, num_layers=2, layer_id=1)
+    y1 = Lup.forward(x, 0, 2, clip_d)
+    y2 = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    w4.w4a4_mx_ffn_forward(Lup.ptr, Ldn.ptr, x, M, 0, 2, clip_d, y2)
+    codes = torch.empty((M, H), dtype=torch.uint8, device=DEV)
+    exps = torch.empty((M, H // 32), dtype=torch.uint8, device=DEV)
+    T = torch.empty((M, r), dtype=torch.float32, device=DEV)
+    w4.w4a4_mx_debug_fused_input(Ldn.ptr, M, codes, exps, T)
+    torch.cuda.synchronize()
+    ctx.check()
+    rng = np.random.default_rng(2)
+    rows = np.array(sorted({0, 127, 128, 255, 256, M - 1, (M - 1) // 256 * 256, *rng.integers(0, M, 3).tolist()}), dtype=np.int32)
+    rt = torch.as_tensor(rows.astype(np.int64), device=DEV)
+    ref = oracle.mx_forward_rows(bits(y1[rt]), np.arange(len(rows), dtype=np.int32), down.lam.numpy(), float(clip[0, 1, 2]),
+                                 bits(down.L1), bits(down.L2), down.wcodes.numpy(), down.wexps.numpy(), None)
+    assert np.array_equal(oracle.e2m1_values(codes[rt].cpu().numpy()), oracle.e2m1_values(ref["codes"])), "elements differ"
+    assert np.array_equal(exps[rt].cpu().numpy(), ref["exps"]), "scale exponents differ"
+    t_gpu, t_ref = T[rt].cpu().numpy().astype(np.float64), ref["T"].astype(np.float64)
+    assert np.all(np.abs(t_gpu - t_ref) <= 1e-4 * np.abs(t_ref).max(axis=1, keepdims=True) + 1e-30), "T differs"
+    y64 = ref["Y64"]
+    rms = float(np.sqrt(np.mean(y64 ** 2)))
+    bound = 2.0 ** -7 * np.abs(y64) + 1e-3 * rms
+    worst = float(np.max(np.abs(y2[rt].to(torch.float64).cpu().numpy() - y64) / bound))
+    assert worst <= 1.0, f"fused output outside tolerance: worst err/bound = {worst:.3f}"
+    Lup.close()
+    Ldn.close()
+    ctx.close()
+
+
 def test_fused_ffn_rejects_small_m():
     import paper_2605_27003_b200 as w4
     x = gen.make_activations(64, 256, outlier_idx=gen.outlier_channels(256, 0, 0, count=2), outlier_gain=10.0, seed=0)
