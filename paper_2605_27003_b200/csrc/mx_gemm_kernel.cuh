@@ -782,12 +782,17 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, ll[4] = {l4.x, l4.y, l4.z, l4.w};
             float xh[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float y = __uint_as_float(v[c][4 * i + e]) + bb[e];
-              if (p.act != 0) y = apply_activation(y, p.act);
-              const float yb = __bfloat162float(__float2bfloat16_rn(y));   // what the plain epilogue would store
-              xh[e] = ch_ok ? __fmul_rn(yb, ll[e]) : 0.0f;                  // smoothing, as kernel 1 does it
+            for (int e = 0; e < 4; e += 2) {
+              float y0 = __uint_as_float(v[c][4 * i + e]) + bb[e], y1 = __uint_as_float(v[c][4 * i + e + 1]) + bb[e + 1];
+              if (p.act != 0) {
+                y0 = apply_activation(y0, p.act);
+                y1 = apply_activation(y1, p.act);
+              }
+              const uint32_t yb = pack_bf16x2(y0, y1);                      // what the plain epilogue would store
+              xh[e] = ch_ok ? __fmul_rn(__uint_as_float(yb << 16), ll[e]) : 0.0f;   // smoothing, as kernel 1 does it
+              xh[e + 1] = ch_ok ? __fmul_rn(__uint_as_float(yb & 0xffff0000u), ll[e + 1]) : 0.0f;
               v[c][4 * i + e] = __float_as_uint(xh[e]);
+              v[c][4 * i + e + 1] = __float_as_uint(xh[e + 1]);
             }
             xw[2 * i] = pack_bf16x2(xh[0], xh[1]);
             xw[2 * i + 1] = pack_bf16x2(xh[2], xh[3]);
