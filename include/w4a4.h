@@ -205,7 +205,9 @@ typedef struct {
 
 /* Copies and repacks one layer's MXFP4 constants (two codes per byte, scale bytes in the tensor core's atom
  * layout).  Synchronous; allocates device memory owned by the handle (and, once per context, the activation
- * scale workspace).  Errors: SHAPE, INVALID_ARG (also: a code above 15, a 0xFF scale byte), ALLOC, CUDA. */
+ * scale workspace and the second workspace of w4a4_mx_ffn_forward: max_M x max_K / 2 bytes of codes, scale atoms,
+ * and max_M x max_r FP32 + BF16 pairs).  Errors: SHAPE, INVALID_ARG (also: a code above 15, a 0xFF scale byte),
+ * ALLOC, CUDA. */
 w4a4_status_t w4a4_mx_pack_weights(w4a4_ctx_t ctx, const w4a4_mx_weight_desc_t* desc, w4a4_mx_handle_t* out);
 void w4a4_mx_destroy(w4a4_mx_handle_t h);
 size_t w4a4_mx_handle_bytes(w4a4_mx_handle_t h);
