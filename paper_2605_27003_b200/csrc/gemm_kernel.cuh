@@ -12,18 +12,19 @@
 // as E4M3 bytes: the activation codes straight from kernel 1, the weight codes from expand_weight_kernel,
 // which runs right before this kernel and turns the layer's nibble-packed weights (their format at rest)
 // into an N x K byte image that stays in L2 for the duration of the GEMM.  Nothing is unpacked on the SM:
-// its issue slots and shared-memory port belong to the epilogue.  Warp roles:
-//   warp 0        producer (one lane): per stage (128 K-codes = two quantization groups) one TMA for the
+// its issue slots and shared-memory port belong to the epilogue.  Every role loops with all 32 lanes of its warp
+// (waits are voted, only the TMA / tcgen05 instructions are predicated on one elected lane), which keeps ring
+// positions, addresses and descriptors warp-uniform for the compiler.  Warp roles:
+//   warp 0        producer: per stage (128 K-codes = two quantization groups) one TMA for the
 //                 128 x 128-byte A tile and one for the B tile, both with the 128-byte swizzle the tensor
 //                 core expects, into a slot of the operand ring, plus the matching 2 x 128 blocks of weight
 //                 scales and of activation scales into the "scale" ring (same mbarrier; that ring is deep
 //                 enough to need no barriers of its own).  The BF16 low-rank operands T and L2 use the
 //                 same ring.
-//   warp 1        MMA issuer (one lane): per stage four tcgen05.mma kind::f8f6f4 (K=32 each), two per group,
+//   warp 1        MMA issuer: per stage four tcgen05.mma kind::f8f6f4 (K=32 each), two per group,
 //                 each group into its own 128-column half of a 256-column TMEM slot (2 slots), so that
 //                 every group's partial sums stay separate; kind::f16 for the low-rank product
-//                 (first slot of a tile).  One barrier round trip per stage, not per group: a single
-//                 thread needs ~300 cycles per wait/issue/commit cycle, more than one group's MMA time.
+//                 (first slot of a tile).  One barrier round trip per stage, not per group.
 //   warp 2        TMEM allocation / release.
 //   warps 4-19    epilogue: TMEM -> registers with the 32x32b shape (a thread reads its own TMEM lane, i.e. one
 //                 token row; by far the fastest of the load shapes: ~830 B/clk/SM against ~250 for the
