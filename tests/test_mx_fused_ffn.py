@@ -74,6 +74,9 @@ def run_fused_case(M, K, H, N2, r1, r2, act, rho1, rho2, bias, seed=0):
     (256, 256, 512, 128, 0, 16, 1, False),     # no low-rank branch upstream, r' = 16
     (300, 512, 768, 512, 32, 64, 0, True),     # r' = 64 (two T buffers of 64 columns), no activation
     (517, 256, 1024, 256, 32, 0, 1, True),     # next layer without a low-rank branch
+    (129, 256, 256, 128, 64, 16, 1, False),    # one row past the first tile, a single column tile, r = 64 upstream
+    (1025, 512, 1536, 384, 16, 32, 1, True),   # nine row tiles (an odd count), six column tiles = one full run
+    (640, 256, 1792, 128, 0, 32, 0, False),    # seven column tiles: a run of six and a run of one
 ])
 def test_fused_ffn_matches_oracle(M, K, H, N2, r1, r2, act, bias):
     run_fused_case(M, K, H, N2, r1, r2, act, 0.9, 0.8, bias, seed=11 + M)
