@@ -385,6 +385,11 @@ __device__ __forceinline__ void tma2_load_2d(uint32_t dst_smem, const CUtensorMa
       ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
       : "memory");
 }
+// Release at cluster scope: for hand-overs of data this thread wrote to memory (the fused epilogue's x_hat rows in
+// shared memory, read by the pair's tensor cores on behalf of the other CTA).
+__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ void tmem_alloc2(uint32_t smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -806,7 +811,7 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (with_t) {
           fence_proxy_async_smem();   // generic-proxy stores -> visible to the tensor core's reads
           __syncwarp();
-          if (lane == 0) mbar_arrive_remote(map_to_cta(bar_xh_full, 0));
+          if (lane == 0) mbar_arrive_remote_release(map_to_cta(bar_xh_full, 0));
         }
         if (row_ok && ch_ok) {
           const float rho2 = __ldg(nx.rho);
