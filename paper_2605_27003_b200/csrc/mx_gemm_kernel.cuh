@@ -441,7 +441,9 @@ static_assert(kMx2StageBytes % 1024 == 0, "operand tiles must stay 1024-byte ali
 // matching 256 rows of L1' (tcgen05.mma kind::f16, M = 256 over the pair, N = r') into a small TMEM accumulator
 // that stays resident while the cluster walks a run of column tiles of one row pair (work is dealt to clusters in
 // such runs), and is added into an FP32 [M, r'] array when the run ends.
-// Shared memory: four stages instead of six, the 64 KiB x_hat tile, 16 KiB for the L1' tile.
+// Shared memory: four stages instead of six, the 64 KiB x_hat tile, 16 KiB for the L1' tile (four K slices of
+// r'/2 rows, packed at whole swizzle atoms; for r' <= 32 they fill the lower half and the upper half holds one
+// 512-byte table per epilogue warp: the bias and the next layer's 1/lambda of the warp's 64 channels).
 // Barriers: xh_full (leader; 32 epilogue warps: "x_hat tile written"), xh_empty (both; committed after the T MMAs:
 // x_hat and L1' tiles may be overwritten), l1_full (leader; TMA bytes of both CTAs' L1' halves), t_full[2] (both;
 // committed after the last T MMA of a row pair), t_empty[2] (leader; 8 warps: "T buffer read").
