@@ -149,3 +149,26 @@ def test_generator_weight_rounding_agrees_with_the_element_rule():
             v = float(np.float32(scaled[k, n].item()))
             if float(scaled[k, n]) == v:  # exactly representable in FP32: same input on both sides
                 assert (oracle.e2m1_rne_sat(v) & 7) == (int(codes[k, n]) & 7)
+
+
+def test_power_of_two_scaling_shifts_exponents_and_blocks_are_independent():
+    # The MX conversion is homogeneous under powers of two: x * 2^k keeps every element code and adds k to every
+    # shared exponent; a block's result depends on that block's 32 values only, so replacing another block of the
+    # row (or another row) changes nothing in it.
+    rng = np.random.default_rng(31)
+    M, K = 5, 128
+    x = torch.tensor(rng.normal(size=(M, K)).astype(np.float32)).to(torch.bfloat16)
+    x[:, 7] *= 25.0
+    lam = (2.0 ** rng.integers(-2, 3, size=K)).astype(np.float32)
+    codes, exps = oracle.mx_quantize(bits(x), lam, 0.9)
+    for k in (-4, 6):
+        ck, ek = oracle.mx_quantize(bits((x.to(torch.float32) * 2.0 ** k).to(torch.bfloat16)), lam, 0.9)
+        assert np.array_equal(oracle.e2m1_values(ck), oracle.e2m1_values(codes))
+        nz = exps > 0
+        assert np.array_equal(ek[nz].astype(np.int32), exps[nz].astype(np.int32) + k)
+    y = x.clone()
+    y[:, 32:64] = torch.tensor(rng.normal(size=(M, 32)).astype(np.float32)).to(torch.bfloat16) * 1000.0
+    y[1:] = y[1:] * 3.0
+    cy, ey = oracle.mx_quantize(bits(y), lam, 0.9)
+    keep = np.r_[0:32, 64:128]
+    assert np.array_equal(cy[0, keep], codes[0, keep]) and np.array_equal(ey[0, [0, 2, 3]], exps[0, [0, 2, 3]])

@@ -316,3 +316,44 @@ def test_generator_residual_rounding_is_on_grid():
     deq = q.astype(np.float64) * np.repeat(layer.wscale.numpy().astype(np.float64), G, axis=0)
     step = np.repeat(layer.wscale.numpy().astype(np.float64), G, axis=0)
     assert np.all(np.abs(deq - layer.R.numpy()) <= 0.5 * step * (1 + 1e-6) + 1e-12)
+
+
+def test_power_of_two_scaling_and_row_independence():
+    # Multiplying the activations by 2^k is exact in BF16 and FP32, so the quantizer must return the same codes with
+    # scales multiplied by 2^k (Eq. 3-5 are homogeneous); rows are quantized independently of one another (Eq. 4's
+    # maximum runs over one token's group only), so any subset or permutation of rows gives the same per-row result.
+    rng = np.random.default_rng(21)
+    M, K = 12, 3 * G
+    x = rng.normal(size=(M, K)).astype(np.float32)
+    x[:, 5] *= 30.0
+    lam = (0.5 + rng.random(K)).astype(np.float32)
+    xb = bf16_bits_of(x)
+    q0, s0 = oracle.quantize(xb, lam, 0.85)
+    for k in (-5, 3):
+        xk = bf16_bits_of(oracle.bf16_bits_to_f64(xb).astype(np.float32) * np.float32(2.0 ** k))
+        qk, sk = oracle.quantize(xk, lam, 0.85)
+        assert np.array_equal(qk, q0)
+        assert np.array_equal(sk, s0 * np.float32(2.0 ** k))
+    perm = rng.permutation(M)
+    qp, sp = oracle.quantize(xb[perm], lam, 0.85)
+    assert np.array_equal(qp, q0[perm]) and np.array_equal(sp, s0[perm])
+    q1, s1 = oracle.quantize(xb[3:4], lam, 0.85)
+    assert np.array_equal(q1, q0[3:4]) and np.array_equal(s1, s0[3:4])
+
+
+def test_smaller_clip_ratio_never_shrinks_a_code():
+    # Eq. 8-9: a smaller rho shrinks the scale, so |x / s| grows: magnitudes of the codes are non-decreasing as rho
+    # falls (until they saturate at 7), and the scale is proportional to rho up to FP32 rounding.
+    rng = np.random.default_rng(22)
+    x = rng.normal(size=(6, 2 * G)).astype(np.float32)
+    lam = np.ones(2 * G, np.float32)
+    xb = bf16_bits_of(x)
+    prev_q, prev_s = None, None
+    for rho in (1.0, 0.9, 0.75, 0.6, 0.5):
+        q, s = oracle.quantize(xb, lam, rho)
+        assert q.min() >= -8 and q.max() <= 7
+        if prev_q is not None:
+            assert np.all(np.abs(q.astype(np.int32)) >= np.abs(prev_q.astype(np.int32))), "a code shrank when rho fell"
+            assert np.all(s <= prev_s)
+        np.testing.assert_allclose(s, oracle.quantize(xb, lam, 1.0)[1] * rho, rtol=3e-7)
+        prev_q, prev_s = q, s
