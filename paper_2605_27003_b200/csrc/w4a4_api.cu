@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "gemm_kernel.cuh"
+#include "gemm_os_kernel.cuh"
 #include "host_common.h"
 #include "quantize_kernel.cuh"
 
@@ -125,6 +126,7 @@ using namespace w4a4;
 struct ExpertData {
   uint8_t* bpacked = nullptr;  // [N, K/2]
   float* wscale = nullptr;     // [G, N]
+  uint8_t* b_sop = nullptr;    // weight scale operands of the scale MMA: [N/128][ceil(G/2)][2][4096]
   float* rlam = nullptr;       // [K]
   uint2* l1frag = nullptr;
   uint16_t* l2dup = nullptr;   // [N, 2r]
@@ -146,6 +148,7 @@ namespace {
 void free_expert(ExpertData& e) {
   cudaFree(e.bpacked);
   cudaFree(e.wscale);
+  cudaFree(e.b_sop);
   cudaFree(e.rlam);
   cudaFree(e.l1frag);
   cudaFree(e.l2dup);
@@ -184,7 +187,8 @@ w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expe
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define W4A4_LAUNCH_Q(R)                                                                                         \
   quantize_kernel<R, quantize_warps(R), kCodesE4M3><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
-                                                 ctx->scales, ctx->scales_ld, ctx->t_hilo, ctx->t_partial)
+                                                 ctx->scales, ctx->scales_ld, ctx->t_hilo, ctx->t_partial,     \
+                                                 reinterpret_cast<uint4*>(ctx->a_sop))
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
     case 16: W4A4_LAUNCH_Q(16); break;
@@ -246,10 +250,25 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   }
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : h->tmB;
-  if (dbg_P) {
-    gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
+  static const bool cuda_core_rescale = [] {
+    const char* v = std::getenv("W4A4_GEMM");
+    return v && std::strcmp(v, "cuda_core_rescale") == 0;
+  }();
+  if (cuda_core_rescale) {
+    if (dbg_P) {
+      gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
+    } else {
+      gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
+    }
   } else {
-    gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
+    OsParams q;
+    q.a_sop = ctx->a_sop;
+    q.b_sop = e.b_sop;
+    if (dbg_P) {
+      gemm_os_kernel<true><<<grid, block, kOsSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, p, q);
+    } else {
+      gemm_os_kernel<false><<<grid, block, kOsSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, p, q);
+    }
   }
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
@@ -312,6 +331,10 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   w4a4_status_t st = dev_alloc(&ctx->codes, static_cast<size_t>(max_M) * max_K, &ctx->bytes);
   if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(ctx->scales_ld) * (max_K / 64), &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->scales, 0, sizeof(float) * ctx->scales_ld * (max_K / 64)) != cudaSuccess) st = W4A4_ERR_CUDA;
+  const size_t a_sop_bytes = static_cast<size_t>((max_M + 127) / 128) * ((max_K / 64 + 1) / 2) * 4096;
+  if (st == W4A4_OK) st = dev_alloc(&ctx->a_sop, a_sop_bytes, &ctx->bytes);
+  // Rows past M and the unused half of an odd last stage are multiplied by zeros: they only have to be finite.
+  if (st == W4A4_OK && cudaMemset(ctx->a_sop, 0, a_sop_bytes) != cudaSuccess) st = W4A4_ERR_CUDA;
   if (st == W4A4_OK) st = dev_alloc(&ctx->t_hilo, static_cast<size_t>(max_M) * 2 * (max_r > 0 ? max_r : 8), &ctx->bytes);
   if (st == W4A4_OK && max_r > 0)
     st = dev_alloc(&ctx->t_partial,
@@ -328,6 +351,8 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
                          static_cast<int>(quantize_smem_bytes(64)));
     cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(gemm_os_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOsSmemBytes);
+    if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(gemm_os_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOsSmemBytes);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       cudaGetLastError();
       st = W4A4_ERR_CUDA;
@@ -353,6 +378,7 @@ void w4a4_ctx_destroy(w4a4_ctx_t ctx) {
   cudaFree(ctx->t_hilo2);
   cudaFree(ctx->t_partial);
   cudaFree(ctx->scales);
+  cudaFree(ctx->a_sop);
   cudaFree(ctx->t_hilo);
   cudaFree(ctx->d_err);
   for (int i = 0; i < 2; ++i) {
@@ -445,6 +471,14 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
 
     const cudaMemcpyKind kind = dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
     if (cudaMemcpy(e.wscale, d->wscale[ei], sizeof(float) * G * N, kind) != cudaSuccess) st = W4A4_ERR_CUDA;
+    const size_t b_sop_bytes = static_cast<size_t>(N / kBN) * ((G + 1) / 2) * kOsSopTile;
+    if (st == W4A4_OK) st = dev_alloc(&e.b_sop, b_sop_bytes, &h->bytes);
+    if (st == W4A4_OK && cudaMemset(e.b_sop, 0, b_sop_bytes) != cudaSuccess) st = W4A4_ERR_CUDA;
+    if (st == W4A4_OK) {
+      const size_t ns = static_cast<size_t>(G) * N;
+      sop_weight_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256>>>(e.wscale, reinterpret_cast<uint4*>(e.b_sop), G, N);
+      if (cudaGetLastError() != cudaSuccess) st = W4A4_ERR_CUDA;
+    }
     if (st == W4A4_OK && bias_src && cudaMemcpy(e.bias, bias_src, sizeof(float) * N, kind) != cudaSuccess)
       st = W4A4_ERR_CUDA;
     if (st != W4A4_OK) break;

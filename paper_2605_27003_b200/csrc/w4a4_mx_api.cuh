@@ -69,7 +69,7 @@ w4a4_status_t mx_launch_quantize_at(w4a4_mx_handle_t h, const void* X, int M, in
   float* sf = reinterpret_cast<float*>(ctx->mx_sfa);
 #define W4A4_LAUNCH_MXQ(R)                                                                                             \
   quantize_kernel<R, quantize_warps(R), kCodesMxfp4><<<grid, block, quantize_smem_bytes(R), stream>>>(                 \
-      x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, sf, h->K / 128, ctx->t_hilo, ctx->t_partial)
+      x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, sf, h->K / 128, ctx->t_hilo, ctx->t_partial, nullptr)
   switch (h->r) {
     case 0: W4A4_LAUNCH_MXQ(0); break;
     case 16: W4A4_LAUNCH_MXQ(16); break;

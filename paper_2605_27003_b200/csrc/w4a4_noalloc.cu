@@ -105,7 +105,7 @@ extern "C" w4a4_status_t w4a4_quantize_noalloc(const void* X, int M, int K, cons
   constexpr int kWarps = w4a4::quantize_warps(0);
   w4a4::quantize_kernel<0, kWarps, w4a4::kCodesPacked><<<(M + w4a4::kQuantRows * kWarps - 1) / (w4a4::kQuantRows * kWarps), 32 * kWarps,
                                      w4a4::quantize_smem_bytes(0), s>>>(
-      static_cast<const uint16_t*>(X), M, K, rlam, clip_table, clip_index, nullptr, ws_codes, ws_scales, ld, nullptr, nullptr);
+      static_cast<const uint16_t*>(X), M, K, rlam, clip_table, clip_index, nullptr, ws_codes, ws_scales, ld, nullptr, nullptr, nullptr);
   const size_t nc = static_cast<size_t>(M) * K, ns = static_cast<size_t>(M) * G;
   noalloc_decode_codes_kernel<<<static_cast<unsigned>((nc + 255) / 256), 256, 0, s>>>(ws_codes, codes, M, K);
   noalloc_decode_scales_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256, 0, s>>>(ws_scales, ld, scales, M, G);
