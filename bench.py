@@ -35,7 +35,8 @@ NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_HBM_GBS = 7700.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries (profiles/);
 # None until a capture exists for that kernel and workload.
-NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 517.3e6, ("quantize", "attn_proj"): 484.7e6}
+# (quantize: 484.7 MB captured before the kernel also wrote the 41.9 MB of scale operands, which are added here.)
+NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 571.6e6, ("quantize", "attn_proj"): 526.6e6}
 
 
 def max_over_ranks(ms: float, dist, device="cpu") -> float:
@@ -310,7 +311,7 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                     for b, alpha in ((0, 0.7), (1, 1.0)):
                         tq, tg = time_layer(w4, layer, xs, [b] * n_x, 0, clip, Y, M, args.steps, max(3, args.warmup), stream)
                         ops = 2.0 * M * K * N
-                        qb = M * (3.0625 * K + 4.0 * r)
+                        qb = M * (3.3125 * K + 4.0 * r)
                         rows.append(dict(M=M, K=K, N=N, r=r, outlier_fraction=frac, alpha=alpha, quantize_ms=tq, gemm_ms=tg,
                                          layer_tops=ops / ((tq + tg) * 1e-3) / 1e12, gemm_tops=ops / (tg * 1e-3) / 1e12,
                                          gemm_frac=ops / (tg * 1e-3) / 1e12 / int8_peak,
@@ -661,7 +662,8 @@ def main():
         tq, tg = statistics.mean(t_q), statistics.mean(t_g)
         int8_peak = 2.0 * peaks["bf16_sustained"]  # dense 8-bit (INT8 or FP8) = 2 x dense BF16 (nominal ratio 4.5 / 2.25)
         gemm_tops = ops / (tg * 1e-3) / 1e12
-        q_bytes = M * (2.0 * K + 1.0 * K + 4.0 * K / 64.0 + 4.0 * r)  # X read, one-byte codes, scales, T as BF16 hi | lo
+        # X read, one-byte codes, FP32 scales, 16-byte scale-operand chunks, T as BF16 hi | lo
+        q_bytes = M * (2.0 * K + 1.0 * K + 4.0 * K / 64.0 + 16.0 * K / 64.0 + 4.0 * r)
         q_gbs = q_bytes / (tq * 1e-3) / 1e9
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
@@ -672,7 +674,7 @@ def main():
                         parallelism="replicas" if world > 1 else "single"),
             roofline=dict(bound="tensor", achieved=gemm_tops, peak=int8_peak, unit="TOP/s", frac=gemm_tops / int8_peak,
                           traffic=NCU_TRAFFIC_BYTES.get(("gemm", args.workload)),
-                          kernel="gemm_kernel (with the 9 us expand_weight_kernel in front of it)", ms=tg,
+                          kernel="gemm_os_kernel (with the 9 us expand_weight_kernel in front of it)", ms=tg,
                           peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 2 "
                                       "(nominal 8-bit:BF16 ratio)",
                           frac_of_nominal_4500=gemm_tops / NOMINAL_INT8_TOPS),
