@@ -6,8 +6,8 @@
 // is an outer product, i.e. a K = 16 BF16 MMA on operands that hold the two scales split into BF16 pieces:
 //     A row (token m, one 8-slot chunk per group):    [h, h, h, m, m, m, l, l]     sx = h + m + l  (BF16 each)
 //     B row (channel n, one 8-slot chunk per group):  [w1, w2, w3, w1, w2, w3, w1, w2]   sw = w1 + w2 + w3
-// so that the MMA's FP32 sum is  h w1 + h w2 + h w3 + m w1 + m w2 + m w3 + l w1 + l w2 = sx * sw  up to the two
-// dropped terms (below 2^-24 of the product) and the FP32 summation.  A K = 16 operand row carries the chunks of the
+// so that the MMA's FP32 sum is  h w1 + h w2 + h w3 + m w1 + m w2 + m w3 + l w1 + l w2 = sx * sw  up to the
+// dropped term l w3 (below 2^-24 of the product) and the FP32 summation.  A K = 16 operand row carries the chunks of the
 // two groups of a stage; the MMA of one group starts both descriptors at that group's chunk and points their second
 // K chunk at a tile of zeros.  The epilogue then does one fused multiply-add per partial sum, acc += P_g * S_g, on two
 // TMEM fragments, and reads no scales from shared memory at all.
