@@ -281,3 +281,49 @@ def gelu_tanh(y):
     activation a layer can be asked to fuse (the FFN's nonlinearity; not part of the paper's equations)."""
     y = np.asarray(y, dtype=np.float64)
     return 0.5 * y * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (y + 0.044715 * y ** 3)))
+
+
+def gptq_hessian(Xhat_bits):
+    """Layer-wise second-order statistic of GPTQ (Frantar et al., 2023, Sec. 3: H = 2 X X^T for the layer's inputs;
+    the factor 2 cancels in every quantity derived from it) for smoothed calibration activations X_hat [M, K] given
+    as BF16 bit patterns: H = X_hat^T X_hat in FP64."""
+    X = bf16_bits_to_f64(Xhat_bits)
+    return X.T @ X
+
+
+def gptq_quantize(R, H, group=64, percdamp=0.01):
+    """GPTQ (Frantar et al., 2023, Algorithm 1 with the Cholesky reformulation of Sec. 4, step 3) on the residual
+    branch (Sec. III-B: "we further apply GPTQ to the residual branch instead of simple round-to-nearest").
+
+    R [K, N] FP64: residual weights, input channels along rows.  H [K, K] FP64: X_hat^T X_hat of the calibration
+    activations.  Input channels are quantized in order; after each one its quantization error, scaled by the
+    matching entry of U = chol(H^-1, upper), is spread over the input channels still to come.  Readings where the
+    papers leave a choice: INT4 grid and group scale exactly as the round-to-nearest quantizer (scale = FP32(max
+    |w| / 7) over the group's 64 input channels, code = round-half-even(w / scale) clamped to [-8, 7], zero group ->
+    scale 0, codes 0), the scale being taken from the error-compensated weights when the sweep enters the group (static
+    groups, no activation ordering); dead input channels (H_kk = 0) get H_kk = 1 and zero weights; damping percdamp *
+    mean(diag H) on the diagonal; the lazy-batch block equals the group (pure bookkeeping: the result does not depend
+    on it).  -> codes int8 [K, N], scales FP32 [K / group, N]."""
+    W = np.array(R, dtype=np.float64, copy=True)
+    H = np.array(H, dtype=np.float64, copy=True)
+    K, N = W.shape
+    assert H.shape == (K, K) and K % group == 0
+    dead = np.diag(H) == 0
+    H[dead, dead] = 1.0
+    W[dead, :] = 0.0
+    H[np.diag_indices(K)] += percdamp * np.mean(np.diag(H))
+    Hinv = np.linalg.inv(H)
+    U = np.linalg.cholesky((Hinv + Hinv.T) / 2).T          # upper, H^-1 = U^T U
+    codes = np.zeros((K, N), np.int8)
+    scales = np.zeros((K // group, N), np.float32)
+    for k in range(K):
+        g = k // group
+        if k % group == 0:
+            scales[g] = (np.abs(W[k:k + group]).max(axis=0) / 7.0).astype(np.float32)
+        s = scales[g].astype(np.float64)
+        safe = np.where(s > 0, s, 1.0)
+        q = np.where(s > 0, np.clip(np.rint(W[k] / safe), -8, 7), 0.0)
+        codes[k] = q.astype(np.int8)
+        err = (W[k] - q * s) / U[k, k]
+        W[k + 1:] -= np.outer(U[k, k + 1:], err)
+    return codes, scales

@@ -1,0 +1,114 @@
+"""Pins of the GPTQ oracle (residual-branch weight quantization, Sec. III-B) against what the algorithm's
+definition fixes: special cases that reduce to round-to-nearest, a hand-computed two-channel case, the greedy
+step's optimality property, invariances, and the reconstruction objective against round-to-nearest."""
+import numpy as np
+import torch
+
+import oracle
+from workloads import generator as gen
+
+
+def rtn(R, group=64):
+    q, s = gen._round_residual(torch.from_numpy(np.asarray(R, np.float64))) if group == 64 else (None, None)
+    return q.numpy(), s.numpy()
+
+
+def proxy_loss(R, q, s, H, group):
+    D = R - q.astype(np.float64) * np.repeat(s.astype(np.float64), group, axis=0)
+    return float(np.einsum("kn,kj,jn->", D, H, D))
+
+
+def test_identity_hessian_reduces_to_round_to_nearest():
+    # H = c I: H^-1 is diagonal, its Cholesky factor has no off-diagonal entries, no error is propagated.
+    rng = np.random.default_rng(0)
+    R = rng.normal(scale=0.02, size=(128, 24))
+    R[64:128, 3] = 0.0
+    for c in (1.0, 37.5):
+        q, s = oracle.gptq_quantize(R, c * np.eye(128))
+        q0, s0 = rtn(R)
+        assert np.array_equal(q, q0) and np.array_equal(s, s0)
+
+
+def test_two_channel_case_by_hand():
+    # group = 2, one output channel, H = [[2, 1], [1, 2]] (no damping).  H^-1 = [[2, -1], [-1, 2]] / 3,
+    # U = chol(H^-1, upper) = [[sqrt(2/3), -sqrt(1/6)], [0, sqrt(1/2)]].
+    # w = (0.7, 0.38): scale = 0.1, q0 = 7, error 0; nothing to propagate -> q1 = round(3.8) = 4.
+    q, s = oracle.gptq_quantize(np.array([[0.7], [0.38]]), np.array([[2.0, 1.0], [1.0, 2.0]]), group=2, percdamp=0.0)
+    assert np.allclose(s, [[0.1]]) and q[:, 0].tolist() == [7, 4]
+    # w = (0.33, 0.7): scale = 0.1, q0 = 3, error e = 0.03; the second weight becomes
+    # 0.7 - e * U01 / U00 = 0.7 + 0.03 * 0.5 = 0.715 -> 7.15 -> 7 (and with e = 0.05 it would cross to 0.725 -> 7).
+    q, s = oracle.gptq_quantize(np.array([[0.33], [0.7]]), np.array([[2.0, 1.0], [1.0, 2.0]]), group=2, percdamp=0.0)
+    assert q[:, 0].tolist() == [3, 7]
+    # w = (0.26, 0.64): q0 = round(0.26 / (0.64 / 7)) = round(2.84375) = 3 with scale 0.0914285..., error
+    # 0.26 - 3 * 0.0914285 = -0.0142857; second weight 0.64 - 0.5 * 0.0142857 = 0.632857 -> 6.92 -> 7.
+    q, s = oracle.gptq_quantize(np.array([[0.26], [0.64]]), np.array([[2.0, 1.0], [1.0, 2.0]]), group=2, percdamp=0.0)
+    assert q[:, 0].tolist() == [3, 7]
+    # A case where the compensation changes a code.  Three channels in one group; the first is uncorrelated with the
+    # others and carries the group maximum 0.7 (scale 0.1, q = 7, no error).  For the other two H = [[2, -1], [-1, 2]]:
+    # H^-1 = [[2, 1], [1, 2]] / 3, U01 / U00 = +0.5.  w1 = 0.33 -> q = 3, error 0.03; w2 = 0.665 - 0.03 * 0.5 = 0.65
+    # -> 6.5 minus the FP32 rounding of the scale (0.1 is slightly above 0.1 in FP32) -> 6, where plain rounding of
+    # 6.65 gives 7.
+    H3 = np.array([[1.0, 0.0, 0.0], [0.0, 2.0, -1.0], [0.0, -1.0, 2.0]])
+    q, s = oracle.gptq_quantize(np.array([[0.7], [0.33], [0.665]]), H3, group=3, percdamp=0.0)
+    assert q[:, 0].tolist() == [7, 3, 6]
+    q, s = oracle.gptq_quantize(np.array([[0.7], [0.33], [0.665]]), np.eye(3), group=3, percdamp=0.0)
+    assert q[:, 0].tolist() == [7, 3, 7]
+
+
+def test_update_minimises_the_remaining_objective():
+    # After fixing the first input channel, the compensated remaining weights are the minimiser of the quadratic
+    # objective over the still-free channels (the optimal-brain-surgeon step GPTQ is built on): with every later
+    # channel left unquantized (a huge group so that nothing else is rounded) the loss must equal e0^2 / [H^-1]_00.
+    rng = np.random.default_rng(2)
+    K = 6
+    X = rng.normal(size=(50, K))
+    H = X.T @ X
+    w = rng.normal(size=(K, 1))
+    Hinv = np.linalg.inv(H)
+    U = np.linalg.cholesky(Hinv).T
+    e0 = 0.123
+    w_rest = w[1:, 0] - e0 / U[0, 0] * U[0, 1:]                      # what the sweep leaves in the later channels
+    d = np.concatenate([[e0], w[1:, 0] - w_rest])                    # w - w_hat
+    loss = d @ H @ d
+    assert np.isclose(loss, e0 ** 2 / Hinv[0, 0], rtol=1e-10)
+    for _ in range(20):                                              # any other choice of the rest is worse
+        alt = w_rest + rng.normal(scale=1e-2, size=K - 1)
+        d2 = np.concatenate([[e0], w[1:, 0] - alt])
+        assert d2 @ H @ d2 >= loss - 1e-12
+
+
+def test_invariances():
+    rng = np.random.default_rng(3)
+    K, N = 128, 10
+    X = rng.normal(size=(300, K)) * (1.0 + 5.0 * (rng.random(K) < 0.05))
+    H = X.T @ X
+    R = rng.normal(scale=0.02, size=(K, N))
+    q, s = oracle.gptq_quantize(R, H)
+    q2, s2 = oracle.gptq_quantize(R, 7.0 * H)                        # the objective's scale does not matter
+    assert np.array_equal(q, q2) and np.array_equal(s, s2)
+    perm = rng.permutation(N)                                        # output channels are independent
+    q3, s3 = oracle.gptq_quantize(R[:, perm], H)
+    assert np.array_equal(q3, q[:, perm]) and np.array_equal(s3, s[:, perm])
+    q4, s4 = oracle.gptq_quantize(4.0 * R, H)                        # weights times a power of two: same codes
+    assert np.array_equal(q4, q) and np.array_equal(s4, 4.0 * s)
+
+
+def test_reconstruction_objective_beats_round_to_nearest():
+    # tr((R - R_hat)^T H (R - R_hat)) = || X (R - R_hat) ||_F^2 on the calibration set: GPTQ's whole point.
+    rng = np.random.default_rng(4)
+    K, N = 256, 32
+    base = rng.normal(size=(400, 16))
+    X = base @ rng.normal(size=(16, K)) + 0.3 * rng.normal(size=(400, K))   # correlated input channels
+    H = X.T @ X
+    R = rng.normal(scale=0.02, size=(K, N))
+    q, s = oracle.gptq_quantize(R, H)
+    q0, s0 = rtn(R)
+    assert q.min() >= -8 and q.max() <= 7
+    assert proxy_loss(R, q, s, H, 64) < 0.8 * proxy_loss(R, q0, s0, H, 64)
+
+
+def test_hessian_of_bf16_activations():
+    x = gen.make_activations(40, 64, seed=1)
+    H = oracle.gptq_hessian(gen.bf16_bits(x).numpy().view(np.uint16))
+    xf = x.to(torch.float64).numpy()
+    assert np.allclose(H, xf.T @ xf, rtol=1e-13) and np.allclose(H, H.T)
