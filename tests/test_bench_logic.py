@@ -4,6 +4,7 @@ import json
 import os
 import subprocess
 import sys
+import tempfile
 
 import torch
 import torch.distributed as dist
@@ -22,17 +23,22 @@ def _worker(rank, world, port, out):
     my_ms = [3.0, 5.0][rank]                        # rank 1 is the slow replica
     slowest = bench.max_over_ranks(my_ms, dist, "cpu")
     value = bench.whole_job_tops(2.0e12, world, slowest)
-    out[rank] = (slowest, value)
+    with open(os.path.join(out, f"rank{rank}.json"), "w") as f:
+        json.dump([slowest, value], f)
     dist.barrier()
     dist.destroy_process_group()
 
 
 def test_replica_aggregation_over_two_gloo_ranks():
     world = 2
-    with mp.Manager() as mgr:
-        out = mgr.dict()
+    # Results come back through files: a manager process would be forked from this one, and a fork leaves the
+    # parent's BLAS thread pool unusable for the LAPACK calls of tests that run later in the same process.
+    with tempfile.TemporaryDirectory() as out:
         mp.spawn(_worker, args=(world, 29731, out), nprocs=world, join=True)
-        res = dict(out)
+        res = {}
+        for rank in range(world):
+            with open(os.path.join(out, f"rank{rank}.json")) as f:
+                res[rank] = tuple(json.load(f))
     for rank in range(world):
         slowest, value = res[rank]
         assert slowest == 5.0                       # every rank sees the max over ranks
