@@ -538,13 +538,65 @@ def run_clip_search(args, w4, dev, local_rank, rank, peaks):
     ctx.close()
 
 
+def run_gptq(args, w4, dev, local_rank, rank, peaks):
+    """GPTQ on the residual branch (Sec. III-B) for one attention-projection layer: statistic from 2048 calibration
+    tokens, factorization, triangular inverse and the sweep, all FP64 on the device.  An offline step: the number is a
+    time per layer, with the FP64 rate it amounts to."""
+    if rank != 0:
+        return
+    K, N, M_cal = 5120, 5120, 2048
+    R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
+    Rd, xd = R.to(dev), xhat.to(dev)
+    codes = torch.empty((K, N), dtype=torch.int8, device=dev)
+    scales = torch.empty((K // 64, N), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(2):
+        w4.w4a4_gptq_quantize(Rd, codes, scales, Xhat=xd)
+    runs = max(1, min(args.steps, 5))
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(runs):
+        w4.w4a4_gptq_quantize(Rd, codes, scales, Xhat=xd)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / runs
+    # FP64 operations the algorithm needs: upper triangle of X^T X, H = V V^T, U = V^-1, the error propagation
+    flops = M_cal * K * K + K ** 3 / 3 + K ** 3 / 3 + float(K) * K * N
+    sm_mhz = clocks.get("sm_max_mhz") or 1965
+    peak = 148 * 64 * 2 * sm_mhz * 1e6 / 1e12      # 64 FP64 fused multiply-adds per SM and clock
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle  # test infrastructure; allowed here for the CPU-baseline leg only
+
+        cols = list(range(0, N, N // 32))[:32]
+        t0 = time.perf_counter()
+        H = oracle.gptq_hessian(bits(xhat))
+        oracle.gptq_quantize(R[:, cols].double().numpy(), H)
+        cpu = dict(value=(time.perf_counter() - t0) * 1e3, unit="ms", cores=torch.get_num_threads(), kind="oracle",
+                   sample="the full statistic and its inverse, the sweep on 32 of the 5120 output channels")
+    groups = K // 64
+    print(json.dumps(dict(
+        metric="gptq_layer_time", value=ms, unit="ms", n_gpus=1, steps=runs, warmup=2, ms_per_step=ms,
+        higher_is_better=False, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+        config=dict(workload="gptq", K=K, N=N, calibration_tokens=M_cal, group=64, percdamp=0.01,
+                    l2="working set of %.0f MB, larger than L2" % ((2 * K * K + K * N) * 8 / 1e6)),
+        roofline=dict(bound="alu", achieved=flops / (ms * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
+                      frac=flops / (ms * 1e-3) / 1e12 / peak, traffic=None,
+                      note="peak = 148 SMs x 64 FP64 FMA per clock x 2 x max SM clock (nominal unit count)"),
+        cpu_baseline=cpu, gpu_launches=(6 + 3 * groups + 3 * groups + 2 * groups) * runs, clocks=clocks)), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search", "mxfp4_attn_proj", "mxfp4_ffn_up",
-                                                            "mxfp4_ffn_down", "mxfp4_ffn"])
+                                                            "mxfp4_ffn_down", "mxfp4_ffn", "gptq"])
     ap.add_argument("--chunk-rows", type=int, default=4096, help="token rows per chunk of the host-buffer forward (e2e)")
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
@@ -593,6 +645,9 @@ def main():
         return
     if args.workload == "clip_search":
         run_clip_search(args, w4, dev, local_rank, rank, peaks)
+        return
+    if args.workload == "gptq":
+        run_gptq(args, w4, dev, local_rank, rank, peaks)
         return
     n_buf = 4
     w = workload_inputs(args.workload, dev, n_buf)

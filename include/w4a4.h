@@ -248,6 +248,27 @@ w4a4_status_t w4a4_mx_ffn_forward(w4a4_mx_handle_t up, w4a4_mx_handle_t down, co
  * uint8 [M, down.K], exps device uint8 [M, down.K/32], T device FP32 [M, down.r] or NULL. */
 w4a4_status_t w4a4_mx_debug_fused_input(w4a4_mx_handle_t down, int M, uint8_t* codes, uint8_t* exps, float* T, void* stream);
 
+/*
+ * GPTQ on the residual branch (Sec. III-B: the residual weights are quantized with GPTQ, not round-to-nearest;
+ * the algorithm is Frantar et al., 2023, Algorithm 1 with the Cholesky reformulation of its Sec. 4).  Offline
+ * step: produces the qweight / wscale inputs of w4a4_pack_weights for one expert of one layer.
+ *   R       device FP32 [K, N] row-major: residual weights, input channels along rows.
+ *   Xhat    device BF16 bit patterns [M_cal, K]: smoothed calibration activations; H = Xhat^T Xhat in FP64; or NULL
+ *   H_in    device FP64 [K, K] row-major, symmetric: the statistic itself (only its upper triangle is read); or NULL.
+ *           Exactly one of Xhat and H_in is given (else W4A4_ERR_INVALID_ARG); M_cal is ignored with H_in.
+ *   percdamp  damping: percdamp * mean(diag H) is added to the diagonal (after dead channels, H_kk = 0, were given
+ *           H_kk = 1 and zero weights).  >= 0.
+ *   codes   device int8 [K, N] (values in [-8, 7]) and scales device FP32 [K/64, N]: outputs.  Group scale =
+ *           FP32(max |w| / 7) over the group's 64 error-compensated input channels when the sweep enters the group;
+ *           code = round-half-even(w / scale) clamped to [-8, 7]; an all-zero group has scale 0 and codes 0.
+ * All arithmetic is FP64.  K a multiple of 64, K <= 16384, N <= 65536 (else W4A4_ERR_SHAPE).  Allocates and frees
+ * its own temporaries (about 16 K^2 + 8 K N + 8 M_cal K bytes; W4A4_ERR_ALLOC), runs on `stream` and returns after
+ * the stream has drained.  A statistic that is not positive definite after damping returns W4A4_ERR_INVALID_ARG
+ * with the outputs undefined.  No context is needed.
+ */
+w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal, const double* H_in,
+                                 int K, int N, double percdamp, int8_t* codes, float* scales, void* stream);
+
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
  * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
 w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);

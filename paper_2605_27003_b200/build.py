@@ -8,7 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libw4a4.so")
-SOURCES = [os.path.join(CSRC, "w4a4_api.cu"), os.path.join(CSRC, "w4a4_noalloc.cu")]
+SOURCES = [os.path.join(CSRC, "w4a4_api.cu"), os.path.join(CSRC, "w4a4_noalloc.cu"),
+           os.path.join(CSRC, "w4a4_gptq.cu")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-shared", "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

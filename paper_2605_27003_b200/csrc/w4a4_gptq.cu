@@ -1,0 +1,335 @@
+// w4a4_gptq_quantize: GPTQ on the residual branch (Sec. III-B), entirely on the device in FP64.
+//
+// The published algorithm (Frantar et al., 2023, Algorithm 1 with the Cholesky reformulation of Sec. 4) quantizes
+// the input channels of R [K, N] in order and spreads each channel's error, scaled by a row of
+// U = chol(H^-1, upper), over the channels still to come, H = X_hat^T X_hat being the second-order statistic of the
+// layer's calibration inputs.  Here:
+//
+//   1. H (upper triangle) = X_hat^T X_hat by a tiled FP64 GEMM; dead channels and damping on the diagonal.
+//   2. U without ever forming H^-1: factor H = V V^T with V UPPER triangular (a Cholesky factorization taken from
+//      the last channel to the first, blocked by 64: diagonal block, panel solve, rank-64 update), then U = V^-1
+//      (blocked triangular inverse, bottom up).  H^-1 = V^-T V^-1 = U^T U with U upper and a positive diagonal,
+//      which is the unique factor the algorithm asks for.
+//   3. The sweep, one 64-channel group at a time: one thread per output channel holds the group's 64 weights in
+//      registers, takes the group scale, quantizes channel after channel and applies the in-group updates; the
+//      group's scaled errors then update all later channels by one more GEMM (the algorithm's lazy batch).
+//
+// Nothing here waits on another block: every dependency is a kernel boundary on one stream.
+#include "../../include/w4a4.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace {
+
+constexpr int kNb = 64;  // block of the factorization = quantization group = lazy batch
+
+// ---------------------------------------------------------------------------------------------------------
+// C[m, n] = beta * C[m, n] + alpha * sum_k A(m, k) * B(k, n), every operand addressed by two strides so that a
+// transposed or sub-matrix operand costs nothing.  64 x 64 tile per block, 16-deep slices, 4 x 4 outputs per
+// thread.  upper_only: blocks whose tile lies entirely below the diagonal return at once.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kBM = 64, kBN = 64, kBK = 16;
+
+__global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int Kd, const double* __restrict__ A, long sa_m,
+                                                    long sa_k, const double* __restrict__ B, long sb_k, long sb_n,
+                                                    double* __restrict__ C, long sc_m, long sc_n, double alpha,
+                                                    double beta, int upper_only) {
+  __shared__ __align__(16) double As[kBK][kBM];
+  __shared__ __align__(16) double Bs[kBK][kBN];
+  const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
+  if (upper_only && m0 >= n0 + kBN) return;
+  const int tid = threadIdx.x, tn = tid & 15, tm = tid >> 4;
+  const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
+  double acc[4][4] = {};
+  for (int k0 = 0; k0 < Kd; k0 += kBK) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int e = tid + i * 256;
+      const int am = a_m_fast ? (e & 63) : (e >> 4), ak = a_m_fast ? (e >> 6) : (e & 15);
+      As[ak][am] = (m0 + am < M && k0 + ak < Kd) ? A[(long)(m0 + am) * sa_m + (long)(k0 + ak) * sa_k] : 0.0;
+      const int bn = b_n_fast ? (e & 63) : (e >> 4), bk = b_n_fast ? (e >> 6) : (e & 15);
+      Bs[bk][bn] = (n0 + bn < N && k0 + bk < Kd) ? B[(long)(k0 + bk) * sb_k + (long)(n0 + bn) * sb_n] : 0.0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kBK; ++k) {
+      double a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[k][tm * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = Bs[k][tn * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + tm * 4 + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tn * 4 + j;
+      if (n >= N) continue;
+      double* c = C + (long)m * sc_m + (long)n * sc_n;
+      *c = (beta == 0.0) ? alpha * acc[i][j] : fma(alpha, acc[i][j], beta * *c);
+    }
+  }
+}
+
+__global__ void bf16_to_f64_kernel(const uint16_t* __restrict__ in, double* __restrict__ out, long n) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = (double)__uint_as_float((uint32_t)in[i] << 16);
+}
+
+// Dead input channels (H_kk = 0) get H_kk = 1, and the mean of the diagonal after that fix goes to *mean_out.
+// One block; the sum runs in a fixed order (thread-strided partial sums, then a tree), so it is deterministic.
+__global__ void gptq_diag_mean_kernel(double* __restrict__ H, int K, unsigned char* __restrict__ dead,
+                                      double* __restrict__ mean_out) {
+  __shared__ double part[256];
+  double s = 0.0;
+  for (int k = threadIdx.x; k < K; k += 256) {
+    double d = H[(long)k * K + k];
+    const bool is_dead = (d == 0.0);
+    if (is_dead) {
+      d = 1.0;
+      H[(long)k * K + k] = 1.0;
+    }
+    dead[k] = is_dead ? 1 : 0;
+    s += d;
+  }
+  part[threadIdx.x] = s;
+  __syncthreads();
+  for (int w = 128; w > 0; w >>= 1) {
+    if (threadIdx.x < w) part[threadIdx.x] += part[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *mean_out = part[0] / (double)K;
+}
+
+__global__ void gptq_damp_kernel(double* __restrict__ H, int K, const double* __restrict__ mean, double percdamp) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < K) H[(long)k * K + k] += percdamp * *mean;
+}
+
+// W = FP64(R) with the rows of dead input channels zeroed.
+__global__ void gptq_init_w_kernel(const float* __restrict__ R, const unsigned char* __restrict__ dead,
+                                   double* __restrict__ W, int K, int N) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < (long)K * N) W[i] = dead[i / N] ? 0.0 : (double)R[i];
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// H = V V^T, V upper triangular, from the last block to the first (A holds H's upper triangle and ends as V).
+// ---------------------------------------------------------------------------------------------------------
+
+// The 64 x 64 diagonal block at j0, whose trailing updates are already applied: column 63 down to column 0.
+// A pivot that is not positive raises *not_pd (the matrix was not positive definite).
+__global__ void __launch_bounds__(kNb) chol_diag_kernel(double* __restrict__ A, long ld, int j0, int* not_pd) {
+  __shared__ double S[kNb][kNb + 1];
+  const int t = threadIdx.x;
+  for (int r = 0; r < kNb; ++r) S[r][t] = A[(long)(j0 + r) * ld + j0 + t];
+  __syncthreads();
+  for (int j = kNb - 1; j >= 0; --j) {
+    if (t == j) {
+      const double d = S[j][j];
+      if (!(d > 0.0)) *not_pd = 1;
+      S[j][j] = sqrt(d);
+    }
+    __syncthreads();
+    if (t < j) S[t][j] /= S[j][j];
+    __syncthreads();
+    if (t < j) {
+      const double f = S[t][j];
+      for (int c = t; c < j; ++c) S[t][c] = fma(-f, S[c][j], S[t][c]);
+    }
+    __syncthreads();
+  }
+  for (int r = 0; r < kNb; ++r) A[(long)(j0 + r) * ld + j0 + t] = (t >= r) ? S[r][t] : 0.0;
+}
+
+// The panel above the diagonal block: each row x of A[0:j0, j0:j0+64] becomes the solution of x D^T = row, D the
+// factored diagonal block.  One thread per row, the row in registers.
+__global__ void __launch_bounds__(kNb) chol_panel_kernel(double* __restrict__ A, long ld, int j0) {
+  __shared__ double D[kNb][kNb + 1];
+  const int t = threadIdx.x;
+  for (int r = 0; r < kNb; ++r) D[r][t] = A[(long)(j0 + r) * ld + j0 + t];
+  __syncthreads();
+  const int row = blockIdx.x * kNb + t;
+  if (row >= j0) return;
+  double* p = A + (long)row * ld + j0;
+  double b[kNb];
+#pragma unroll
+  for (int c = 0; c < kNb; ++c) b[c] = p[c];
+#pragma unroll
+  for (int c = kNb - 1; c >= 0; --c) {
+    b[c] = b[c] / D[c][c];
+#pragma unroll
+    for (int c2 = 0; c2 < c; ++c2) b[c2] = fma(-b[c], D[c2][c], b[c2]);
+  }
+#pragma unroll
+  for (int c = 0; c < kNb; ++c) p[c] = b[c];
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// U = V^-1 (both upper triangular), block row by block row from the bottom.
+// ---------------------------------------------------------------------------------------------------------
+
+// Inverse of the diagonal block of V at i0 into the same place of U: thread c solves D x = e_c.
+__global__ void __launch_bounds__(kNb) triinv_diag_kernel(const double* __restrict__ V, double* __restrict__ U,
+                                                          long ld, int i0) {
+  __shared__ double D[kNb][kNb + 1];
+  const int t = threadIdx.x;
+  for (int r = 0; r < kNb; ++r) D[r][t] = V[(long)(i0 + r) * ld + i0 + t];
+  __syncthreads();
+  double b[kNb];
+#pragma unroll
+  for (int r = 0; r < kNb; ++r) b[r] = (r == t) ? 1.0 : 0.0;
+#pragma unroll
+  for (int k = kNb - 1; k >= 0; --k) {
+    b[k] = b[k] / D[k][k];
+#pragma unroll
+    for (int r = 0; r < k; ++r) b[r] = fma(-D[r][k], b[k], b[r]);
+  }
+#pragma unroll
+  for (int r = 0; r < kNb; ++r) U[(long)(i0 + r) * ld + i0 + t] = b[r];
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// The sweep over one group of 64 input channels starting at k0 (Algorithm 1's inner loop): thread = output channel.
+// scale = FP32(max |w| / 7) over the group as it stands on entry; per channel code = clamp(round-half-even(w /
+// scale), -8, 7) (0 for an all-zero group), err = (w - code * scale) / U_kk, later channels of the group -= err *
+// U_kj.  Err [64, N] keeps the scaled errors for the update of the groups still to come.
+// ---------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kNb) gptq_group_kernel(const double* __restrict__ W, int N,
+                                                         const double* __restrict__ U, long ldu, int k0,
+                                                         int8_t* __restrict__ codes, float* __restrict__ scales,
+                                                         double* __restrict__ Err) {
+  __shared__ double D[kNb][kNb + 1];
+  const int t = threadIdx.x;
+  for (int r = 0; r < kNb; ++r) D[r][t] = U[(long)(k0 + r) * ldu + k0 + t];
+  __syncthreads();
+  const int n = blockIdx.x * kNb + t;
+  if (n >= N) return;
+  double w[kNb];
+  double amax = 0.0;
+#pragma unroll
+  for (int k = 0; k < kNb; ++k) {
+    w[k] = W[(long)(k0 + k) * N + n];
+    amax = fmax(amax, fabs(w[k]));
+  }
+  const float s32 = (float)(amax / 7.0);  // FP64 quotient rounded once to FP32
+  scales[(long)(k0 / kNb) * N + n] = s32;
+  const double s = (double)s32;
+#pragma unroll
+  for (int k = 0; k < kNb; ++k) {
+    double q = 0.0;
+    if (s > 0.0) q = fmin(fmax(rint(w[k] / s), -8.0), 7.0);
+    codes[(long)(k0 + k) * N + n] = (int8_t)q;
+    const double e = (w[k] - q * s) / D[k][k];
+    Err[(long)k * N + n] = e;
+#pragma unroll
+    for (int j = k + 1; j < kNb; ++j) w[j] -= e * D[k][j];
+  }
+}
+
+struct DeviceBuffers {
+  double *H = nullptr, *U = nullptr, *Xd = nullptr, *W = nullptr, *Err = nullptr, *T = nullptr, *mean = nullptr;
+  unsigned char* dead = nullptr;
+  int* not_pd = nullptr;
+  ~DeviceBuffers() {
+    cudaFree(H), cudaFree(U), cudaFree(Xd), cudaFree(W), cudaFree(Err), cudaFree(T), cudaFree(mean);
+    cudaFree(dead), cudaFree(not_pd);
+  }
+};
+
+void dgemm(cudaStream_t st, int M, int N, int Kd, const double* A, long sa_m, long sa_k, const double* B, long sb_k,
+           long sb_n, double* C, long sc_m, long sc_n, double alpha, double beta, bool upper_only = false) {
+  if (M <= 0 || N <= 0) return;
+  dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM);
+  dgemm_kernel<<<grid, 256, 0, st>>>(M, N, Kd, A, sa_m, sa_k, B, sb_k, sb_n, C, sc_m, sc_n, alpha, beta,
+                                     upper_only ? 1 : 0);
+}
+
+}  // namespace
+
+extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal,
+                                            const double* H_in, int K, int N, double percdamp, int8_t* codes,
+                                            float* scales, void* stream) {
+  if (R == nullptr || codes == nullptr || scales == nullptr) return W4A4_ERR_INVALID_ARG;
+  if ((Xhat == nullptr) == (H_in == nullptr)) return W4A4_ERR_INVALID_ARG;  // exactly one source of H
+  if (K <= 0 || N <= 0 || K % kNb != 0 || K > 16384 || N > 65536) return W4A4_ERR_SHAPE;
+  if (Xhat != nullptr && M_cal <= 0) return W4A4_ERR_SHAPE;
+  if (!(percdamp >= 0.0)) return W4A4_ERR_INVALID_ARG;
+  if (cudaSetDevice(device) != cudaSuccess) return W4A4_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return W4A4_ERR_CUDA;
+  if (prop.major != 10) return W4A4_ERR_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  DeviceBuffers d;
+  const size_t kk = (size_t)K * K * sizeof(double);
+  bool ok = cudaMalloc(&d.H, kk) == cudaSuccess && cudaMalloc(&d.U, kk) == cudaSuccess &&
+            cudaMalloc(&d.W, (size_t)K * N * sizeof(double)) == cudaSuccess &&
+            cudaMalloc(&d.Err, (size_t)kNb * N * sizeof(double)) == cudaSuccess &&
+            cudaMalloc(&d.T, (size_t)kNb * K * sizeof(double)) == cudaSuccess &&
+            cudaMalloc(&d.mean, sizeof(double)) == cudaSuccess && cudaMalloc(&d.dead, K) == cudaSuccess &&
+            cudaMalloc(&d.not_pd, sizeof(int)) == cudaSuccess;
+  if (ok && Xhat != nullptr) ok = cudaMalloc(&d.Xd, (size_t)M_cal * K * sizeof(double)) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return W4A4_ERR_ALLOC;
+  }
+  cudaMemsetAsync(d.not_pd, 0, sizeof(int), st);
+  cudaMemsetAsync(d.U, 0, kk, st);
+
+  // 1. H, its dead channels and damping.
+  if (Xhat != nullptr) {
+    const long n = (long)M_cal * K;
+    bf16_to_f64_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(Xhat, d.Xd, n);
+    cudaMemsetAsync(d.H, 0, kk, st);
+    dgemm(st, K, K, M_cal, d.Xd, 1, K, d.Xd, K, 1, d.H, K, 1, 1.0, 0.0, /*upper_only=*/true);
+  } else {
+    cudaMemcpyAsync(d.H, H_in, kk, cudaMemcpyDeviceToDevice, st);
+  }
+  gptq_diag_mean_kernel<<<1, 256, 0, st>>>(d.H, K, d.dead, d.mean);
+  gptq_damp_kernel<<<(K + 255) / 256, 256, 0, st>>>(d.H, K, d.mean, percdamp);
+  {
+    const long n = (long)K * N;
+    gptq_init_w_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(R, d.dead, d.W, K, N);
+  }
+
+  // 2a. H = V V^T in place, last block first.
+  for (int j0 = K - kNb; j0 >= 0; j0 -= kNb) {
+    chol_diag_kernel<<<1, kNb, 0, st>>>(d.H, K, j0, d.not_pd);
+    if (j0 == 0) break;
+    chol_panel_kernel<<<(j0 + kNb - 1) / kNb, kNb, 0, st>>>(d.H, K, j0);
+    // H[0:j0, 0:j0] -= P P^T, P = the panel just solved (upper triangle only).
+    dgemm(st, j0, j0, kNb, d.H + j0, K, 1, d.H + j0, 1, K, d.H, K, 1, -1.0, 1.0, /*upper_only=*/true);
+  }
+  // 2b. U = V^-1, last block row first: U[i, rest] = -inv(V_ii) (V[i, rest] U[rest, rest]).
+  for (int i0 = K - kNb; i0 >= 0; i0 -= kNb) {
+    triinv_diag_kernel<<<1, kNb, 0, st>>>(d.H, d.U, K, i0);
+    const int r0 = i0 + kNb, rest = K - r0;
+    if (rest == 0) continue;
+    dgemm(st, kNb, rest, rest, d.H + (long)i0 * K + r0, K, 1, d.U + (long)r0 * K + r0, K, 1, d.T, K, 1, 1.0, 0.0);
+    dgemm(st, kNb, rest, kNb, d.U + (long)i0 * K + i0, K, 1, d.T, K, 1, d.U + (long)i0 * K + r0, K, 1, -1.0, 0.0);
+  }
+
+  // 3. The sweep: group by group, then the groups still to come -= U[group, later]^T Err.
+  for (int k0 = 0; k0 < K; k0 += kNb) {
+    gptq_group_kernel<<<(N + kNb - 1) / kNb, kNb, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, d.Err);
+    const int r0 = k0 + kNb, rest = K - r0;
+    dgemm(st, rest, N, kNb, d.U + (long)k0 * K + r0, 1, K, d.Err, N, 1, d.W + (long)r0 * N, N, 1, -1.0, 1.0);
+  }
+
+  int not_pd = 0;
+  if (cudaMemcpyAsync(&not_pd, d.not_pd, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+    return W4A4_ERR_CUDA;
+  return not_pd ? W4A4_ERR_INVALID_ARG : W4A4_OK;
+}

@@ -1,0 +1,119 @@
+"""GPTQ on the residual branch (Sec. III-B) on the GPU against the FP64 oracle, through the C ABI (GPU only).
+
+Both sides work in FP64 but reach U = chol(H^-1, upper) by different routes (the oracle inverts H and factors the
+inverse; the library factors H from the last channel to the first and inverts the triangular factor), so their
+error-compensated weights differ by rounding noise, about 1e-10 relative.  A weight that sits that close to a
+rounding boundary may take the neighbouring code on one side, and every later input channel of that OUTPUT channel
+then follows a different but equally valid trajectory; output channels do not interact.  The tests therefore demand
+bit-equal codes and scales on all but a handful of output channels and, on those, an objective value as good as the
+oracle's."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from workloads import generator as gen
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def bits(t):
+    return gen.bf16_bits(t.cpu()).numpy().view(np.uint16)
+
+
+def gpu_gptq(R, xhat=None, H=None, percdamp=0.01):
+    import paper_2605_27003_b200 as w4
+    K, N = R.shape
+    codes = torch.full((K, N), 99, dtype=torch.int8, device=DEV)
+    scales = torch.full((K // 64, N), -1.0, dtype=torch.float32, device=DEV)
+    w4.w4a4_gptq_quantize(R.to(DEV), codes, scales, Xhat=None if xhat is None else xhat.to(DEV),
+                          H=None if H is None else torch.from_numpy(H).to(DEV), percdamp=percdamp)
+    return codes.cpu().numpy(), scales.cpu().numpy()
+
+
+def objective(R, q, s, H):
+    D = R - q.astype(np.float64) * np.repeat(s.astype(np.float64), 64, axis=0)
+    return np.einsum("kn,kj,jn->n", D, H, D)
+
+
+def compare(R64, H, q_gpu, s_gpu, q_ref, s_ref, max_bad_columns):
+    bad = np.flatnonzero((q_gpu != q_ref).any(axis=0) | (s_gpu != s_ref).any(axis=0))
+    assert bad.size <= max_bad_columns, f"{bad.size} output channels differ"
+    if bad.size:
+        o_gpu = objective(R64[:, bad], q_gpu[:, bad], s_gpu[:, bad], H)
+        o_ref = objective(R64[:, bad], q_ref[:, bad], s_ref[:, bad], H)
+        assert np.all(o_gpu <= o_ref * 1.05), (o_gpu, o_ref)
+    assert q_gpu.min() >= -8 and q_gpu.max() <= 7
+
+
+def test_identity_statistic_is_round_to_nearest():
+    # H = c I: nothing is propagated, so the result is the plain group quantizer's, bit for bit.
+    R, _ = gen.make_gptq_inputs(256, 200, 8, seed=1)
+    R[64:128, 5] = 0.0
+    q0, s0 = gen._round_residual(R.double())
+    for c in (1.0, 12.5):
+        q, s = gpu_gptq(R, H=c * np.eye(256))
+        assert np.array_equal(q, q0.numpy()) and np.array_equal(s, s0.numpy())
+
+
+@pytest.mark.parametrize("K,N,M_cal,dead,percdamp", [
+    (64, 40, 96, (), 0.01),                # a single group: no update between groups
+    (256, 96, 300, (), 0.01),
+    (512, 130, 384, (3, 200), 0.01),       # ragged N, dead input channels
+    (320, 257, 100, (), 0.05),             # fewer calibration tokens than channels: H is singular before damping
+    (1024, 512, 1500, (1023,), 0.002),
+])
+def test_matches_oracle(K, N, M_cal, dead, percdamp):
+    R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=K + N, dead=dead)
+    R64 = R.double().numpy()
+    H = oracle.gptq_hessian(bits(xhat))
+    q_ref, s_ref = oracle.gptq_quantize(R64, H, percdamp=percdamp)
+    q, s = gpu_gptq(R, xhat=xhat, percdamp=percdamp)
+    compare(R64, H, q, s, q_ref, s_ref, max_bad_columns=max(1, N // 200))
+    # the compensation must have mattered: the plain quantizer gives different codes and a worse objective
+    q0, s0 = gen._round_residual(R.double())
+    assert (q != q0.numpy()).mean() > 0.05
+    Rz = R64.copy()
+    Rz[list(dead), :] = 0.0
+    assert objective(Rz, q, s, H).sum() < 0.9 * objective(Rz, q0.numpy(), s0.numpy(), H).sum()
+    # and the statistic handed over directly gives the same result as the activations
+    q2, s2 = gpu_gptq(R, H=H, percdamp=percdamp)
+    compare(R64, H, q2, s2, q_ref, s_ref, max_bad_columns=max(1, N // 200))
+
+
+def test_full_size_layer_on_sampled_output_channels():
+    # The size the bench times (K = N = 5120, 2048 calibration tokens).  Output channels are independent, so the
+    # oracle runs on a sample of them with the full statistic.
+    K, N, M_cal = 5120, 5120, 2048
+    R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
+    q, s = gpu_gptq(R, xhat=xhat)
+    cols = np.sort(np.random.default_rng(3).choice(N, 40, replace=False))
+    R64 = R[:, cols].double().numpy()
+    H = oracle.gptq_hessian(bits(xhat))
+    q_ref, s_ref = oracle.gptq_quantize(R64, H)
+    compare(R64, H, q[:, cols], s[:, cols], q_ref, s_ref, max_bad_columns=2)
+
+
+def test_argument_errors():
+    import paper_2605_27003_b200 as w4
+    lib = w4.load_library()
+    R = torch.zeros(64, 8, device=DEV)
+    codes = torch.zeros(64, 8, dtype=torch.int8, device=DEV)
+    scales = torch.zeros(1, 8, device=DEV)
+    H = torch.eye(64, dtype=torch.float64, device=DEV)
+    x = torch.zeros(4, 64, dtype=torch.bfloat16, device=DEV)
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    call = lambda *a: lib.w4a4_gptq_quantize(*a)
+    assert call(0, p(R), None, 0, None, 64, 8, 0.01, p(codes), p(scales), None) == 1        # no statistic
+    assert call(0, p(R), p(x), 4, p(H), 64, 8, 0.01, p(codes), p(scales), None) == 1        # two statistics
+    assert call(0, None, None, 0, p(H), 64, 8, 0.01, p(codes), p(scales), None) == 1
+    assert call(0, p(R), None, 0, p(H), 96, 8, 0.01, p(codes), p(scales), None) == 2        # K not a multiple of 64
+    assert call(0, p(R), p(x), 0, None, 64, 8, 0.01, p(codes), p(scales), None) == 2        # no calibration tokens
+    assert call(0, p(R), None, 0, p(H), 64, 8, -1.0, p(codes), p(scales), None) == 1
+    # not positive definite (and no damping): reported, not a fault
+    Hbad = -torch.eye(64, dtype=torch.float64, device=DEV)
+    assert call(0, p(R), None, 0, p(Hbad), 64, 8, 0.0, p(codes), p(scales), None) == 1
+    torch.cuda.synchronize()

@@ -103,6 +103,24 @@ def make_activations(M: int, K: int, *, sigma: float = 1.0, outlier_idx: Optiona
     return x.to(torch.bfloat16)
 
 
+def make_gptq_inputs(K: int, N: int, M_cal: int, *, seed: int = 0, shared: int = 8, dead: Sequence[int] = (),
+                     w_std: float = 0.02):
+    """Inputs of the residual-branch weight quantization: residual weights R [K, N] (FP32 values) and smoothed
+    calibration activations [M_cal, K] in BF16 whose channels are correlated (a few shared directions on top of
+    independent noise, a few channels scaled up), so that the second-order statistic is far from diagonal.  Channels
+    listed in `dead` are zero in every calibration token."""
+    g = _gen(seed * 15485863 + 3, "cpu")
+    R = (torch.randn(K, N, generator=g, dtype=torch.float32) * w_std)
+    z = torch.randn(M_cal, K, generator=g, dtype=torch.float32)
+    mix = torch.randn(shared, K, generator=g, dtype=torch.float32)
+    x = z + 0.8 * torch.randn(M_cal, shared, generator=g, dtype=torch.float32) @ mix
+    idx = outlier_channels(K, 0, seed, count=max(2, K // 128))
+    x[:, idx] *= 6.0
+    for k in dead:
+        x[:, k] = 0.0
+    return R, x.to(torch.bfloat16)
+
+
 def make_clip_table(num_experts: int, num_layers: int, num_bins: int,
                     ranges: Sequence[Sequence[float]], seed: int = 0) -> torch.Tensor:
     """FP32 clip ratios [E, L, B]; expert e draws uniformly from ranges[e] = (lo, hi)."""
