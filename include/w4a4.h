@@ -261,13 +261,19 @@ w4a4_status_t w4a4_mx_debug_fused_input(w4a4_mx_handle_t down, int M, uint8_t* c
  *   codes   device int8 [K, N] (values in [-8, 7]) and scales device FP32 [K/64, N]: outputs.  Group scale =
  *           FP32(max |w| / 7) over the group's 64 error-compensated input channels when the sweep enters the group;
  *           code = round-half-even(w / scale) clamped to [-8, 7]; an all-zero group has scale 0 and codes 0.
- * All arithmetic is FP64.  K a multiple of 64, K <= 16384, N <= 65536 (else W4A4_ERR_SHAPE).  Allocates and frees
- * its own temporaries (about 16 K^2 + 8 K N + 8 M_cal K bytes; W4A4_ERR_ALLOC), runs on `stream` and returns after
- * the stream has drained.  A statistic that is not positive definite after damping returns W4A4_ERR_INVALID_ARG
- * with the outputs undefined.  No context is needed.
+ *   workspace  device memory for the temporaries (FP64 copies of the statistic, its factor, the weights), 256-byte
+ *           aligned, at least w4a4_gptq_workspace_bytes(K, N, M_cal) bytes (M_cal = 0 with H_in), owned by the caller
+ *           and free again when the call returns; too small or misaligned returns W4A4_ERR_INVALID_ARG.  NULL: the
+ *           call allocates and frees the same amount itself (W4A4_ERR_ALLOC if that fails).
+ * All arithmetic is FP64.  K a multiple of 64, K <= 16384, N <= 65536, M_cal <= 2^20 (else W4A4_ERR_SHAPE;
+ * w4a4_gptq_workspace_bytes returns 0 for such a shape).  The workspace is about 16 K^2 + 8 K N + 8 M_cal K bytes.
+ * Runs on `stream` and returns after the stream has drained.  A statistic that is not positive definite after
+ * damping returns W4A4_ERR_INVALID_ARG with the outputs undefined.  No context is needed.
  */
+size_t w4a4_gptq_workspace_bytes(int K, int N, int M_cal);
 w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal, const double* H_in,
-                                 int K, int N, double percdamp, int8_t* codes, float* scales, void* stream);
+                                 int K, int N, double percdamp, int8_t* codes, float* scales, void* workspace,
+                                 size_t workspace_bytes, void* stream);
 
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
  * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */

@@ -23,53 +23,66 @@
 
 namespace {
 
-constexpr int kNb = 64;  // block of the factorization = quantization group = lazy batch
+constexpr int kNb = 64;     // block of the factorization = quantization group = lazy batch
+constexpr int kBand = 512;  // columns per band of the factorization, rows per band of the triangular inverse
+constexpr int kLazy = 256;  // input channels per lazy batch of the sweep
 
 // ---------------------------------------------------------------------------------------------------------
 // C[m, n] = beta * C[m, n] + alpha * sum_k A(m, k) * B(k, n), every operand addressed by two strides so that a
-// transposed or sub-matrix operand costs nothing.  64 x 64 tile per block, 16-deep slices, 4 x 4 outputs per
-// thread.  upper_only: blocks whose tile lies entirely below the diagonal return at once.
+// transposed or sub-matrix operand costs nothing.  (16 TM) x 64 tile per block, 16-deep slices, TM x 4 outputs per
+// thread.  Structure flags: kUpperOut -- blocks whose tile lies entirely below the diagonal return at once (only the
+// upper triangle of C is wanted); kAUpper -- A(m, k) = 0 for k < m, so the sum starts at the tile's first row;
+// kBUpper -- B(k, n) = 0 for k > n, so the sum ends at the tile's last column.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kBM = 64, kBN = 64, kBK = 16;
+constexpr int kBN = 64, kBK = 16;
+enum : int { kUpperOut = 1, kAUpper = 2, kBUpper = 4 };
 
-__global__ void __launch_bounds__(256) dgemm_kernel(int M, int N, int Kd, const double* __restrict__ A, long sa_m,
+template <int TM>
+__global__ void __launch_bounds__(256, 2) dgemm_kernel(int M, int N, int Kd, const double* __restrict__ A, long sa_m,
                                                     long sa_k, const double* __restrict__ B, long sb_k, long sb_n,
                                                     double* __restrict__ C, long sc_m, long sc_n, double alpha,
-                                                    double beta, int upper_only) {
-  __shared__ __align__(16) double As[kBK][kBM];
+                                                    double beta, int flags) {
+  constexpr int BM = 16 * TM;
+  __shared__ __align__(16) double As[kBK][BM];
   __shared__ __align__(16) double Bs[kBK][kBN];
-  const int m0 = blockIdx.y * kBM, n0 = blockIdx.x * kBN;
-  if (upper_only && m0 >= n0 + kBN) return;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * kBN;
+  if ((flags & kUpperOut) && m0 >= n0 + kBN) return;
   const int tid = threadIdx.x, tn = tid & 15, tm = tid >> 4;
   const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
-  double acc[4][4] = {};
-  for (int k0 = 0; k0 < Kd; k0 += kBK) {
+  const int k_begin = (flags & kAUpper) ? m0 : 0;  // m0 is a multiple of 16
+  const int k_end = (flags & kBUpper) ? min(Kd, n0 + kBN) : Kd;
+  double acc[TM][4] = {};
+  for (int k0 = k_begin; k0 < k_end; k0 += kBK) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+      const int e = tid + i * 256;
+      const int am = a_m_fast ? (e % BM) : (e >> 4), ak = a_m_fast ? (e / BM) : (e & 15);
+      As[ak][am] = (m0 + am < M && k0 + ak < Kd) ? A[(long)(m0 + am) * sa_m + (long)(k0 + ak) * sa_k] : 0.0;
+    }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int e = tid + i * 256;
-      const int am = a_m_fast ? (e & 63) : (e >> 4), ak = a_m_fast ? (e >> 6) : (e & 15);
-      As[ak][am] = (m0 + am < M && k0 + ak < Kd) ? A[(long)(m0 + am) * sa_m + (long)(k0 + ak) * sa_k] : 0.0;
       const int bn = b_n_fast ? (e & 63) : (e >> 4), bk = b_n_fast ? (e >> 6) : (e & 15);
       Bs[bk][bn] = (n0 + bn < N && k0 + bk < Kd) ? B[(long)(k0 + bk) * sb_k + (long)(n0 + bn) * sb_n] : 0.0;
     }
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < kBK; ++k) {
-      double a[4], b[4];
+      double a[TM], b[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = As[k][tm * 4 + i];
+      for (int i = 0; i < TM; ++i) a[i] = As[k][tm * TM + i];
 #pragma unroll
       for (int j = 0; j < 4; ++j) b[j] = Bs[k][tn * 4 + j];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int m = m0 + tm * 4 + i;
+  for (int i = 0; i < TM; ++i) {
+    const int m = m0 + tm * TM + i;
     if (m >= M) continue;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -129,27 +142,27 @@ __global__ void gptq_init_w_kernel(const float* __restrict__ R, const unsigned c
 
 // The 64 x 64 diagonal block at j0, whose trailing updates are already applied: column 63 down to column 0.
 // A pivot that is not positive raises *not_pd (the matrix was not positive definite).
-__global__ void __launch_bounds__(kNb) chol_diag_kernel(double* __restrict__ A, long ld, int j0, int* not_pd) {
+__global__ void __launch_bounds__(4 * kNb) chol_diag_kernel(double* __restrict__ A, long ld, int j0, int* not_pd) {
   __shared__ double S[kNb][kNb + 1];
-  const int t = threadIdx.x;
-  for (int r = 0; r < kNb; ++r) S[r][t] = A[(long)(j0 + r) * ld + j0 + t];
+  const int t = threadIdx.x & (kNb - 1), part = threadIdx.x >> 6;  // four threads share a row's update
+  for (int r = part; r < kNb; r += 4) S[r][t] = A[(long)(j0 + r) * ld + j0 + t];
   __syncthreads();
   for (int j = kNb - 1; j >= 0; --j) {
-    if (t == j) {
+    if (threadIdx.x == j) {
       const double d = S[j][j];
       if (!(d > 0.0)) *not_pd = 1;
       S[j][j] = sqrt(d);
     }
     __syncthreads();
-    if (t < j) S[t][j] /= S[j][j];
+    if (part == 0 && t < j) S[t][j] /= S[j][j];
     __syncthreads();
     if (t < j) {
       const double f = S[t][j];
-      for (int c = t; c < j; ++c) S[t][c] = fma(-f, S[c][j], S[t][c]);
+      for (int c = t + part; c < j; c += 4) S[t][c] = fma(-f, S[c][j], S[t][c]);
     }
     __syncthreads();
   }
-  for (int r = 0; r < kNb; ++r) A[(long)(j0 + r) * ld + j0 + t] = (t >= r) ? S[r][t] : 0.0;
+  for (int r = part; r < kNb; r += 4) A[(long)(j0 + r) * ld + j0 + t] = (t >= r) ? S[r][t] : 0.0;
 }
 
 // The panel above the diagonal block: each row x of A[0:j0, j0:j0+64] becomes the solution of x D^T = row, D the
@@ -179,11 +192,12 @@ __global__ void __launch_bounds__(kNb) chol_panel_kernel(double* __restrict__ A,
 // U = V^-1 (both upper triangular), block row by block row from the bottom.
 // ---------------------------------------------------------------------------------------------------------
 
-// Inverse of the diagonal block of V at i0 into the same place of U: thread c solves D x = e_c.
+// Inverse of every 64 x 64 diagonal block of V into the same place of U (one block of threads each): thread c
+// solves D x = e_c.
 __global__ void __launch_bounds__(kNb) triinv_diag_kernel(const double* __restrict__ V, double* __restrict__ U,
-                                                          long ld, int i0) {
+                                                          long ld) {
   __shared__ double D[kNb][kNb + 1];
-  const int t = threadIdx.x;
+  const int t = threadIdx.x, i0 = blockIdx.x * kNb;
   for (int r = 0; r < kNb; ++r) D[r][t] = V[(long)(i0 + r) * ld + i0 + t];
   __syncthreads();
   double b[kNb];
@@ -237,53 +251,90 @@ __global__ void __launch_bounds__(kNb) gptq_group_kernel(const double* __restric
   }
 }
 
-struct DeviceBuffers {
-  double *H = nullptr, *U = nullptr, *Xd = nullptr, *W = nullptr, *Err = nullptr, *T = nullptr, *mean = nullptr;
-  unsigned char* dead = nullptr;
-  int* not_pd = nullptr;
-  ~DeviceBuffers() {
-    cudaFree(H), cudaFree(U), cudaFree(Xd), cudaFree(W), cudaFree(Err), cudaFree(T), cudaFree(mean);
-    cudaFree(dead), cudaFree(not_pd);
+// The temporaries of one call, carved out of one workspace (256-byte aligned pieces).
+struct Workspace {
+  double *H, *U, *Xd, *W, *Err, *T, *mean;
+  unsigned char* dead;
+  int* not_pd;
+  size_t bytes;
+  Workspace(unsigned char* base, int K, int N, int M_cal) {
+    size_t off = 0;
+    auto take = [&](size_t n) {
+      unsigned char* p = reinterpret_cast<unsigned char*>(reinterpret_cast<uintptr_t>(base) + off);
+      off += (n + 255) & ~static_cast<size_t>(255);
+      return p;
+    };
+    const size_t kk = (size_t)K * K * sizeof(double);
+    H = reinterpret_cast<double*>(take(kk));
+    U = reinterpret_cast<double*>(take(kk));
+    W = reinterpret_cast<double*>(take((size_t)K * N * sizeof(double)));
+    Err = reinterpret_cast<double*>(take((size_t)kLazy * N * sizeof(double)));
+    T = reinterpret_cast<double*>(take((size_t)kBand * K * sizeof(double)));
+    Xd = reinterpret_cast<double*>(take((size_t)M_cal * K * sizeof(double)));
+    mean = reinterpret_cast<double*>(take(sizeof(double)));
+    dead = take((size_t)K);
+    not_pd = reinterpret_cast<int*>(take(sizeof(int)));
+    bytes = off;
   }
 };
 
+struct OwnedAllocation {
+  void* p = nullptr;
+  ~OwnedAllocation() { cudaFree(p); }
+};
+
 void dgemm(cudaStream_t st, int M, int N, int Kd, const double* A, long sa_m, long sa_k, const double* B, long sb_k,
-           long sb_n, double* C, long sc_m, long sc_n, double alpha, double beta, bool upper_only = false) {
+           long sb_n, double* C, long sc_m, long sc_n, double alpha, double beta, int flags = 0) {
   if (M <= 0 || N <= 0) return;
-  dim3 grid((N + kBN - 1) / kBN, (M + kBM - 1) / kBM);
-  dgemm_kernel<<<grid, 256, 0, st>>>(M, N, Kd, A, sa_m, sa_k, B, sb_k, sb_n, C, sc_m, sc_n, alpha, beta,
-                                     upper_only ? 1 : 0);
+  if (M > 64) {
+    dim3 grid((N + kBN - 1) / kBN, (M + 127) / 128);
+    dgemm_kernel<8><<<grid, 256, 0, st>>>(M, N, Kd, A, sa_m, sa_k, B, sb_k, sb_n, C, sc_m, sc_n, alpha, beta, flags);
+  } else {
+    dim3 grid((N + kBN - 1) / kBN, 1);
+    dgemm_kernel<4><<<grid, 256, 0, st>>>(M, N, Kd, A, sa_m, sa_k, B, sb_k, sb_n, C, sc_m, sc_n, alpha, beta, flags);
+  }
+}
+
+
+bool gptq_shape_ok(int K, int N, int M_cal) {
+  return K > 0 && N > 0 && K % kNb == 0 && K <= 16384 && N <= 65536 && M_cal >= 0 && M_cal <= (1 << 20);
 }
 
 }  // namespace
 
+extern "C" size_t w4a4_gptq_workspace_bytes(int K, int N, int M_cal) {
+  if (!gptq_shape_ok(K, N, M_cal)) return 0;
+  return Workspace(nullptr, K, N, M_cal).bytes;
+}
+
 extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal,
                                             const double* H_in, int K, int N, double percdamp, int8_t* codes,
-                                            float* scales, void* stream) {
+                                            float* scales, void* workspace, size_t workspace_bytes, void* stream) {
   if (R == nullptr || codes == nullptr || scales == nullptr) return W4A4_ERR_INVALID_ARG;
   if ((Xhat == nullptr) == (H_in == nullptr)) return W4A4_ERR_INVALID_ARG;  // exactly one source of H
-  if (K <= 0 || N <= 0 || K % kNb != 0 || K > 16384 || N > 65536) return W4A4_ERR_SHAPE;
+  if (Xhat == nullptr) M_cal = 0;
+  if (!gptq_shape_ok(K, N, M_cal)) return W4A4_ERR_SHAPE;
   if (Xhat != nullptr && M_cal <= 0) return W4A4_ERR_SHAPE;
   if (!(percdamp >= 0.0)) return W4A4_ERR_INVALID_ARG;
+  const size_t need = Workspace(nullptr, K, N, M_cal).bytes;
+  if (workspace != nullptr && (workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0))
+    return W4A4_ERR_INVALID_ARG;
   if (cudaSetDevice(device) != cudaSuccess) return W4A4_ERR_CUDA;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return W4A4_ERR_CUDA;
   if (prop.major != 10) return W4A4_ERR_ARCH;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-  DeviceBuffers d;
-  const size_t kk = (size_t)K * K * sizeof(double);
-  bool ok = cudaMalloc(&d.H, kk) == cudaSuccess && cudaMalloc(&d.U, kk) == cudaSuccess &&
-            cudaMalloc(&d.W, (size_t)K * N * sizeof(double)) == cudaSuccess &&
-            cudaMalloc(&d.Err, (size_t)kNb * N * sizeof(double)) == cudaSuccess &&
-            cudaMalloc(&d.T, (size_t)kNb * K * sizeof(double)) == cudaSuccess &&
-            cudaMalloc(&d.mean, sizeof(double)) == cudaSuccess && cudaMalloc(&d.dead, K) == cudaSuccess &&
-            cudaMalloc(&d.not_pd, sizeof(int)) == cudaSuccess;
-  if (ok && Xhat != nullptr) ok = cudaMalloc(&d.Xd, (size_t)M_cal * K * sizeof(double)) == cudaSuccess;
-  if (!ok) {
-    cudaGetLastError();
-    return W4A4_ERR_ALLOC;
+  OwnedAllocation own;
+  if (workspace == nullptr) {
+    if (cudaMalloc(&own.p, need) != cudaSuccess) {
+      cudaGetLastError();
+      return W4A4_ERR_ALLOC;
+    }
+    workspace = own.p;
   }
+  const Workspace d(static_cast<unsigned char*>(workspace), K, N, M_cal);
+  const size_t kk = (size_t)K * K * sizeof(double);
   cudaMemsetAsync(d.not_pd, 0, sizeof(int), st);
   cudaMemsetAsync(d.U, 0, kk, st);
 
@@ -292,7 +343,7 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
     const long n = (long)M_cal * K;
     bf16_to_f64_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(Xhat, d.Xd, n);
     cudaMemsetAsync(d.H, 0, kk, st);
-    dgemm(st, K, K, M_cal, d.Xd, 1, K, d.Xd, K, 1, d.H, K, 1, 1.0, 0.0, /*upper_only=*/true);
+    dgemm(st, K, K, M_cal, d.Xd, 1, K, d.Xd, K, 1, d.H, K, 1, 1.0, 0.0, kUpperOut);
   } else {
     cudaMemcpyAsync(d.H, H_in, kk, cudaMemcpyDeviceToDevice, st);
   }
@@ -303,28 +354,56 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
     gptq_init_w_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(R, d.dead, d.W, K, N);
   }
 
-  // 2a. H = V V^T in place, last block first.
-  for (int j0 = K - kNb; j0 >= 0; j0 -= kNb) {
-    chol_diag_kernel<<<1, kNb, 0, st>>>(d.H, K, j0, d.not_pd);
-    if (j0 == 0) break;
-    chol_panel_kernel<<<(j0 + kNb - 1) / kNb, kNb, 0, st>>>(d.H, K, j0);
-    // H[0:j0, 0:j0] -= P P^T, P = the panel just solved (upper triangle only).
-    dgemm(st, j0, j0, kNb, d.H + j0, K, 1, d.H + j0, 1, K, d.H, K, 1, -1.0, 1.0, /*upper_only=*/true);
+  // 2a. H = V V^T in place, last block first, in bands of kBand columns: inside a band every 64-column block is
+  // factored, solved against all rows above it and applied to the band's columns still to come; the columns to the
+  // left of the band take the whole band's panels in one product that is kBand deep.
+  for (int hi = K; hi > 0;) {
+    const int lo = hi - kBand > 0 ? hi - kBand : 0;
+    for (int j0 = hi - kNb; j0 >= lo; j0 -= kNb) {
+      chol_diag_kernel<<<1, 4 * kNb, 0, st>>>(d.H, K, j0, d.not_pd);
+      if (j0 == 0) break;
+      chol_panel_kernel<<<(j0 + kNb - 1) / kNb, kNb, 0, st>>>(d.H, K, j0);
+      // H[0:j0, lo:j0] -= P P[lo:j0]^T, P = the panel just solved
+      dgemm(st, j0, j0 - lo, kNb, d.H + j0, K, 1, d.H + (long)lo * K + j0, 1, K, d.H + lo, K, 1, -1.0, 1.0);
+    }
+    // H[0:lo, 0:lo] -= P P^T over the band's panels (upper triangle only)
+    dgemm(st, lo, lo, hi - lo, d.H + lo, K, 1, d.H + lo, 1, K, d.H, K, 1, -1.0, 1.0, kUpperOut);
+    hi = lo;
   }
-  // 2b. U = V^-1, last block row first: U[i, rest] = -inv(V_ii) (V[i, rest] U[rest, rest]).
-  for (int i0 = K - kNb; i0 >= 0; i0 -= kNb) {
-    triinv_diag_kernel<<<1, kNb, 0, st>>>(d.H, d.U, K, i0);
-    const int r0 = i0 + kNb, rest = K - r0;
-    if (rest == 0) continue;
-    dgemm(st, kNb, rest, rest, d.H + (long)i0 * K + r0, K, 1, d.U + (long)r0 * K + r0, K, 1, d.T, K, 1, 1.0, 0.0);
-    dgemm(st, kNb, rest, kNb, d.U + (long)i0 * K + i0, K, 1, d.T, K, 1, d.U + (long)i0 * K + r0, K, 1, -1.0, 0.0);
+  // 2b. U = V^-1 in two levels, last rows first.  Within a band of kBand rows the diagonal part is inverted block by
+  // block (U[i, rest] = -inv(V_ii) (V[i, rest] U[rest, rest]) with 64-row products); the band's part to the right of
+  // it then takes two products that are kBand rows high, so that they fill the machine.
+  triinv_diag_kernel<<<K / kNb, kNb, 0, st>>>(d.H, d.U, K);
+  for (int hi = K; hi > 0;) {
+    const int lo = hi - kBand > 0 ? hi - kBand : 0;
+    for (int i0 = hi - 2 * kNb; i0 >= lo; i0 -= kNb) {
+      const int r0 = i0 + kNb, rest = hi - r0;
+      dgemm(st, kNb, rest, rest, d.H + (long)i0 * K + r0, K, 1, d.U + (long)r0 * K + r0, K, 1, d.T, K, 1, 1.0, 0.0,
+            kBUpper);
+      dgemm(st, kNb, rest, kNb, d.U + (long)i0 * K + i0, K, 1, d.T, K, 1, d.U + (long)i0 * K + r0, K, 1, -1.0, 0.0);
+    }
+    const int band = hi - lo, right = K - hi;
+    if (right > 0) {
+      dgemm(st, band, right, right, d.H + (long)lo * K + hi, K, 1, d.U + (long)hi * K + hi, K, 1, d.T, K, 1, 1.0, 0.0,
+            kBUpper);
+      dgemm(st, band, right, band, d.U + (long)lo * K + lo, K, 1, d.T, K, 1, d.U + (long)lo * K + hi, K, 1, -1.0, 0.0,
+            kAUpper);
+    }
+    hi = lo;
   }
 
-  // 3. The sweep: group by group, then the groups still to come -= U[group, later]^T Err.
-  for (int k0 = 0; k0 < K; k0 += kNb) {
-    gptq_group_kernel<<<(N + kNb - 1) / kNb, kNb, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, d.Err);
-    const int r0 = k0 + kNb, rest = K - r0;
-    dgemm(st, rest, N, kNb, d.U + (long)k0 * K + r0, 1, K, d.Err, N, 1, d.W + (long)r0 * N, N, 1, -1.0, 1.0);
+  // 3. The sweep, group by group.  Inside a lazy batch of kLazy input channels each group's scaled errors update the
+  // batch's groups still to come; the channels after the batch take the whole batch in one product: W[later] -=
+  // U[batch, later]^T Err.
+  for (int b0 = 0; b0 < K; b0 += kLazy) {
+    const int b1 = b0 + kLazy < K ? b0 + kLazy : K;
+    for (int k0 = b0; k0 < b1; k0 += kNb) {
+      double* err = d.Err + (long)(k0 - b0) * N;
+      gptq_group_kernel<<<(N + kNb - 1) / kNb, kNb, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
+      const int r0 = k0 + kNb;
+      dgemm(st, b1 - r0, N, kNb, d.U + (long)k0 * K + r0, 1, K, err, N, 1, d.W + (long)r0 * N, N, 1, -1.0, 1.0);
+    }
+    dgemm(st, K - b1, N, b1 - b0, d.U + (long)b0 * K + b1, 1, K, d.Err, N, 1, d.W + (long)b1 * N, N, 1, -1.0, 1.0);
   }
 
   int not_pd = 0;

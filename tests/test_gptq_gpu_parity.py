@@ -24,13 +24,17 @@ def bits(t):
     return gen.bf16_bits(t.cpu()).numpy().view(np.uint16)
 
 
-def gpu_gptq(R, xhat=None, H=None, percdamp=0.01):
+def gpu_gptq(R, xhat=None, H=None, percdamp=0.01, own_workspace=False):
     import paper_2605_27003_b200 as w4
     K, N = R.shape
+    ws = None
+    if own_workspace:
+        ws = torch.empty(w4.w4a4_gptq_workspace_bytes(K, N, 0 if xhat is None else xhat.shape[0]), dtype=torch.uint8,
+                         device=DEV)
     codes = torch.full((K, N), 99, dtype=torch.int8, device=DEV)
     scales = torch.full((K // 64, N), -1.0, dtype=torch.float32, device=DEV)
     w4.w4a4_gptq_quantize(R.to(DEV), codes, scales, Xhat=None if xhat is None else xhat.to(DEV),
-                          H=None if H is None else torch.from_numpy(H).to(DEV), percdamp=percdamp)
+                          H=None if H is None else torch.from_numpy(H).to(DEV), percdamp=percdamp, workspace=ws)
     return codes.cpu().numpy(), scales.cpu().numpy()
 
 
@@ -82,6 +86,9 @@ def test_matches_oracle(K, N, M_cal, dead, percdamp):
     # and the statistic handed over directly gives the same result as the activations
     q2, s2 = gpu_gptq(R, H=H, percdamp=percdamp)
     compare(R64, H, q2, s2, q_ref, s_ref, max_bad_columns=max(1, N // 200))
+    # a caller-owned workspace changes nothing, bit for bit
+    q3, s3 = gpu_gptq(R, xhat=xhat, percdamp=percdamp, own_workspace=True)
+    assert np.array_equal(q3, q) and np.array_equal(s3, s)
 
 
 def test_full_size_layer_on_sampled_output_channels():
@@ -106,14 +113,19 @@ def test_argument_errors():
     H = torch.eye(64, dtype=torch.float64, device=DEV)
     x = torch.zeros(4, 64, dtype=torch.bfloat16, device=DEV)
     p = lambda t: ctypes.c_void_p(t.data_ptr())
-    call = lambda *a: lib.w4a4_gptq_quantize(*a)
-    assert call(0, p(R), None, 0, None, 64, 8, 0.01, p(codes), p(scales), None) == 1        # no statistic
-    assert call(0, p(R), p(x), 4, p(H), 64, 8, 0.01, p(codes), p(scales), None) == 1        # two statistics
-    assert call(0, None, None, 0, p(H), 64, 8, 0.01, p(codes), p(scales), None) == 1
-    assert call(0, p(R), None, 0, p(H), 96, 8, 0.01, p(codes), p(scales), None) == 2        # K not a multiple of 64
-    assert call(0, p(R), p(x), 0, None, 64, 8, 0.01, p(codes), p(scales), None) == 2        # no calibration tokens
-    assert call(0, p(R), None, 0, p(H), 64, 8, -1.0, p(codes), p(scales), None) == 1
+    call = lambda *a: lib.w4a4_gptq_quantize(*a, None, 0, None)
+    assert call(0, p(R), None, 0, None, 64, 8, 0.01, p(codes), p(scales)) == 1        # no statistic
+    assert call(0, p(R), p(x), 4, p(H), 64, 8, 0.01, p(codes), p(scales)) == 1        # two statistics
+    assert call(0, None, None, 0, p(H), 64, 8, 0.01, p(codes), p(scales)) == 1
+    assert call(0, p(R), None, 0, p(H), 96, 8, 0.01, p(codes), p(scales)) == 2        # K not a multiple of 64
+    assert call(0, p(R), p(x), 0, None, 64, 8, 0.01, p(codes), p(scales)) == 2        # no calibration tokens
+    assert call(0, p(R), None, 0, p(H), 64, 8, -1.0, p(codes), p(scales)) == 1
+    need = w4.w4a4_gptq_workspace_bytes(64, 8, 0)
+    assert need > 0 and w4.w4a4_gptq_workspace_bytes(96, 8, 0) == 0
+    small = torch.empty(need - 256, dtype=torch.uint8, device=DEV)
+    assert lib.w4a4_gptq_quantize(0, p(R), None, 0, p(H), 64, 8, 0.01, p(codes), p(scales), p(small), need - 256,
+                                  None) == 1                                              # workspace too small
     # not positive definite (and no damping): reported, not a fault
     Hbad = -torch.eye(64, dtype=torch.float64, device=DEV)
-    assert call(0, p(R), None, 0, p(Hbad), 64, 8, 0.0, p(codes), p(scales), None) == 1
+    assert call(0, p(R), None, 0, p(Hbad), 64, 8, 0.0, p(codes), p(scales)) == 1
     torch.cuda.synchronize()
