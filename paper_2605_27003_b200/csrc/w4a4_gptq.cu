@@ -30,7 +30,7 @@ constexpr int kLazy = 256;  // input channels per lazy batch of the sweep
 // ---------------------------------------------------------------------------------------------------------
 // C[m, n] = beta * C[m, n] + alpha * sum_k A(m, k) * B(k, n), every operand addressed by two strides so that a
 // transposed or sub-matrix operand costs nothing.  (16 TM) x 64 tile per block, 16-deep slices, TM x 4 outputs per
-// thread.  Structure flags: kUpperOut -- blocks whose tile lies entirely below the diagonal return at once (only the
+// thread (TM consecutive rows, four columns 16 apart).  Structure flags: kUpperOut -- blocks whose tile lies entirely below the diagonal return at once (only the
 // upper triangle of C is wanted); kAUpper -- A(m, k) = 0 for k < m, so the sum starts at the tile's first row;
 // kBUpper -- B(k, n) = 0 for k > n, so the sum ends at the tile's last column.
 // ---------------------------------------------------------------------------------------------------------
@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(256, 2) dgemm_kernel(int M, int N, int Kd, con
 #pragma unroll
       for (int i = 0; i < TM; ++i) a[i] = As[k][tm * TM + i];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) b[j] = Bs[k][tn * 4 + j];
+      for (int j = 0; j < 4; ++j) b[j] = Bs[k][tn + 16 * j];  // neighbouring threads, neighbouring words: no bank conflict
 #pragma unroll
       for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(256, 2) dgemm_kernel(int M, int N, int Kd, con
     if (m >= M) continue;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int n = n0 + tn * 4 + j;
+      const int n = n0 + tn + 16 * j;
       if (n >= N) continue;
       double* c = C + (long)m * sc_m + (long)n * sc_n;
       *c = (beta == 0.0) ? alpha * acc[i][j] : fma(alpha, acc[i][j], beta * *c);
