@@ -129,3 +129,35 @@ def test_argument_errors():
     Hbad = -torch.eye(64, dtype=torch.float64, device=DEV)
     assert call(0, p(R), None, 0, p(Hbad), 64, 8, 0.0, p(codes), p(scales)) == 1
     torch.cuda.synchronize()
+
+
+def test_gptq_codes_lower_the_layer_error_on_held_out_tokens():
+    # The point of the step (Sec. III-B): with the statistic of calibration tokens, the residual's quantization error
+    # as seen through fresh tokens of the same distribution is far below round-to-nearest's -- for the weights alone
+    # (FP64 check of the codes the GPU produced) and through the real W4A4 forward, where the 4-bit activations add
+    # the same noise to both.
+    import paper_2605_27003_b200 as w4
+    K, N, M_cal, M_eval = 512, 256, 1024, 512
+    R, x = gen.make_gptq_inputs(K, N, M_cal + M_eval, seed=11)
+    cal, ev = x[:M_cal].contiguous(), x[M_cal:].contiguous()
+    q, s = gpu_gptq(R, xhat=cal)
+    q0, s0 = gen._round_residual(R.double())
+    q0, s0 = q0.numpy(), s0.numpy()
+    deq = lambda c, sc: c.astype(np.float64) * np.repeat(sc.astype(np.float64), 64, axis=0)
+    Xe, R64 = ev.double().numpy(), R.double().numpy()
+    target = Xe @ R64
+    err_w = lambda c, sc: float(((Xe @ deq(c, sc) - target) ** 2).sum())
+    assert err_w(q, s) < 0.5 * err_w(q0, s0)
+
+    ctx = w4.Context(0, M_eval, K, 0)
+    clip = torch.ones((1, 1, 1), dtype=torch.float32, device=DEV)
+    errs = []
+    for codes, scales in ((q, s), (q0, s0)):
+        lay = gen.LayerInputs(K, N, 0, torch.ones(K), None, None, torch.from_numpy(codes), torch.from_numpy(scales), None)
+        L = w4.Layer(ctx, [lay.to(DEV)], num_bins=1)
+        Y = L.forward(ev.to(DEV), 0, 0, clip).double().cpu().numpy()
+        ctx.check()
+        L.close()
+        errs.append(float(((Y - target) ** 2).sum()))
+    ctx.close()
+    assert errs[0] < 0.9 * errs[1], errs
