@@ -29,13 +29,27 @@ constexpr int kLazy = 256;  // input channels per lazy batch of the sweep
 
 // ---------------------------------------------------------------------------------------------------------
 // C[m, n] = beta * C[m, n] + alpha * sum_k A(m, k) * B(k, n), every operand addressed by two strides so that a
-// transposed or sub-matrix operand costs nothing.  (16 TM) x 64 tile per block, 16-deep slices, TM x 4 outputs per
-// thread (TM consecutive rows, four columns 16 apart).  Structure flags: kUpperOut -- blocks whose tile lies entirely below the diagonal return at once (only the
+// transposed or sub-matrix operand costs nothing.  (16 TM) x 64 tile per block in 16-deep slices, double-buffered in
+// shared memory by asynchronous copies; eight warps, each a (4 TM) x 32 corner as 8 x 8 x 4 FP64 tensor-core steps.  Structure flags: kUpperOut -- blocks whose tile lies entirely below the diagonal return at once (only the
 // upper triangle of C is wanted); kAUpper -- A(m, k) = 0 for k < m, so the sum starts at the tile's first row;
 // kBUpper -- B(k, n) = 0 for k > n, so the sum ends at the tile's last column.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kBN = 64, kBK = 16;
 enum : int { kUpperOut = 1, kAUpper = 2, kBUpper = 4 };
+
+// 8-byte asynchronous copy global -> shared; with `valid` false nothing is read and zeros are written.
+__device__ __forceinline__ void async_copy8(double* smem_dst, const double* gmem_src, bool valid) {
+  const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+  const int src_bytes = valid ? 8 : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(gmem_src), "r"(src_bytes) : "memory");
+}
+
+// D (8 x 8) += A (8 x 4) B (4 x 8) on the FP64 tensor core; per lane one element of A and B, two of D.
+__device__ __forceinline__ void dmma_8x8x4(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d[0]), "+d"(d[1])
+               : "d"(a), "d"(b));
+}
 
 template <int TM>
 __global__ void __launch_bounds__(256, 2) dgemm_kernel(int M, int N, int Kd, const double* __restrict__ A, long sa_m,
@@ -43,55 +57,94 @@ __global__ void __launch_bounds__(256, 2) dgemm_kernel(int M, int N, int Kd, con
                                                     double* __restrict__ C, long sc_m, long sc_n, double alpha,
                                                     double beta, int flags) {
   constexpr int BM = 16 * TM;
-  __shared__ __align__(16) double As[kBK][BM];
-  __shared__ __align__(16) double Bs[kBK][kBN];
+  constexpr int MT = TM / 2;  // 8 x 8 tensor-core tiles per warp along M (four along N)
+  // Two slices of each operand: the next one arrives while this one is used.  Element (k, x) sits at column
+  // x ^ ((k & 3) << 2): a fragment load touches four k rows times four neighbouring columns per half warp, and the
+  // swap of 4-column groups by k spreads them over all banks.
+  __shared__ __align__(16) double As[2][kBK][BM];
+  __shared__ __align__(16) double Bs[2][kBK][kBN];
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * kBN;
   if ((flags & kUpperOut) && m0 >= n0 + kBN) return;
-  const int tid = threadIdx.x, tn = tid & 15, tm = tid >> 4;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = (warp & 3) * (8 * MT), wn = (warp >> 2) * 32;  // the warp's corner inside the block's tile
+  const int fr = lane >> 2, fk = lane & 3;                      // fragment row (or column) and k index of this lane
   const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
   const int k_begin = (flags & kAUpper) ? m0 : 0;  // m0 is a multiple of 16
   const int k_end = (flags & kBUpper) ? min(Kd, n0 + kBN) : Kd;
-  double acc[TM][4] = {};
-  for (int k0 = k_begin; k0 < k_end; k0 += kBK) {
+  // One slice of both operands, global -> shared without passing through registers; elements outside the
+  // operands are written as zeros (source size 0).
+  auto fetch_slice = [&](int buf, int k0) {
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
       const int e = tid + i * 256;
       const int am = a_m_fast ? (e % BM) : (e >> 4), ak = a_m_fast ? (e / BM) : (e & 15);
-      As[ak][am] = (m0 + am < M && k0 + ak < Kd) ? A[(long)(m0 + am) * sa_m + (long)(k0 + ak) * sa_k] : 0.0;
+      const bool in = (m0 + am < M && k0 + ak < Kd);
+      async_copy8(&As[buf][ak][am ^ ((ak & 3) << 2)], in ? A + (long)(m0 + am) * sa_m + (long)(k0 + ak) * sa_k : A, in);
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int e = tid + i * 256;
       const int bn = b_n_fast ? (e & 63) : (e >> 4), bk = b_n_fast ? (e >> 6) : (e & 15);
-      Bs[bk][bn] = (n0 + bn < N && k0 + bk < Kd) ? B[(long)(k0 + bk) * sb_k + (long)(n0 + bn) * sb_n] : 0.0;
+      const bool in = (n0 + bn < N && k0 + bk < Kd);
+      async_copy8(&Bs[buf][bk][bn ^ ((bk & 3) << 2)], in ? B + (long)(k0 + bk) * sb_k + (long)(n0 + bn) * sb_n : B, in);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  double acc[MT][4][2] = {};
+  if (k_begin < k_end) fetch_slice(0, k_begin);
+  int buf = 0;
+  for (int k0 = k_begin; k0 < k_end; k0 += kBK, buf ^= 1) {
+    if (k0 + kBK < k_end) {
+      fetch_slice(buf ^ 1, k0 + kBK);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
 #pragma unroll
-    for (int k = 0; k < kBK; ++k) {
-      double a[TM], b[4];
+    for (int k = 0; k < kBK; k += 4) {
+      // FP64 tensor-core step (8 x 8 x 4): this lane holds A[row fr][k fk] and B[k fk][column fr] of each tile
+      double a[MT], b[4];
 #pragma unroll
-      for (int i = 0; i < TM; ++i) a[i] = As[k][tm * TM + i];
+      for (int i = 0; i < MT; ++i) a[i] = As[buf][k + fk][(wm + 8 * i + fr) ^ (fk << 2)];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) b[j] = Bs[k][tn + 16 * j];  // neighbouring threads, neighbouring words: no bank conflict
+      for (int j = 0; j < 4; ++j) b[j] = Bs[buf][k + fk][(wn + 8 * j + fr) ^ (fk << 2)];
 #pragma unroll
-      for (int i = 0; i < TM; ++i)
+      for (int i = 0; i < MT; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+        for (int j = 0; j < 4; ++j) dmma_8x8x4(acc[i][j], a[i], b[j]);
     }
-    __syncthreads();
+    __syncthreads();  // everyone is done with this slice before the next fetch overwrites it
+  }
+  // Accumulator layout: rows fr, columns 2 fk and 2 fk + 1 of each 8 x 8 tile.  Two passes over the outputs, all
+  // loads of C before the first store: with run-time strides the compiler cannot tell that the addresses differ, and
+  // a load placed after a store would wait for it, one memory round trip each.
+  if (beta != 0.0) {
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          const int m = m0 + wm + 8 * i + fr, n = n0 + wn + 8 * j + 2 * fk + c;
+          const double v = (m < M && n < N) ? C[(long)m * sc_m + (long)n * sc_n] : 0.0;
+          acc[i][j][c] = fma(alpha, acc[i][j][c], beta * v);
+        }
+  } else {
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j][0] *= alpha, acc[i][j][1] *= alpha;
   }
 #pragma unroll
-  for (int i = 0; i < TM; ++i) {
-    const int m = m0 + tm * TM + i;
-    if (m >= M) continue;
+  for (int i = 0; i < MT; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int n = n0 + tn + 16 * j;
-      if (n >= N) continue;
-      double* c = C + (long)m * sc_m + (long)n * sc_n;
-      *c = (beta == 0.0) ? alpha * acc[i][j] : fma(alpha, acc[i][j], beta * *c);
-    }
-  }
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int m = m0 + wm + 8 * i + fr, n = n0 + wn + 8 * j + 2 * fk + c;
+        if (m < M && n < N) C[(long)m * sc_m + (long)n * sc_n] = acc[i][j][c];
+      }
 }
 
 __global__ void bf16_to_f64_kernel(const uint16_t* __restrict__ in, double* __restrict__ out, long n) {
