@@ -193,29 +193,35 @@ __global__ void gptq_init_w_kernel(const float* __restrict__ R, const unsigned c
 // H = V V^T, V upper triangular, from the last block to the first (A holds H's upper triangle and ends as V).
 // ---------------------------------------------------------------------------------------------------------
 
-// The 64 x 64 diagonal block at j0, whose trailing updates are already applied: column 63 down to column 0.
-// A pivot that is not positive raises *not_pd (the matrix was not positive definite).
-__global__ void __launch_bounds__(4 * kNb) chol_diag_kernel(double* __restrict__ A, long ld, int j0, int* not_pd) {
+// The 64 x 64 diagonal block at j0, whose trailing updates are already applied: column 63 down to column 0, one
+// barrier per column.  Four threads share a row.  At column j every thread forms 1 / sqrt(pivot) itself, scales
+// the entries of column j it needs on the fly (they stay unscaled in shared memory; the scaled column goes straight
+// to global memory, nobody reads it again here) and updates its part of the columns to the left, so reads (column j)
+// and writes (columns < j) of one step never meet.  A pivot that is not positive raises *not_pd.
+constexpr int kDiagParts = 4;  // threads per row: more of them only repeat the square root and the division
+constexpr int kDiagThreads = kDiagParts * kNb;
+__global__ void __launch_bounds__(kDiagThreads) chol_diag_kernel(double* __restrict__ A, long ld, int j0, int* not_pd) {
   __shared__ double S[kNb][kNb + 1];
-  const int t = threadIdx.x & (kNb - 1), part = threadIdx.x >> 6;  // four threads share a row's update
-  for (int r = part; r < kNb; r += 4) S[r][t] = A[(long)(j0 + r) * ld + j0 + t];
+  const int t = threadIdx.x & (kNb - 1), part = threadIdx.x >> 6;
+  for (int r = part; r < kNb; r += kDiagParts) S[r][t] = A[(long)(j0 + r) * ld + j0 + t];
   __syncthreads();
   for (int j = kNb - 1; j >= 0; --j) {
+    const double d = S[j][j];
+    const double root = sqrt(d), inv = 1.0 / root;
     if (threadIdx.x == j) {
-      const double d = S[j][j];
       if (!(d > 0.0)) *not_pd = 1;
-      S[j][j] = sqrt(d);
+      A[(long)(j0 + j) * ld + j0 + j] = root;
     }
-    __syncthreads();
-    if (part == 0 && t < j) S[t][j] /= S[j][j];
-    __syncthreads();
     if (t < j) {
-      const double f = S[t][j];
-      for (int c = t + part; c < j; c += 4) S[t][c] = fma(-f, S[c][j], S[t][c]);
+      const double f = S[t][j] * inv;
+      if (part == 0) A[(long)(j0 + t) * ld + j0 + j] = f;
+      for (int c = t + part; c < j; c += kDiagParts) S[t][c] = fma(-f, S[c][j] * inv, S[t][c]);
     }
     __syncthreads();
   }
-  for (int r = part; r < kNb; r += 4) A[(long)(j0 + r) * ld + j0 + t] = (t >= r) ? S[r][t] : 0.0;
+  // below the diagonal: zeros (the triangular inverse reads the whole block)
+  for (int r = part; r < kNb; r += kDiagParts)
+    if (t < r) A[(long)(j0 + r) * ld + j0 + t] = 0.0;
 }
 
 // The panel above the diagonal block: each row x of A[0:j0, j0:j0+64] becomes the solution of x D^T = row, D the
@@ -413,7 +419,7 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
   for (int hi = K; hi > 0;) {
     const int lo = hi - kBand > 0 ? hi - kBand : 0;
     for (int j0 = hi - kNb; j0 >= lo; j0 -= kNb) {
-      chol_diag_kernel<<<1, 4 * kNb, 0, st>>>(d.H, K, j0, d.not_pd);
+      chol_diag_kernel<<<1, kDiagThreads, 0, st>>>(d.H, K, j0, d.not_pd);
       if (j0 == 0) break;
       chol_panel_kernel<<<(j0 + kNb - 1) / kNb, kNb, 0, st>>>(d.H, K, j0);
       // H[0:j0, lo:j0] -= P P[lo:j0]^T, P = the panel just solved
