@@ -553,10 +553,10 @@ def gptq_launch_count(K: int, nb: int = 64, band: int = 512, lazy: int = 256) ->
             n += 1 + (1 if j0 > lo else 0)          # panel, in-band update
         n += 1 if lo > 0 else 0
         hi = lo
-    n += 1                                          # all diagonal inverses
     hi = K
     while hi > 0:                                   # U = V^-1
         lo = max(0, hi - band)
+        n += 1                                      # the band's diagonal inverses
         n += 2 * len(range(hi - 2 * nb, lo - 1, -nb))
         n += 2 if K - hi > 0 else 0
         hi = lo
@@ -564,7 +564,9 @@ def gptq_launch_count(K: int, nb: int = 64, band: int = 512, lazy: int = 256) ->
         b1 = min(K, b0 + lazy)
         for k0 in range(b0, b1, nb):
             n += 1 + (1 if b1 - k0 - nb > 0 else 0)
-        n += 1 if K - b1 > 0 else 0
+        if b1 < K:
+            b2 = min(K, b1 + lazy)
+            n += 1 + (1 if K - b2 > 0 else 0)       # next batch's rows, then the rest
     return n
 
 

@@ -14,7 +14,8 @@
 //      registers, takes the group scale, quantizes channel after channel and applies the in-group updates; the
 //      group's scaled errors then update all later channels by one more GEMM (the algorithm's lazy batch).
 //
-// Nothing here waits on another block: every dependency is a kernel boundary on one stream.
+// Nothing here waits on another block: every dependency is a kernel boundary, on the caller's stream or on an event
+// between it and one side stream of the call's own.
 #include "../../include/w4a4.h"
 
 #include <cuda_runtime.h>
@@ -251,12 +252,12 @@ __global__ void __launch_bounds__(kNb) chol_panel_kernel(double* __restrict__ A,
 // U = V^-1 (both upper triangular), block row by block row from the bottom.
 // ---------------------------------------------------------------------------------------------------------
 
-// Inverse of every 64 x 64 diagonal block of V into the same place of U (one block of threads each): thread c
-// solves D x = e_c.
+// Inverse of the 64 x 64 diagonal blocks of V from row `first` on (one block of threads each) into the same place of
+// U: thread c solves D x = e_c.
 __global__ void __launch_bounds__(kNb) triinv_diag_kernel(const double* __restrict__ V, double* __restrict__ U,
-                                                          long ld) {
+                                                          long ld, int first) {
   __shared__ double D[kNb][kNb + 1];
-  const int t = threadIdx.x, i0 = blockIdx.x * kNb;
+  const int t = threadIdx.x, i0 = first + blockIdx.x * kNb;
   for (int r = 0; r < kNb; ++r) D[r][t] = V[(long)(i0 + r) * ld + i0 + t];
   __syncthreads();
   double b[kNb];
@@ -327,13 +328,29 @@ struct Workspace {
     H = reinterpret_cast<double*>(take(kk));
     U = reinterpret_cast<double*>(take(kk));
     W = reinterpret_cast<double*>(take((size_t)K * N * sizeof(double)));
-    Err = reinterpret_cast<double*>(take((size_t)kLazy * N * sizeof(double)));
+    Err = reinterpret_cast<double*>(take((size_t)2 * kLazy * N * sizeof(double)));  // two error batches
     T = reinterpret_cast<double*>(take((size_t)kBand * K * sizeof(double)));
     Xd = reinterpret_cast<double*>(take((size_t)M_cal * K * sizeof(double)));
     mean = reinterpret_cast<double*>(take(sizeof(double)));
     dead = take((size_t)K);
     not_pd = reinterpret_cast<int*>(take(sizeof(int)));
     bytes = off;
+  }
+};
+
+// The second stream of a call and the two events that order it against the caller's stream.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t ev_main = nullptr, ev_side = nullptr;
+  bool create() {
+    return cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev_main, cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ev_side, cudaEventDisableTiming) == cudaSuccess;
+  }
+  ~SideStream() {
+    if (ev_main) cudaEventDestroy(ev_main);
+    if (ev_side) cudaEventDestroy(ev_side);
+    if (stream) cudaStreamDestroy(stream);
   }
 };
 
@@ -393,6 +410,11 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
     workspace = own.p;
   }
   const Workspace d(static_cast<unsigned char*>(workspace), K, N, M_cal);
+  SideStream side;
+  if (!side.create()) {
+    cudaGetLastError();
+    return W4A4_ERR_CUDA;
+  }
   const size_t kk = (size_t)K * K * sizeof(double);
   cudaMemsetAsync(d.not_pd, 0, sizeof(int), st);
   cudaMemsetAsync(d.U, 0, kk, st);
@@ -413,9 +435,16 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
     gptq_init_w_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(R, d.dead, d.W, K, N);
   }
 
-  // 2a. H = V V^T in place, last block first, in bands of kBand columns: inside a band every 64-column block is
-  // factored, solved against all rows above it and applied to the band's columns still to come; the columns to the
-  // left of the band take the whole band's panels in one product that is kBand deep.
+  // 2. H = V V^T in place (main stream) and U = V^-1 (side stream), band by band from the last channels.
+  // Factorization: inside a band of kBand columns every 64-column block is factored, solved against all rows above
+  // it and applied to the band's columns still to come; the columns to the left of the band then take the whole
+  // band's panels in one product that is kBand deep.  Rows lo..hi of V are final once the band's blocks are done (the
+  // product that follows only touches rows and columns below lo), so the side stream inverts that band meanwhile:
+  // the diagonal part block by block (U[i, rest] = -inv(V_ii) (V[i, rest] U[rest, rest]), 64-row products), the
+  // part to the right of it in two products that are kBand rows high.  The factorization's chain of small kernels
+  // and the inverse's large products overlap.
+  cudaEventRecord(side.ev_main, st);  // U is zeroed
+  cudaStreamWaitEvent(side.stream, side.ev_main, 0);
   for (int hi = K; hi > 0;) {
     const int lo = hi - kBand > 0 ? hi - kBand : 0;
     for (int j0 = hi - kNb; j0 >= lo; j0 -= kNb) {
@@ -425,49 +454,62 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
       // H[0:j0, lo:j0] -= P P[lo:j0]^T, P = the panel just solved
       dgemm(st, j0, j0 - lo, kNb, d.H + j0, K, 1, d.H + (long)lo * K + j0, 1, K, d.H + lo, K, 1, -1.0, 1.0);
     }
+    cudaEventRecord(side.ev_main, st);
     // H[0:lo, 0:lo] -= P P^T over the band's panels (upper triangle only)
     dgemm(st, lo, lo, hi - lo, d.H + lo, K, 1, d.H + lo, 1, K, d.H, K, 1, -1.0, 1.0, kUpperOut);
-    hi = lo;
-  }
-  // 2b. U = V^-1 in two levels, last rows first.  Within a band of kBand rows the diagonal part is inverted block by
-  // block (U[i, rest] = -inv(V_ii) (V[i, rest] U[rest, rest]) with 64-row products); the band's part to the right of
-  // it then takes two products that are kBand rows high, so that they fill the machine.
-  triinv_diag_kernel<<<K / kNb, kNb, 0, st>>>(d.H, d.U, K);
-  for (int hi = K; hi > 0;) {
-    const int lo = hi - kBand > 0 ? hi - kBand : 0;
+
+    cudaStream_t s2 = side.stream;
+    cudaStreamWaitEvent(s2, side.ev_main, 0);
+    triinv_diag_kernel<<<(hi - lo) / kNb, kNb, 0, s2>>>(d.H, d.U, K, lo);
     for (int i0 = hi - 2 * kNb; i0 >= lo; i0 -= kNb) {
       const int r0 = i0 + kNb, rest = hi - r0;
-      dgemm(st, kNb, rest, rest, d.H + (long)i0 * K + r0, K, 1, d.U + (long)r0 * K + r0, K, 1, d.T, K, 1, 1.0, 0.0,
+      dgemm(s2, kNb, rest, rest, d.H + (long)i0 * K + r0, K, 1, d.U + (long)r0 * K + r0, K, 1, d.T, K, 1, 1.0, 0.0,
             kBUpper);
-      dgemm(st, kNb, rest, kNb, d.U + (long)i0 * K + i0, K, 1, d.T, K, 1, d.U + (long)i0 * K + r0, K, 1, -1.0, 0.0);
+      dgemm(s2, kNb, rest, kNb, d.U + (long)i0 * K + i0, K, 1, d.T, K, 1, d.U + (long)i0 * K + r0, K, 1, -1.0, 0.0);
     }
     const int band = hi - lo, right = K - hi;
     if (right > 0) {
-      dgemm(st, band, right, right, d.H + (long)lo * K + hi, K, 1, d.U + (long)hi * K + hi, K, 1, d.T, K, 1, 1.0, 0.0,
+      dgemm(s2, band, right, right, d.H + (long)lo * K + hi, K, 1, d.U + (long)hi * K + hi, K, 1, d.T, K, 1, 1.0, 0.0,
             kBUpper);
-      dgemm(st, band, right, band, d.U + (long)lo * K + lo, K, 1, d.T, K, 1, d.U + (long)lo * K + hi, K, 1, -1.0, 0.0,
+      dgemm(s2, band, right, band, d.U + (long)lo * K + lo, K, 1, d.T, K, 1, d.U + (long)lo * K + hi, K, 1, -1.0, 0.0,
             kAUpper);
     }
     hi = lo;
   }
+  cudaEventRecord(side.ev_side, side.stream);
+  cudaStreamWaitEvent(st, side.ev_side, 0);  // U is complete
 
   // 3. The sweep, group by group.  Inside a lazy batch of kLazy input channels each group's scaled errors update the
-  // batch's groups still to come; the channels after the batch take the whole batch in one product: W[later] -=
-  // U[batch, later]^T Err.
-  for (int b0 = 0; b0 < K; b0 += kLazy) {
+  // batch's groups still to come.  The channels after the batch take the whole batch in one product, W[later] -=
+  // U[batch, later]^T Err, split in two: the next batch's channels on the main stream, the rest on the side stream
+  // while the next batch is swept.  Both touch the same rows as the next batch's own products, so each main-stream
+  // product first waits for the side stream's previous one; the error batches alternate between two buffers.
+  int batch = 0;
+  for (int b0 = 0; b0 < K; b0 += kLazy, ++batch) {
     const int b1 = b0 + kLazy < K ? b0 + kLazy : K;
+    double* err_batch = d.Err + (long)(batch & 1) * kLazy * N;
     for (int k0 = b0; k0 < b1; k0 += kNb) {
-      double* err = d.Err + (long)(k0 - b0) * N;
+      double* err = err_batch + (long)(k0 - b0) * N;
       gptq_group_kernel<<<(N + kNb - 1) / kNb, kNb, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
       const int r0 = k0 + kNb;
       dgemm(st, b1 - r0, N, kNb, d.U + (long)k0 * K + r0, 1, K, err, N, 1, d.W + (long)r0 * N, N, 1, -1.0, 1.0);
     }
-    dgemm(st, K - b1, N, b1 - b0, d.U + (long)b0 * K + b1, 1, K, d.Err, N, 1, d.W + (long)b1 * N, N, 1, -1.0, 1.0);
+    if (b1 == K) break;
+    const int b2 = b1 + kLazy < K ? b1 + kLazy : K;  // end of the next batch
+    cudaStreamWaitEvent(st, side.ev_side, 0);        // the side stream's product of the batch before
+    dgemm(st, b2 - b1, N, b1 - b0, d.U + (long)b0 * K + b1, 1, K, err_batch, N, 1, d.W + (long)b1 * N, N, 1, -1.0, 1.0);
+    cudaEventRecord(side.ev_main, st);
+    cudaStreamWaitEvent(side.stream, side.ev_main, 0);
+    dgemm(side.stream, K - b2, N, b1 - b0, d.U + (long)b0 * K + b2, 1, K, err_batch, N, 1, d.W + (long)b2 * N, N, 1,
+          -1.0, 1.0);
+    cudaEventRecord(side.ev_side, side.stream);
   }
+  cudaStreamWaitEvent(st, side.ev_side, 0);
 
   int not_pd = 0;
   if (cudaMemcpyAsync(&not_pd, d.not_pd, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess)
+      cudaStreamSynchronize(st) != cudaSuccess || cudaStreamSynchronize(side.stream) != cudaSuccess ||
+      cudaGetLastError() != cudaSuccess)
     return W4A4_ERR_CUDA;
   return not_pd ? W4A4_ERR_INVALID_ARG : W4A4_OK;
 }
