@@ -576,7 +576,8 @@ def run_gptq(args, w4, dev, local_rank, rank, peaks):
     time per layer, with the FP64 rate it amounts to."""
     if rank != 0:
         return
-    K, N, M_cal = 5120, 5120, 2048
+    K, N = {"gptq": (5120, 5120), "gptq_ffn_up": (5120, 13824), "gptq_ffn_down": (13824, 5120)}[args.workload]
+    M_cal = 2048
     R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
     Rd, xd = R.to(dev), xhat.to(dev)
     codes = torch.empty((K, N), dtype=torch.int8, device=dev)
@@ -605,16 +606,16 @@ def run_gptq(args, w4, dev, local_rank, rank, peaks):
     if not args.no_cpu_baseline:
         import oracle  # test infrastructure; allowed here for the CPU-baseline leg only
 
-        cols = list(range(0, N, N // 32))[:32]
+        cols = list(range(0, N, N // 32))[:32]   # (the statistic's inverse dominates: minutes at K = 13824)
         t0 = time.perf_counter()
         H = oracle.gptq_hessian(bits(xhat))
         oracle.gptq_quantize(R[:, cols].double().numpy(), H)
         cpu = dict(value=(time.perf_counter() - t0) * 1e3, unit="ms", cores=torch.get_num_threads(), kind="oracle",
-                   sample="the full statistic and its inverse, the sweep on 32 of the 5120 output channels")
+                   sample="the full statistic and its inverse, the sweep on 32 of the %d output channels" % N)
     print(json.dumps(dict(
         metric="gptq_layer_time", value=ms, unit="ms", n_gpus=1, steps=runs, warmup=2, ms_per_step=ms,
         higher_is_better=False, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-        config=dict(workload="gptq", K=K, N=N, calibration_tokens=M_cal, group=64, percdamp=0.01,
+        config=dict(workload=args.workload, K=K, N=N, calibration_tokens=M_cal, group=64, percdamp=0.01,
                     l2="working set of %.0f MB, larger than L2" % ((2 * K * K + K * N) * 8 / 1e6)),
         roofline=dict(bound="alu", achieved=flops / (ms * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
                       frac=flops / (ms * 1e-3) / 1e12 / peak, traffic=None,
@@ -628,7 +629,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search", "mxfp4_attn_proj", "mxfp4_ffn_up",
-                                                            "mxfp4_ffn_down", "mxfp4_ffn", "gptq"])
+                                                            "mxfp4_ffn_down", "mxfp4_ffn", "gptq", "gptq_ffn_up", "gptq_ffn_down"])
     ap.add_argument("--chunk-rows", type=int, default=4096, help="token rows per chunk of the host-buffer forward (e2e)")
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
@@ -678,7 +679,7 @@ def main():
     if args.workload == "clip_search":
         run_clip_search(args, w4, dev, local_rank, rank, peaks)
         return
-    if args.workload == "gptq":
+    if args.workload.startswith("gptq"):
         run_gptq(args, w4, dev, local_rank, rank, peaks)
         return
     n_buf = 4

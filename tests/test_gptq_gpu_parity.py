@@ -91,13 +91,14 @@ def test_matches_oracle(K, N, M_cal, dead, percdamp):
     assert np.array_equal(q3, q) and np.array_equal(s3, s)
 
 
-def test_full_size_layer_on_sampled_output_channels():
-    # The size the bench times (K = N = 5120, 2048 calibration tokens).  Output channels are independent, so the
-    # oracle runs on a sample of them with the full statistic.
-    K, N, M_cal = 5120, 5120, 2048
+@pytest.mark.parametrize("K,N,n_cols", [(5120, 5120, 40), (13824, 5120, 8)])
+def test_full_size_layer_on_sampled_output_channels(K, N, n_cols):
+    # The sizes the bench times (attention projection and FFN down-projection, 2048 calibration tokens).  Output
+    # channels are independent, so the oracle runs on a sample of them with the full statistic.
+    M_cal = 2048
     R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
     q, s = gpu_gptq(R, xhat=xhat)
-    cols = np.sort(np.random.default_rng(3).choice(N, 40, replace=False))
+    cols = np.sort(np.random.default_rng(3).choice(N, n_cols, replace=False))
     R64 = R[:, cols].double().numpy()
     H = oracle.gptq_hessian(bits(xhat))
     q_ref, s_ref = oracle.gptq_quantize(R64, H)
