@@ -112,3 +112,35 @@ def test_hessian_of_bf16_activations():
     H = oracle.gptq_hessian(gen.bf16_bits(x).numpy().view(np.uint16))
     xf = x.to(torch.float64).numpy()
     assert np.allclose(H, xf.T @ xf, rtol=1e-13) and np.allclose(H, H.T)
+
+
+def test_equals_the_defining_recursion_with_explicit_inverse_downdates():
+    # The algorithm's definition before its Cholesky reformulation (Frantar et al., 2023, Eq. 2-3 applied in a fixed
+    # order): quantize the first free channel, move the free channels by
+    #   delta = -(w_q - quant(w_q)) / [Hf^-1]_qq * (Hf^-1)[:, q],
+    # then remove q from the inverse by one step of Gaussian elimination,
+    #   Hf^-1 <- Hf^-1 - (Hf^-1)[:, q] (Hf^-1)[q, :] / [Hf^-1]_qq   (row and column q dropped).
+    # Written here with no Cholesky factor at all; the oracle must produce the same codes and scales.
+    rng = np.random.default_rng(5)
+    K, N, group = 128, 6, 64
+    X = rng.normal(size=(200, 8)) @ rng.normal(size=(8, K)) + 0.5 * rng.normal(size=(200, K))
+    H = X.T @ X
+    R = rng.normal(scale=0.02, size=(K, N))
+    Hd = H + 0.01 * np.mean(np.diag(H)) * np.eye(K)
+    Hinv = np.linalg.inv(Hd)
+    W = R.copy()
+    codes = np.zeros((K, N), np.int8)
+    scales = np.zeros((K // group, N), np.float32)
+    for k in range(K):
+        if k % group == 0:
+            scales[k // group] = (np.abs(W[k:k + group]).max(axis=0) / 7.0).astype(np.float32)
+        s = scales[k // group].astype(np.float64)
+        q = np.clip(np.rint(W[k] / s), -8, 7)
+        codes[k] = q.astype(np.int8)
+        err = W[k] - q * s
+        # free channels are k..K-1; Hinv holds their inverse with index 0 = channel k
+        W[k:] -= np.outer(Hinv[:, 0] / Hinv[0, 0], err)
+        Hinv = (Hinv - np.outer(Hinv[:, 0], Hinv[0, :]) / Hinv[0, 0])[1:, 1:]
+    q_o, s_o = oracle.gptq_quantize(R, H, group=group, percdamp=0.01)
+    assert np.array_equal(s_o, scales)
+    assert np.array_equal(q_o, codes)
