@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kDiagThreads) chol_diag_kernel(double* __restr
   __syncthreads();
   for (int j = kNb - 1; j >= 0; --j) {
     const double d = S[j][j];
-    const double root = sqrt(d), inv = 1.0 / root;
+    const double inv = rsqrt(d), root = d * inv;  // one short chain per column instead of a root and a division
     if (threadIdx.x == j) {
       if (!(d > 0.0)) *not_pd = 1;
       A[(long)(j0 + j) * ld + j0 + j] = root;
@@ -229,8 +229,10 @@ __global__ void __launch_bounds__(kDiagThreads) chol_diag_kernel(double* __restr
 // factored diagonal block.  One thread per row, the row in registers.
 __global__ void __launch_bounds__(kNb) chol_panel_kernel(double* __restrict__ A, long ld, int j0) {
   __shared__ double D[kNb][kNb + 1];
+  __shared__ double rD[kNb];  // reciprocal diagonal: a product per column instead of a division in the serial chain
   const int t = threadIdx.x;
   for (int r = 0; r < kNb; ++r) D[r][t] = A[(long)(j0 + r) * ld + j0 + t];
+  rD[t] = 1.0 / A[(long)(j0 + t) * ld + j0 + t];
   __syncthreads();
   const int row = blockIdx.x * kNb + t;
   if (row >= j0) return;
@@ -240,7 +242,7 @@ __global__ void __launch_bounds__(kNb) chol_panel_kernel(double* __restrict__ A,
   for (int c = 0; c < kNb; ++c) b[c] = p[c];
 #pragma unroll
   for (int c = kNb - 1; c >= 0; --c) {
-    b[c] = b[c] / D[c][c];
+    b[c] = b[c] * rD[c];
 #pragma unroll
     for (int c2 = 0; c2 < c; ++c2) b[c2] = fma(-b[c], D[c2][c], b[c2]);
   }
@@ -274,40 +276,57 @@ __global__ void __launch_bounds__(kNb) triinv_diag_kernel(const double* __restri
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// The sweep over one group of 64 input channels starting at k0 (Algorithm 1's inner loop): thread = output channel.
+// The sweep over one group of 64 input channels starting at k0 (Algorithm 1's inner loop).
 // scale = FP32(max |w| / 7) over the group as it stands on entry; per channel code = clamp(round-half-even(w /
 // scale), -8, 7) (0 for an all-zero group), err = (w - code * scale) / U_kk, later channels of the group -= err *
 // U_kj.  Err [64, N] keeps the scaled errors for the update of the groups still to come.
+// Two neighbouring lanes share an output channel: the even lane keeps the group's even input channels in registers,
+// the odd lane the odd ones.  At step k both get w_k from its owner by a shuffle and compute code and error alike
+// (same operations, same results), and each updates its own later channels: half the multiply-adds and half the
+// unrolled code per thread.
 // ---------------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kNb) gptq_group_kernel(const double* __restrict__ W, int N,
-                                                         const double* __restrict__ U, long ldu, int k0,
-                                                         int8_t* __restrict__ codes, float* __restrict__ scales,
-                                                         double* __restrict__ Err) {
+constexpr int kGroupCols = 32;  // output channels per block of 64 threads
+__global__ void __launch_bounds__(2 * kGroupCols) gptq_group_kernel(const double* __restrict__ W, int N,
+                                                                    const double* __restrict__ U, long ldu, int k0,
+                                                                    int8_t* __restrict__ codes,
+                                                                    float* __restrict__ scales,
+                                                                    double* __restrict__ Err) {
   __shared__ double D[kNb][kNb + 1];
+  __shared__ double rD[kNb];  // 1 / U_kk: the error is scaled by a product, which keeps one division out of the
+                              // chain from one input channel to the next (the code is still decided by w / s)
   const int t = threadIdx.x;
   for (int r = 0; r < kNb; ++r) D[r][t] = U[(long)(k0 + r) * ldu + k0 + t];
+  rD[t] = 1.0 / U[(long)(k0 + t) * ldu + k0 + t];
   __syncthreads();
-  const int n = blockIdx.x * kNb + t;
-  if (n >= N) return;
-  double w[kNb];
+  const int lane = t & 31, p = t & 1;
+  const int col = blockIdx.x * kGroupCols + (t >> 1);
+  const bool valid = col < N;           // both lanes of a pair agree; nobody leaves before the last shuffle
+  const int n = valid ? col : N - 1;
+  double w[kNb / 2];                    // input channels 2 i + p
   double amax = 0.0;
 #pragma unroll
-  for (int k = 0; k < kNb; ++k) {
-    w[k] = W[(long)(k0 + k) * N + n];
-    amax = fmax(amax, fabs(w[k]));
+  for (int i = 0; i < kNb / 2; ++i) {
+    w[i] = W[(long)(k0 + 2 * i + p) * N + n];
+    amax = fmax(amax, fabs(w[i]));
   }
+  amax = fmax(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
   const float s32 = (float)(amax / 7.0);  // FP64 quotient rounded once to FP32
-  scales[(long)(k0 / kNb) * N + n] = s32;
+  if (valid && p == 0) scales[(long)(k0 / kNb) * N + n] = s32;
   const double s = (double)s32;
 #pragma unroll
   for (int k = 0; k < kNb; ++k) {
+    const int i = k >> 1;
+    const double wk = __shfl_sync(0xffffffffu, w[i], (lane & ~1) | (k & 1));
     double q = 0.0;
-    if (s > 0.0) q = fmin(fmax(rint(w[k] / s), -8.0), 7.0);
-    codes[(long)(k0 + k) * N + n] = (int8_t)q;
-    const double e = (w[k] - q * s) / D[k][k];
-    Err[(long)k * N + n] = e;
+    if (s > 0.0) q = fmin(fmax(rint(wk / s), -8.0), 7.0);
+    const double e = (wk - q * s) * rD[k];
+    if (valid && p == (k & 1)) {
+      codes[(long)(k0 + k) * N + n] = (int8_t)q;
+      Err[(long)k * N + n] = e;
+    }
+    if ((k & 1) == 0 && p == 1) w[i] -= e * D[k][k + 1];  // channel k + 1 lives in the odd lane
 #pragma unroll
-    for (int j = k + 1; j < kNb; ++j) w[j] -= e * D[k][j];
+    for (int i2 = i + 1; i2 < kNb / 2; ++i2) w[i2] -= e * D[k][2 * i2 + p];
   }
 }
 
@@ -490,7 +509,7 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
     double* err_batch = d.Err + (long)(batch & 1) * kLazy * N;
     for (int k0 = b0; k0 < b1; k0 += kNb) {
       double* err = err_batch + (long)(k0 - b0) * N;
-      gptq_group_kernel<<<(N + kNb - 1) / kNb, kNb, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
+      gptq_group_kernel<<<(N + kGroupCols - 1) / kGroupCols, 2 * kGroupCols, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
       const int r0 = k0 + kNb;
       dgemm(st, b1 - r0, N, kNb, d.U + (long)k0 * K + r0, 1, K, err, N, 1, d.W + (long)r0 * N, N, 1, -1.0, 1.0);
     }
