@@ -327,3 +327,55 @@ def gptq_quantize(R, H, group=64, percdamp=0.01):
         err = (W[k] - q * s) / U[k, k]
         W[k + 1:] -= np.outer(U[k, k + 1:], err)
     return codes, scales
+
+
+def _mx_block_exponent(amax):
+    """Shared exponent of an MXFP4 block (OCP MX v1.0, Sec. 6.3): floor(log2(largest magnitude)) minus the largest
+    E2M1 exponent (2), kept within E8M0's range; an all-zero block gets the smallest exponent.  amax FP64 array."""
+    m, ex = np.frexp(amax)                                 # amax = m * 2^ex, 0.5 <= m < 1  ->  floor(log2) = ex - 1
+    e = np.where(amax > 0, ex - 1 - 2, -127)
+    return np.clip(e, -127, 125).astype(np.int64)
+
+
+def _e2m1_round_index(v):
+    """Nearest E2M1 magnitude index for v >= 0 (saturating at 6), ties to the even index: one comparison per
+    midpoint, strict where the lower neighbour is the even one."""
+    idx = np.zeros(v.shape, np.int64)
+    for i in range(7):
+        mid = 0.5 * (E2M1_VALUES[i] + E2M1_VALUES[i + 1])
+        idx += ((v > mid) | ((v == mid) & (i % 2 == 1))).astype(np.int64)
+    return idx
+
+
+def gptq_quantize_mx(R, H, percdamp=0.01):
+    """GPTQ (as gptq_quantize: Frantar et al., 2023, Algorithm 1 with the Cholesky reformulation) on the residual
+    branch with the MXFP4 grid of the MX variant instead of INT4: per 32 input channels and output channel one E8M0
+    exponent, taken from the error-compensated weights when the sweep enters the block (floor(log2 max|w|) - 2), and
+    E2M1 elements, nearest with ties to the even code, saturating at 6, sign bit from the compensated weight.  Dead
+    channels, damping and the order of the sweep as in gptq_quantize.
+    -> codes uint8 [K, N] (bit 3 sign, bits 0-2 magnitude index), exps uint8 [K / 32, N] (exponent + 127)."""
+    W = np.array(R, dtype=np.float64, copy=True)
+    H = np.array(H, dtype=np.float64, copy=True)
+    K, N = W.shape
+    assert H.shape == (K, K) and K % 32 == 0
+    dead = np.diag(H) == 0
+    H[dead, dead] = 1.0
+    W[dead, :] = 0.0
+    H[np.diag_indices(K)] += percdamp * np.mean(np.diag(H))
+    Hinv = np.linalg.inv(H)
+    U = np.linalg.cholesky((Hinv + Hinv.T) / 2).T          # upper, H^-1 = U^T U
+    codes = np.zeros((K, N), np.uint8)
+    exps = np.zeros((K // 32, N), np.uint8)
+    e = np.zeros(N, np.int64)
+    for k in range(K):
+        if k % 32 == 0:
+            e = _mx_block_exponent(np.abs(W[k:k + 32]).max(axis=0))
+            exps[k // 32] = (e + 127).astype(np.uint8)
+        scale = np.ldexp(1.0, e)
+        idx = _e2m1_round_index(np.minimum(np.abs(W[k]) / scale, 6.0))
+        codes[k] = (idx + 8 * (W[k] < 0)).astype(np.uint8)
+        deq = np.where(W[k] < 0, -1.0, 1.0) * E2M1_VALUES[idx] * scale
+        err = (W[k] - deq) / U[k, k]
+        W[k + 1:] -= np.outer(U[k, k + 1:], err)
+    return codes, exps
+

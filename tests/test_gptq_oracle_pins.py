@@ -144,3 +144,89 @@ def test_equals_the_defining_recursion_with_explicit_inverse_downdates():
     q_o, s_o = oracle.gptq_quantize(R, H, group=group, percdamp=0.01)
     assert np.array_equal(s_o, scales)
     assert np.array_equal(q_o, codes)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The same sweep on the MXFP4 grid (E2M1 elements, E8M0 exponent per 32 input channels)
+# ---------------------------------------------------------------------------------------------------------------
+E2M1 = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def nearest_e2m1_by_search(v):
+    # brute force over the eight magnitudes: smallest distance, and of two equally near ones the even index
+    d = np.abs(v[..., None] - E2M1)
+    best = d.min(axis=-1, keepdims=True)
+    cand = np.where(d == best, np.arange(8), 99)
+    lo = cand.min(axis=-1)
+    hi = np.where(d == best, np.arange(8), -1).max(axis=-1)
+    return np.where(lo == hi, lo, np.where(lo % 2 == 0, lo, hi))
+
+
+def test_mx_identity_hessian_reduces_to_the_plain_mxfp4_conversion():
+    rng = np.random.default_rng(6)
+    R = rng.normal(scale=0.02, size=(128, 20))
+    R[32:64, 3] = 0.0                                   # an all-zero block
+    R[5, 7] = 0.0                                       # a zero element inside a block
+    q0, e0 = gen._round_residual_mx(torch.from_numpy(R))
+    for c in (1.0, 9.0):
+        q, e = oracle.gptq_quantize_mx(R, c * np.eye(128))
+        assert np.array_equal(q, q0.numpy()) and np.array_equal(e, e0.numpy())
+
+
+def test_mx_hand_cases():
+    # One block of 32 channels, one output channel, all weights zero except the first three.
+    # w0 = 6.0 -> exponent floor(log2 6) - 2 = 0, scale 1, code 7 (value 6), no error.
+    # H couples channels 1 and 2 as in the INT4 hand case ([[2, -1], [-1, 2]] -> U12 / U11 = +0.5).
+    # w1 = 1.3 -> nearest 1.5 (index 3), error -0.2; w2 = 2.45 - (-0.2) * 0.5 = 2.55 -> nearest 3 (index 5), where
+    # plain rounding of 2.45 gives 2 (index 4).
+    K = 32
+    H = np.eye(K)
+    H[1:3, 1:3] = [[2.0, -1.0], [-1.0, 2.0]]
+    w = np.zeros((K, 1))
+    w[:3, 0] = [6.0, 1.3, 2.45]
+    q, e = oracle.gptq_quantize_mx(w, H, percdamp=0.0)
+    assert e[0, 0] == 127 and q[:3, 0].tolist() == [7, 3, 5]
+    q, e = oracle.gptq_quantize_mx(w, np.eye(K), percdamp=0.0)
+    assert q[:3, 0].tolist() == [7, 3, 4]
+    # negative weights carry bit 3; the exponent follows the block's largest magnitude: 0.2 -> floor(log2 0.2) - 2 = -5
+    w = np.zeros((K, 1))
+    w[:2, 0] = [-0.2, 0.05]
+    q, e = oracle.gptq_quantize_mx(w, np.eye(K), percdamp=0.0)
+    assert e[0, 0] == 127 - 5 and q[:2, 0].tolist() == [8 + 7, 3]     # 0.2 * 32 = 6.4 -> 6 (saturates); 0.05 * 32 = 1.6 -> 1.5
+
+
+def test_mx_equals_the_defining_recursion_with_explicit_inverse_downdates():
+    rng = np.random.default_rng(7)
+    K, N = 96, 5
+    X = rng.normal(size=(150, 6)) @ rng.normal(size=(6, K)) + 0.5 * rng.normal(size=(150, K))
+    H = X.T @ X
+    R = rng.normal(scale=0.02, size=(K, N))
+    Hinv = np.linalg.inv(H + 0.01 * np.mean(np.diag(H)) * np.eye(K))
+    W = R.copy()
+    codes = np.zeros((K, N), np.uint8)
+    exps = np.zeros((K // 32, N), np.uint8)
+    for k in range(K):
+        if k % 32 == 0:
+            ex = np.floor(np.log2(np.abs(W[k:k + 32]).max(axis=0))) - 2
+            exps[k // 32] = (ex + 127).astype(np.uint8)
+        scale = 2.0 ** ex
+        idx = nearest_e2m1_by_search(np.minimum(np.abs(W[k]) / scale, 6.0))
+        codes[k] = idx + 8 * (W[k] < 0)
+        err = W[k] - np.sign(W[k]) * E2M1[idx] * scale
+        W[k:] -= np.outer(Hinv[:, 0] / Hinv[0, 0], err)
+        Hinv = (Hinv - np.outer(Hinv[:, 0], Hinv[0, :]) / Hinv[0, 0])[1:, 1:]
+    q_o, e_o = oracle.gptq_quantize_mx(R, H, percdamp=0.01)
+    assert np.array_equal(e_o, exps) and np.array_equal(q_o, codes)
+
+
+def test_mx_objective_beats_the_plain_conversion():
+    rng = np.random.default_rng(8)
+    K, N = 256, 24
+    X = rng.normal(size=(400, 16)) @ rng.normal(size=(16, K)) + 0.3 * rng.normal(size=(400, K))
+    H = X.T @ X
+    R = rng.normal(scale=0.02, size=(K, N))
+    q, e = oracle.gptq_quantize_mx(R, H)
+    q0, e0 = gen._round_residual_mx(torch.from_numpy(R))
+    deq = lambda c, x: gen.mx_dequantize(torch.from_numpy(np.asarray(c)), torch.from_numpy(np.asarray(x))).numpy()
+    loss = lambda D: float(np.einsum("kn,kj,jn->", D, H, D))
+    assert loss(R - deq(q, e)) < 0.8 * loss(R - deq(q0.numpy(), e0.numpy()))
