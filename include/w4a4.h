@@ -275,6 +275,16 @@ w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xha
                                  int K, int N, double percdamp, int8_t* codes, float* scales, void* workspace,
                                  size_t workspace_bytes, void* stream);
 
+/* The same step on the MX variant's grid (Sec. III-B with the MXFP4 quantizer of w4a4_mx_pack_weights; OCP MX v1.0):
+ * codes device uint8 [K, N] (E2M1: bit 3 sign, bits 0-2 magnitude index of {0, 0.5, 1, 1.5, 2, 3, 4, 6}) and exps
+ * device uint8 [K/32, N] (E8M0: scale 2^(e - 127)).  A block's exponent is floor(log2 max|w|) - 2 over its 32
+ * error-compensated input channels when the sweep enters the block (an all-zero block: 0); elements are the nearest
+ * E2M1 value of w / 2^e, ties to the even code, saturating at 6, sign bit from the compensated weight.  Everything
+ * else (arguments, workspace, limits, errors) as w4a4_gptq_quantize. */
+w4a4_status_t w4a4_mx_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal, const double* H_in,
+                                    int K, int N, double percdamp, uint8_t* codes, uint8_t* exps, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
  * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
 w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);

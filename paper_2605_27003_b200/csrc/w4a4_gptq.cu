@@ -285,11 +285,15 @@ __global__ void __launch_bounds__(kNb) triinv_diag_kernel(const double* __restri
 // (same operations, same results), and each updates its own later channels: half the multiply-adds and half the
 // unrolled code per thread.
 // ---------------------------------------------------------------------------------------------------------
+// MX: the same sweep on the MXFP4 grid of the MX variant (OCP MX v1.0): one E8M0 exponent per 32 input channels,
+// floor(log2 max|w|) - 2 over the block as it stands when the sweep enters it, and E2M1 elements {0, 0.5, 1, 1.5, 2,
+// 3, 4, 6} * 2^e, nearest with ties to the even code, saturating at 6, sign bit from the compensated weight.
 constexpr int kGroupCols = 32;  // output channels per block of 64 threads
+template <bool MX>
 __global__ void __launch_bounds__(2 * kGroupCols) gptq_group_kernel(const double* __restrict__ W, int N,
                                                                     const double* __restrict__ U, long ldu, int k0,
-                                                                    int8_t* __restrict__ codes,
-                                                                    float* __restrict__ scales,
+                                                                    void* __restrict__ codes_out,
+                                                                    void* __restrict__ scales_out,
                                                                     double* __restrict__ Err) {
   __shared__ double D[kNb][kNb + 1];
   __shared__ double rD[kNb];  // 1 / U_kk: the error is scaled by a product, which keeps one division out of the
@@ -303,25 +307,54 @@ __global__ void __launch_bounds__(2 * kGroupCols) gptq_group_kernel(const double
   const bool valid = col < N;           // both lanes of a pair agree; nobody leaves before the last shuffle
   const int n = valid ? col : N - 1;
   double w[kNb / 2];                    // input channels 2 i + p
-  double amax = 0.0;
 #pragma unroll
-  for (int i = 0; i < kNb / 2; ++i) {
-    w[i] = W[(long)(k0 + 2 * i + p) * N + n];
-    amax = fmax(amax, fabs(w[i]));
+  for (int i = 0; i < kNb / 2; ++i) w[i] = W[(long)(k0 + 2 * i + p) * N + n];
+  double s = 0.0, inv_s = 0.0;          // INT4: the group's scale.  MX: 2^e of the running block and its reciprocal
+  if constexpr (!MX) {
+    double amax = 0.0;
+#pragma unroll
+    for (int i = 0; i < kNb / 2; ++i) amax = fmax(amax, fabs(w[i]));
+    amax = fmax(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    const float s32 = (float)(amax / 7.0);  // FP64 quotient rounded once to FP32
+    if (valid && p == 0) static_cast<float*>(scales_out)[(long)(k0 / kNb) * N + n] = s32;
+    s = (double)s32;
   }
-  amax = fmax(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-  const float s32 = (float)(amax / 7.0);  // FP64 quotient rounded once to FP32
-  if (valid && p == 0) scales[(long)(k0 / kNb) * N + n] = s32;
-  const double s = (double)s32;
 #pragma unroll
   for (int k = 0; k < kNb; ++k) {
     const int i = k >> 1;
+    if constexpr (MX) {
+      if ((k & 31) == 0) {  // entering a block of 32 input channels: its exponent from the weights as they stand
+        double amax = 0.0;
+#pragma unroll
+        for (int i2 = 0; i2 < 16; ++i2) amax = fmax(amax, fabs(w[i + i2]));
+        amax = fmax(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        int e = amax > 0.0 ? ilogb(amax) - 2 : -127;
+        e = max(-127, min(125, e));
+        s = scalbn(1.0, e);
+        inv_s = scalbn(1.0, -e);
+        if (valid && p == 0) static_cast<uint8_t*>(scales_out)[(long)((k0 + k) / 32) * N + n] = (uint8_t)(e + 127);
+      }
+    }
     const double wk = __shfl_sync(0xffffffffu, w[i], (lane & ~1) | (k & 1));
-    double q = 0.0;
-    if (s > 0.0) q = fmin(fmax(rint(wk / s), -8.0), 7.0);
-    const double e = (wk - q * s) * rD[k];
+    double deq;
+    int code;
+    if constexpr (MX) {
+      const double v = fmin(fabs(wk) * inv_s, 6.0);  // exact: the scale is a power of two
+      // one comparison per midpoint between neighbouring magnitudes, strict where the lower neighbour is the even code
+      const int idx = (v > 0.25) + (v >= 0.75) + (v > 1.25) + (v >= 1.75) + (v > 2.5) + (v >= 3.5) + (v > 5.0);
+      const double mag = idx < 4 ? 0.5 * idx : (idx < 6 ? idx - 2.0 : 2.0 * idx - 8.0);
+      deq = (wk < 0.0 ? -mag : mag) * s;
+      code = idx + (wk < 0.0 ? 8 : 0);
+    } else {
+      double q = 0.0;
+      if (s > 0.0) q = fmin(fmax(rint(wk / s), -8.0), 7.0);
+      deq = q * s;
+      code = (int)q;
+    }
+    const double e = (wk - deq) * rD[k];
     if (valid && p == (k & 1)) {
-      codes[(long)(k0 + k) * N + n] = (int8_t)q;
+      if constexpr (MX) static_cast<uint8_t*>(codes_out)[(long)(k0 + k) * N + n] = (uint8_t)code;
+      else static_cast<int8_t*>(codes_out)[(long)(k0 + k) * N + n] = (int8_t)code;
       Err[(long)k * N + n] = e;
     }
     if ((k & 1) == 0 && p == 1) w[i] -= e * D[k][k + 1];  // channel k + 1 lives in the odd lane
@@ -402,9 +435,11 @@ extern "C" size_t w4a4_gptq_workspace_bytes(int K, int N, int M_cal) {
   return Workspace(nullptr, K, N, M_cal).bytes;
 }
 
-extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal,
-                                            const double* H_in, int K, int N, double percdamp, int8_t* codes,
-                                            float* scales, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+
+w4a4_status_t gptq_run(bool mx, int device, const float* R, const uint16_t* Xhat, int M_cal, const double* H_in, int K,
+                       int N, double percdamp, void* codes, void* scales, void* workspace, size_t workspace_bytes,
+                       void* stream) {
   if (R == nullptr || codes == nullptr || scales == nullptr) return W4A4_ERR_INVALID_ARG;
   if ((Xhat == nullptr) == (H_in == nullptr)) return W4A4_ERR_INVALID_ARG;  // exactly one source of H
   if (Xhat == nullptr) M_cal = 0;
@@ -509,7 +544,9 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
     double* err_batch = d.Err + (long)(batch & 1) * kLazy * N;
     for (int k0 = b0; k0 < b1; k0 += kNb) {
       double* err = err_batch + (long)(k0 - b0) * N;
-      gptq_group_kernel<<<(N + kGroupCols - 1) / kGroupCols, 2 * kGroupCols, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
+      const dim3 grid((N + kGroupCols - 1) / kGroupCols);
+      if (mx) gptq_group_kernel<true><<<grid, 2 * kGroupCols, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
+      else gptq_group_kernel<false><<<grid, 2 * kGroupCols, 0, st>>>(d.W, N, d.U, K, k0, codes, scales, err);
       const int r0 = k0 + kNb;
       dgemm(st, b1 - r0, N, kNb, d.U + (long)k0 * K + r0, 1, K, err, N, 1, d.W + (long)r0 * N, N, 1, -1.0, 1.0);
     }
@@ -531,4 +568,18 @@ extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const ui
       cudaGetLastError() != cudaSuccess)
     return W4A4_ERR_CUDA;
   return not_pd ? W4A4_ERR_INVALID_ARG : W4A4_OK;
+}
+
+}  // namespace
+
+extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal,
+                                            const double* H_in, int K, int N, double percdamp, int8_t* codes,
+                                            float* scales, void* workspace, size_t workspace_bytes, void* stream) {
+  return gptq_run(false, device, R, Xhat, M_cal, H_in, K, N, percdamp, codes, scales, workspace, workspace_bytes, stream);
+}
+
+extern "C" w4a4_status_t w4a4_mx_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal,
+                                               const double* H_in, int K, int N, double percdamp, uint8_t* codes,
+                                               uint8_t* exps, void* workspace, size_t workspace_bytes, void* stream) {
+  return gptq_run(true, device, R, Xhat, M_cal, H_in, K, N, percdamp, codes, exps, workspace, workspace_bytes, stream);
 }

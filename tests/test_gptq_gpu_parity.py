@@ -162,3 +162,79 @@ def test_gptq_codes_lower_the_layer_error_on_held_out_tokens():
         errs.append(float(((Y - target) ** 2).sum()))
     ctx.close()
     assert errs[0] < 0.9 * errs[1], errs
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The same step on the MXFP4 grid (w4a4_mx_gptq_quantize)
+# ---------------------------------------------------------------------------------------------------------------
+def gpu_gptq_mx(R, xhat=None, H=None, percdamp=0.01):
+    import paper_2605_27003_b200 as w4
+    K, N = R.shape
+    codes = torch.full((K, N), 99, dtype=torch.uint8, device=DEV)
+    exps = torch.full((K // 32, N), 77, dtype=torch.uint8, device=DEV)
+    w4.w4a4_mx_gptq_quantize(R.to(DEV), codes, exps, Xhat=None if xhat is None else xhat.to(DEV),
+                             H=None if H is None else torch.from_numpy(H).to(DEV), percdamp=percdamp)
+    return codes.cpu().numpy(), exps.cpu().numpy()
+
+
+def mx_deq(c, e):
+    return gen.mx_dequantize(torch.from_numpy(c), torch.from_numpy(e)).numpy()
+
+
+def test_mx_identity_statistic_is_the_plain_conversion():
+    R, _ = gen.make_gptq_inputs(256, 150, 8, seed=2)
+    R[32:64, 5] = 0.0
+    R[7, 9] = 0.0
+    q0, e0 = gen._round_residual_mx(R.double())
+    q, e = gpu_gptq_mx(R, H=3.0 * np.eye(256))
+    assert np.array_equal(q, q0.numpy()) and np.array_equal(e, e0.numpy())
+
+
+@pytest.mark.parametrize("K,N,M_cal,dead,percdamp", [
+    (64, 33, 96, (), 0.01),
+    (512, 130, 384, (3, 200), 0.01),
+    (1024, 300, 1500, (1023,), 0.002),
+])
+def test_mx_matches_oracle(K, N, M_cal, dead, percdamp):
+    R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=K + N + 1, dead=dead)
+    R64 = R.double().numpy()
+    H = oracle.gptq_hessian(bits(xhat))
+    q_ref, e_ref = oracle.gptq_quantize_mx(R64, H, percdamp=percdamp)
+    q, e = gpu_gptq_mx(R, xhat=xhat, percdamp=percdamp)
+    bad = np.flatnonzero((q != q_ref).any(axis=0) | (e != e_ref).any(axis=0))
+    assert bad.size <= max(1, N // 200), f"{bad.size} output channels differ"
+    obj = lambda c, x, cols: np.einsum("kn,kj,jn->n", R64[:, cols] - mx_deq(c, x)[:, cols], H, R64[:, cols] - mx_deq(c, x)[:, cols])
+    if bad.size:
+        assert np.all(obj(q, e, bad) <= 1.05 * obj(q_ref, e_ref, bad))
+    q0, e0 = gen._round_residual_mx(R.double())
+    Rz = R64.copy()
+    Rz[list(dead), :] = 0.0
+    D, D0 = Rz - mx_deq(q, e), Rz - mx_deq(q0.numpy(), e0.numpy())
+    assert np.einsum("kn,kj,jn->", D, H, D) < 0.9 * np.einsum("kn,kj,jn->", D0, H, D0)
+    assert q.max() <= 15
+
+
+def test_mx_gptq_codes_lower_the_layer_error_on_held_out_tokens():
+    import paper_2605_27003_b200 as w4
+    K, N, M_cal, M_eval = 512, 256, 1024, 512
+    R, x = gen.make_gptq_inputs(K, N, M_cal + M_eval, seed=12)
+    cal, ev = x[:M_cal].contiguous(), x[M_cal:].contiguous()
+    q, e = gpu_gptq_mx(R, xhat=cal)
+    q0, e0 = gen._round_residual_mx(R.double())
+    q0, e0 = q0.numpy(), e0.numpy()
+    Xe, R64 = ev.double().numpy(), R.double().numpy()
+    target = Xe @ R64
+    err_w = lambda c, x_: float(((Xe @ mx_deq(c, x_) - target) ** 2).sum())
+    assert err_w(q, e) < 0.6 * err_w(q0, e0)
+    ctx = w4.Context(0, M_eval, K, 0)
+    clip = torch.ones((1, 1, 1), dtype=torch.float32, device=DEV)
+    errs = []
+    for codes, exps in ((q, e), (q0, e0)):
+        lay = gen.MxLayerInputs(K, N, 0, torch.ones(K), None, None, torch.from_numpy(codes), torch.from_numpy(exps), None)
+        L = w4.MxLayer(ctx, [lay.to(DEV)], num_bins=1)
+        Y = L.forward(ev.to(DEV), 0, 0, clip).double().cpu().numpy()
+        ctx.check()
+        L.close()
+        errs.append(float(((Y - target) ** 2).sum()))
+    ctx.close()
+    assert errs[0] < 0.95 * errs[1], errs
