@@ -322,7 +322,7 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                 ctx.close()
                 del Y
                 torch.cuda.empty_cache()
-    out = args.out or os.path.join(ROOT, "gpurun_out", "sweep.json")
+    out = args.out or os.path.join(ROOT, "bench_out", "sweep.json")
     os.makedirs(os.path.dirname(out), exist_ok=True)
     with open(out, "w") as f:
         json.dump(rows, f)
