@@ -179,6 +179,13 @@ def run_reference(args, rank):
     """--impl reference: the CPU oracle timed on host cores; each step is a bounded row sample."""
     if rank != 0:
         return
+    if args.workload.startswith("gptq"):
+        run_reference_gptq(args)
+        return
+    if args.workload not in gen.CONFIG_SHAPES:
+        print(json.dumps(dict(impl="reference", unavailable="the reference arm (the CPU oracle) covers the single-layer "
+                              "workloads and gptq*; %s has no oracle-timed counterpart" % args.workload)), flush=True)
+        return
     w = workload_inputs(args.workload, "cpu" if not torch.cuda.is_available() else "cuda:0", 1)
     t_probe, n_probe = oracle_time_rows(w, 2)
     budget = 90.0 / max(1, args.steps + args.warmup)
@@ -197,6 +204,34 @@ def run_reference(args, rank):
                                   sample=f"{n} sampled token rows per step, all output columns"),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line), flush=True)
+
+
+def run_reference_gptq(args):
+    """--impl reference for the gptq workloads: the FP64 oracle on host cores.  A step is the full statistic, its
+    inverse and Cholesky factor, and the sweep on a sample of 32 output channels (the sweep over all of them would take
+    minutes; the part that does not depend on the output channels is done in full)."""
+    import oracle  # test infrastructure; allowed here for the reference leg only
+
+    K, N = {"gptq": (5120, 5120), "gptq_ffn_up": (5120, 13824), "gptq_ffn_down": (13824, 5120)}[args.workload]
+    M_cal = 2048
+    R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
+    cols = list(range(0, N, N // 32))[:32]
+    Rs, xb = R[:, cols].double().numpy(), bits(xhat)
+    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.gptq_quantize(Rs, oracle.gptq_hessian(xb))
+        if i >= warmup:
+            times.append((time.perf_counter() - t0) * 1e3)
+    ms = statistics.median(times)
+    sample = "the full statistic and its inverse, the sweep on 32 of the %d output channels" % N
+    print(json.dumps(dict(
+        metric="gptq_layer_time", value=ms, unit="ms", n_gpus=args.gpus, steps=steps, warmup=warmup, ms_per_step=ms,
+        higher_is_better=False, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
+        config=dict(workload=args.workload, K=K, N=N, calibration_tokens=M_cal, group=64, percdamp=0.01),
+        cpu_baseline=dict(value=ms, unit="ms", cores=torch.get_num_threads(), kind="oracle", sample=sample),
+        e2e=dict(value=ms, unit="ms", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)), flush=True)
 
 
 def time_layer(w4, layer, xs, bins, expert, clip, Y, M, iters, warmup, stream):
