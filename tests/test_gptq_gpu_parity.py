@@ -238,3 +238,14 @@ def test_mx_gptq_codes_lower_the_layer_error_on_held_out_tokens():
         errs.append(float(((Y - target) ** 2).sum()))
     ctx.close()
     assert errs[0] < 0.95 * errs[1], errs
+
+
+def test_mx_full_size_layer_on_sampled_output_channels():
+    K, N, M_cal = 5120, 5120, 2048
+    R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=8)
+    q, e = gpu_gptq_mx(R, xhat=xhat)
+    cols = np.sort(np.random.default_rng(4).choice(N, 24, replace=False))
+    H = oracle.gptq_hessian(bits(xhat))
+    q_ref, e_ref = oracle.gptq_quantize_mx(R[:, cols].double().numpy(), H)
+    bad = np.flatnonzero((q[:, cols] != q_ref).any(axis=0) | (e[:, cols] != e_ref).any(axis=0))
+    assert bad.size <= 1, f"{bad.size} of the sampled output channels differ"
