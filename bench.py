@@ -212,8 +212,10 @@ def run_reference_gptq(args):
     minutes; the part that does not depend on the output channels is done in full)."""
     import oracle  # test infrastructure; allowed here for the reference leg only
 
-    K, N = {"gptq": (5120, 5120), "gptq_ffn_up": (5120, 13824), "gptq_ffn_down": (13824, 5120)}[args.workload]
+    K, N = {"gptq": (5120, 5120), "gptq_mx": (5120, 5120), "gptq_ffn_up": (5120, 13824),
+            "gptq_ffn_down": (13824, 5120)}[args.workload]
     M_cal = 2048
+    sweep = oracle.gptq_quantize_mx if args.workload == "gptq_mx" else oracle.gptq_quantize
     R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
     cols = list(range(0, N, N // 32))[:32]
     Rs, xb = R[:, cols].double().numpy(), bits(xhat)
@@ -221,7 +223,7 @@ def run_reference_gptq(args):
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        oracle.gptq_quantize(Rs, oracle.gptq_hessian(xb))
+        sweep(Rs, oracle.gptq_hessian(xb))
         if i >= warmup:
             times.append((time.perf_counter() - t0) * 1e3)
     ms = statistics.median(times)
@@ -611,16 +613,20 @@ def run_gptq(args, w4, dev, local_rank, rank, peaks):
     time per layer, with the FP64 rate it amounts to."""
     if rank != 0:
         return
-    K, N = {"gptq": (5120, 5120), "gptq_ffn_up": (5120, 13824), "gptq_ffn_down": (13824, 5120)}[args.workload]
+    K, N = {"gptq": (5120, 5120), "gptq_mx": (5120, 5120), "gptq_ffn_up": (5120, 13824),
+            "gptq_ffn_down": (13824, 5120)}[args.workload]
     M_cal = 2048
+    mx = args.workload == "gptq_mx"                 # the MX variant's grid: E2M1 codes, E8M0 exponents per 32 channels
+    quantize = w4.w4a4_mx_gptq_quantize if mx else w4.w4a4_gptq_quantize
     R, xhat = gen.make_gptq_inputs(K, N, M_cal, seed=7)
     Rd, xd = R.to(dev), xhat.to(dev)
-    codes = torch.empty((K, N), dtype=torch.int8, device=dev)
-    scales = torch.empty((K // 64, N), dtype=torch.float32, device=dev)
+    codes = torch.empty((K, N), dtype=torch.uint8 if mx else torch.int8, device=dev)
+    scales = (torch.empty((K // 32, N), dtype=torch.uint8, device=dev) if mx
+              else torch.empty((K // 64, N), dtype=torch.float32, device=dev))
     ws = torch.empty(w4.w4a4_gptq_workspace_bytes(K, N, M_cal), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
     for _ in range(2):
-        w4.w4a4_gptq_quantize(Rd, codes, scales, Xhat=xd, workspace=ws)
+        quantize(Rd, codes, scales, Xhat=xd, workspace=ws)
     runs = max(1, min(args.steps, 9))
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -629,7 +635,7 @@ def run_gptq(args, w4, dev, local_rank, rank, peaks):
     for _ in range(runs):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        w4.w4a4_gptq_quantize(Rd, codes, scales, Xhat=xd, workspace=ws)
+        quantize(Rd, codes, scales, Xhat=xd, workspace=ws)
         e1.record(stream)
         torch.cuda.synchronize()
         per_call.append(e0.elapsed_time(e1))
@@ -648,7 +654,7 @@ def run_gptq(args, w4, dev, local_rank, rank, peaks):
         cols = list(range(0, N, N // 32))[:32]   # (the statistic's inverse dominates: minutes at K = 13824)
         t0 = time.perf_counter()
         H = oracle.gptq_hessian(bits(xhat))
-        oracle.gptq_quantize(R[:, cols].double().numpy(), H)
+        (oracle.gptq_quantize_mx if mx else oracle.gptq_quantize)(R[:, cols].double().numpy(), H)
         cpu = dict(value=(time.perf_counter() - t0) * 1e3, unit="ms", cores=torch.get_num_threads(), kind="oracle",
                    sample="the full statistic and its inverse, the sweep on 32 of the %d output channels" % N)
     print(json.dumps(dict(
@@ -669,7 +675,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="attn_proj", choices=sorted(gen.CONFIG_SHAPES) + ["dit_step", "sweep", "clip_search", "mxfp4_attn_proj", "mxfp4_ffn_up",
-                                                            "mxfp4_ffn_down", "mxfp4_ffn", "gptq", "gptq_ffn_up", "gptq_ffn_down"])
+                                                            "mxfp4_ffn_down", "mxfp4_ffn", "gptq", "gptq_mx", "gptq_ffn_up", "gptq_ffn_down"])
     ap.add_argument("--chunk-rows", type=int, default=4096, help="token rows per chunk of the host-buffer forward (e2e)")
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
