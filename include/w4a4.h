@@ -275,6 +275,14 @@ w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xha
                                  int K, int N, double percdamp, int8_t* codes, float* scales, void* workspace,
                                  size_t workspace_bytes, void* stream);
 
+/* The statistic of GPTQ over several batches of calibration tokens (Sec. III-B; Frantar et al., 2023, Sec. 3: the
+ * layer-wise Hessian is a sum over calibration inputs): H += Xhat^T Xhat in FP64.  Xhat device BF16 bit patterns
+ * [M_cal, K]; H device FP64 [K, K] row-major, zeroed by the caller before the first batch.  Only the tiles on and above
+ * the diagonal are updated (64 x 128 granularity), which is the part w4a4_gptq_quantize reads from H_in.  K a multiple
+ * of 64, K <= 16384, 0 < M_cal <= 2^20 (W4A4_ERR_SHAPE).  Allocates and frees 8 * min(M_cal, 4096) * K bytes
+ * (W4A4_ERR_ALLOC); runs on `stream` and returns after it has drained. */
+w4a4_status_t w4a4_gptq_accumulate(int device, const uint16_t* Xhat, int M_cal, int K, double* H, void* stream);
+
 /* The same step on the MX variant's grid (Sec. III-B with the MXFP4 quantizer of w4a4_mx_pack_weights; OCP MX v1.0):
  * codes device uint8 [K, N] (E2M1: bit 3 sign, bits 0-2 magnitude index of {0, 0.5, 1, 1.5, 2, 3, 4, 6}) and exps
  * device uint8 [K/32, N] (E8M0: scale 2^(e - 127)).  A block's exponent is floor(log2 max|w|) - 2 over its 32

@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search",
     "w4a4_mx_pack_weights", "w4a4_mx_destroy", "w4a4_mx_handle_bytes", "w4a4_mx_linear_forward",
     "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_mx_clip_search",
-    "w4a4_mx_ffn_forward", "w4a4_mx_debug_fused_input", "w4a4_gptq_quantize", "w4a4_mx_gptq_quantize", "w4a4_gptq_workspace_bytes", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
+    "w4a4_mx_ffn_forward", "w4a4_mx_debug_fused_input", "w4a4_gptq_quantize", "w4a4_mx_gptq_quantize", "w4a4_gptq_accumulate", "w4a4_gptq_workspace_bytes", "w4a4_query_status", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
 
@@ -103,6 +103,7 @@ def _lib():
         lib.w4a4_mx_clip_search.argtypes = lib.w4a4_clip_search.argtypes
         lib.w4a4_gptq_quantize.argtypes = [ci, vp, vp, ci, vp, ci, ci, ctypes.c_double, vp, vp, vp, ctypes.c_size_t, vp]
         lib.w4a4_mx_gptq_quantize.argtypes = lib.w4a4_gptq_quantize.argtypes
+        lib.w4a4_gptq_accumulate.argtypes = [ci, vp, ci, ci, vp, vp]
         lib.w4a4_gptq_workspace_bytes.argtypes = [ci, ci, ci]
         lib.w4a4_gptq_workspace_bytes.restype = ctypes.c_size_t
         lib.w4a4_tile_shape.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci)]
@@ -352,6 +353,13 @@ def w4a4_gptq_quantize(R, codes, scales, Xhat=None, H=None, percdamp=0.01, works
     _check(_lib().w4a4_gptq_quantize(R.device.index or 0, _ptr(R), _ptr(Xhat), M_cal, _ptr(H), K, N, float(percdamp),
                                      _ptr(codes), _ptr(scales), _ptr(workspace), ws_bytes, _stream(stream)),
            "w4a4_gptq_quantize")
+
+
+def w4a4_gptq_accumulate(Xhat, H, stream=None):
+    """H (device FP64 [K, K], upper triangle) += Xhat^T Xhat for one batch of calibration tokens (device BF16 [M, K])."""
+    M_cal, K = Xhat.shape
+    _check(_lib().w4a4_gptq_accumulate(Xhat.device.index or 0, _ptr(Xhat), M_cal, K, _ptr(H), _stream(stream)),
+           "w4a4_gptq_accumulate")
 
 
 def w4a4_mx_gptq_quantize(R, codes, exps, Xhat=None, H=None, percdamp=0.01, workspace=None, stream=None):

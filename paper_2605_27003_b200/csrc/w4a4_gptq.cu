@@ -572,6 +572,33 @@ w4a4_status_t gptq_run(bool mx, int device, const float* R, const uint16_t* Xhat
 
 }  // namespace
 
+extern "C" w4a4_status_t w4a4_gptq_accumulate(int device, const uint16_t* Xhat, int M_cal, int K, double* H,
+                                              void* stream) {
+  if (Xhat == nullptr || H == nullptr) return W4A4_ERR_INVALID_ARG;
+  if (!gptq_shape_ok(K, 1, M_cal) || M_cal <= 0) return W4A4_ERR_SHAPE;
+  if (cudaSetDevice(device) != cudaSuccess) return W4A4_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return W4A4_ERR_CUDA;
+  if (prop.major != 10) return W4A4_ERR_ARCH;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  constexpr int kChunkRows = 4096;  // tokens converted to FP64 at a time
+  const int chunk = M_cal < kChunkRows ? M_cal : kChunkRows;
+  OwnedAllocation xd;
+  if (cudaMalloc(&xd.p, (size_t)chunk * K * sizeof(double)) != cudaSuccess) {
+    cudaGetLastError();
+    return W4A4_ERR_ALLOC;
+  }
+  double* Xd = static_cast<double*>(xd.p);
+  for (int m0 = 0; m0 < M_cal; m0 += chunk) {
+    const int rows = M_cal - m0 < chunk ? M_cal - m0 : chunk;
+    const long n = (long)rows * K;
+    bf16_to_f64_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(Xhat + (size_t)m0 * K, Xd, n);
+    dgemm(st, K, K, rows, Xd, 1, K, Xd, K, 1, H, K, 1, 1.0, 1.0, kUpperOut);
+  }
+  if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) return W4A4_ERR_CUDA;
+  return W4A4_OK;
+}
+
 extern "C" w4a4_status_t w4a4_gptq_quantize(int device, const float* R, const uint16_t* Xhat, int M_cal,
                                             const double* H_in, int K, int N, double percdamp, int8_t* codes,
                                             float* scales, void* workspace, size_t workspace_bytes, void* stream) {

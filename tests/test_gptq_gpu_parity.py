@@ -249,3 +249,29 @@ def test_mx_full_size_layer_on_sampled_output_channels():
     q_ref, e_ref = oracle.gptq_quantize_mx(R[:, cols].double().numpy(), H)
     bad = np.flatnonzero((q[:, cols] != q_ref).any(axis=0) | (e[:, cols] != e_ref).any(axis=0))
     assert bad.size <= 1, f"{bad.size} of the sampled output channels differ"
+
+
+def test_statistic_accumulated_over_batches():
+    # Calibration tokens arrive in batches: H += Xhat^T Xhat per batch, then the sweep on the accumulated statistic.
+    import paper_2605_27003_b200 as w4
+    K, N = 320, 150
+    sizes = (100, 4096 + 37, 300)                  # the middle batch is longer than the library's conversion chunk
+    R, x = gen.make_gptq_inputs(K, N, sum(sizes), seed=21)
+    H = torch.zeros((K, K), dtype=torch.float64, device=DEV)
+    m0 = 0
+    for m in sizes:
+        w4.w4a4_gptq_accumulate(x[m0:m0 + m].contiguous().to(DEV), H)
+        m0 += m
+    H_ref = oracle.gptq_hessian(bits(x))
+    Hg = H.cpu().numpy()
+    iu = np.triu_indices(K)
+    assert np.allclose(Hg[iu], H_ref[iu], rtol=1e-12, atol=1e-9 * np.abs(H_ref).max())
+    # the sweep reads only the upper triangle: garbage below the diagonal must not matter
+    Hd = H.clone()
+    Hd[np.tril_indices(K, -1)] = float("nan")
+    codes = torch.empty((K, N), dtype=torch.int8, device=DEV)
+    scales = torch.empty((K // 64, N), dtype=torch.float32, device=DEV)
+    w4.w4a4_gptq_quantize(R.to(DEV), codes, scales, H=Hd)
+    R64 = R.double().numpy()
+    q_ref, s_ref = oracle.gptq_quantize(R64, H_ref)
+    compare(R64, H_ref, codes.cpu().numpy(), scales.cpu().numpy(), q_ref, s_ref, max_bad_columns=1)
