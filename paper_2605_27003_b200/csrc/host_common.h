@@ -16,7 +16,7 @@ struct w4a4_ctx {
   int max_M = 0, max_K = 0, max_r = 0;
   uint8_t* codes = nullptr;   // [max_M, K] activation codes, one E4M3 byte each (pitch K of the running layer)
   float* scales = nullptr;    // [K/64, scales_ld] group-major activation scales
-  uint8_t* a_sop = nullptr;   // activation scale operands of the scale MMA: [ceil(max_M/128)][ceil(G/2)][4096]
+  uint8_t* a_sop = nullptr;   // token-side scale operands of the GEMM's scale MMA: [ceil(max_M/128)][ceil(G/2)][2048]
   int scales_ld = 0;          // max_M rounded up to a multiple of 4 (16-byte rows for TMA)
   uint16_t* t_hilo = nullptr; // [max_M, 2r] BF16 high | low parts of Xh L1
   uint8_t* b8 = nullptr;      // [N, K] E4M3 image of the running layer's weight codes (rewritten by every forward)

@@ -30,13 +30,13 @@
 //               for the epilogue to drain it before the next tile: sixteen warps pull the whole accumulator into
 //               registers at once and hand it back before they convert and store.
 //
-// Every wait is bounded exactly as in gemm_kernel.cuh (whose Ring / bounded_wait helpers are used here).
+// Every wait is bounded (pipeline.cuh).
 #pragma once
 
 #include <cuda_bf16.h>
 #include <stdint.h>
 
-#include "gemm_kernel.cuh"
+#include "pipeline.cuh"
 #include "ptx.cuh"
 #include "quantize_kernel.cuh"
 
@@ -134,7 +134,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
   const int atoms_k = p.K / 128;
   const int num_tiles = p.tiles_m * p.tiles_n;
-  const WaitEnv env{p.err, s_abort};
+  const WaitEnv env{p.err, s_abort, kWaitLimitNs};
 
   if (threadIdx.x == 0) {
     *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
@@ -357,46 +357,6 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 //   acc_empty  (leader)   all 32 epilogue warps of the pair have pulled their part of the accumulator.
 // Scale factors: every CTA needs the A scales of its own rows and the B scales of all 256 columns in its own TMEM;
 // tcgen05.cp.cta_group::2 copies them from each CTA's own shared memory.
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Relaxed on purpose: the arrive only hands TMEM columns back (tcgen05.wait::ld has completed the reads, the
-// tcgen05 fence orders them); a release at cluster scope would also wait for the warp's earlier global stores
-// (the previous tile's outputs) to become visible, which cost about 1200 clocks per tile.
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// 2D tiled load into this CTA's shared memory whose byte count is reported to `bar_cluster_addr`, a barrier of
-// this CTA or of the other CTA of the pair.
-__device__ __forceinline__ void tma2_load_2d(uint32_t dst_smem, const CUtensorMap* tm, uint32_t bar_cluster_addr, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
-      : "memory");
-}
-// Release at cluster scope: for hand-overs of data this thread wrote to memory (the fused epilogue's x_hat rows in
-// shared memory, read by the pair's tensor cores on behalf of the other CTA).
-__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc2(uint32_t smem_result, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
 __device__ __forceinline__ void tmem_cp2_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
   asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
@@ -411,21 +371,6 @@ __device__ __forceinline__ void umma2_mxf4(uint32_t d_tmem, uint64_t a_desc, uin
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
       : "memory");
 }
-__device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Arrives on the mbarrier at `cluster_addr` (this CTA's or the neighbour's) once the pair's MMAs issued so far are done.
-__device__ __forceinline__ void umma2_commit(uint32_t cluster_addr) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
-}
-
 constexpr int kMx2Stages = 6;
 constexpr uint32_t kMx2BHalf = kMxBTile / 2;                                  // 16 KiB: this CTA's 128 rows of B
 constexpr uint32_t kMx2StageBytes = kMxATile + kMx2BHalf + 3 * kMxSfTile;      // 35 KiB
@@ -532,7 +477,7 @@ mx_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int runs_per_pair = (p.tiles_n + run - 1) / run;
   const int num_runs = ((p.tiles_m + 1) / 2) * runs_per_pair;
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
-  const WaitEnv env{p.err, s_abort};
+  const WaitEnv env{p.err, s_abort, kWaitLimitNs};
   if (threadIdx.x == 0) {
     *s_abort = (*reinterpret_cast<volatile int*>(p.err) != 0) ? 1 : 0;
     for (int i = 0; i < STAGES; ++i) {

@@ -146,6 +146,88 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&v)
 
 
 
+// ------------------------------------------------------------------------------------ CTA pairs (cta_group::2)
+// A thread-block cluster of two CTAs runs one tcgen05.mma over both SMs: A rows 0..127 / 128..255 and B rows
+// (output columns) of the first / second half lie in the shared memory of CTA 0 / CTA 1 at the same offsets, and
+// the accumulator rows land in the TMEM of the CTA that holds the A rows.  CTA 0 issues for the pair.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Relaxed on purpose: the arrive only hands TMEM columns back (tcgen05.wait::ld has completed the reads, the
+// tcgen05 fence orders them); a release at cluster scope would also wait for the warp's earlier global stores
+// (the previous tile's outputs) to become visible, which cost about 1200 clocks per tile.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// 2D tiled load into this CTA's shared memory whose byte count is reported to `bar_cluster_addr`, a barrier of
+// this CTA or of the other CTA of the pair.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst_smem, const CUtensorMap* tm, uint32_t bar_cluster_addr, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
+// Release at cluster scope: for hand-overs of data this thread wrote to memory (the fused epilogue's x_hat rows in
+// shared memory, read by the pair's tensor cores on behalf of the other CTA).
+__device__ __forceinline__ void mbar_arrive_remote_release(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier at `cluster_addr` (this CTA's or the neighbour's) once the pair's MMAs issued so far are done.
+__device__ __forceinline__ void umma2_commit(uint32_t cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__device__ __forceinline__ void umma2_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Shared-memory operand descriptor, K-major tile without swizzle (canonical layout: core matrices of 8 rows x
+// 16 bytes, each 128 contiguous bytes).  `k_step` is the byte distance from a core matrix to the next one along K
+// (leading byte offset), `mn_step` the distance to the next 8-row group (stride byte offset).
+__device__ __forceinline__ uint64_t umma_desc_k_plain(uint32_t smem_addr, uint32_t k_step, uint32_t mn_step) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr >> 4) & 0x3FFFu);
+  d |= static_cast<uint64_t>((k_step >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((mn_step >> 4) & 0x3FFFu) << 32;
+  d |= static_cast<uint64_t>(1u) << 46;
+  return d;
+}
+
 // Shared-memory operand descriptor, K-major tile with the 128-byte swizzle: rows of 128 bytes,
 // 8-row swizzle atoms of 1024 bytes stacked along M/N (stride-byte-offset 1024), tile base aligned
 // to 1024 bytes.  `byte_offset_in_row` selects the K slice (multiple of 32 bytes) inside the row.

@@ -199,15 +199,13 @@ __device__ __forceinline__ uint32_t mxfp4_block16(const float* xh, float rho, ui
   return ex;
 }
 
-// One 16-byte chunk of the activation-side scale operand of the GEMM's scale MMA: s = h + m + l in BF16 pieces,
-// laid out [h, h, h, m, m, m, l, l] against the weight side's [w1, w2, w3, w1, w2, w3, w1, w2].
-__device__ __forceinline__ uint4 sop_chunk_activation(float s) {
+// The token side of the GEMM's scale MMA for one (row, group): the scale as two BF16 pieces, s = h + m up to 2^-16
+// relative, laid out [h, h, m, m] against the channel side's [w1, w2, w1, w2].
+__device__ __forceinline__ uint2 sop_slots_activation(float s) {
   const __nv_bfloat16 h = __float2bfloat16_rn(s);
-  const float r1 = s - __bfloat162float(h);
-  const __nv_bfloat16 m = __float2bfloat16_rn(r1);
-  const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
-  const uint32_t hb = __bfloat16_as_ushort(h), mb = __bfloat16_as_ushort(m), lb = __bfloat16_as_ushort(l);
-  return make_uint4(hb | (hb << 16), hb | (mb << 16), mb | (mb << 16), lb | (lb << 16));
+  const __nv_bfloat16 m = __float2bfloat16_rn(s - __bfloat162float(h));
+  const uint32_t hb = __bfloat16_as_ushort(h), mb = __bfloat16_as_ushort(m);
+  return make_uint2(hb | (hb << 16), mb | (mb << 16));
 }
 
 template <int R, int WARPS, int FORMAT>
@@ -215,7 +213,7 @@ __global__ void __launch_bounds__(32 * WARPS)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
                 uint8_t* __restrict__ codes, float* __restrict__ scales, int scales_ld,
-                uint16_t* __restrict__ t_hilo, float* __restrict__ t_partial, uint4* __restrict__ a_sop) {
+                uint16_t* __restrict__ t_hilo, float* __restrict__ t_partial, uint2* __restrict__ a_sop) {
   constexpr int NT = R / 8;                          // n-tiles of the m16n8k16 MMA
   constexpr int kFragBytes = 4 * NT * 32 * 8;        // L1 fragments of one group (4 KiB at r = 32)
   constexpr int kFragChunks = kFragBytes / 16;
@@ -353,11 +351,11 @@ quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __res
     if (qj == 0 && okA) scales[static_cast<size_t>(g) * scales_ld + rowA] = s_mine;
     if (qj == 1 && okB) scales[static_cast<size_t>(g) * scales_ld + rowB] = s_mine;
     if (a_sop != nullptr && ((qj == 0 && okA) || (qj == 1 && okB))) {
-      // The scale once more, as one 16-byte chunk of the operand from which the GEMM's tensor core forms
-      // sx * sw: 4 KiB shared-memory images per (128 rows, 2 groups), [8-row group][group parity][8 rows][16 bytes].
+      // The scale once more, as four BF16 slots of the operand from which the GEMM's tensor core forms sx * sw:
+      // 2 KiB shared-memory images per (128 rows, 2 groups), [8-row group][8 rows][group parity][8 bytes].
       const int row = qj == 0 ? rowA : rowB;
       const size_t image = static_cast<size_t>(row >> 7) * ((G + 1) >> 1) + (g >> 1);
-      a_sop[image * 256 + ((row & 127) >> 3) * 16 + (g & 1) * 8 + (row & 7)] = sop_chunk_activation(s_mine);
+      a_sop[image * 256 + ((row & 127) >> 3) * 16 + (row & 7) * 2 + (g & 1)] = sop_slots_activation(s_mine);
     }
     }
 

@@ -8,13 +8,11 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
 
-#include "gemm_kernel.cuh"
-#include "gemm_os_kernel.cuh"
+#include "gemm_w4a4_kernel.cuh"
 #include "host_common.h"
 #include "quantize_kernel.cuh"
 
@@ -126,19 +124,19 @@ using namespace w4a4;
 struct ExpertData {
   uint8_t* bpacked = nullptr;  // [N, K/2]
   float* wscale = nullptr;     // [G, N]
-  uint8_t* b_sop = nullptr;    // weight scale operands of the scale MMA: [N/128][ceil(G/2)][2][4096]
+  uint8_t* b_sop = nullptr;    // weight scale operands of the scale MMA: [N/128][ceil(G/2)][4096]
   float* rlam = nullptr;       // [K]
   uint2* l1frag = nullptr;
   uint16_t* l2dup = nullptr;   // [N, 2r]
   float* bias = nullptr;       // [N] or null
-  CUtensorMap tmSW, tmL2;
+  CUtensorMap tmL2, tmSopB;
 };
 
 struct w4a4_layer {
   w4a4_ctx* ctx = nullptr;
   int K = 0, N = 0, r = 0, E = 0, B = 0, L = 0, layer_id = 0, act = 0;
   std::vector<ExpertData> experts;
-  CUtensorMap tmA, tmSA, tmT, tmB;
+  CUtensorMap tmA, tmSopA, tmT, tmB;
   const uint8_t* tmB_base = nullptr;  // the context's weight-byte scratch this handle's tmB was encoded for
   size_t bytes = 0;
 };
@@ -188,7 +186,7 @@ w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expe
 #define W4A4_LAUNCH_Q(R)                                                                                         \
   quantize_kernel<R, quantize_warps(R), kCodesE4M3><<<grid, block, quantize_smem_bytes(R), stream>>>(x, M, h->K, e.rlam, clip_table, clip_index, e.l1frag, ctx->codes, \
                                                  ctx->scales, ctx->scales_ld, ctx->t_hilo, ctx->t_partial,     \
-                                                 reinterpret_cast<uint4*>(ctx->a_sop))
+                                                 reinterpret_cast<uint2*>(ctx->a_sop))
   switch (h->r) {
     case 0: W4A4_LAUNCH_Q(0); break;
     case 16: W4A4_LAUNCH_Q(16); break;
@@ -228,14 +226,13 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   p.tiles_m = (M + kBM - 1) / kBM;
   p.tiles_n = h->N / kBN;
   p.err = ctx->d_err;
+  p.wait_limit_ns = kWaitLimitNs;
   p.dbg_P = dbg_P;
   p.dbg_m0 = dbg_m0;
   p.dbg_n0 = dbg_n0;
   p.yref = static_cast<const uint16_t*>(yref);
   p.sq_err = sq_err;
   p.act = h->act;
-  const int num_tiles = p.tiles_m * p.tiles_n;
-  const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
   // The context's weight-byte scratch may have been reallocated (a larger layer packed since): re-aim the map.
   if (h->tmB_base != ctx->b8) {
     if (!encode_2d(ctx->encode, &h->tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, ctx->b8, h->K, h->N, h->K, kBK, kBN,
@@ -248,29 +245,18 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
     expand_weight_kernel<<<static_cast<unsigned>((chunks + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<const uint4*>(e.bpacked), reinterpret_cast<uint4*>(ctx->b8), chunks);
   }
+  // Persistent: one CTA per SM walks the 128 x 128 tiles.
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : h->tmB;
-  static const bool cuda_core_rescale = [] {
-    const char* v = std::getenv("W4A4_GEMM");
-    return v && std::strcmp(v, "cuda_core_rescale") == 0;
-  }();
-  if (cuda_core_rescale) {
-    if (dbg_P) {
-      gemm_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
-    } else {
-      gemm_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, e.tmSW, h->tmSA, tmT, tmL2, p);
-    }
+  if (dbg_P) {
+    gemm_w4a4_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, h->tmSopA, e.tmSopB, p);
   } else {
-    OsParams q;
-    q.a_sop = ctx->a_sop;
-    q.b_sop = e.b_sop;
-    if (dbg_P) {
-      gemm_os_kernel<true><<<grid, block, kOsSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, p, q);
-    } else {
-      gemm_os_kernel<false><<<grid, block, kOsSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, p, q);
-    }
+    gemm_w4a4_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, h->tmSopA, e.tmSopB, p);
   }
-  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+  const cudaError_t le = cudaGetLastError();
+  return le == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
 }
 
 }  // namespace
@@ -331,7 +317,7 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   w4a4_status_t st = dev_alloc(&ctx->codes, static_cast<size_t>(max_M) * max_K, &ctx->bytes);
   if (st == W4A4_OK) st = dev_alloc(&ctx->scales, static_cast<size_t>(ctx->scales_ld) * (max_K / 64), &ctx->bytes);
   if (st == W4A4_OK && cudaMemset(ctx->scales, 0, sizeof(float) * ctx->scales_ld * (max_K / 64)) != cudaSuccess) st = W4A4_ERR_CUDA;
-  const size_t a_sop_bytes = static_cast<size_t>((max_M + 127) / 128) * ((max_K / 64 + 1) / 2) * 4096;
+  const size_t a_sop_bytes = static_cast<size_t>((max_M + 127) / 128) * ((max_K / 64 + 1) / 2) * kSopATile;
   if (st == W4A4_OK) st = dev_alloc(&ctx->a_sop, a_sop_bytes, &ctx->bytes);
   // Rows past M and the unused half of an odd last stage are multiplied by zeros: they only have to be finite.
   if (st == W4A4_OK && cudaMemset(ctx->a_sop, 0, a_sop_bytes) != cudaSuccess) st = W4A4_ERR_CUDA;
@@ -349,10 +335,8 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   if (st == W4A4_OK) {
     cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesE4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          static_cast<int>(quantize_smem_bytes(64)));
-    cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
-    cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
-    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(gemm_os_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOsSmemBytes);
-    if (e2 == cudaSuccess) e2 = cudaFuncSetAttribute(gemm_os_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kOsSmemBytes);
+    const cudaError_t e1 = cudaFuncSetAttribute(gemm_w4a4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
+    const cudaError_t e2 = cudaFuncSetAttribute(gemm_w4a4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
       cudaGetLastError();
       st = W4A4_ERR_CUDA;
@@ -471,7 +455,7 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
 
     const cudaMemcpyKind kind = dev ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
     if (cudaMemcpy(e.wscale, d->wscale[ei], sizeof(float) * G * N, kind) != cudaSuccess) st = W4A4_ERR_CUDA;
-    const size_t b_sop_bytes = static_cast<size_t>(N / kBN) * ((G + 1) / 2) * kOsSopTile;
+    const size_t b_sop_bytes = static_cast<size_t>(N / kBN) * ((G + 1) / 2) * kSopBTile;
     if (st == W4A4_OK) st = dev_alloc(&e.b_sop, b_sop_bytes, &h->bytes);
     if (st == W4A4_OK && cudaMemset(e.b_sop, 0, b_sop_bytes) != cudaSuccess) st = W4A4_ERR_CUDA;
     if (st == W4A4_OK) {
@@ -510,8 +494,9 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
     cudaFree(l2_own);
     if (st != W4A4_OK) break;
 
-    if (!encode_2d(ctx->encode, &e.tmSW, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, e.wscale, N, G, static_cast<uint64_t>(N) * 4,
-                   kBN, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
+    // Scale operand images as rows of 32-bit words (one row per 128 output channels), fetched in boxes of 1 KiB.
+    if (!encode_2d(ctx->encode, &e.tmSopB, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, e.b_sop, static_cast<uint64_t>((G + 1) / 2) * (kSopBTile / 4),
+                   N / kBN, static_cast<uint64_t>((G + 1) / 2) * kSopBTile, 256, 1, CU_TENSOR_MAP_SWIZZLE_NONE))
       st = W4A4_ERR_CUDA;
     if (st == W4A4_OK && r > 0 &&
         !encode_2d(ctx->encode, &e.tmL2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, e.l2dup, 2 * r, N, 4 * r, 64, kBN,
@@ -529,8 +514,8 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
                  CU_TENSOR_MAP_SWIZZLE_128B))
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK &&
-      !encode_2d(ctx->encode, &h->tmSA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ctx->scales, ctx->scales_ld, G,
-                 static_cast<uint64_t>(ctx->scales_ld) * 4, kBM, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
+      !encode_2d(ctx->encode, &h->tmSopA, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, ctx->a_sop, static_cast<uint64_t>((G + 1) / 2) * (kSopATile / 4),
+                 (ctx->max_M + kBM - 1) / kBM, static_cast<uint64_t>((G + 1) / 2) * kSopATile, 256, 1, CU_TENSOR_MAP_SWIZZLE_NONE))
     st = W4A4_ERR_CUDA;
   if (st == W4A4_OK && r > 0 &&
       !encode_2d(ctx->encode, &h->tmT, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ctx->t_hilo, 2 * r, ctx->max_M, 4 * r, 64,

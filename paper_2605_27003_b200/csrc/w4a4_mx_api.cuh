@@ -123,11 +123,7 @@ w4a4_status_t mx_launch_gemm(w4a4_mx_handle_t h, int M, int expert_id, void* Y, 
   const CUtensorMap& tmT = h->r > 0 ? (second_ws ? h->tmT2 : h->tmT) : tmA;  // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : e.tmB;
   // CTA pairs (cta_group::2) need at least two row tiles and an even number of CTAs.
-  static const bool pair_allowed = [] {
-    const char* v = std::getenv("W4A4_MX_GEMM");
-    return !(v && std::strcmp(v, "single") == 0);
-  }();
-  if (pair_allowed && p.tiles_m >= 2 && ctx->num_sms >= 2) {
+  if (p.tiles_m >= 2 && ctx->num_sms >= 2) {
     const int runs = ((p.tiles_m + 1) / 2) * ((p.tiles_n + p.run - 1) / p.run);
     const int ctas = 2 * runs < ctx->num_sms ? 2 * runs : (ctx->num_sms & ~1);
     cudaLaunchConfig_t cfg = {};

@@ -283,25 +283,6 @@ def test_host_buffer_forward_equals_device_forward():
     ctx.close()
 
 
-@pytest.mark.parametrize("env,module,call", [
-    ("W4A4_GEMM=cuda_core_rescale", "test_gpu_parity",
-     "x, lay = m.tiny_inputs(333, 768, 256, 32, seed=5, bias=True); m.run_case(x, [lay], torch.full((1, 1, 1), 0.8), 0, 0)"),
-    ("W4A4_MX_GEMM=single", "test_mx_gpu_parity",
-     "x, lay = m.mx_inputs(333, 768, 256, 32, seed=5, bias=True); m.run_mx_case(x, [lay], torch.full((1, 1, 1), 0.8), 0, 0)"),
-])
-def test_alternative_kernels_selected_by_environment(env, module, call):
-    """The first form of the INT4 GEMM (rescale on the CUDA cores) and the single-CTA MXFP4 GEMM stay selectable for
-    A/B timing; the switch is read once per process, so each runs in a process of its own."""
-    import subprocess
-    import sys
-    key, value = env.split("=")
-    code = f"import sys, torch; sys.path.insert(0, 'tests'); import {module} as m; {call}; print('parity ok')"
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    out = subprocess.run([sys.executable, "-c", code], cwd=root, env={**os.environ, key: value}, capture_output=True,
-                         text=True, timeout=600)
-    assert out.returncode == 0 and "parity ok" in out.stdout, out.stdout[-2000:] + out.stderr[-2000:]
-
-
 def test_qkv_packed_as_one_layer_shares_one_activation_pass():
     # q, k and v read the same input with the same smoothing vector and the same clipping-ratio entry, so their
     # activation quantization and low-rank down-projection can be done once: pack the three projections as ONE layer
