@@ -33,10 +33,9 @@ METRIC = "w4a4_lowrank_linear_effective_tops"
 UNIT = "TOPS"
 NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_HBM_GBS = 7700.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summaries (profiles/);
-# None until a capture exists for that kernel and workload.
-# (quantize: 484.7 MB captured before the kernel also wrote the 41.9 MB of scale operands, which are added here.)
-NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 571.6e6, ("quantize", "attn_proj"): 526.6e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, each from one single-launch ncu capture of the kernel as
+# it stands (summaries under profiles/); None where no capture exists for that kernel and workload.
+NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): None, ("quantize", "attn_proj"): 502.0e6}
 
 
 def max_over_ranks(ms: float, dist, device="cpu") -> float:
@@ -67,6 +66,81 @@ def load_peaks():
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
                     bf16_sustained=float(p["bf16_tflops_sustained"]), source="measured")
     return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def _time_loop(fn, stream, seconds: float):
+    """(best single-call ms over 10 calls, mean ms of calls issued back to back for about `seconds`)."""
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    reps = max(10, int(seconds * 1e3 / best))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return best, e0.elapsed_time(e1) / reps
+
+
+def measure_tensor_peaks(dev, seconds: float = 3.0):
+    """Dense 8-bit tensor-core peaks of this GPU from library GEMMs (8192^3), taken the way MEASURED_PEAKS.json's
+    BF16 figures were: best of 10 calls (burst) and a seconds-long back-to-back loop (sustained).  Library calls are
+    fine for a peak probe; nothing here is on the layer's path or inside a timed region of it."""
+    n = 8192
+    ops = 2.0 * n ** 3
+    stream = torch.cuda.current_stream()
+    out = {}
+    try:
+        a = torch.randn(n, n, device=dev).to(torch.float8_e4m3fn)
+        b = torch.randn(n, n, device=dev).to(torch.float8_e4m3fn).t()
+        one = torch.ones((), device=dev, dtype=torch.float32)
+        best, mean = _time_loop(lambda: torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16), stream, seconds)
+        out["fp8_tops_burst"], out["fp8_tops_sustained"] = ops / (best * 1e-3) / 1e12, ops / (mean * 1e-3) / 1e12
+        del a, b
+    except Exception as e:  # noqa: BLE001
+        out["fp8_error"] = repr(e)[:200]
+    try:
+        a = torch.randint(-8, 8, (n, n), device=dev, dtype=torch.int8)
+        b = torch.randint(-8, 8, (n, n), device=dev, dtype=torch.int8).t().contiguous().t()
+        best, mean = _time_loop(lambda: torch._int_mm(a, b), stream, seconds)
+        out["int8_tops_burst"], out["int8_tops_sustained"] = ops / (best * 1e-3) / 1e12, ops / (mean * 1e-3) / 1e12
+        del a, b
+    except Exception as e:  # noqa: BLE001
+        out["int8_error"] = repr(e)[:200]
+    out["how"] = "torch._scaled_mm (E4M3) and torch._int_mm (INT8) at 8192^3: best of 10 and a %.0f s back-to-back loop" % seconds
+    torch.cuda.empty_cache()
+    return out
+
+
+def tensor_roofline(gemm_tops: float, timed_seconds: float, peaks: dict, tp: dict, fp4: bool = False) -> dict:
+    """Fractions of the dense tensor peak of the contraction's own type.  8-bit (the INT4-exact path runs on the FP8
+    pipe): the FP8 figures measured in this run when they exist, else 2 x the measured BF16 figures (nominal ratio).
+    FP4 (the MXFP4 variant): no library FP4 GEMM is timed, so 2 x the 8-bit figure (nominal ratio 9 : 4.5).  The burst
+    figure serves a timed region shorter than a second, the sustained one a longer region."""
+    if tp and "fp8_tops_burst" in tp:
+        burst, sustained, src = tp["fp8_tops_burst"], tp["fp8_tops_sustained"], "library FP8 GEMM 8192^3 measured in this run"
+    else:
+        burst, sustained = 2.0 * peaks["bf16_burst"], 2.0 * peaks["bf16_sustained"]
+        src = f"{peaks['source']} BF16 figures x 2 (nominal 8-bit : BF16 ratio; no 8-bit library GEMM could be timed)"
+    nominal = NOMINAL_INT8_TOPS
+    if fp4:
+        burst, sustained, nominal, src = 2.0 * burst, 2.0 * sustained, 2.0 * NOMINAL_INT8_TOPS, src + ", x 2 (nominal FP4 : 8-bit ratio)"
+    use_burst = timed_seconds < 1.0
+    peak = burst if use_burst else sustained
+    out = dict(bound="tensor", achieved=gemm_tops, peak=peak, unit="TOP/s", frac=gemm_tops / peak,
+               peak_kind="burst" if use_burst else "sustained", peak_source=src,
+               frac_burst=gemm_tops / burst, frac_sustained=gemm_tops / sustained)
+    out["frac_of_nominal_%d" % nominal] = gemm_tops / nominal
+    return out
 
 
 class ClockSampler:
@@ -253,11 +327,12 @@ def time_layer(w4, layer, xs, bins, expert, clip, Y, M, iters, warmup, stream):
     return (statistics.mean(e[0].elapsed_time(e[1]) for e in ev), statistics.mean(e[1].elapsed_time(e[2]) for e in ev))
 
 
-def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks):
-    """One denoising step's quantized linears of a 40-block, 5120-hidden DiT at M = 32760, r = 32, with both
-    experts' weight sets resident; step s uses expert (s >= 20) and timestep bin s // 5 (40-step schedule)."""
+def measure_dit_step(w4, dev, local_rank, steps, warmup, blocks, dist=None):
+    """One denoising step's quantized linears of a `blocks`-block, 5120-hidden DiT at M = 32760, r = 32, with both
+    experts' weight sets resident; step s uses expert (s >= 20) and timestep bin s // 5 (40-step schedule).
+    Returns this rank's device time per step and what the step holds."""
     M, r, bins, experts = 32760, 32, 8, 2
-    shapes = dit_step_layers(args.blocks)
+    shapes = dit_step_layers(blocks)
     L = len(shapes)
     ctx = w4.Context(local_rank, M, 13824, r)
     layers = []
@@ -285,7 +360,7 @@ def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for s in range(args.warmup):
+    for s in range(warmup):
         step(s)
     barrier()
     ctx.check()
@@ -294,44 +369,68 @@ def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record(stream)
-    for s in range(args.steps):
+    for s in range(steps):
         step(18 + s)  # straddles the expert switch at step 20
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
     ctx.check()
-    total_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
-    ms_per_step = total_ms / args.steps
-    ops = sum(2.0 * M * K * N for (K, N) in shapes)
-    if rank == 0:
-        int8_peak = 2.0 * peaks["bf16_sustained"]
-        tops = whole_job_tops(ops, world, ms_per_step)
-        line = dict(metric=METRIC, value=tops, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-                    ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e4m3",
-                    data="synthetic",
-                    config=dict(workload="dit_step", M=M, r=r, group=64, blocks=args.blocks, linears=L, experts=experts,
-                                bins=bins, resident_weight_gb=weight_bytes / 1e9, tera_ops_per_step=ops / 1e12,
-                                l2="inputs larger than L2: 3 rotating activation buffers per shape (335 / 906 MB)",
-                                parallelism="replicas" if world > 1 else "single"),
-                    ms_per_dit_step=ms_per_step,
-                    roofline=dict(bound="tensor", achieved=tops / world, peak=int8_peak, unit="TOP/s",
-                                  frac=tops / world / int8_peak, traffic=None, kernel="quantize + gemm, whole step",
-                                  peak_source=f"{peaks['source']} sustained BF16 x 2"),
-                    gpu_launches=3 * L * args.steps, clocks=clocks)
-        print(json.dumps(line), flush=True)
+    total_ms = e0.elapsed_time(e1)
     for l in layers:
         l.close()
     ctx.close()
+    del xs, Y
+    torch.cuda.empty_cache()
+    return dict(total_ms=total_ms, ops=sum(2.0 * M * K * N for (K, N) in shapes), M=M, r=r, experts=experts, bins=bins,
+                linears=L, weight_bytes=weight_bytes, clocks=clocks)
+
+
+def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks, tp):
+    d = measure_dit_step(w4, dev, local_rank, args.steps, args.warmup, args.blocks, dist)
+    total_ms = max_over_ranks(d["total_ms"], dist, dev)
+    ms_per_step = total_ms / args.steps
+    if rank == 0:
+        tops = whole_job_tops(d["ops"], world, ms_per_step)
+        roof = tensor_roofline(tops / world, total_ms * 1e-3, peaks, tp)
+        roof.update(traffic=None, kernel="quantize + expand + gemm of every layer, whole step")
+        line = dict(metric=METRIC, value=tops, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                    ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e4m3",
+                    data="synthetic",
+                    config=dict(workload="dit_step", M=d["M"], r=d["r"], group=64, blocks=args.blocks, linears=d["linears"],
+                                experts=d["experts"], bins=d["bins"], resident_weight_gb=d["weight_bytes"] / 1e9,
+                                tera_ops_per_step=d["ops"] / 1e12,
+                                l2="inputs larger than L2: 3 rotating activation buffers per shape (335 / 906 MB)",
+                                parallelism="replicas" if world > 1 else "single"),
+                    ms_per_dit_step=ms_per_step, roofline=roof, tensor_peaks=tp,
+                    gpu_launches=3 * d["linears"] * args.steps, clocks=d["clocks"])
+        print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
 
 
-def run_sweep(args, w4, dev, local_rank, rank, peaks):
+def measure_single_layer(w4, dev, local_rank, name, iters, warmup):
+    """Mean kernel times of one of the single-layer workloads (used for the second shape the performance target names)."""
+    w = workload_inputs(name, dev, 3)
+    M, K, N, r = w["M"], w["K"], w["N"], w["r"]
+    ctx = w4.Context(local_rank, M, K, r)
+    layer = w4.Layer(ctx, [w["layer"]], num_bins=w["num_bins"])
+    clip = w["clip"].to(dev)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+    tq, tg = time_layer(w4, layer, w["xs"], w["bins"], 0, clip, Y, M, iters, warmup, torch.cuda.current_stream())
+    ctx.check()
+    layer.close()
+    ctx.close()
+    del w, Y
+    torch.cuda.empty_cache()
+    return dict(M=M, K=K, N=N, r=r, quantize_ms=tq, gemm_ms=tg, iters=iters)
+
+
+def run_sweep(args, w4, dev, local_rank, rank, peaks, tp):
     """Shape sweep: M x (K, N) x r x outlier fraction x clip ratio, TOPS and roofline fractions per point."""
     if rank != 0:
         return
-    int8_peak = 2.0 * peaks["bf16_sustained"]
+    int8_peak = tp.get("fp8_tops_sustained", 2.0 * peaks["bf16_sustained"])   # hours of back-to-back kernels: the sustained figure
     rows = []
     stream = torch.cuda.current_stream()
     for (K, N) in ((5120, 5120), (5120, 13824), (13824, 5120)):
@@ -348,7 +447,7 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                     for b, alpha in ((0, 0.7), (1, 1.0)):
                         tq, tg = time_layer(w4, layer, xs, [b] * n_x, 0, clip, Y, M, args.steps, max(3, args.warmup), stream)
                         ops = 2.0 * M * K * N
-                        qb = M * (3.3125 * K + 4.0 * r)
+                        qb = M * (2.5625 * K + 2.0 * r)   # X, 4-bit codes, FP32 scales, BF16 T: the bytes the step needs, not the layout's
                         rows.append(dict(M=M, K=K, N=N, r=r, outlier_fraction=frac, alpha=alpha, quantize_ms=tq, gemm_ms=tg,
                                          layer_tops=ops / ((tq + tg) * 1e-3) / 1e12, gemm_tops=ops / (tg * 1e-3) / 1e12,
                                          gemm_frac=ops / (tg * 1e-3) / 1e12 / int8_peak,
@@ -370,7 +469,7 @@ def run_sweep(args, w4, dev, local_rank, rank, peaks):
                           best_point=best, gpu_launches=3 * args.steps * len(rows))), flush=True)
 
 
-def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
+def run_mxfp4(args, w4, dev, local_rank, rank, peaks, tp):
     """The MXFP4 variant of the layer (E2M1 elements, E8M0 block scales applied inside the tensor core) on the
     shape of one of the single-layer workloads: `--workload mxfp4_attn_proj | mxfp4_ffn_up | mxfp4_ffn_down`."""
     if rank != 0:
@@ -417,8 +516,9 @@ def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
     tq = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     tg = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
     ops = 2.0 * M * K * N
-    fp4_peak = 4.0 * peaks["bf16_sustained"]  # dense FP4 = 4 x dense BF16 (nominal ratio 9 / 2.25)
     gemm_tops = ops / (tg * 1e-3) / 1e12
+    roof = tensor_roofline(gemm_tops, tg * 1e-3 * len(ev), peaks, tp, fp4=True)
+    roof.update(traffic=None, kernel="mx_gemm2_kernel (CTA pairs; mx_gemm_kernel when M <= 128)", ms=tg)
     q_bytes = M * (2.0 * K + K / 2.0 + K / 32.0 + 4.0 * r)  # X read, packed codes, scale bytes, T hi | lo
     print(json.dumps(dict(
         metric=METRIC, value=ops / (ms * 1e-3) / 1e12, unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
@@ -426,10 +526,7 @@ def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
         data="synthetic",
         config=dict(workload=args.workload, M=M, K=K, N=N, r=r, block=32, experts=1, bins=num_bins,
                     l2="inputs larger than L2: 4 rotating activation buffers of %.0f MB" % (M * K * 2 / 1e6)),
-        roofline=dict(bound="tensor", achieved=gemm_tops, peak=fp4_peak, unit="TOP/s", frac=gemm_tops / fp4_peak,
-                      traffic=None, kernel="mx_gemm2_kernel (CTA pairs; mx_gemm_kernel when M <= 128)", ms=tg,
-                      peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 4 "
-                                  "(nominal FP4:BF16 ratio)", frac_of_nominal_9000=gemm_tops / 9000.0),
+        roofline=roof,
         roofline_quantize=dict(bound="hbm", achieved=q_bytes / (tq * 1e-3) / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
                                frac=q_bytes / (tq * 1e-3) / 1e9 / peaks["hbm_gbs"], kernel="quantize_kernel (MXFP4 format)",
                                ms=tq, algorithmic_bytes=q_bytes, peak_source=peaks["source"]),
@@ -438,7 +535,7 @@ def run_mxfp4(args, w4, dev, local_rank, rank, peaks):
     ctx.close()
 
 
-def run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks):
+def run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks, tp):
     """The FFN of the MXFP4 variant, 5120 -> 13824 (GELU) -> 5120 at M = 32760: the fused call (the up-projection's
     epilogue quantizes for the down-projection; the hidden activation never reaches memory) against the same two
     layers as two calls (`--workload mxfp4_ffn`)."""
@@ -487,18 +584,15 @@ def run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks):
     clocks = sampler.stop()
     ctx.check()
     ops = 2.0 * M * K * H + 2.0 * M * H * N
-    fp4_peak = 4.0 * peaks["bf16_sustained"]
+    roof = tensor_roofline(ops / (ms * 1e-3) / 1e12, ms * 1e-3 * args.steps, peaks, tp, fp4=True)
+    roof.update(traffic=None, kernel="whole fused call: quantize, mx_gemm2_kernel<fused epilogue>, T finish, mx_gemm2_kernel")
     print(json.dumps(dict(
         metric=METRIC, value=ops / (ms * 1e-3) / 1e12, unit=UNIT, n_gpus=1, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e2m1 x e8m0 (mxfp4)",
         data="synthetic",
         config=dict(workload=args.workload, M=M, K=K, hidden=H, N=N, r=r, block=32, activation="gelu_tanh",
                     l2="inputs larger than L2: 4 rotating activation buffers of %.0f MB" % (M * K * 2 / 1e6)),
-        roofline=dict(bound="tensor", achieved=ops / (ms * 1e-3) / 1e12, peak=fp4_peak, unit="TOP/s",
-                      frac=ops / (ms * 1e-3) / 1e12 / fp4_peak, traffic=None,
-                      kernel="whole fused call: quantize, mx_gemm2_kernel<fused epilogue>, T finish, mx_gemm2_kernel",
-                      peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 4 "
-                                  "(nominal FP4:BF16 ratio)"),
+        roofline=roof,
         two_calls=dict(ms_per_step=ms_two, value=ops / (ms_two * 1e-3) / 1e12, unit=UNIT,
                        note="same layers as w4a4_mx_linear_forward twice (hidden activation stored and re-read)"),
         e2e=None, gpu_launches=5 * args.steps, clocks=clocks)), flush=True)
@@ -681,6 +775,8 @@ def main():
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the library peak probe, the second target shape and the short DiT-step run (profiling runs)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -710,17 +806,19 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     peaks = load_peaks()
+    # Library 8-bit GEMM peaks of this GPU, before (and outside) every timed region of the layer.
+    tp = {} if (args.no_extras or args.workload.startswith("gptq") or args.workload == "tiny") else measure_tensor_peaks(dev)
     if args.workload == "dit_step":
-        run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks)
+        run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks, tp)
         return
     if args.workload == "sweep":
-        run_sweep(args, w4, dev, local_rank, rank, peaks)
+        run_sweep(args, w4, dev, local_rank, rank, peaks, tp)
         return
     if args.workload == "mxfp4_ffn":
-        run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks)
+        run_mxfp4_ffn(args, w4, dev, local_rank, rank, peaks, tp)
         return
     if args.workload.startswith("mxfp4_"):
-        run_mxfp4(args, w4, dev, local_rank, rank, peaks)
+        run_mxfp4(args, w4, dev, local_rank, rank, peaks, tp)
         return
     if args.workload == "clip_search":
         run_clip_search(args, w4, dev, local_rank, rank, peaks)
@@ -792,43 +890,63 @@ def main():
     e2e_value = whole_job_tops(ops, world, e2e_ms / e2e_steps)
     ctx.check()
 
+    mx_ctx = mxfp4_context(w4, ctx, w, clip, Y, stream) if (rank == 0 and args.workload != "tiny") else None
+    layer.close()
+    ctx.close()
+    w_small = dict(M=M, K=K, N=N, r=r, num_bins=w["num_bins"], xs=w["xs"][:1], bins=w["bins"][:1], layer=w["layer"], clip=w["clip"])
+    del w, Y, xh, yh
+    torch.cuda.empty_cache()
+
     if rank == 0:
         tq, tg = statistics.mean(t_q), statistics.mean(t_g)
-        int8_peak = 2.0 * peaks["bf16_sustained"]  # dense 8-bit (INT8 or FP8) = 2 x dense BF16 (nominal ratio 4.5 / 2.25)
         gemm_tops = ops / (tg * 1e-3) / 1e12
-        # X read, one-byte codes, FP32 scales, 16-byte scale-operand chunks, T as BF16 hi | lo
-        q_bytes = M * (2.0 * K + 1.0 * K + 4.0 * K / 64.0 + 16.0 * K / 64.0 + 4.0 * r)
-        q_gbs = q_bytes / (tq * 1e-3) / 1e9
+        roof = tensor_roofline(gemm_tops, total_ms * 1e-3, peaks, tp)
+        roof.update(traffic=NCU_TRAFFIC_BYTES.get(("gemm", args.workload)),
+                    kernel="gemm_w4a4_kernel (with the 9 us expand_weight_kernel in front of it)", ms=tg)
+        # Bytes the activation step needs by its definition (X read; 4-bit codes, FP32 group scales and BF16 T written)
+        # and bytes this layout moves (one E4M3 byte per code, FP32 scales plus the 8-byte scale operand of the GEMM's
+        # scale MMA per (token, group), T as a BF16 high | low pair).
+        q_alg = M * (2.0 * K + 0.5 * K + 4.0 * K / 64.0 + 2.0 * r)
+        q_layout = M * (2.0 * K + 1.0 * K + 4.0 * K / 64.0 + 8.0 * K / 64.0 + 4.0 * r)
+        q_gbs = q_alg / (tq * 1e-3) / 1e9
         line = dict(
             metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
             ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e4m3",
             data="synthetic",
-            config=dict(workload=args.workload, M=M, K=K, N=N, r=r, group=64, experts=1, bins=w["num_bins"],
+            config=dict(workload=args.workload, M=M, K=K, N=N, r=r, group=64, experts=1, bins=w_small["num_bins"],
                         l2="inputs larger than L2: 4 rotating activation buffers of %.0f MB" % (M * K * 2 / 1e6),
                         parallelism="replicas" if world > 1 else "single"),
-            roofline=dict(bound="tensor", achieved=gemm_tops, peak=int8_peak, unit="TOP/s", frac=gemm_tops / int8_peak,
-                          traffic=NCU_TRAFFIC_BYTES.get(("gemm", args.workload)),
-                          kernel="gemm_os_kernel (with the 9 us expand_weight_kernel in front of it)", ms=tg,
-                          peak_source=f"{peaks['source']} sustained BF16 {peaks['bf16_sustained']} TFLOP/s x 2 "
-                                      "(nominal 8-bit:BF16 ratio)",
-                          frac_of_nominal_4500=gemm_tops / NOMINAL_INT8_TOPS),
+            roofline=roof,
             roofline_quantize=dict(bound="hbm", achieved=q_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
                                    frac=q_gbs / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES.get(("quantize", args.workload)),
-                                   kernel="quantize_kernel", ms=tq, algorithmic_bytes=q_bytes,
-                                   peak_source=peaks["source"]),
+                                   kernel="quantize_kernel", ms=tq, algorithmic_bytes=q_alg,
+                                   bytes_note="algorithmic = X + 4-bit codes + FP32 scales + BF16 T (13,184 B per token at K = 5120, r = 32)",
+                                   layout_bytes=q_layout, frac_of_layout_bytes=q_layout / (tq * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                   frac_of_nominal_7700=q_gbs / NOMINAL_HBM_GBS, peak_source=peaks["source"]),
             kernel_ms=dict(quantize_mean=tq, quantize_min=min(t_q), gemm_mean=tg, gemm_min=min(t_g)),
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=M * K * 2, d2h_bytes_per_step=M * N * 2,
                      ms_per_step=e2e_ms / e2e_steps, steps=e2e_steps,
                      path="w4a4_linear_forward_host: pinned host X -> %d-row chunks over 3 streams -> pinned host Y"
                           % chunk_rows),
-            gpu_launches=3 * args.steps, clocks=clocks)
-        if args.workload != "tiny":
-            line["mxfp4_variant"] = mxfp4_context(w4, ctx, w, clip, Y, stream)
+            gpu_launches=3 * args.steps, clocks=clocks, tensor_peaks=tp)
+        if mx_ctx is not None:
+            line["mxfp4_variant"] = mx_ctx
+        if not args.no_extras and args.workload == "attn_proj" and world == 1:
+            # The second shape of the performance target and a short run of one denoising step's 320 linears.
+            up = measure_single_layer(w4, dev, local_rank, "ffn_up", 20, 3)
+            up_tops = 2.0 * up["M"] * up["K"] * up["N"] / (up["gemm_ms"] * 1e-3) / 1e12
+            up["roofline"] = tensor_roofline(up_tops, up["gemm_ms"] * 1e-3 * up["iters"], peaks, tp)
+            up["layer_tops"] = 2.0 * up["M"] * up["K"] * up["N"] / ((up["gemm_ms"] + up["quantize_ms"]) * 1e-3) / 1e12
+            line["ffn_up"] = up
+            d = measure_dit_step(w4, dev, local_rank, 3, 3, 40)
+            d_ms = d["total_ms"] / 3
+            d_tops = d["ops"] / (d_ms * 1e-3) / 1e12
+            line["dit_step"] = dict(ms_per_dit_step=d_ms, steps=3, warmup=3, value=d_tops, unit=UNIT, linears=d["linears"],
+                                    tera_ops_per_step=d["ops"] / 1e12, resident_weight_gb=d["weight_bytes"] / 1e9,
+                                    roofline=tensor_roofline(d_tops, d["total_ms"] * 1e-3, peaks, tp), clocks=d["clocks"])
         if not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(w)
+            line["cpu_baseline"] = cpu_baseline(w_small)
         print(json.dumps(line), flush=True)
-    layer.close()
-    ctx.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
