@@ -99,7 +99,8 @@ void w4a4_destroy(w4a4_handle_t h);
  *   clip_table  device FP32 [num_experts, num_layers, num_bins], values in [1e-4, 1]
  *   stream      a cudaStream_t (as void*); three kernels are enqueued (activation quantization, expansion of
  *               the layer's 4-bit weights to bytes, GEMM), no host synchronisation.
- * M may be 0 (nothing is launched).  Errors: INVALID_ARG, SHAPE (M > max_M), CUDA. */
+ * M may be 0 (nothing is launched).  Errors: INVALID_ARG, SHAPE (M > max_M), CUDA.  A pipeline wait that
+ * gives up on the device is not visible here (the call does not synchronise): see w4a4_query_status. */
 w4a4_status_t w4a4_linear_forward(w4a4_handle_t h, const void* X, int M, int expert_id, int timestep_bin,
                                   const float* clip_table, void* Y, void* stream);
 
@@ -294,8 +295,25 @@ w4a4_status_t w4a4_mx_gptq_quantize(int device, const float* R, const uint16_t* 
                                     size_t workspace_bytes, void* stream);
 
 /* Synchronises the context's device and reports W4A4_ERR_TIMEOUT if any kernel launched through this
- * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA. */
+ * context gave up on a bounded wait since the last query (the flag is cleared), else W4A4_OK / ERR_CUDA.
+ * The flag is sticky on the device: from the moment one CTA records a give-up, every other CTA of that kernel
+ * and every GEMM launched on the context afterwards leaves its pipeline at its next wait (within microseconds)
+ * and stores nothing more, so outputs enqueued between the failure and this query are undefined.  A caller
+ * that must trust an output queries the status after the work that produced it; a W4A4_ERR_TIMEOUT answer means
+ * "re-run everything enqueued since the last W4A4_OK".  The context stays usable after the query. */
 w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);
+
+/* Test hooks for the two failure paths that no healthy run reaches (no counterpart in the paper).
+ * w4a4_debug_wait_probe enqueues a one-warp kernel that waits, with the library's bounded wait, for an mbarrier
+ * phase nobody completes; it uses no copy engine, tensor core or tensor memory.  After limit_ns (1 .. 1e8, else
+ * W4A4_ERR_INVALID_ARG) the wait gives up and sets the context's device error word exactly as a stuck GEMM
+ * pipeline would: the next w4a4_query_status returns W4A4_ERR_TIMEOUT, the one after it W4A4_OK.
+ * w4a4_debug_fail_allocation_after(n) makes the (n + 1)-th device allocation that w4a4_ctx_create,
+ * w4a4_ctx_enable_host_io, w4a4_pack_weights, w4a4_mx_pack_weights or the clip-ratio searches attempt from now on
+ * fail once, as if cudaMalloc had refused it (the call then returns W4A4_ERR_ALLOC after releasing what it had
+ * allocated); n < 0 disarms.  Process-wide; not for use while other threads call the library. */
+w4a4_status_t w4a4_debug_wait_probe(w4a4_ctx_t ctx, uint64_t limit_ns, void* stream);
+void w4a4_debug_fail_allocation_after(int n);
 
 /* Bytes of device memory held by a handle / a context. */
 size_t w4a4_handle_bytes(w4a4_handle_t h);

@@ -39,6 +39,7 @@
 // "quantization disabled" reductions to a plain FP64 matrix product).  The paper prints no worked
 // numbers for this path, so nothing here is pinned against the authors' own code.
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -378,21 +379,28 @@ int oracle_mx_forward_rows(const uint16_t* X, const int* rows, int num_rows, int
   reciprocal_lambda(lambda, K, rl);
   std::vector<uint8_t> crow(static_cast<size_t>(K)), erow(static_cast<size_t>(B));
   std::vector<float> trow(static_cast<size_t>(r > 0 ? r : 1));
+  std::vector<double> yrow(static_cast<size_t>(N)), dot(static_cast<size_t>(N));
   for (int i = 0; i < num_rows; ++i) {
     const uint16_t* x = X + static_cast<size_t>(rows[i]) * K;
     mx_quantize_row(x, rl.data(), rho, K, crow.data(), erow.data());
     if (r > 0) lowrank_down_row(x, rl.data(), L1, K, r, trow.data());
-    for (int n = 0; n < N; ++n) {
-      double y = 0.0;
-      for (int b = 0; b < B; ++b) {
-        double dot = 0.0;  // multiples of 0.25, at most 32 * 36: exact
-        for (int j = 0; j < kMxBlock; ++j) {
-          const int k = b * kMxBlock + j;
-          dot += e2m1_value(crow[k]) * e2m1_value(wcodes[static_cast<size_t>(k) * N + n]);
-        }
-        y += dot * std::ldexp(1.0, static_cast<int>(erow[b]) - 127) *
-             std::ldexp(1.0, static_cast<int>(wexps[static_cast<size_t>(b) * N + n]) - 127);
+    // Every output channel n sums its blocks b in ascending order, and inside a block its 32 products in
+    // ascending k; the loops run with n innermost only so that the [K, N] weight arrays are read along rows.
+    std::fill(yrow.begin(), yrow.end(), 0.0);
+    for (int b = 0; b < B; ++b) {
+      std::fill(dot.begin(), dot.end(), 0.0);  // multiples of 0.25, at most 32 * 36: exact
+      for (int j = 0; j < kMxBlock; ++j) {
+        const int k = b * kMxBlock + j;
+        const double a = e2m1_value(crow[k]);
+        for (int n = 0; n < N; ++n) dot[n] += a * e2m1_value(wcodes[static_cast<size_t>(k) * N + n]);
       }
+      const double sa = std::ldexp(1.0, static_cast<int>(erow[b]) - 127);
+      for (int n = 0; n < N; ++n) {
+        yrow[n] += dot[n] * sa * std::ldexp(1.0, static_cast<int>(wexps[static_cast<size_t>(b) * N + n]) - 127);
+      }
+    }
+    for (int n = 0; n < N; ++n) {
+      double y = yrow[n];
       for (int j = 0; j < r; ++j) {
         y += static_cast<double>(trow[j]) * static_cast<double>(bf16_to_f32(L2[static_cast<size_t>(j) * N + n]));
       }

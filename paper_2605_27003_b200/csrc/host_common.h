@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/w4a4.h"
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -42,6 +44,19 @@ struct w4a4_ctx {
   cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
 };
 
+// Test hook for the allocation-failure paths (w4a4_debug_fail_allocation_after): a countdown over the device
+// allocations of the whole library, -1 when idle.  The allocation that finds it at 0 fails once, exactly as a refused
+// cudaMalloc would, and the hook disarms itself.  One definition, in w4a4_api.cu.
+extern std::atomic<int> g_w4a4_alloc_countdown;
+
+inline bool alloc_failure_injected() {
+  int c = g_w4a4_alloc_countdown.load(std::memory_order_relaxed);
+  while (c >= 0) {
+    if (g_w4a4_alloc_countdown.compare_exchange_weak(c, c - 1, std::memory_order_relaxed)) return c == 0;
+  }
+  return false;
+}
+
 namespace {
 
 struct DeviceGuard {
@@ -64,7 +79,7 @@ w4a4_status_t dev_alloc(T** p, size_t count, size_t* tally) {
   *p = nullptr;
   if (count == 0) return W4A4_OK;
   void* q = nullptr;
-  if (cudaMalloc(&q, count * sizeof(T)) != cudaSuccess) {
+  if (alloc_failure_injected() || cudaMalloc(&q, count * sizeof(T)) != cudaSuccess) {
     cudaGetLastError();
     return W4A4_ERR_ALLOC;
   }

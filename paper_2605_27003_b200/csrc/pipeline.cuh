@@ -160,4 +160,20 @@ __device__ __forceinline__ void drain_after_abort(volatile int* s_abort) {
   }
 }
 
+// Exercises the give-up path of bounded_wait without any pipeline around it: one warp waits for a phase of an
+// mbarrier that nobody ever completes.  No copy, tensor-core operation or TMEM allocation is involved, so there is
+// nothing to drain: after limit_ns the wait records kErrProbeWait in *err and the kernel returns normally.
+__global__ void wait_probe_kernel(int* err, uint64_t limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  const WaitEnv env{err, &s_abort, limit_ns};
+  bounded_wait<0, 9>(smem_u32(&bar), 0, env, kErrProbeWait);
+}
+
 }  // namespace w4a4

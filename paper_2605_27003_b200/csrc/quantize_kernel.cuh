@@ -48,13 +48,7 @@ constexpr int kCodesPacked = 0, kCodesE4M3 = 1, kCodesMxfp4 = 2;
 constexpr int kQuantRows = 16;      // token rows per CTA
 // Warps per CTA (16 rows each).  Small CTAs spread evenly over the 148 SMs; the widest rank shares its
 // larger L1 fragments among more warps.
-#ifndef QW
-#define QW 2
-#endif
-#ifndef QMINB
-#define QMINB 1
-#endif
-constexpr int quantize_warps(int R) { return R >= 64 ? 4 : QW; }
+constexpr int quantize_warps(int R) { return R >= 64 ? 4 : 2; }
 constexpr int kStages = 3;          // depth of the cp.async rings (groups in flight = kStages - 1)
 
 // Dynamic shared memory of quantize_kernel<R>: activation rings, smoothing-factor ring, L1 fragment ring.
@@ -215,7 +209,7 @@ __device__ __forceinline__ uint2 sop_slots_activation(float s) {
 }
 
 template <int R, int WARPS, int FORMAT>
-__global__ void __launch_bounds__(32 * WARPS, QMINB)
+__global__ void __launch_bounds__(32 * WARPS, 1)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
                 uint8_t* __restrict__ codes, float* __restrict__ scales, int scales_ld,

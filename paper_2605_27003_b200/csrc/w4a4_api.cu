@@ -262,6 +262,8 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
 }  // namespace
 
 // ------------------------------------------------------------------------------------ C ABI
+std::atomic<int> g_w4a4_alloc_countdown{-1};
+
 extern "C" {
 
 const char* w4a4_status_string(w4a4_status_t s) {
@@ -741,6 +743,17 @@ w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx) {
   }
   return W4A4_OK;
 }
+
+w4a4_status_t w4a4_debug_wait_probe(w4a4_ctx_t ctx, uint64_t limit_ns, void* stream) {
+  if (!ctx) return W4A4_ERR_INVALID_ARG;
+  if (limit_ns == 0 || limit_ns > 100000000ull) return W4A4_ERR_INVALID_ARG;  // at most 0.1 s
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+  wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_err, limit_ns);
+  return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+void w4a4_debug_fail_allocation_after(int n) { g_w4a4_alloc_countdown.store(n < 0 ? -1 : n); }
 
 }  // extern "C"
 

@@ -49,9 +49,25 @@ def oracle_rows(x_rows: torch.Tensor, layer, rho: float, want_partials=False):
         None if layer.bias is None else layer.bias.cpu().numpy(), want_partials=want_partials)
 
 
+GUARD = 3   # sentinel rows in front of and behind every output buffer of run_case
+
+
+def guarded(shape, dtype, sentinel):
+    """A tensor of `shape` cut out of a larger allocation whose GUARD leading and trailing rows hold `sentinel`."""
+    rows = shape[0]
+    buf = torch.full((rows + 2 * GUARD,) + tuple(shape[1:]), sentinel, dtype=dtype, device=DEV)
+    return buf, buf[GUARD:GUARD + rows]
+
+
+def guards_intact(buf, sentinel):
+    ref = torch.full_like(buf[:GUARD], sentinel)
+    return torch.equal(buf[:GUARD], ref) and torch.equal(buf[buf.shape[0] - GUARD:], ref)
+
+
 def run_case(x: torch.Tensor, experts, clip: torch.Tensor, expert_id: int, bin_id: int, rows=None,
              check_partials_tiles=(), layer_id=0, num_layers=1, max_M=None):
-    """Runs quantize tap + forward (+ partial taps) on the GPU and compares with the oracle on `rows`."""
+    """Runs quantize tap + forward (+ partial taps) on the GPU and compares with the oracle on `rows`.  Every output
+    buffer sits between sentinel guard rows that must come back untouched."""
     M, K = x.shape
     lay = experts[expert_id]
     N, r = lay.N, lay.r
@@ -60,17 +76,21 @@ def run_case(x: torch.Tensor, experts, clip: torch.Tensor, expert_id: int, bin_i
     clip_d = clip.to(DEV)
     rho = float(clip[expert_id, layer_id, bin_id])
     xd = x.to(DEV)
-    codes = torch.full((M, K), 99, dtype=torch.int8, device=DEV)
-    scales = torch.full((M, K // G), -1.0, dtype=torch.float32, device=DEV)
-    T = torch.zeros((M, max(r, 1)), dtype=torch.float32, device=DEV)
+    codes_buf, codes = guarded((M, K), torch.int8, 99)
+    scales_buf, scales = guarded((M, K // G), torch.float32, -1.0)
+    t_buf, T = guarded((M, max(r, 1)), torch.float32, -7.0)
+    y_buf, Y = guarded((M, N), torch.bfloat16, 1234.0)
     w4.w4a4_debug_quantize(L.ptr, xd, M, expert_id, bin_id, clip_d, codes, scales, T if r > 0 else None)
-    Y = L.forward(xd, expert_id, bin_id, clip_d)
+    w4.w4a4_linear_forward(L.ptr, xd, M, expert_id, bin_id, clip_d, Y)
     torch.cuda.synchronize()
     ctx.check()
+    assert guards_intact(codes_buf, 99) and guards_intact(scales_buf, -1.0) and guards_intact(t_buf, -7.0), \
+        "the quantize tap wrote outside its buffers"
+    assert guards_intact(y_buf, 1234.0), "the forward wrote outside Y"
     if rows is None:
         rows = np.arange(M)
     rows = np.asarray(rows)
-    ref = oracle_rows(x[rows], lay, rho, want_partials=bool(check_partials_tiles))
+    ref = oracle_rows(x[rows], lay, rho)
     rt = torch.from_numpy(rows).to(DEV)
     assert np.array_equal(codes[rt].cpu().numpy(), ref["q"]), "activation codes differ"
     assert np.array_equal(scales[rt].cpu().numpy().view(np.uint32), ref["s"].view(np.uint32)), "scales differ"
@@ -83,17 +103,21 @@ def run_case(x: torch.Tensor, experts, clip: torch.Tensor, expert_id: int, bin_i
     assert worst <= 1.0, f"output outside tolerance: worst err/bound = {worst:.3f} (rms {rms:.4g})"
     bm, bn = w4.w4a4_tile_shape()
     for (m0, n0) in check_partials_tiles:
-        P = torch.zeros((bm, K // G, bn), dtype=torch.int32, device=DEV)
-        Y2 = torch.empty_like(Y)
+        p_buf, P = guarded((bm, K // G, bn), torch.int32, -5)
+        y2_buf, Y2 = guarded((M, N), torch.bfloat16, 1234.0)
         w4.w4a4_debug_partials(L.ptr, xd, M, expert_id, bin_id, clip_d, Y2, m0, n0, P)
         torch.cuda.synchronize()
         ctx.check()
+        assert guards_intact(p_buf, -5) and guards_intact(y2_buf, 1234.0), "the partial-sum tap wrote outside its buffers"
         assert torch.equal(Y2, Y), "the debug-tap forward must give the same output"
-        sel = [(i, int(rw)) for i, rw in enumerate(rows) if m0 <= rw < min(m0 + bm, M)]
+        # The oracle's partial sums of the compared rows that fall into the tile (at most 12 of them: the array
+        # is [rows, G, N] int32).
+        sel = [int(rw) for rw in rows if m0 <= rw < min(m0 + bm, M)][:12]
         assert sel, "no compared row falls into the requested tile"
+        pref = oracle_rows(x[np.array(sel)], lay, rho, want_partials=True)["P"]
         Pg = P.cpu().numpy()
-        for i, rw in sel:
-            assert np.array_equal(Pg[rw - m0], ref["P"][i][:, n0:n0 + bn]), f"partials differ at row {rw}"
+        for i, rw in enumerate(sel):
+            assert np.array_equal(Pg[rw - m0], pref[i][:, n0:n0 + bn]), f"partials differ at row {rw}"
     L.close()
     ctx.close()
     return worst
@@ -180,6 +204,8 @@ def test_empty_batch_and_argument_errors():
 
 # ----------------------------------------------------------------------------- full-size workloads, sampled rows
 def sampled_rows(M, n_random, seed):
+    """The tile-boundary rows (first and last row, both sides of the first tile boundary and of the last one) plus
+    n_random seeded rows: rows are independent, so the oracle on a row subset is exact for those rows."""
     fixed = [0, 127, 128, M - 1, (M - 1) // 128 * 128, (M - 1) // 128 * 128 - 1]
     rng = np.random.default_rng(seed)
     rnd = rng.choice(M, size=n_random, replace=False).tolist()
@@ -202,7 +228,7 @@ def test_attention_projection_full_size_sampled_rows():
     for b in (0, 5):
         x = gen.make_activations(M, K, sigma=gen.sigma_for_bin(b), outlier_idx=idx, outlier_gain=50.0, seed=2002 + b,
                                  device=DEV).cpu()
-        rows = sampled_rows(M, 24, b)
+        rows = sampled_rows(M, 256, b)
         last = (M - 1) // 128 * 128
         run_case(x, [layer], clip, 0, b, rows=rows, check_partials_tiles=[(0, 0), (last, N - 128)])
 
@@ -218,7 +244,7 @@ def test_ffn_pair_full_size_sampled_rows():
     calib = gen.make_activations(1024, K, sigma=1.0, outlier_idx=idx, outlier_gain=50.0, seed=3000, device=DEV)
     up = big_layer(K, N, r, calib, 3001)
     x = gen.make_activations(M, K, sigma=1.0, outlier_idx=idx, outlier_gain=50.0, seed=3002, device=DEV).cpu()
-    rows = sampled_rows(M, 10, 31)
+    rows = sampled_rows(M, 256, 31)
     run_case(x, [up, up], clip, 1, 4, rows=rows, check_partials_tiles=[((M - 1) // 128 * 128, 0)])
     del x, up
     # down projection
@@ -235,7 +261,7 @@ def test_dit_step_layers_both_experts_sampled_rows():
     # the clip table): the step index picks expert (s >= 20) and bin s // 5; parity per distinct shape.
     M, r = 32760, 32
     clip = gen.make_clip_table(2, 4, 8, [(0.6, 1.0), (0.8, 1.0)], seed=4)
-    rows = sampled_rows(M, 6, 41)
+    rows = sampled_rows(M, 24, 41)
     for layer_id, (K, N, step) in enumerate(((5120, 5120, 3), (5120, 13824, 22), (13824, 5120, 39))):
         expert, b = (1 if step >= 20 else 0), step // 5
         experts = [gen.make_layer_direct(K, N, r, seed=4000 + 2 * layer_id + e, device=DEV).to("cpu") for e in range(2)]
@@ -247,17 +273,22 @@ def test_dit_step_layers_both_experts_sampled_rows():
         del x, experts
 
 
-@pytest.mark.parametrize("M,K,N,r,frac,alpha", [
-    (1560, 5120, 5120, 0, 0.0, 0.7),      # one latent frame, no low-rank branch, no outliers
-    (1560, 13824, 5120, 64, 0.05, 1.0),   # widest K, widest rank, 5% outlier channels
-    (75600, 5120, 13824, 16, 0.01, 0.7),  # the largest token count (21 x 45 x 80 grid)
-])
+SWEEP_POINTS = [(1560, K, N, r, frac, alpha)            # one latent frame: every (K, N, r) of the sweep
+                for (K, N) in ((5120, 5120), (5120, 13824), (13824, 5120))
+                for (r, frac, alpha) in ((0, 0.0, 0.7), (16, 0.01, 1.0), (32, 0.05, 0.7), (64, 0.01, 1.0))] + [
+    (32760, 5120, 5120, 64, 0.05, 1.0),    # the widest rank at the main token count
+    (75600, 5120, 13824, 16, 0.01, 0.7),   # the largest token count (21 x 45 x 80 grid)
+    (75600, 13824, 5120, 0, 0.0, 1.0),
+]
+
+
+@pytest.mark.parametrize("M,K,N,r,frac,alpha", SWEEP_POINTS)
 def test_sweep_points_sampled_rows(M, K, N, r, frac, alpha):
     layer = gen.make_layer_direct(K, N, r, seed=5000 + r + K // 64, device=DEV).to("cpu")
     x = gen.make_activations(M, K, outlier_idx=gen.outlier_channels(K, frac, 50), outlier_gain=50.0, seed=5100,
                              device=DEV).cpu()
     clip = torch.tensor([[[alpha]]], dtype=torch.float32)
-    run_case(x, [layer], clip, 0, 0, rows=sampled_rows(M, 6, 51), check_partials_tiles=[(0, 0)])
+    run_case(x, [layer], clip, 0, 0, rows=sampled_rows(M, 18, 51), check_partials_tiles=[(0, 0)])
 
 
 def test_host_buffer_forward_equals_device_forward():

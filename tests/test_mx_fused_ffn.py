@@ -48,6 +48,10 @@ def run_fused_case(M, K, H, N2, r1, r2, act, rho1, rho2, bias, seed=0):
     torch.cuda.synchronize()
     ctx.check()
     rows = np.arange(M).astype(np.int32)
+    # The oracle's second layer is fed the GPU's own first-layer output y1 here (itself checked against the oracle in
+    # test_mx_gpu_parity.py): codes and exponents are compared bit for bit, and a first-layer output that differs
+    # from the oracle's by one BF16 ulp -- which the layer's tolerance allows -- legitimately changes them.  The
+    # chain with no GPU intermediate is test_fused_ffn_against_the_oracle_only_chain below.
     ref = oracle.mx_forward_rows(bits(y1), rows, down.lam.numpy(), float(rho2),
                                  None if r2 == 0 else bits(down.L1), None if r2 == 0 else bits(down.L2),
                                  down.wcodes.numpy(), down.wexps.numpy(), None if down.bias is None else down.bias.numpy())
@@ -80,6 +84,58 @@ def run_fused_case(M, K, H, N2, r1, r2, act, rho1, rho2, bias, seed=0):
 ])
 def test_fused_ffn_matches_oracle(M, K, H, N2, r1, r2, act, bias):
     run_fused_case(M, K, H, N2, r1, r2, act, 0.9, 0.8, bias, seed=11 + M)
+
+
+def test_fused_ffn_against_the_oracle_only_chain():
+    """Oracle layer 1 -> GELU -> BF16 -> oracle layer 2, no GPU value anywhere in the expected result.  The GPU's
+    hidden activation may differ from the oracle's by a BF16 ulp where the layer tolerance allows it, and the second
+    layer's quantizer is not continuous, so the bound has two parts: the layer tolerance around the oracle-only
+    result, plus D = |oracle layer 2 on the GPU's hidden - oracle layer 2 on the oracle's hidden|, the oracle's own
+    sensitivity to that difference (both terms of D are CPU results; the GPU only supplies an input of one of them)."""
+    import paper_2605_27003_b200 as w4
+    M, K, H, N2, r1, r2, rho1, rho2 = 333, 512, 768, 256, 16, 32, 0.9, 0.8
+    idx = gen.outlier_channels(K, 0, 3, count=4)
+    x = gen.make_activations(M, K, outlier_idx=idx, outlier_gain=40.0, seed=3)
+    up = gen.make_layer_mx_svd(K, H, r1, x, seed=4, bias_std=0.01)
+    hid = gen.make_activations(M, H, outlier_idx=gen.outlier_channels(H, 0, 5, count=6), outlier_gain=20.0, seed=5)
+    down = gen.make_layer_mx_svd(H, N2, r2, hid, seed=6, bias_std=0.01)
+    rows = np.arange(M).astype(np.int32)
+
+    def second_layer(h_bits):
+        return oracle.mx_forward_rows(h_bits, rows, down.lam.numpy(), rho2, bits(down.L1), bits(down.L2), down.wcodes.numpy(),
+                                      down.wexps.numpy(), down.bias.numpy())["Y64"]
+
+    r1o = oracle.mx_forward_rows(bits(x), rows, up.lam.numpy(), rho1, bits(up.L1), bits(up.L2), up.wcodes.numpy(),
+                                 up.wexps.numpy(), up.bias.numpy())
+    h_or = torch.from_numpy(oracle.gelu_tanh(r1o["Y64"]).astype(np.float32)).to(torch.bfloat16)
+    y64_chain = second_layer(bits(h_or))
+
+    ctx = w4.Context(0, M, max(K, H), max(r1, r2))
+    clip = torch.full((1, 2, 1), rho1)
+    clip[0, 1, 0] = rho2
+    clip_d = clip.to(DEV)
+    Lup = w4.MxLayer(ctx, [up.to(DEV)], num_bins=1, num_layers=2, layer_id=0, output_activation=1)
+    Ldn = w4.MxLayer(ctx, [down.to(DEV)], num_bins=1, num_layers=2, layer_id=1)
+    xd = x.to(DEV)
+    h_gpu = Lup.forward(xd, 0, 0, clip_d)
+    y2 = torch.empty(M, N2, dtype=torch.bfloat16, device=DEV)
+    w4.w4a4_mx_ffn_forward(Lup.ptr, Ldn.ptr, xd, M, 0, 0, clip_d, y2)
+    torch.cuda.synchronize()
+    ctx.check()
+    # the hidden activations: equal on nearly every element, within the first layer's tolerance everywhere
+    g64 = oracle.gelu_tanh(r1o["Y64"])
+    tol1 = 1.13 * (2.0 ** -7 * np.abs(r1o["Y64"]) + 1e-3 * float(np.sqrt(np.mean(r1o["Y64"] ** 2)))) + 2.0 ** -8 * np.abs(g64)
+    assert np.all(np.abs(h_gpu.to(torch.float64).cpu().numpy() - g64) <= tol1)
+    assert (h_gpu.cpu() == h_or).float().mean().item() > 0.99
+    sens = np.abs(second_layer(bits(h_gpu)) - y64_chain)
+    rms = float(np.sqrt(np.mean(y64_chain ** 2)))
+    bound = 2.0 ** -7 * np.abs(y64_chain) + 1e-3 * rms + sens
+    worst = float(np.max(np.abs(y2.to(torch.float64).cpu().numpy() - y64_chain) / bound))
+    assert worst <= 1.0, f"fused output outside tolerance of the oracle-only chain: worst err/bound = {worst:.3f}"
+    assert float(np.sqrt(np.mean(sens ** 2))) < 0.02 * rms   # the sensitivity term stays a small correction
+    Lup.close()
+    Ldn.close()
+    ctx.close()
 
 
 def test_fused_ffn_many_tiles():

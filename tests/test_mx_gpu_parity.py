@@ -15,7 +15,7 @@ def bits(t):
 
 
 def y_within_tolerance(y_gpu_bf16, y64):
-    """spec tolerance: |Y_gpu - Y64| <= 2^-7 |Y64| + 1e-3 rms(Y64), rms over the compared outputs."""
+    """Output tolerance of the layer: |Y_gpu - Y64| <= 2^-7 |Y64| + 1e-3 rms(Y64), rms over the compared outputs."""
     yg = y_gpu_bf16.to(torch.float64).cpu().numpy()
     rms = float(np.sqrt(np.mean(y64 ** 2)))
     bound = 2.0 ** -7 * np.abs(y64) + 1e-3 * rms
@@ -123,13 +123,19 @@ def test_mx_argument_errors():
     ctx.close()
 
 
-def test_mx_full_size_attention_projection_sampled_rows():
-    shape = gen.CONFIG_SHAPES["attn_proj"]
+@pytest.mark.parametrize("name", ["attn_proj", "ffn_up", "ffn_down"])
+def test_mx_full_size_sampled_rows(name):
+    # The three layer shapes of the DiT at M = 32760: tile-boundary rows (the pair kernel's 256-row tiles included)
+    # plus 256 seeded random rows, all output columns.
+    shape = gen.CONFIG_SHAPES[name]
     M, K, N, r = shape["M"], shape["K"], shape["N"], shape["r"]
-    x = gen.make_activations(M, K, sigma=gen.sigma_for_bin(2), outlier_idx=gen.outlier_channels(K, 0.01, 7),
-                             outlier_gain=50.0, seed=31, device=DEV).cpu()
+    dist = "gelu" if name == "ffn_down" else "normal"
+    x = gen.make_activations(M, K, sigma=1.0 if dist == "gelu" else gen.sigma_for_bin(2), dist=dist,
+                             outlier_idx=gen.outlier_channels(K, 0.01, 7), outlier_gain=80.0 if dist == "gelu" else 50.0,
+                             seed=31, device=DEV).cpu()
     layer = gen.make_layer_mx_direct(K, N, r, seed=32)
     rng = np.random.default_rng(1)
-    rows = sorted({0, 127, 128, M - 1, (M - 1) // 128 * 128, *rng.integers(0, M, 3).tolist()})
+    last = (M - 1) // 128 * 128
+    rows = sorted({0, 127, 128, 255, 256, last - 1, last, M - 1, *rng.choice(M, 256, replace=False).tolist()})
     clip = gen.make_clip_table(1, 1, 8, [(0.6, 1.0)], seed=6)
     run_mx_case(x, [layer], clip, 0, 2, rows=rows)
