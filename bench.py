@@ -35,7 +35,7 @@ NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_HBM_GBS = 7700.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, each from one single-launch ncu capture of the kernel as
 # it stands (summaries under profiles/); None where no capture exists for that kernel and workload.
-NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): None, ("quantize", "attn_proj"): 502.0e6}
+NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 537.9e6, ("quantize", "attn_proj"): 503.3e6}
 
 
 def max_over_ranks(ms: float, dist, device="cpu") -> float:
@@ -130,7 +130,7 @@ def tensor_roofline(gemm_tops: float, timed_seconds: float, peaks: dict, tp: dic
         burst, sustained, src = tp["fp8_tops_burst"], tp["fp8_tops_sustained"], "library FP8 GEMM 8192^3 measured in this run"
     else:
         burst, sustained = 2.0 * peaks["bf16_burst"], 2.0 * peaks["bf16_sustained"]
-        src = f"{peaks['source']} BF16 figures x 2 (nominal 8-bit : BF16 ratio; no 8-bit library GEMM could be timed)"
+        src = f"{peaks['source']} BF16 figures x 2 (nominal 8-bit : BF16 ratio; no 8-bit library GEMM was timed in this run)"
     nominal = NOMINAL_INT8_TOPS
     if fp4:
         burst, sustained, nominal, src = 2.0 * burst, 2.0 * sustained, 2.0 * NOMINAL_INT8_TOPS, src + ", x 2 (nominal FP4 : 8-bit ratio)"
