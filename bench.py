@@ -52,9 +52,14 @@ def whole_job_tops(ops_per_step_per_rank: float, world: int, ms_per_step: float)
     return world * ops_per_step_per_rank / (ms_per_step * 1e-3) / 1e12
 
 
-def dit_step_layers(blocks: int = 40):
-    """(K, N) of the quantized linears of one denoising step: per block q, k, v, o, cross q, cross o, ffn up, ffn down."""
-    per_block = [(5120, 5120)] * 6 + [(5120, 13824), (13824, 5120)]
+def dit_step_layers(blocks: int = 40, qkv_packed: bool = False):
+    """(K, N, r) of the quantized linears of one denoising step: per block q, k, v, o, cross q, cross o, ffn up,
+    ffn down at r = 32.  With qkv_packed the self-attention q, k and v (one input, one smoothing vector, one clip entry)
+    are one layer 5120 -> 15360 of joint rank 96 whose L2 is block-diagonal: one activation pass instead of three."""
+    if qkv_packed:
+        per_block = [(5120, 15360, 96)] + [(5120, 5120, 32)] * 3 + [(5120, 13824, 32), (13824, 5120, 32)]
+    else:
+        per_block = [(5120, 5120, 32)] * 6 + [(5120, 13824, 32), (13824, 5120, 32)]
     return per_block * blocks
 
 
@@ -327,17 +332,23 @@ def time_layer(w4, layer, xs, bins, expert, clip, Y, M, iters, warmup, stream):
     return (statistics.mean(e[0].elapsed_time(e[1]) for e in ev), statistics.mean(e[1].elapsed_time(e[2]) for e in ev))
 
 
-def measure_dit_step(w4, dev, local_rank, steps, warmup, blocks, dist=None):
+def measure_dit_step(w4, dev, local_rank, steps, warmup, blocks, dist=None, qkv_packed=False):
     """One denoising step's quantized linears of a `blocks`-block, 5120-hidden DiT at M = 32760, r = 32, with both
     experts' weight sets resident; step s uses expert (s >= 20) and timestep bin s // 5 (40-step schedule).
     Returns this rank's device time per step and what the step holds."""
     M, r, bins, experts = 32760, 32, 8, 2
-    shapes = dit_step_layers(blocks)
+    shapes = dit_step_layers(blocks, qkv_packed)
     L = len(shapes)
-    ctx = w4.Context(local_rank, M, 13824, r)
+    ctx = w4.Context(local_rank, M, 13824, 96 if qkv_packed else r)
     layers = []
-    for li, (K, N) in enumerate(shapes):
-        ex = [gen.make_layer_direct(K, N, r, seed=4000 + 2 * li + e, device=dev) for e in range(experts)]
+    for li, (K, N, rl) in enumerate(shapes):
+        ex = [gen.make_layer_direct(K, N, rl, seed=4000 + 2 * li + e, device=dev) for e in range(experts)]
+        if rl == 96:  # three projections side by side: each reads only its own 32 columns of T
+            for lay in ex:
+                for i in range(3):
+                    for j in range(3):
+                        if i != j:
+                            lay.L2[32 * i:32 * (i + 1), 5120 * j:5120 * (j + 1)] = 0
         layers.append(w4.Layer(ctx, ex, num_bins=bins, num_layers=L, layer_id=li))
         del ex
     weight_bytes = sum(w4.w4a4_handle_bytes(l.ptr) for l in layers)
@@ -347,12 +358,12 @@ def measure_dit_step(w4, dev, local_rank, steps, warmup, blocks, dist=None):
                                       device=dev) for i in range(3)],
           13824: [gen.make_activations(M, 13824, dist="gelu", outlier_idx=idx[13824], outlier_gain=80.0, seed=4200 + i,
                                        device=dev) for i in range(3)]}
-    Y = {n: torch.empty(M, n, dtype=torch.bfloat16, device=dev) for n in (5120, 13824)}
+    Y = {n: torch.empty(M, n, dtype=torch.bfloat16, device=dev) for n in (5120, 13824, 15360)[:3 if qkv_packed else 2]}
     stream = torch.cuda.current_stream()
 
     def step(s):
         expert, b = (1 if (s % 40) >= 20 else 0), (s % 40) // 5
-        for li, (K, N) in enumerate(shapes):
+        for li, (K, N, _) in enumerate(shapes):
             w4.w4a4_linear_forward(layers[li].ptr, xs[K][(s + li) % 3], M, expert, b, clip, Y[N], stream)
 
     def barrier():
@@ -381,12 +392,12 @@ def measure_dit_step(w4, dev, local_rank, steps, warmup, blocks, dist=None):
     ctx.close()
     del xs, Y
     torch.cuda.empty_cache()
-    return dict(total_ms=total_ms, ops=sum(2.0 * M * K * N for (K, N) in shapes), M=M, r=r, experts=experts, bins=bins,
-                linears=L, weight_bytes=weight_bytes, clocks=clocks)
+    return dict(total_ms=total_ms, ops=sum(2.0 * M * K * N for (K, N, _) in shapes), M=M, r=r, experts=experts, bins=bins,
+                linears=L, weight_bytes=weight_bytes, clocks=clocks, qkv_packed=qkv_packed)
 
 
 def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks, tp):
-    d = measure_dit_step(w4, dev, local_rank, args.steps, args.warmup, args.blocks, dist)
+    d = measure_dit_step(w4, dev, local_rank, args.steps, args.warmup, args.blocks, dist, args.qkv_packed)
     total_ms = max_over_ranks(d["total_ms"], dist, dev)
     ms_per_step = total_ms / args.steps
     if rank == 0:
@@ -397,6 +408,7 @@ def run_dit_step(args, w4, dev, local_rank, rank, world, dist, peaks, tp):
                     ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="e4m3",
                     data="synthetic",
                     config=dict(workload="dit_step", M=d["M"], r=d["r"], group=64, blocks=args.blocks, linears=d["linears"],
+                                qkv="one packed layer 5120 -> 15360, joint rank 96" if d["qkv_packed"] else "three layers",
                                 experts=d["experts"], bins=d["bins"], resident_weight_gb=d["weight_bytes"] / 1e9,
                                 tera_ops_per_step=d["ops"] / 1e12,
                                 l2="inputs larger than L2: 3 rotating activation buffers per shape (335 / 906 MB)",
@@ -772,6 +784,8 @@ def main():
                                                             "mxfp4_ffn_down", "mxfp4_ffn", "gptq", "gptq_mx", "gptq_ffn_up", "gptq_ffn_down"])
     ap.add_argument("--chunk-rows", type=int, default=4096, help="token rows per chunk of the host-buffer forward (e2e)")
     ap.add_argument("--blocks", type=int, default=40, help="DiT blocks for --workload dit_step")
+    ap.add_argument("--qkv-packed", action="store_true",
+                    help="dit_step: self-attention q, k, v as one layer packed along N (one activation pass for the three)")
     ap.add_argument("--out", default=None, help="file for the per-point table of --workload sweep")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -61,7 +61,7 @@ typedef struct w4a4_layer* w4a4_handle_t; /* one layer position: packed constant
 typedef struct {
   int K;           /* input channels C_in, multiple of 64 */
   int N;           /* output channels C_out, multiple of 128 */
-  int r;           /* low-rank width: 0, 16, 32 or 64 */
+  int r;           /* low-rank width: 0, 16, 32, 64 or 96 (96: three rank-32 projections packed along N) */
   int group;       /* quantization group along K: must be 64 */
   int num_experts; /* >= 1 */
   int num_bins;    /* timestep bins per (expert, layer) in the clip table */

@@ -84,14 +84,11 @@ __device__ __forceinline__ uint4 ldg_stream_v4(const void* p) {
 
 // Smooth 8 BF16 values (one 16-byte load) with 8 reciprocals.
 __device__ __forceinline__ void smooth8(const uint4& raw, const float4& r0, const float4& r1, float* xh) {
-  xh[0] = __fmul_rn(__uint_as_float(raw.x << 16), r0.x);
-  xh[1] = __fmul_rn(__uint_as_float(raw.x & 0xffff0000u), r0.y);
-  xh[2] = __fmul_rn(__uint_as_float(raw.y << 16), r0.z);
-  xh[3] = __fmul_rn(__uint_as_float(raw.y & 0xffff0000u), r0.w);
-  xh[4] = __fmul_rn(__uint_as_float(raw.z << 16), r1.x);
-  xh[5] = __fmul_rn(__uint_as_float(raw.z & 0xffff0000u), r1.y);
-  xh[6] = __fmul_rn(__uint_as_float(raw.w << 16), r1.z);
-  xh[7] = __fmul_rn(__uint_as_float(raw.w & 0xffff0000u), r1.w);
+  const float2 a = __fmul2_rn(make_float2(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u)), make_float2(r0.x, r0.y));
+  const float2 b = __fmul2_rn(make_float2(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u)), make_float2(r0.z, r0.w));
+  const float2 c = __fmul2_rn(make_float2(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xffff0000u)), make_float2(r1.x, r1.y));
+  const float2 d = __fmul2_rn(make_float2(__uint_as_float(raw.w << 16), __uint_as_float(raw.w & 0xffff0000u)), make_float2(r1.z, r1.w));
+  xh[0] = a.x; xh[1] = a.y; xh[2] = b.x; xh[3] = b.y; xh[4] = c.x; xh[5] = c.y; xh[6] = d.x; xh[7] = d.y;
 }
 
 // Group absolute maximum of the lane's 16 smoothed values, combined over the quad (= 64 channels).
@@ -131,16 +128,28 @@ __device__ __forceinline__ void quantize16_offset(const float* xh, float is, uin
 // Quantize the lane's 16 values and return them as E4M3 bytes: .x/.y = elements 0..7 (channels coff .. +7),
 // .z/.w = elements 8..15 (channels coff + 16 .. +23).
 __device__ __forceinline__ uint4 quantize16_bytes(const float* xh, float is) {
-  uint32_t u[16];
-  quantize16_offset(xh, is, u);
-  uint32_t n0 = u[0], n1 = u[8];  // eight nibbles each, element e in nibble e % 8
+  // Eq. 3: z = xh * is rounded to FP32, then to the nearest integer with ties to even (cvt.rni), then clamped to
+  // [-8, 7]: cvt.pack.sat.s4 saturates two integers to 4 bits and shifts them in under the nibbles packed so far,
+  // so the eight codes of a word take four instructions, element 0 in the lowest nibble.
+  uint32_t n[2];
 #pragma unroll
-  for (int e = 1; e < 8; ++e) {
-    n0 += u[e] << (4 * e);
-    n1 += u[8 + e] << (4 * e);
+  for (int hh = 0; hh < 2; ++hh) {
+    int v[8];
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+      const float2 z = __fmul2_rn(make_float2(xh[8 * hh + e], xh[8 * hh + e + 1]), make_float2(is, is));
+      v[e] = __float2int_rn(z.x);
+      v[e + 1] = __float2int_rn(z.y);
+    }
+    uint32_t w;
+    asm("cvt.pack.sat.s4.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v[7]), "r"(v[6]), "r"(0));
+    asm("cvt.pack.sat.s4.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v[5]), "r"(v[4]), "r"(w));
+    asm("cvt.pack.sat.s4.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v[3]), "r"(v[2]), "r"(w));
+    asm("cvt.pack.sat.s4.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(v[1]), "r"(v[0]), "r"(w));
+    n[hh] = w ^ 0x88888888u;   // two's complement nibbles -> code + 8, the index the byte lookup takes
   }
-  return make_uint4(e4m3_of_offset_nibbles4(n0), e4m3_of_offset_nibbles4(n0 >> 16), e4m3_of_offset_nibbles4(n1),
-                    e4m3_of_offset_nibbles4(n1 >> 16));
+  return make_uint4(e4m3_of_offset_nibbles4(n[0]), e4m3_of_offset_nibbles4(n[0] >> 16), e4m3_of_offset_nibbles4(n[1]),
+                    e4m3_of_offset_nibbles4(n[1] >> 16));
 }
 
 // Quantize the lane's 16 smoothed values of one row (Eq. 3) and return its two packed words.

@@ -192,6 +192,7 @@ w4a4_status_t launch_quantize_at(w4a4_handle_t h, const void* X, int M, int expe
     case 16: W4A4_LAUNCH_Q(16); break;
     case 32: W4A4_LAUNCH_Q(32); break;
     case 64: W4A4_LAUNCH_Q(64); break;
+    case 96: W4A4_LAUNCH_Q(96); break;
     default: return W4A4_ERR_SHAPE;
   }
 #undef W4A4_LAUNCH_Q
@@ -287,7 +288,7 @@ void w4a4_tile_shape(int* tile_m, int* tile_n) {
 w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_ctx_t* out) {
   if (!out) return W4A4_ERR_INVALID_ARG;
   *out = nullptr;
-  if (max_M <= 0 || max_K <= 0 || max_K % 64 != 0 || max_r < 0 || max_r > 64) return W4A4_ERR_SHAPE;
+  if (max_M <= 0 || max_K <= 0 || max_K % 64 != 0 || max_r < 0 || max_r > 96) return W4A4_ERR_SHAPE;
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
     cudaGetLastError();
@@ -337,6 +338,8 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   if (st == W4A4_OK) {
     cudaFuncSetAttribute(quantize_kernel<64, quantize_warps(64), kCodesE4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          static_cast<int>(quantize_smem_bytes(64)));
+    cudaFuncSetAttribute(quantize_kernel<96, quantize_warps(96), kCodesE4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         static_cast<int>(quantize_smem_bytes(96)));
     const cudaError_t e1 = cudaFuncSetAttribute(gemm_w4a4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     const cudaError_t e2 = cudaFuncSetAttribute(gemm_w4a4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmemBytes);
     if (e1 != cudaSuccess || e2 != cudaSuccess) {
@@ -399,7 +402,7 @@ w4a4_status_t w4a4_pack_weights(w4a4_ctx_t ctx, const w4a4_weight_desc_t* d, w4a
   *out = nullptr;
   if (!ctx || !d) return W4A4_ERR_INVALID_ARG;
   if (d->group != 64 || d->K <= 0 || d->K % 64 != 0 || d->N <= 0 || d->N % kBN != 0) return W4A4_ERR_SHAPE;
-  if (!(d->r == 0 || d->r == 16 || d->r == 32 || d->r == 64)) return W4A4_ERR_SHAPE;
+  if (!(d->r == 0 || d->r == 16 || d->r == 32 || d->r == 64 || d->r == 96)) return W4A4_ERR_SHAPE;
   if (d->K > ctx->max_K || d->r > ctx->max_r) return W4A4_ERR_SHAPE;
   if (d->num_experts < 1 || d->num_bins < 1 || d->num_layers < 1 || d->layer_id < 0 || d->layer_id >= d->num_layers)
     return W4A4_ERR_INVALID_ARG;

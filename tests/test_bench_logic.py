@@ -50,9 +50,13 @@ def test_replica_aggregation_over_two_gloo_ranks():
 def test_dit_step_layer_list_matches_the_workload_definition():
     shapes = bench.dit_step_layers(40)
     assert len(shapes) == 320
-    assert shapes.count((5120, 5120)) == 240 and shapes.count((5120, 13824)) == 40 and shapes.count((13824, 5120)) == 40
-    tera_ops = sum(2.0 * 32760 * k * n for k, n in shapes) / 1e12
+    assert shapes.count((5120, 5120, 32)) == 240 and shapes.count((5120, 13824, 32)) == 40 and \
+        shapes.count((13824, 5120, 32)) == 40
+    tera_ops = sum(2.0 * 32760 * k * n for k, n, _ in shapes) / 1e12
     assert abs(tera_ops - 783.2) < 0.5              # the per-step operation count quoted for this workload
+    packed = bench.dit_step_layers(40, qkv_packed=True)   # q, k, v as one layer: same operations, 80 fewer layers
+    assert len(packed) == 240 and packed.count((5120, 15360, 96)) == 40
+    assert sum(k * n for k, n, _ in packed) == sum(k * n for k, n, _ in shapes)
 
 
 def test_reference_arm_prints_one_contract_line_on_the_tiny_workload():

@@ -314,33 +314,40 @@ def test_host_buffer_forward_equals_device_forward():
     ctx.close()
 
 
-def test_qkv_packed_as_one_layer_shares_one_activation_pass():
+@pytest.mark.parametrize("M,K,N,r", [(300, 512, 256, 16), (391, 1024, 384, 32)])
+def test_qkv_packed_as_one_layer_shares_one_activation_pass(M, K, N, r):
     # q, k and v read the same input with the same smoothing vector and the same clipping-ratio entry, so their
     # activation quantization and low-rank down-projection can be done once: pack the three projections as ONE layer
-    # along N (codes, scales and bias side by side; L1 side by side, L2 block-diagonal, joint rank <= 64).  The packed
-    # layer must give what the three layers give (same codes and scales by construction; the output within the
-    # layer's tolerance, because the low-rank sum now runs over 64 instead of 16 terms, most of them exact zeros),
-    # and what the oracle gives for the packed constants.
-    M, K, N, r = 300, 512, 256, 16
+    # along N (codes, scales and bias side by side; L1 side by side, L2 block-diagonal; joint rank 3 r, padded to 64
+    # at r = 16 and 96 at the rank the DiT workload uses).  The packed layer must give what the three layers give
+    # (same codes and scales by construction; the output within the layer's tolerance, because the low-rank sum now
+    # runs over 3 r terms, two thirds of them exact zeros), and what the oracle gives for the packed constants.
+    R = 64 if r == 16 else 3 * r
     idx = gen.outlier_channels(K, 0, 5, count=4)
     x = gen.make_activations(M, K, outlier_idx=idx, outlier_gain=40.0, seed=5)
     parts = [gen.make_layer_svd(K, N, r, x, seed=50 + i, bias_std=0.01) for i in range(3)]
     lam = parts[0].lam
     for p_ in parts:                               # one smoothing vector for the three projections
         p_.lam = lam
-    L1 = torch.zeros((K, 64), dtype=torch.bfloat16)
-    L2 = torch.zeros((64, 3 * N), dtype=torch.bfloat16)
+    L1 = torch.zeros((K, R), dtype=torch.bfloat16)
+    L2 = torch.zeros((R, 3 * N), dtype=torch.bfloat16)
     for i, p_ in enumerate(parts):
         L1[:, r * i:r * (i + 1)] = p_.L1
         L2[r * i:r * (i + 1), N * i:N * (i + 1)] = p_.L2
-    packed = gen.LayerInputs(K, 3 * N, 64, lam, L1, L2, torch.cat([p_.qweight for p_ in parts], dim=1),
+    packed = gen.LayerInputs(K, 3 * N, R, lam, L1, L2, torch.cat([p_.qweight for p_ in parts], dim=1),
                              torch.cat([p_.wscale for p_ in parts], dim=1), torch.cat([p_.bias for p_ in parts]))
     clip = torch.full((1, 1, 2), 0.85)
-    ctx = w4.Context(0, M, K, 64)
+    ctx = w4.Context(0, M, K, R)
     clip_d, xd = clip.to(DEV), x.to(DEV)
     Lp = w4.Layer(ctx, [packed.to(DEV)], num_bins=2)
     Yp = Lp.forward(xd, 0, 1, clip_d).float().cpu().numpy()
     ctx.check()
+    # the joint down-projection against the oracle's, column block by column block
+    codes = torch.empty((M, K), dtype=torch.int8, device=DEV)
+    scales = torch.empty((M, K // G), dtype=torch.float32, device=DEV)
+    T = torch.empty((M, R), dtype=torch.float32, device=DEV)
+    w4.w4a4_debug_quantize(Lp.ptr, xd, M, 0, 1, clip_d, codes, scales, T)
+    torch.cuda.synchronize()
     Lp.close()
     ys = []
     for p_ in parts:
@@ -351,6 +358,10 @@ def test_qkv_packed_as_one_layer_shares_one_activation_pass():
     ctx.close()
     Ys = np.concatenate(ys, axis=1)
     ref = oracle_rows(x, packed, 0.85)
+    assert np.array_equal(codes.cpu().numpy(), ref["q"]) and \
+        np.array_equal(scales.cpu().numpy().view(np.uint32), ref["s"].view(np.uint32))
+    t_ref = ref["T"].astype(np.float64)
+    assert np.all(np.abs(T.cpu().numpy() - t_ref) <= 1e-4 * np.abs(t_ref).max(axis=1, keepdims=True) + 1e-30)
     Y64 = ref["Y64"]
     bound = 2.0 ** -7 * np.abs(Y64) + 1e-3 * np.sqrt(np.mean(Y64 ** 2))
     assert np.all(np.abs(Yp - Y64) <= bound) and np.all(np.abs(Ys - Y64) <= bound)
