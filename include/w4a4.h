@@ -180,8 +180,8 @@ w4a4_status_t w4a4_quantize_noalloc(const void* X, int M, int K, const float* la
                                     int clip_index, int8_t* codes, float* scales, void* stream);
 
 /* ---- MXFP4 variant of the same layer -------------------------------------------------------------------------
- * The caption of the paper's Table 1 states that all its 4-bit runs use the MXFP4 data format, and Sec. IV-D asks
- * for "native FP4/MXFP4 tensor operations".  This variant computes Eq. 11 with both 4-bit operands in MXFP4 as
+ * The caption of the paper's Table 1 states that all its 4-bit runs use the MXFP4 data format, and Sec. IV-D names
+ * the hardware's own 4-bit floating-point tensor path as the way forward.  This variant computes Eq. 11 with both 4-bit operands in MXFP4 as
  * the OCP Microscaling Formats specification v1.0 defines it: E2M1 elements (+-{0, 0.5, 1, 1.5, 2, 3, 4, 6}), one
  * E8M0 scale (a byte e, value 2^(e-127)) per block of 32 consecutive input channels, conversion by shared exponent
  * floor(log2(block maximum)) - 2 and round-to-nearest-even with saturation.  The clipping ratio of Eq. 8-9 scales the

@@ -300,8 +300,8 @@ def gptq_quantize(R, H, group=64, percdamp=0.01):
     matching entry of U = chol(H^-1, upper), is spread over the input channels still to come.  Readings where the
     papers leave a choice: INT4 grid and group scale exactly as the round-to-nearest quantizer (scale = FP32(max
     |w| / 7) over the group's 64 input channels, code = round-half-even(w / scale) clamped to [-8, 7], zero group ->
-    scale 0, codes 0), the scale being taken from the error-compensated weights when the sweep enters the group (static
-    groups, no activation ordering); dead input channels (H_kk = 0) get H_kk = 1 and zero weights; damping percdamp *
+    scale 0, codes 0), the scale being taken from the error-compensated weights when the sweep enters the group (not
+    fixed from the original weights beforehand), input channels in natural order (no activation ordering); dead input channels (H_kk = 0) get H_kk = 1 and zero weights; damping percdamp *
     mean(diag H) on the diagonal; the lazy-batch block equals the group (pure bookkeeping: the result does not depend
     on it).  -> codes int8 [K, N], scales FP32 [K / group, N]."""
     W = np.array(R, dtype=np.float64, copy=True)

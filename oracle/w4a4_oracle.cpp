@@ -28,7 +28,7 @@
 // rho is the clipping ratio fetched from the (expert, layer, timestep-bin) table (Sec. III-C); the
 // reference magnitude m_{l,k} of Eq. 8 is taken dynamically as the group's absolute maximum.
 //
-// Readings where the paper is silent are listed in the repository's design notes; in short: INT4
+// Readings where the paper is silent: INT4
 // two's complement codes, q_max = 7 for the scale and [-8, 7] for the clip, ties to even, group 64,
 // multiplication by a reciprocal in place of the division inside Eq. 3, bias added at the end.
 //
@@ -271,7 +271,7 @@ uint16_t oracle_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
 
 // =====================================================================================================
 // MXFP4 variant of the same layer (the data format the paper's Table 1 says its 4-bit runs used, and the
-// "native FP4/MXFP4 tensor operations" its Sec. IV-D asks for).  Element and scale formats and the
+// hardware 4-bit floating-point path that Sec. IV-D names as the way forward).  Element and scale formats and the
 // conversion rule are those of the OCP Microscaling Formats (MX) specification v1.0:
 //
 //   block          32 consecutive input channels of one token (activations) / of one output column (weights)

@@ -76,7 +76,7 @@ struct MxGemmParams {
 // One lane of a converged warp.  The MMA warp runs its loop with all lanes (waits included) and only predicates
 // the tcgen05 instructions on this: everything they take as operands then stays warp-uniform for the compiler,
 // which keeps descriptors and addresses in uniform registers instead of converting them per instruction
-// (elect_one_lane() comes from gemm_kernel.cuh).
+// (elect_one_lane() comes from pipeline.cuh).
 
 // Shared-memory descriptor of one scale atom (32 rows x 16 bytes, rows contiguous): K-major, no swizzle, 8-row
 // core matrices 128 bytes apart.
