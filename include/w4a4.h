@@ -311,8 +311,16 @@ w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);
  * w4a4_debug_fail_allocation_after(n) makes the (n + 1)-th device allocation that w4a4_ctx_create,
  * w4a4_ctx_enable_host_io, w4a4_pack_weights, w4a4_mx_pack_weights or the clip-ratio searches attempt from now on
  * fail once, as if cudaMalloc had refused it (the call then returns W4A4_ERR_ALLOC after releasing what it had
- * allocated); n < 0 disarms.  Process-wide; not for use while other threads call the library. */
+ * allocated); n < 0 disarms.  Process-wide; not for use while other threads call the library.
+ * w4a4_debug_stalled_gemm runs the GEMM of w4a4_gemm_from_workspace (its parity-tap instantiation) on whatever the
+ * workspace holds, with the wait limit set to limit_ns (1 .. 1e8) and with one operand stage (number stall_stage >= 0
+ * of every CTA's sequence) never loaded: the consumers of that stage run into the limit, every role of the CTA
+ * leaves through the kernel's common tail (error word, a drain period for copies in flight, release of tensor
+ * memory), and Y is left partly written.  The next w4a4_query_status returns W4A4_ERR_TIMEOUT, and the context must
+ * compute correctly afterwards.  Nothing faults or traps. */
 w4a4_status_t w4a4_debug_wait_probe(w4a4_ctx_t ctx, uint64_t limit_ns, void* stream);
+w4a4_status_t w4a4_debug_stalled_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, int stall_stage,
+                                      uint64_t limit_ns, void* stream);
 void w4a4_debug_fail_allocation_after(int n);
 
 /* Bytes of device memory held by a handle / a context. */

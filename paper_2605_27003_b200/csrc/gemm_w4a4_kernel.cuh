@@ -190,12 +190,21 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const bool issuer = elect_one_lane();
       Ring<kGemmStages> op;
       bool ok = true;
+      int stage_no = 0;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
         const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
         const int m0 = tm * kBM, n0 = tn * kBN;
         for (int st = 0; st < n_lr_stages + n_int_stages; ++st) {
           ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_op_empty + 8 * op.slot, op.parity ^ 1u, env, kErrProducerWait));
           if (!ok) break;
+          if (DEBUG) {
+            // Test hook: one stage is never loaded, so its consumers' waits run into their limit and every role of
+            // the CTA leaves through the common tail (error word, drain, TMEM release).
+            if (stage_no++ == p.dbg_stall_stage) {
+              op.advance();
+              continue;
+            }
+          }
           const uint32_t full = bar_op_full + 8 * op.slot;
           const uint32_t dst = smem_base + op.slot * kStageBytes;
           if (st < n_lr_stages) {

@@ -130,6 +130,7 @@ struct GemmParams {
   uint64_t wait_limit_ns;
   int32_t* dbg_P;       // debug tap: [kBM, G, kBN] or nullptr
   int dbg_m0, dbg_n0;
+  int dbg_stall_stage;  // test hook of the tap instantiation: every CTA's producer skips its stage of this number (-1: none)
   // Clip-ratio search (Eq. 10): when yref is set, Y is not stored; the squared distance between the layer's
   // BF16 output and yref is accumulated into *sq_err instead.
   const uint16_t* yref; // [M, N] BF16 or nullptr

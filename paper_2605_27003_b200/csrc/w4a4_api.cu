@@ -213,7 +213,7 @@ w4a4_status_t launch_quantize(w4a4_handle_t h, const void* X, int M, int expert_
 // *sq_err instead of storing Y.
 w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaStream_t stream, int32_t* dbg_P,
                           int dbg_m0, int dbg_n0, const void* yref = nullptr, double* sq_err = nullptr,
-                          bool expand = true) {
+                          bool expand = true, int stall_stage = -1, uint64_t wait_limit_ns = kWaitLimitNs) {
   if (M == 0) return W4A4_OK;
   w4a4_ctx* ctx = h->ctx;
   const ExpertData& e = h->experts[expert_id];
@@ -227,7 +227,8 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   p.tiles_m = (M + kBM - 1) / kBM;
   p.tiles_n = h->N / kBN;
   p.err = ctx->d_err;
-  p.wait_limit_ns = kWaitLimitNs;
+  p.wait_limit_ns = wait_limit_ns;
+  p.dbg_stall_stage = stall_stage;
   p.dbg_P = dbg_P;
   p.dbg_m0 = dbg_m0;
   p.dbg_n0 = dbg_n0;
@@ -251,7 +252,7 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   const dim3 grid(num_tiles < ctx->num_sms ? num_tiles : ctx->num_sms), block(kGemmThreads);
   const CUtensorMap& tmT = h->r > 0 ? h->tmT : h->tmA;   // unused when r == 0
   const CUtensorMap& tmL2 = h->r > 0 ? e.tmL2 : h->tmB;
-  if (dbg_P) {
+  if (dbg_P || stall_stage >= 0) {
     gemm_w4a4_kernel<true><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, h->tmSopA, e.tmSopB, p);
   } else {
     gemm_w4a4_kernel<false><<<grid, block, kGemmSmemBytes, stream>>>(h->tmA, h->tmB, tmT, tmL2, h->tmSopA, e.tmSopB, p);
@@ -754,6 +755,18 @@ w4a4_status_t w4a4_debug_wait_probe(w4a4_ctx_t ctx, uint64_t limit_ns, void* str
   if (!guard.ok) return W4A4_ERR_CUDA;
   wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_err, limit_ns);
   return cudaGetLastError() == cudaSuccess ? W4A4_OK : W4A4_ERR_CUDA;
+}
+
+w4a4_status_t w4a4_debug_stalled_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, int stall_stage,
+                                      uint64_t limit_ns, void* stream) {
+  w4a4_status_t st = check_forward_args(h, nullptr, M, expert_id, 0, nullptr, false);
+  if (st != W4A4_OK) return st;
+  if (!Y || !aligned16(Y) || stall_stage < 0) return W4A4_ERR_INVALID_ARG;
+  if (limit_ns == 0 || limit_ns > 100000000ull) return W4A4_ERR_INVALID_ARG;  // at most 0.1 s
+  DeviceGuard guard(h->ctx->device);
+  if (!guard.ok) return W4A4_ERR_CUDA;
+  return launch_gemm(h, M, expert_id, Y, static_cast<cudaStream_t>(stream), nullptr, 0, 0, nullptr, nullptr, true,
+                     stall_stage, limit_ns);
 }
 
 void w4a4_debug_fail_allocation_after(int n) { g_w4a4_alloc_countdown.store(n < 0 ? -1 : n); }

@@ -6,6 +6,9 @@
    operation, no tensor memory), with a limit of a millisecond or less.  What is checked is the contract the header
    states: the next status query reports W4A4_ERR_TIMEOUT once, the one after it W4A4_OK, and the context still
    computes correct results afterwards.
+   The same is then done to the real GEMM: `w4a4_debug_stalled_gemm` withholds one operand stage from every CTA, so
+   that the producer, both MMA-issuing warps and the epilogue warps all run into a 1 ms limit and leave through the
+   kernel's common tail (drain of copies in flight, release of tensor memory).
 2. Allocation failures.  A countdown hook makes the n-th device allocation fail as a refused cudaMalloc would.  Walking
    n over every allocation of w4a4_ctx_create and w4a4_pack_weights checks that each partial construction returns
    W4A4_ERR_ALLOC, leaks nothing (device memory in use returns to where it was) and leaves the library usable.
@@ -71,6 +74,36 @@ def test_the_context_computes_correctly_after_a_reported_timeout():
         ctx.check()
     assert ei.value.status == ERR_TIMEOUT
     assert forward_matches_oracle(ctx, L, layer, M, seed=8)
+    ctx.check()
+    L.close()
+    ctx.close()
+
+
+def test_a_stalled_gemm_pipeline_gives_up_cleans_up_and_the_context_recovers():
+    # The real GEMM (TMA producer, two MMA-issuing warps, sixteen epilogue warps, TMEM) with one operand stage
+    # withheld and a 1 ms wait limit: every role's wait runs out, the CTAs leave through the common tail (error
+    # word, drain, TMEM release) and the kernel ends by itself.  Then: TIMEOUT once, OK after, and a forward on
+    # the same context (which needs all 512 TMEM columns of every SM again) matches the oracle.
+    pkg_build.build()
+    w4.load_library()
+    M, K, N, r = 700, 1024, 512, 32
+    layer = gen.make_layer_direct(K, N, r, seed=6).to(DEV)
+    ctx = w4.Context(0, M, K, r)
+    L = w4.Layer(ctx, [layer], num_bins=1)
+    x = gen.make_activations(M, K, seed=12).to(DEV)
+    clip = torch.ones((1, 1, 1), dtype=torch.float32, device=DEV)
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device=DEV)
+    w4.w4a4_quantize_activations(L.ptr, x, M, 0, 0, clip)
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    w4.w4a4_debug_stalled_gemm(L.ptr, M, 0, y, 3, 1_000_000)
+    ev1.record()
+    torch.cuda.synchronize()
+    assert ev0.elapsed_time(ev1) < 500.0, "the stalled kernel must end by itself shortly after its limit"
+    assert w4.w4a4_query_status(ctx.ptr) == ERR_TIMEOUT
+    assert w4.w4a4_query_status(ctx.ptr) == 0
+    assert forward_matches_oracle(ctx, L, layer, M, seed=13)
     ctx.check()
     L.close()
     ctx.close()
