@@ -111,29 +111,6 @@ __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.
 
 // TMEM -> registers, shape 32x32b: thread i of the warp reads TMEM lane (base lane + i), 16 consecutive 32-bit
 // columns starting at the base column; v[c] is column c.  The load is asynchronous until tcgen05.wait::ld.
-//
-// The "_before" / "_after" variants carry scheduling pins for software pipelining.  A TMEM load writes its
-// registers at some point before the wait, so (1) it must not be moved above the last read of the buffer it
-// overwrites: `pin` is a register the caller still reads from that buffer, tied as an in/out operand; and
-// (2) arithmetic the caller wants to overlap with the load must not sink below the wait: the wait takes the
-// accumulators that arithmetic produces as in/out operands.
-__device__ __forceinline__ void tmem_ld_32x32b_x16_before(uint32_t taddr, uint32_t (&v)[16], uint32_t& pin) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%17];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "+r"(pin)
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld_after(float2 (&a)[8]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+f"(a[0].x), "+f"(a[0].y), "+f"(a[1].x), "+f"(a[1].y), "+f"(a[2].x), "+f"(a[2].y), "+f"(a[3].x),
-                 "+f"(a[3].y), "+f"(a[4].x), "+f"(a[4].y), "+f"(a[5].x), "+f"(a[5].y), "+f"(a[6].x), "+f"(a[6].y),
-                 "+f"(a[7].x), "+f"(a[7].y)
-               :
-               : "memory");
-}
 __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -203,17 +180,6 @@ __device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint
 // Arrives on the mbarrier at `cluster_addr` (this CTA's or the neighbour's) once the pair's MMAs issued so far are done.
 __device__ __forceinline__ void umma2_commit(uint32_t cluster_addr) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_addr) : "memory");
-}
-
-__device__ __forceinline__ void umma2_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n"
-      "}\n" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
 }
 
 // Shared-memory operand descriptor, K-major tile without swizzle (canonical layout: core matrices of 8 rows x
