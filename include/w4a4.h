@@ -317,8 +317,13 @@ w4a4_status_t w4a4_query_status(w4a4_ctx_t ctx);
  * of every CTA's sequence) never loaded: the consumers of that stage run into the limit, every role of the CTA
  * leaves through the kernel's common tail (error word, a drain period for copies in flight, release of tensor
  * memory), and Y is left partly written.  The next w4a4_query_status returns W4A4_ERR_TIMEOUT, and the context must
- * compute correctly afterwards.  Nothing faults or traps. */
+ * compute correctly afterwards.  Nothing faults or traps.
+ * w4a4_debug_set_tile_order forces the width, in 128-channel column tiles, of the super-columns in which the INT4
+ * GEMM walks its output tiles (all row blocks of one super-column before the next; the width is otherwise chosen so
+ * that a super-column's weight bytes take about two ninths of the L2); 0 restores the automatic choice.  Results do
+ * not depend on it; the tests use it to run every shape of the order on small layers. */
 w4a4_status_t w4a4_debug_wait_probe(w4a4_ctx_t ctx, uint64_t limit_ns, void* stream);
+w4a4_status_t w4a4_debug_set_tile_order(w4a4_ctx_t ctx, int super_column_tiles);
 w4a4_status_t w4a4_debug_stalled_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, int stall_stage,
                                       uint64_t limit_ns, void* stream);
 void w4a4_debug_fail_allocation_after(int n);

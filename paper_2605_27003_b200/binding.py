@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "w4a4_tile_shape", "w4a4_quantize_noalloc", "w4a4_clip_search",
     "w4a4_mx_pack_weights", "w4a4_mx_destroy", "w4a4_mx_handle_bytes", "w4a4_mx_linear_forward",
     "w4a4_mx_quantize_activations", "w4a4_mx_gemm_from_workspace", "w4a4_mx_debug_quantize", "w4a4_mx_clip_search",
-    "w4a4_mx_ffn_forward", "w4a4_mx_debug_fused_input", "w4a4_gptq_quantize", "w4a4_mx_gptq_quantize", "w4a4_gptq_accumulate", "w4a4_gptq_workspace_bytes", "w4a4_query_status", "w4a4_debug_wait_probe", "w4a4_debug_stalled_gemm",
+    "w4a4_mx_ffn_forward", "w4a4_mx_debug_fused_input", "w4a4_gptq_quantize", "w4a4_mx_gptq_quantize", "w4a4_gptq_accumulate", "w4a4_gptq_workspace_bytes", "w4a4_query_status", "w4a4_debug_wait_probe", "w4a4_debug_stalled_gemm", "w4a4_debug_set_tile_order",
     "w4a4_debug_fail_allocation_after", "w4a4_handle_bytes", "w4a4_ctx_bytes", "w4a4_status_string",
 )
 
@@ -113,6 +113,7 @@ def _lib():
         lib.w4a4_debug_wait_probe.argtypes = [vp, ctypes.c_uint64, vp]
         lib.w4a4_debug_stalled_gemm.argtypes = [vp, ci, ci, vp, ci, ctypes.c_uint64, vp]
         lib.w4a4_debug_fail_allocation_after.argtypes = [ci]
+        lib.w4a4_debug_set_tile_order.argtypes = [vp, ci]
         lib.w4a4_debug_fail_allocation_after.restype = None
         lib.w4a4_handle_bytes.argtypes = [vp]
         lib.w4a4_handle_bytes.restype = ctypes.c_size_t
@@ -391,6 +392,11 @@ def w4a4_debug_stalled_gemm(handle, M: int, expert_id: int, Y, stall_stage: int,
     """Test hook: the GEMM on the current workspace with one operand stage withheld and a short wait limit."""
     _check(_lib().w4a4_debug_stalled_gemm(handle, M, expert_id, _ptr(Y), int(stall_stage), int(limit_ns),
                                           _stream(stream)), "w4a4_debug_stalled_gemm")
+
+
+def w4a4_debug_set_tile_order(ctx, super_column_tiles: int):
+    """Test hook: forces the super-column width of the INT4 GEMM's tile order (0: automatic)."""
+    _check(_lib().w4a4_debug_set_tile_order(ctx, int(super_column_tiles)), "w4a4_debug_set_tile_order")
 
 
 def w4a4_debug_fail_allocation_after(n: int):

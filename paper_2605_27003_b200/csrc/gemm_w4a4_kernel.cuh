@@ -23,7 +23,7 @@
 // its S is the constant 1 (an MMA on a tile of ones), so the epilogue has a single loop.
 //
 // Persistent, one CTA (640 threads) per SM, 128 x 128 tiles, column tile fastest (the CTAs running at any moment
-// share a few row blocks of A and all of B through L2).  TMEM: two slots of 256 columns, one per group in flight:
+// share a few row blocks of A and a super-column of B through L2).  TMEM: two slots of 256 columns, one per group in flight:
 // columns 0..127 P_g, columns 128..255 S_g.  Warp roles:
 //   warp 0      producer: per stage of 128 K-codes (two groups) TMA loads of the A and B code tiles (16 KiB each,
 //               128-byte swizzle) and of the two scale-operand images, all onto the stage's mbarrier;
@@ -31,15 +31,25 @@
 //               commit onto tmem_full[slot];
 //   warp 3      scale-MMA issuer: per group one tcgen05.mma kind::f16 (K = 16) into the slot's S columns and a commit
 //               onto the same barrier (it counts two arrivals).  Two issuing threads because the issue of a
-//               tcgen05.mma waits for room in the tensor pipe's queue and an mbarrier test costs its thread well over a
-//               hundred cycles: one thread would put all of that on the hand-over path of every slot;
+//               tcgen05.mma waits for room in the tensor pipe's queue: one thread would put all of that on the
+//               hand-over path of every slot;
 //   warp 2      TMEM allocation;
 //   warps 4-19  epilogue: a thread owns one token row and 32 output channels.  Per group two round trips of two
 //               tcgen05.ld.32x32b.x16 (P and S of 16 columns) with the eight packed multiply-adds of the first half
 //               in between; the slot goes back to the issuing warps (tmem_empty[slot], 16 arrivals) as soon as the
 //               second half is in registers.  Measured alternatives (all four loads in one round trip; the second
 //               half's loads issued ahead of the first half's arithmetic; warps of a scheduler skewed against one
-//               another) were slower: a TMEM load in flight holds up the arithmetic behind it.
+//               another) were slower.
+// What bounds the kernel is the round trip of a TMEM slot (two slots, so two round trips overlap): epilogue releases it
+// -> issuing warps see that -> MMAs run -> commit -> epilogue sees that -> loads.  A lone warp's dependent instructions
+// cost 10-15 cycles each and a branch on a fresh mbarrier result ~70, so the hops are written as single instruction
+// sequences: wait_issue_* (try_wait loop, fence, predicated MMAs, commit: nothing between the barrier's answer and the
+// tcgen05.mma), wait_then_ld16 (try_wait loop, fence, first TMEM load), descriptors computed before the wait, and
+// predicated instead of branched single-lane instructions (umma_*_if, mbar_arrive_if).  A wait that outlasts the short
+// inline run falls back to the bounded wait of pipeline.cuh and the same instructions issued from C++.
+// Tile order: column tiles are walked in super-columns (GemmParams::sc_tiles column tiles wide, all row blocks of a
+// super-column before the next) sized so that the weight bytes a wave of CTAs touches stay in L2; with the plain
+// row-major order the 71 MB weight image of the FFN shapes streamed from DRAM once per 1.4 row blocks.
 // Every role loops warp-uniformly (waits are voted, only the TMA / tcgen05 instructions are predicated on one elected
 // lane), which keeps ring positions, addresses and descriptors in uniform registers.  All waits are bounded
 // (pipeline.cuh).  Finally + bias -> optional GELU -> BF16, or the squared error against a reference (clip search).
@@ -71,6 +81,114 @@ static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligne
 // warp and four epilogue warps).  Moving registers from the control warps to the epilogue with setmaxnreg was
 // measured and does not pay: at 104 the time is the same, at 112 the compiler's freer scheduling of the TMEM loads
 // against the multiply-adds made the kernel 7 % slower.
+
+// Wait for a TMEM slot and issue its MMAs in one instruction sequence: a short run of try_waits; on success the fence,
+// the (predicated) MMAs and the commit follow at once.  Returns 0 if the barrier did not complete within the run (the
+// caller then takes the bounded wait and issues from C++).
+__device__ __forceinline__ uint32_t wait_issue_f8x2(uint32_t go, uint32_t bar, uint32_t parity, uint32_t d_tmem, uint64_t a0, uint64_t b0,
+                                                    uint64_t a1, uint64_t b1, uint32_t idesc, uint32_t full_bar) {
+  uint32_t done;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q, r;\n"
+      ".reg .u32 n;\n"
+      "setp.ne.b32 q, %6, 0;\n"
+      "mov.u32 n, 32;\n"
+      "LAB_WAIT:\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "@p bra LAB_GO;\n"
+      "sub.u32 n, n, 1;\n"
+      "setp.ne.u32 r, n, 0;\n"
+      "@r bra LAB_WAIT;\n"
+      "mov.u32 %0, 0;\n"
+      "bra LAB_END;\n"
+      "LAB_GO:\n"
+      "tcgen05.fence::after_thread_sync;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%3], %4, %5, %7, 0;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%3], %8, %9, %7, 1;\n"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%10];\n"
+      "mov.u32 %0, 1;\n"
+      "LAB_END:\n"
+      "}\n"
+      : "=r"(done)
+      : "r"(bar), "r"(parity), "r"(d_tmem), "l"(a0), "l"(b0), "r"(go), "r"(idesc), "l"(a1), "l"(b1), "r"(full_bar)
+      : "memory");
+  return done;
+}
+__device__ __forceinline__ uint32_t wait_issue_f16(uint32_t go, uint32_t bar, uint32_t parity, uint32_t d_tmem, uint64_t a0, uint64_t b0,
+                                                   uint32_t idesc, uint32_t full_bar) {
+  uint32_t done;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, q, r;\n"
+      ".reg .u32 n;\n"
+      "setp.ne.b32 q, %6, 0;\n"
+      "mov.u32 n, 32;\n"
+      "LAB_WAIT:\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "@p bra LAB_GO;\n"
+      "sub.u32 n, n, 1;\n"
+      "setp.ne.u32 r, n, 0;\n"
+      "@r bra LAB_WAIT;\n"
+      "mov.u32 %0, 0;\n"
+      "bra LAB_END;\n"
+      "LAB_GO:\n"
+      "tcgen05.fence::after_thread_sync;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %7, 0;\n"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
+      "mov.u32 %0, 1;\n"
+      "LAB_END:\n"
+      "}\n"
+      : "=r"(done)
+      : "r"(bar), "r"(parity), "r"(d_tmem), "l"(a0), "l"(b0), "r"(go), "r"(idesc), "r"(full_bar)
+      : "memory");
+  return done;
+}
+
+// Wait for a full TMEM slot and start its first load in one instruction sequence.  Returns 0 if the barrier did not
+// complete within the run of try_waits (nothing was loaded then).
+__device__ __forceinline__ uint32_t wait_then_ld16(uint32_t bar, uint32_t parity, uint32_t taddr, uint32_t (&v)[16]) {
+  uint32_t done;
+  asm volatile(
+      "{\n"
+      ".reg .pred p, r;\n"
+      ".reg .u32 n;\n"
+      "mov.u32 n, 32;\n"
+      "LAB_WAIT:\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%17], %18;\n"
+      "@p bra LAB_GO;\n"
+      "sub.u32 n, n, 1;\n"
+      "setp.ne.u32 r, n, 0;\n"
+      "@r bra LAB_WAIT;\n"
+      "mov.u32 %16, 0;\n"
+      "bra LAB_END;\n"
+      "LAB_GO:\n"
+      "tcgen05.fence::after_thread_sync;\n"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%19];\n"
+      "mov.u32 %16, 1;\n"
+      "LAB_END:\n"
+      "}\n"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(done)
+      : "r"(bar), "r"(parity), "r"(taddr)
+      : "memory");
+  return done;
+}
+
+// Tile raster: column tiles are walked in super-columns of `sc` tiles (all row blocks of one super-column before the
+// next), so that the weight bytes a wave of CTAs touches stay in L2.  sc == tiles_n: plain row-major order.
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int sc, int& tm, int& tn) {
+  const int per_sc = tiles_m * sc;
+  const int full = tiles_n / sc;
+  int s_idx = tile / per_sc, rem = tile - s_idx * per_sc, width = sc;
+  if (s_idx >= full) {
+    s_idx = full;
+    rem = tile - full * per_sc;
+    width = tiles_n - full * sc;
+  }
+  tm = rem / width;
+  tn = s_idx * sc + (rem - tm * width);
+}
 
 // Ties a fragment to the tcgen05.wait::ld in front of it: the registers count as written there, so nothing that
 // reads them can be scheduled above the wait (an asm statement takes at most 30 operands, hence one statement per
@@ -145,6 +263,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int n_int_stages = (G + 1) >> 1;
   const int n_lr_stages = p.r > 0 ? (2 * p.r + 63) / 64 : 0;
   const int num_tiles = p.tiles_m * p.tiles_n;
+  const int sc_tiles = p.sc_tiles;
   const WaitEnv env{p.err, s_abort, p.wait_limit_ns};
 
   if (threadIdx.x == 0) {
@@ -192,7 +311,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       bool ok = true;
       int stage_no = 0;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+        int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, sc_tiles, tm, tn);
         const int m0 = tm * kBM, n0 = tn * kBN;
         for (int st = 0; st < n_lr_stages + n_int_stages; ++st) {
           ok = __all_sync(0xffffffffu, bounded_wait<64>(bar_op_empty + 8 * op.slot, op.parity ^ 1u, env, kErrProducerWait));
@@ -233,6 +353,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       constexpr uint32_t idesc_f8 = umma_idesc(1, 0, kBM, kBN);
       constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
       const bool issuer = elect_one_lane();
+      const uint32_t go = issuer ? 1u : 0u;
+      const int issue_lane = __ffs(__ballot_sync(0xffffffffu, issuer)) - 1;   // the decision below is the issuing lane's
       Ring<kGemmStages> op;
       Ring<kTmemSlots> tm;
       bool ok = true;
@@ -264,21 +386,23 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint32_t a = smem_base + op.slot * kStageBytes, b = a + kOpATile;
           const int groups = (2 * st + 1 < G) ? 2 : 1;
           for (int v = 0; v < groups; ++v) {
-            ok = __all_sync(0xffffffffu, bounded_wait<0, 1>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait));
-            if (!ok) break;
-            tc_fence_after_sync();
+            // everything the issue needs is ready before the wait that sits on the slot's round trip
             const uint32_t d = tmem_base + tm.slot * 2 * kBN;
             const uint32_t full_bar = bar_tmem_full + 8 * tm.slot;
-            tm.advance();
-            if (issuer) {
-              // bytes [64 v, 64 v + 64) of every code row: group v of the stage, two MMAs of K = 32
-              umma_f8(d, umma_desc_k_sw128(a, 64 * v), umma_desc_k_sw128(b, 64 * v), idesc_f8, 0u);
-              umma_f8(d, umma_desc_k_sw128(a, 64 * v + 32), umma_desc_k_sw128(b, 64 * v + 32), idesc_f8, 1u);
-              umma_commit(full_bar);
+            const uint64_t da0 = umma_desc_k_sw128(a, 64 * v), db0 = umma_desc_k_sw128(b, 64 * v);
+            const uint64_t da1 = umma_desc_k_sw128(a, 64 * v + 32), db1 = umma_desc_k_sw128(b, 64 * v + 32);
+            if (__shfl_sync(0xffffffffu, wait_issue_f8x2(go, bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, d, da0, db0, da1, db1, idesc_f8, full_bar), issue_lane) == 0) {
+              ok = __all_sync(0xffffffffu, bounded_wait<0, 1>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait));
+              if (!ok) break;
+              tc_fence_after_sync();
+              umma_f8_if(go, d, da0, db0, idesc_f8, 0u);
+              umma_f8_if(go, d, da1, db1, idesc_f8, 1u);
+              umma_commit_if(go, full_bar);
             }
+            tm.advance();
           }
           if (!ok) break;
-          if (issuer) umma_commit(bar_op_empty + 8 * op.slot);
+          umma_commit_if(go, bar_op_empty + 8 * op.slot);
           op.advance();
         }
       }
@@ -287,6 +411,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       // Walks the same slot uses as the code-MMA warp: S = 1 for the low-rank entry, S_g for the groups.
       constexpr uint32_t idesc_bf16 = umma_idesc(1, 1, kBM, kBN);
       const bool issuer = elect_one_lane();
+      const uint32_t go = issuer ? 1u : 0u;
+      const int issue_lane = __ffs(__ballot_sync(0xffffffffu, issuer)) - 1;   // the decision below is the issuing lane's
       Ring<kGemmStages> op;
       Ring<kTmemSlots> tm;
       bool ok = true;
@@ -315,20 +441,21 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           const uint32_t sa = smem_base + op.slot * kStageBytes + kOpATile + kOpBTile, sb = sa + kSopATile;
           const int groups = (2 * st + 1 < G) ? 2 : 1;
           for (int v = 0; v < groups; ++v) {
-            ok = __all_sync(0xffffffffu, bounded_wait<0, 1>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait));
-            if (!ok) break;
-            tc_fence_after_sync();
             const uint32_t d = tmem_base + tm.slot * 2 * kBN + kBN;
             const uint32_t full_bar = bar_tmem_full + 8 * tm.slot;
-            tm.advance();
-            if (issuer) {
-              const uint32_t cb = sb + (kSopBTile / 2) * v;   // the channel side's chunk of this group
-              umma_f16(d, umma_desc_k_plain(sa, zero_base - sa, 128), umma_desc_k_plain(cb, zero_base - cb, 128), idesc_bf16, 0u);
-              umma_commit(full_bar);
+            const uint32_t cb = sb + (kSopBTile / 2) * v;   // the channel side's chunk of this group
+            const uint64_t dsa = umma_desc_k_plain(sa, zero_base - sa, 128), dsb = umma_desc_k_plain(cb, zero_base - cb, 128);
+            if (__shfl_sync(0xffffffffu, wait_issue_f16(go, bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, d, dsa, dsb, idesc_bf16, full_bar), issue_lane) == 0) {
+              ok = __all_sync(0xffffffffu, bounded_wait<0, 1>(bar_tmem_empty + 8 * tm.slot, tm.parity ^ 1u, env, kErrMmaWait));
+              if (!ok) break;
+              tc_fence_after_sync();
+              umma_f16_if(go, d, dsa, dsb, idesc_bf16, 0u);
+              umma_commit_if(go, full_bar);
             }
+            tm.advance();
           }
           if (!ok) break;
-          if (issuer) umma_commit(bar_op_empty + 8 * op.slot);
+          umma_commit_if(go, bar_op_empty + 8 * op.slot);
           op.advance();
         }
       }
@@ -345,23 +472,27 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       Ring<kTmemSlots> tm;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+        int tm_e, tn_e;
+        tile_coords(tile, p.tiles_m, p.tiles_n, sc_tiles, tm_e, tn_e);
+        const int m0 = tm_e * kBM, n0 = tn_e * kBN;
         const bool dbg_tile = DEBUG && p.dbg_P != nullptr && m0 == p.dbg_m0 && n0 == p.dbg_n0;
         float2 acc[16];  // pair k: channels ch0 + 2 k, ch0 + 2 k + 1
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc[j] = make_float2(0.0f, 0.0f);
         for (int e = 0; e < entries; ++e) {
-          ok = __all_sync(0xffffffffu, bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait));
-          if (!ok) break;
-          tc_fence_after_sync();
           const uint32_t t = t_lane + tm.slot * 2 * kBN;
+          uint32_t pv[16], sv[16];
+          if (!__all_sync(0xffffffffu, wait_then_ld16(bar_tmem_full + 8 * tm.slot, tm.parity, t, pv) != 0)) {
+            ok = __all_sync(0xffffffffu, bounded_wait(bar_tmem_full + 8 * tm.slot, tm.parity, env, kErrEpilogueWait));
+            if (!ok) break;
+            tc_fence_after_sync();
+            tmem_ld_32x32b_x16(t, pv);
+          }
           int32_t* d0 = nullptr;
           if (DEBUG) {
             const int g = e - (n_lr_stages > 0 ? 1 : 0);
             if (dbg_tile && g >= 0) d0 = p.dbg_P + (static_cast<size_t>(32 * quarter + lane) * G + g) * kBN + kEpiCols * colblk;
           }
-          uint32_t pv[16], sv[16];
-          tmem_ld_32x32b_x16(t, pv);
           tmem_ld_32x32b_x16(t + kBN, sv);
           tmem_wait_ld();
           tie_fragment(pv);
@@ -375,7 +506,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           // The whole slot is in registers: hand it back to the MMA warps.
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(bar_tmem_empty + 8 * tm.slot);
+          mbar_arrive_if(lane == 0 ? 1u : 0u, bar_tmem_empty + 8 * tm.slot);
           tm.advance();
           fma_fragment<DEBUG>(pv, sv, acc + 8, DEBUG && d0 ? d0 + 16 : nullptr);
         }

@@ -34,6 +34,8 @@ struct w4a4_ctx {
   int* d_err = nullptr;       // device error word
   size_t bytes = 0;
   int num_sms = 0;
+  size_t l2_bytes = 0;        // size of the device's L2 (sizes the GEMM's tile order)
+  int debug_sc_tiles = 0;     // test hook: forced super-column width of the GEMM's tile order (0: automatic)
   EncodeTiledFn encode = nullptr;
   // Host-buffer forward (w4a4_linear_forward_host): staging buffers, copy streams and events.
   int host_chunk_rows = 0, host_max_N = 0;

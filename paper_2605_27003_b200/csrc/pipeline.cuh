@@ -126,6 +126,7 @@ struct GemmParams {
   uint16_t* Y;          // [M, N] BF16
   int M, N, K, r;
   int tiles_m, tiles_n;
+  int sc_tiles;         // column tiles per super-column of the tile order (tiles_n: plain row-major order)
   int* err;
   uint64_t wait_limit_ns;
   int32_t* dbg_P;       // debug tap: [kBM, G, kBN] or nullptr

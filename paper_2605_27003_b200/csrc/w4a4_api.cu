@@ -226,6 +226,21 @@ w4a4_status_t launch_gemm(w4a4_handle_t h, int M, int expert_id, void* Y, cudaSt
   p.r = h->r;
   p.tiles_m = (M + kBM - 1) / kBM;
   p.tiles_n = h->N / kBN;
+  // Tile order: super-columns whose weight bytes (kBN x K per column tile) take about two ninths of L2 (28 MB of
+  // 126), of equal width; a weight image that fits such a budget as a whole keeps the plain row-major order.
+  {
+    const size_t budget = ctx->l2_bytes * 2 / 9;
+    int sc = static_cast<int>(budget / (static_cast<size_t>(kBN) * h->K));
+    if (sc < 1) sc = 1;
+    if (sc >= p.tiles_n) {
+      sc = p.tiles_n;
+    } else {
+      const int ns = (p.tiles_n + sc - 1) / sc;
+      sc = (p.tiles_n + ns - 1) / ns;
+    }
+    if (ctx->debug_sc_tiles > 0) sc = ctx->debug_sc_tiles < p.tiles_n ? ctx->debug_sc_tiles : p.tiles_n;
+    p.sc_tiles = sc;
+  }
   p.err = ctx->d_err;
   p.wait_limit_ns = wait_limit_ns;
   p.dbg_stall_stage = stall_stage;
@@ -309,6 +324,7 @@ w4a4_status_t w4a4_ctx_create(int device, int max_M, int max_K, int max_r, w4a4_
   ctx->max_K = max_K;
   ctx->max_r = max_r;
   ctx->num_sms = prop.multiProcessorCount;
+  ctx->l2_bytes = static_cast<size_t>(prop.l2CacheSize);
   ctx->scales_ld = (max_M + 3) & ~3;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -767,6 +783,12 @@ w4a4_status_t w4a4_debug_stalled_gemm(w4a4_handle_t h, int M, int expert_id, voi
   if (!guard.ok) return W4A4_ERR_CUDA;
   return launch_gemm(h, M, expert_id, Y, static_cast<cudaStream_t>(stream), nullptr, 0, 0, nullptr, nullptr, true,
                      stall_stage, limit_ns);
+}
+
+w4a4_status_t w4a4_debug_set_tile_order(w4a4_ctx_t ctx, int super_column_tiles) {
+  if (!ctx || super_column_tiles < 0) return W4A4_ERR_INVALID_ARG;
+  ctx->debug_sc_tiles = super_column_tiles;
+  return W4A4_OK;
 }
 
 void w4a4_debug_fail_allocation_after(int n) { g_w4a4_alloc_countdown.store(n < 0 ? -1 : n); }

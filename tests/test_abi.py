@@ -45,6 +45,7 @@ def test_null_and_bad_arguments_are_rejected_without_a_device():
     assert lib.w4a4_query_status(None) == 1
     assert lib.w4a4_debug_wait_probe(None, 1000, None) == 1
     assert lib.w4a4_debug_stalled_gemm(None, 1, 0, None, 0, 1000, None) == 1
+    assert lib.w4a4_debug_set_tile_order(None, 2) == 1
     lib.w4a4_debug_fail_allocation_after(-1)                          # disarming needs no device
     lib.w4a4_destroy(None)
     lib.w4a4_ctx_destroy(None)

@@ -130,6 +130,35 @@ def tiny_inputs(M=256, K=512, N=512, r=16, seed=0, bias=False):
     return x, layer
 
 
+@pytest.mark.parametrize("sc", [1, 2, 3, 5])
+def test_tile_order_in_super_columns_gives_the_same_result(sc):
+    # The GEMM walks its output tiles in super-columns (all row blocks of `sc` column tiles before the next `sc`), sized
+    # for the L2 at full scale.  Forced here on a layer of 3 row blocks x 5 column tiles: widths that divide the
+    # column count, that leave a narrower last super-column, and the plain order; every tile's output against the
+    # oracle and the partial sums of the first and last tile.
+    M, K, N, r = 300, 256, 640, 16
+    x, layer = tiny_inputs(M, K, N, r, seed=21, bias=True)
+    clip = torch.full((1, 1, 1), 0.8, dtype=torch.float32)
+    ctx = w4.Context(0, M, K, r)
+    w4.w4a4_debug_set_tile_order(ctx.ptr, sc)
+    L = w4.Layer(ctx, [layer.to(DEV)], num_bins=1)
+    y = L.forward(x.to(DEV), 0, 0, clip.to(DEV))
+    bm, bn = w4.w4a4_tile_shape()
+    P = torch.full((bm, K // G, bn), -5, dtype=torch.int32, device=DEV)
+    y2 = torch.empty_like(y)
+    w4.w4a4_debug_partials(L.ptr, x.to(DEV), M, 0, 0, clip.to(DEV), y2, 256, 512, P)
+    torch.cuda.synchronize()
+    ctx.check()
+    ref = oracle_rows(x, layer, 0.8, want_partials=True)
+    worst, _ = y_within_tolerance(y, ref["Y64"])
+    assert worst <= 1.0 and torch.equal(y, y2)
+    Pg = P.cpu().numpy()
+    for row in range(256, M):
+        assert np.array_equal(Pg[row - 256], ref["P"][row][:, 512:640])
+    L.close()
+    ctx.close()
+
+
 def test_tiny_config_full_parity():
     # M=256, K=N=512, r=16, one bin with rho=0.9, no bias; every row, every tile's partial sums.
     x, layer = tiny_inputs()
