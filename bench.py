@@ -35,7 +35,7 @@ NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_HBM_GBS = 7700.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, each from one single-launch ncu capture of the kernel as
 # it stands (summaries under profiles/); None where no capture exists for that kernel and workload.
-NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 537.9e6, ("quantize", "attn_proj"): 503.3e6}
+NCU_TRAFFIC_BYTES = {("gemm", "attn_proj"): 545.9e6, ("quantize", "attn_proj"): 503.3e6}
 
 
 def max_over_ranks(ms: float, dist, device="cpu") -> float:
