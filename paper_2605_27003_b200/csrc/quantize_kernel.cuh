@@ -218,7 +218,9 @@ __device__ __forceinline__ uint2 sop_slots_activation(float s) {
 }
 
 template <int R, int WARPS, int FORMAT>
-__global__ void __launch_bounds__(32 * WARPS, 1)
+// Sixteen resident warps per SM (at most 128 registers) at every rank, so that the 2048 warps of row blocks of the
+// DiT shapes fit one wave: at 130-160 registers the wide ranks ran 1.15 waves.
+__global__ void __launch_bounds__(32 * WARPS, 16 / WARPS)
 quantize_kernel(const uint16_t* __restrict__ X, int M, int K, const float* __restrict__ rlam,
                 const float* __restrict__ clip_table, int clip_index, const uint2* __restrict__ l1frag,
                 uint8_t* __restrict__ codes, float* __restrict__ scales, int scales_ld,
