@@ -43,10 +43,10 @@
 // What bounds the kernel is the round trip of a TMEM slot (two slots, so two round trips overlap): epilogue releases it
 // -> issuing warps see that -> MMAs run -> commit -> epilogue sees that -> loads.  A lone warp's dependent instructions
 // cost 10-15 cycles each and a branch on a fresh mbarrier result ~70, so the hops are written as single instruction
-// sequences: wait_issue_* (try_wait loop, fence, predicated MMAs, commit: nothing between the barrier's answer and the
-// tcgen05.mma), wait_then_ld16 (try_wait loop, fence, first TMEM load), descriptors computed before the wait, and
-// predicated instead of branched single-lane instructions (umma_*_if, mbar_arrive_if).  A wait that outlasts the short
-// inline run falls back to the bounded wait of pipeline.cuh and the same instructions issued from C++.
+// sequences without branches: wait_issue_* (try_wait, then fence, MMAs and commit predicated on its answer),
+// wait_then_ld16 (try_wait, then fence and first TMEM load predicated on its answer), descriptors computed before the wait, and
+// predicated instead of branched single-lane instructions (umma_*_if, mbar_arrive_if).  A wait that outlasts the
+// try_wait falls back to the bounded wait of pipeline.cuh and the same instructions issued from C++.
 // Tile order: column tiles are walked in super-columns (GemmParams::sc_tiles column tiles wide, all row blocks of a
 // super-column before the next) sized so that the weight bytes a wave of CTAs touches stay in L2; with the plain
 // row-major order the 71 MB weight image of the FFN shapes streamed from DRAM once per 1.4 row blocks.
@@ -82,33 +82,25 @@ static_assert(kStageBytes % 1024 == 0, "operand tiles must stay 1024-byte aligne
 // measured and does not pay: at 104 the time is the same, at 112 the compiler's freer scheduling of the TMEM loads
 // against the multiply-adds made the kernel 7 % slower.
 
-// Wait for a TMEM slot and issue its MMAs in one instruction sequence: a short run of try_waits; on success the fence,
-// the (predicated) MMAs and the commit follow at once.  Returns 0 if the barrier did not complete within the run (the
-// caller then takes the bounded wait and issues from C++).
+// Wait for a TMEM slot and issue its MMAs in one branch-free instruction sequence: one try_wait (it blocks in hardware
+// for a while before it gives up), then the fence, the MMAs and the commit predicated on its answer.  A branch on the
+// fresh answer would hold the warp ~70 cycles; a second try_wait predicated on the first one's failure costs its
+// latency even when it is skipped (both measured slower).  Returns 0 if the barrier did not complete (the caller then
+// takes the bounded wait and issues from C++).
 __device__ __forceinline__ uint32_t wait_issue_f8x2(uint32_t go, uint32_t bar, uint32_t parity, uint32_t d_tmem, uint64_t a0, uint64_t b0,
                                                     uint64_t a1, uint64_t b1, uint32_t idesc, uint32_t full_bar) {
   uint32_t done;
   asm volatile(
       "{\n"
-      ".reg .pred p, q, r;\n"
-      ".reg .u32 n;\n"
+      ".reg .pred p, q, pq;\n"
       "setp.ne.b32 q, %6, 0;\n"
-      "mov.u32 n, 32;\n"
-      "LAB_WAIT:\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "@p bra LAB_GO;\n"
-      "sub.u32 n, n, 1;\n"
-      "setp.ne.u32 r, n, 0;\n"
-      "@r bra LAB_WAIT;\n"
-      "mov.u32 %0, 0;\n"
-      "bra LAB_END;\n"
-      "LAB_GO:\n"
-      "tcgen05.fence::after_thread_sync;\n"
-      "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%3], %4, %5, %7, 0;\n"
-      "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%3], %8, %9, %7, 1;\n"
-      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%10];\n"
-      "mov.u32 %0, 1;\n"
-      "LAB_END:\n"
+      "and.pred pq, p, q;\n"
+      "@p tcgen05.fence::after_thread_sync;\n"
+      "@pq tcgen05.mma.cta_group::1.kind::f8f6f4 [%3], %4, %5, %7, 0;\n"
+      "@pq tcgen05.mma.cta_group::1.kind::f8f6f4 [%3], %8, %9, %7, 1;\n"
+      "@pq tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%10];\n"
+      "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(done)
       : "r"(bar), "r"(parity), "r"(d_tmem), "l"(a0), "l"(b0), "r"(go), "r"(idesc), "l"(a1), "l"(b1), "r"(full_bar)
@@ -120,24 +112,14 @@ __device__ __forceinline__ uint32_t wait_issue_f16(uint32_t go, uint32_t bar, ui
   uint32_t done;
   asm volatile(
       "{\n"
-      ".reg .pred p, q, r;\n"
-      ".reg .u32 n;\n"
+      ".reg .pred p, q, pq;\n"
       "setp.ne.b32 q, %6, 0;\n"
-      "mov.u32 n, 32;\n"
-      "LAB_WAIT:\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "@p bra LAB_GO;\n"
-      "sub.u32 n, n, 1;\n"
-      "setp.ne.u32 r, n, 0;\n"
-      "@r bra LAB_WAIT;\n"
-      "mov.u32 %0, 0;\n"
-      "bra LAB_END;\n"
-      "LAB_GO:\n"
-      "tcgen05.fence::after_thread_sync;\n"
-      "@q tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %7, 0;\n"
-      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
-      "mov.u32 %0, 1;\n"
-      "LAB_END:\n"
+      "and.pred pq, p, q;\n"
+      "@p tcgen05.fence::after_thread_sync;\n"
+      "@pq tcgen05.mma.cta_group::1.kind::f16 [%3], %4, %5, %7, 0;\n"
+      "@pq tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%8];\n"
+      "selp.u32 %0, 1, 0, p;\n"
       "}\n"
       : "=r"(done)
       : "r"(bar), "r"(parity), "r"(d_tmem), "l"(a0), "l"(b0), "r"(go), "r"(idesc), "r"(full_bar)
@@ -145,28 +127,17 @@ __device__ __forceinline__ uint32_t wait_issue_f16(uint32_t go, uint32_t bar, ui
   return done;
 }
 
-// Wait for a full TMEM slot and start its first load in one instruction sequence.  Returns 0 if the barrier did not
-// complete within the run of try_waits (nothing was loaded then).
+// Wait for a full TMEM slot and start its first load in one branch-free instruction sequence.  Returns 0 if the barrier
+// did not complete within the try_wait (nothing was loaded then).
 __device__ __forceinline__ uint32_t wait_then_ld16(uint32_t bar, uint32_t parity, uint32_t taddr, uint32_t (&v)[16]) {
   uint32_t done;
   asm volatile(
       "{\n"
-      ".reg .pred p, r;\n"
-      ".reg .u32 n;\n"
-      "mov.u32 n, 32;\n"
-      "LAB_WAIT:\n"
+      ".reg .pred p;\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%17], %18;\n"
-      "@p bra LAB_GO;\n"
-      "sub.u32 n, n, 1;\n"
-      "setp.ne.u32 r, n, 0;\n"
-      "@r bra LAB_WAIT;\n"
-      "mov.u32 %16, 0;\n"
-      "bra LAB_END;\n"
-      "LAB_GO:\n"
-      "tcgen05.fence::after_thread_sync;\n"
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%19];\n"
-      "mov.u32 %16, 1;\n"
-      "LAB_END:\n"
+      "@p tcgen05.fence::after_thread_sync;\n"
+      "@p tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%19];\n"
+      "selp.u32 %16, 1, 0, p;\n"
       "}\n"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(done)
