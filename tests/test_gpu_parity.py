@@ -262,6 +262,25 @@ def test_attention_projection_full_size_sampled_rows():
         run_case(x, [layer], clip, 0, b, rows=rows, check_partials_tiles=[(0, 0), (last, N - 128)])
 
 
+def test_packed_qkv_full_size_sampled_rows():
+    # The self-attention q, k and v of the DiT workload as one layer: M = 32760, K = 5120, N = 3 x 5120, joint rank 96
+    # (three rank-32 projections; L2 block-diagonal), direct-recipe constants.  At this size the activation kernel runs
+    # its widest instantiation, the GEMM three low-rank stages per tile and two super-columns of 60 column tiles.
+    M, K, N1, r = 32760, 5120, 5120, 32
+    lay = gen.make_layer_direct(K, 3 * N1, 3 * r, seed=4400, device=DEV)
+    for i in range(3):
+        for j in range(3):
+            if i != j:
+                lay.L2[r * i:r * (i + 1), N1 * j:N1 * (j + 1)] = 0
+    lay = lay.to("cpu")
+    clip = gen.make_clip_table(1, 1, 8, [(0.6, 1.0)], seed=5)
+    x = gen.make_activations(M, K, sigma=gen.sigma_for_bin(2), outlier_idx=gen.outlier_channels(K, 0.01, 44), outlier_gain=50.0,
+                             seed=4401, device=DEV).cpu()
+    rows = sampled_rows(M, 64, 9)
+    last = (M - 1) // 128 * 128
+    run_case(x, [lay], clip, 0, 2, rows=rows, check_partials_tiles=[(0, 0), (last, 3 * N1 - 128)])
+
+
 def test_ffn_pair_full_size_sampled_rows():
     # up 5120 -> 13824 and down 13824 -> 5120 at M = 32760; the down input is GELU of a Gaussian with
     # 1% outlier channels x80; two experts with their own clip tables.
